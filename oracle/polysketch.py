@@ -1,0 +1,280 @@
+"""CPU oracle for causal polynomial-sketch (Polysketch) attention, fp64.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain reference that the
+CUDA library is checked against.  It shares no code with the CUDA path and the
+product never imports it: only the tests, the smoke check and the benchmark's
+CPU-baseline leg may call it.
+
+Everything here works on ONE (batch, head) slice: Q, K, V are (n, h) arrays,
+G1, G2 are (h, r).  Arithmetic is float64 throughout.  Matrix products use
+numpy's matmul as a library primitive; nothing is blocked, fused or reordered
+beyond what the cited definition or algorithm states.
+
+Notation (paper -> here)
+  M = A^{(x)2} S               half sketch, Section 2.2 / Algorithm 1 (p = 2 level)
+  phi'(A) = M^{(x)2}           self-tensored features, Algorithm 1 (PolySketchNonNegative)
+  lt(.)                        keep the lower triangle INCLUDING the diagonal (Section 1.2)
+  D~ = diag(1 + lt(..) 1)      row normaliser of Section 3 (the "1 +" is part of it)
+  H_l, Z_l, P_l                per-block state, exclusive prefix, diagonal block (Section 3.1)
+
+Pins (tests/test_oracle_*.py): exact-feature case against looped (q.k)^4
+attention, hand-worked rational example, G = I closed form, Monte-Carlo mean and
+closed-form variance of the sketch, V = 1 closed form, n = 1 closed form,
+causality, block-size invariance, lt-multiply against a dense triangle, central
+finite differences for every gradient, dV against the explicit weight matrix.
+No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _f64(x):
+    return np.asarray(x, dtype=F64)
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 1
+# ---------------------------------------------------------------------------
+def polysketch_with_negativity(A, gaussians, p):
+    """Algorithm 1, PolySketchWithNegativity(A, r, p): A^{(x)p} S.
+
+    `gaussians` supplies the matrices the algorithm would sample, in the order
+    the recursion consumes them (left sub-call first, then right sub-call, then
+    this level's own G1, G2), so that the same S can be applied to Q and to K
+    (Definition 2.1 uses one S on both sides).  p = 1 returns A; p = 2 uses two
+    (m x r) matrices; p = 4 uses 2 + 2 (m x r) and then two (r x r).
+    """
+    A = _f64(A)
+    if p == 1:
+        return A, gaussians
+    if p < 1 or p % 2:
+        raise ValueError("p must be a power of two")
+    M1, rest = polysketch_with_negativity(A, gaussians, p // 2)
+    M2, rest = polysketch_with_negativity(A, rest, p // 2)
+    G1, G2 = _f64(rest[0]), _f64(rest[1])
+    r = G1.shape[1]
+    return np.sqrt(1.0 / r) * ((M1 @ G1) * (M2 @ G2)), rest[2:]
+
+
+def half_sketch(X, G1, G2):
+    """Degree-2 level of Algorithm 1 (Section 2.2): sqrt(1/r) [(X G1) * (X G2)]."""
+    M, rest = polysketch_with_negativity(X, [G1, G2], 2)
+    assert len(rest) == 0
+    return M
+
+
+def self_tensor(M):
+    """Row-wise M^{(x)2}: entry (a, b) of the Kronecker square sits at a*r + b
+    (the ordering of the Kronecker product in Section 1.2)."""
+    M = _f64(M)
+    n, r = M.shape
+    return (M[:, :, None] * M[:, None, :]).reshape(n, r * r)
+
+
+def polysketch_non_negative(A, G1, G2):
+    """Algorithm 1, PolySketchNonNegative(A, r, 4): phi'(A) = (A^{(x)2} S)^{(x)2}."""
+    return self_tensor(half_sketch(A, G1, G2))
+
+
+# ---------------------------------------------------------------------------
+# Definitions: Section 2.1 (exact polynomial attention), Section 3 (causal
+# Polysketch attention).  Quadratic in n; these are the plain definitions.
+# ---------------------------------------------------------------------------
+def lt(M):
+    """Lower-triangular part including the diagonal (j <= i), Section 1.2."""
+    return np.tril(_f64(M))
+
+
+def causal_attention_from_features(PhiQ, PhiK, V):
+    """Section 3: D~^{-1} lt(phi'(Q) phi'(K)^T) V with D~ = diag(1 + lt(..) 1).
+
+    Returns (O, d) with d the diagonal of D~.
+    """
+    W = lt(_f64(PhiQ) @ _f64(PhiK).T)
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
+def causal_polysketch_attention(Q, K, V, G1, G2):
+    """Section 3 with phi' from Algorithm 1 (p = 4), features materialised."""
+    return causal_attention_from_features(
+        polysketch_non_negative(Q, G1, G2), polysketch_non_negative(K, G1, G2), V)
+
+
+def causal_weights(Q, K, G1, G2):
+    """lt(phi'(Q) phi'(K)^T) through the identity <a^{(x)2}, b^{(x)2}> = <a,b>^2
+    (Section 2.2): entries (m(q_i) . m(k_j))^2 for j <= i, zero above."""
+    s = half_sketch(Q, G1, G2) @ half_sketch(K, G1, G2).T
+    return lt(s * s)
+
+
+def causal_exact_polynomial_attention(Q, K, V, p):
+    """Section 2.1 with a causal mask: weights <q_i,k_j>^p / (1 + sum_{j'<=i} <q_i,k_j'>^p)."""
+    W = lt((_f64(Q) @ _f64(K).T) ** p)
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
+# ---------------------------------------------------------------------------
+# Section 3.1: block lower-triangular multiplication
+# ---------------------------------------------------------------------------
+def lt_multiply_blocked(A, B, C, b, diag_block=None):
+    """lt(A B^T) C by the block algorithm of Section 3.1.
+
+    Blocks of b consecutive rows (n = t*b).  H_l = sum_{i in block l} b_i c_i^T,
+    Z_l = sum_{j<l} H_j (sequential prefix, as the authors use),
+    P_l = lt(A_l B_l^T) C_l, and rows of block l are P_l + A_l Z_l.
+    `diag_block(l)` may return lt(A_l B_l^T) computed some other way (the
+    (L R^T)^2 shortcut of Section 3.1); default is the direct product.
+    """
+    A, B, C = _f64(A), _f64(B), _f64(C)
+    n, m = A.shape
+    k = C.shape[1]
+    if n % b:
+        raise ValueError("n must be a multiple of the block size")
+    t = n // b
+    out = np.empty((n, k), dtype=F64)
+    Z = np.zeros((m, k), dtype=F64)
+    for l in range(t):
+        rows = slice(l * b, (l + 1) * b)
+        Al, Bl, Cl = A[rows], B[rows], C[rows]
+        T = lt(Al @ Bl.T) if diag_block is None else diag_block(l)
+        P = T @ Cl
+        out[rows] = P + Al @ Z
+        H = Bl.T @ Cl
+        Z = Z + H
+    return out
+
+
+def causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal="LR"):
+    """Causal Polysketch attention in time linear in n (Section 3.1).
+
+    A = phi'(Q), B = phi'(K), C = [V | 1_n]; the last output column is the
+    normaliser without its "1 +".  diagonal="phi" forms the diagonal blocks from
+    the r^2-dimensional features, diagonal="LR" from (L R^T)^2 with L, R the
+    b x r half sketches of the block.
+    """
+    V = _f64(V)
+    n, h = V.shape
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    C = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    if diagonal == "phi":
+        diag_block = None
+    elif diagonal == "LR":
+        def diag_block(l):
+            L, R = Mq[l * b:(l + 1) * b], Mk[l * b:(l + 1) * b]
+            return lt((L @ R.T) ** 2)
+    else:
+        raise ValueError(diagonal)
+    N = lt_multiply_blocked(self_tensor(Mq), self_tensor(Mk), C, b, diag_block)
+    d = 1.0 + N[:, h]
+    return N[:, :h] / d[:, None], d
+
+
+# ---------------------------------------------------------------------------
+# Backward.  The paper differentiates automatically and prints no formulas;
+# these are the derivatives of the definitions above, taken by hand:
+#   O_i = N_i / d_i,  N_i = sum_{j<=i} W_ij v_j,  d_i = 1 + sum_{j<=i} W_ij,
+#   W_ij = s_ij^2,  s_ij = m(q_i) . m(k_j),  m(x) = (x G1)*(x G2)/sqrt(r).
+# With g = dL/dO:  dL/dN_i = g_i/d_i,  dL/dd_i = -(g_i . O_i)/d_i, so with
+#   E_i = [ g_i/d_i | -(g_i . O_i)/d_i ]  and  V~_j = [ v_j | 1 ]
+# dL/dW_ij = E_i . V~_j for j <= i.
+# ---------------------------------------------------------------------------
+def _backward_rows(O, d, dO):
+    O, d, dO = _f64(O), _f64(d), _f64(dO)
+    return np.concatenate([dO / d[:, None],
+                           -((dO * O).sum(axis=1) / d)[:, None]], axis=1)
+
+
+def _sketch_backward(X, G1, G2, dM):
+    """Chain rule through m(x): dX = ((dM*A2) G1^T + (dM*A1) G2^T)/sqrt(r)."""
+    X, G1, G2 = _f64(X), _f64(G1), _f64(G2)
+    r = G1.shape[1]
+    A1, A2 = X @ G1, X @ G2
+    return ((dM * A2) @ G1.T + (dM * A1) @ G2.T) / np.sqrt(r)
+
+
+def causal_polysketch_attention_backward(Q, K, V, G1, G2, dO):
+    """Gradients (dQ, dK, dV) of sum(dO * O) through the quadratic definition."""
+    V = _f64(V)
+    n, h = V.shape
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    s = Mq @ Mk.T
+    W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = lt(E @ Vt.T)
+    dV = W.T @ E[:, :h]
+    ds = 2.0 * s * dW
+    dMq = ds @ Mk
+    dMk = ds.T @ Mq
+    return (_sketch_backward(Q, G1, G2, dMq), _sketch_backward(K, G1, G2, dMk), dV)
+
+
+def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b):
+    """Same gradients in time linear in n, in the style of Section 3.1.
+
+    Forward sweep carries Z_l = sum_{blocks < l} phi'(K)^T V~ (the forward's
+    own prefix); reverse sweep carries R_l = sum_{blocks > l} phi'(Q)^T E.
+    For a row in block l:  d phi'(q_i) = Z_l E_i,  d phi'(k_j) = R_l V~_j,
+    dV~_j = R_l^T phi'(k_j); the same-block pairs go through the b x b tile
+    exactly as in the forward.  d m = (mat(d phi') + mat(d phi')^T) m because
+    phi'(m)[a*r+b] = m_a m_b.
+    """
+    V = _f64(V)
+    n, h = V.shape
+    if n % b:
+        raise ValueError("n must be a multiple of the block size")
+    t = n // b
+    G1 = _f64(G1)
+    r = G1.shape[1]
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    O, d = causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal="LR")
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    PhiQ, PhiK = self_tensor(Mq), self_tensor(Mk)
+    dMq = np.zeros_like(Mq)
+    dMk = np.zeros_like(Mk)
+    dVt = np.zeros_like(Vt)
+
+    def untensor(dPhi, M):
+        T = dPhi.reshape(-1, r, r)
+        return np.einsum("nab,nb->na", T + T.transpose(0, 2, 1), M)
+
+    # same-block pairs and the forward sweep (earlier blocks -> queries)
+    Z = np.zeros((r * r, h + 1), dtype=F64)
+    for l in range(t):
+        rows = slice(l * b, (l + 1) * b)
+        s = Mq[rows] @ Mk[rows].T
+        W = lt(s * s)
+        dW = lt(E[rows] @ Vt[rows].T)
+        ds = 2.0 * s * dW
+        dMq[rows] += ds @ Mk[rows]
+        dMk[rows] += ds.T @ Mq[rows]
+        dVt[rows] += W.T @ E[rows]
+        dMq[rows] += untensor(E[rows] @ Z.T, Mq[rows])
+        Z = Z + PhiK[rows].T @ Vt[rows]
+    # reverse sweep (later blocks -> keys and values)
+    R = np.zeros((r * r, h + 1), dtype=F64)
+    for l in range(t - 1, -1, -1):
+        rows = slice(l * b, (l + 1) * b)
+        dMk[rows] += untensor(Vt[rows] @ R.T, Mk[rows])
+        dVt[rows] += PhiK[rows] @ R
+        R = R + PhiQ[rows].T @ E[rows]
+    return (_sketch_backward(Q, G1, G2, dMq), _sketch_backward(K, G1, G2, dMk), dVt[:, :h])
+
+
+# ---------------------------------------------------------------------------
+# Error metric used by the parity tests and the benchmark
+# ---------------------------------------------------------------------------
+def rel_l2(x, ref):
+    """|| x - ref ||_2 / || ref ||_2 over the whole tensor (fp64)."""
+    x, ref = _f64(x), _f64(ref)
+    den = np.linalg.norm(ref.ravel())
+    num = np.linalg.norm((x - ref).ravel())
+    return num / den if den > 0 else num
