@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of causal Polysketch attention (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl psk|reference]
+
+One "step" is one pass of the whole hot path over one batch: psk_causal_attn_fwd
+followed by psk_causal_attn_bwd (forward only for forward-only workloads).  Prints ONE
+JSON line (rank 0).  Inputs are synthetic (seeded Gaussians with row-normalised Q, K).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "causal polysketch attn fwd+bwd tokens/s at n=32k GPT-2-small shape; % bf16 TC peak"
+UNIT = "model-tokens/s"
+
+
+# ---------------------------------------------------------------------------
+# flop model (GEMM flops only, per head-token); "nominal" follows the paper's statement
+# of the algorithm (r^2 features, h+1 columns, full b x b diagonal tiles)
+# ---------------------------------------------------------------------------
+def nominal_flops_per_head_token(w):
+    h, r, b = w.h, w.r, w.b
+    fwd = 8 * h * r + 4 * r * r * (h + 1) + 2 * b * (r + h + 1)
+    bwd = 10 * r * r * (h + 1) + 6 * b * r + 4 * b * (h + 1) + 16 * h * r
+    return fwd, (bwd if w.backward else 0)
+
+
+def kernel_flops_per_head_token(name, w):
+    """Executed flops of one launch of a library kernel, per head-token it covers."""
+    h, r, b = w.h, w.r, w.b
+    k = h + 1
+    half = (b + 1) / 2.0                       # causal pairs per row inside a block
+    table = {
+        # CUDA-core path
+        "sketch_kernel": 4 * h * r,
+        "rows_prep_kernel": 2 * h,
+        "state_kernel": 2 * r * r * k + r * r,
+        "scan_kernel": r * r * k / b,
+        "fwd_out_kernel": 2 * r * r * k + r * r + half * 2 * (r + k),
+        "bwd_q_kernel": 2 * r * r * k + 2 * r * r + half * 2 * (2 * r + k),
+        "bwd_k_kernel": 4 * r * r * k + 3 * r * r + half * 2 * (2 * r + 2 * k),
+        "sketch_bwd_kernel": 8 * h * r,
+    }
+    return table.get(name)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
+ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for nm, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_step(w, inp_host, head):
+    """One bounded sample of the workload for the CPU oracle: forward (+ backward) of one
+    (batch, head) slice at full n.  Returns seconds."""
+    from oracle import polysketch as orc
+    Q, K, V, dO, G1, G2 = inp_host[head]
+    t0 = time.perf_counter()
+    orc.causal_polysketch_attention_blocked(Q, K, V, G1, G2, w.b)
+    if w.backward:
+        orc.causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, w.b)
+    return time.perf_counter() - t0
+
+
+def host_head_inputs(w, heads):
+    """Oracle inputs for a few heads, drawn on the host with the workload's recipe."""
+    import numpy as np
+    import torch
+    from paper_2310_01655_b200 import inputs as wl
+    small = wl.Workload(w.name, 1, len(heads), w.n, w.h, w.r, w.p, w.b, w.dtype, w.backward,
+                        w.data_seed, w.g_seed, w.correlated)
+    inp = wl.make_inputs(small, "cpu", with_dO=True)
+    out = []
+    for i, _ in enumerate(heads):
+        f = lambda k: inp[k][0, i].to(torch.float64).numpy()
+        out.append((f("Q"), f("K"), f("V"), f("dO"), inp["G1"][i].double().numpy(), inp["G2"][i].double().numpy()))
+    return out
+
+
+def cpu_threads():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle, as it stands, on bounded samples of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    heads = list(range(max(1, min(2, args.steps + args.warmup))))
+    data = host_head_inputs(w, heads)
+    for i in range(args.warmup):
+        oracle_step(w, data, i % len(data))
+    times = [oracle_step(w, data, i % len(data)) for i in range(args.steps)]
+    total = sum(times)
+    value = (w.n * args.steps / total) / w.H          # head-tokens/s -> model-tokens/s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
+                   "passes": "fwd+bwd" if w.backward else "fwd",
+                   "step": "oracle on one (batch, head) slice at full n; value extrapolated over heads"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                         "sample": "%d steps x 1 head slice of %s at n=%d" % (args.steps, w.name, w.n)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--impl", default="psk", choices=["psk", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "cuda_cores", "tensor_cores"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-heads", type=int, default=3, help="head slices the CPU baseline leg times")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2310_01655_b200 import inputs as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2310_01655_b200 as psk
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the library")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    psk.lib()
+    path = {"auto": psk.PATH_AUTO, "cuda_cores": psk.PATH_CUDA_CORES, "tensor_cores": psk.PATH_TENSOR_CORES}[args.path]
+
+    # every rank holds its own batch of the workload (independent (batch, head) problems:
+    # no data-path collective), seeded differently per rank
+    wr = wl.Workload(**dict(w.asdict(), data_seed=w.data_seed + 7919 * rank))
+    inp = wl.make_inputs(wr, "cuda", with_dO=True)
+    Q, K, V, dO, G1, G2 = (inp[k] for k in ("Q", "K", "V", "dO", "G1", "G2"))
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path)
+    ws_bytes = max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True) if w.backward else 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    O = torch.empty_like(Q)
+    den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
+    grads = tuple(torch.empty_like(Q) for _ in range(3)) if w.backward else None
+    launches = [0]
+
+    def step():
+        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den)
+        n = psk.last_launch_count()
+        if w.backward:
+            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, path, ws, grads)
+            n += psk.last_launch_count()
+        launches[0] += n
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if psk.check(ws) != 0:
+        raise RuntimeError("device-side error during warm-up")
+
+    # ---- timed region: K steps, CUDA events on the launch stream, per-kernel events on ----
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    psk.profile_enable(True)
+    launches[0] = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    records = psk.profile_records()
+    psk.profile_enable(False)
+    if psk.check(ws) != 0:
+        raise RuntimeError("device-side error during the timed region")
+    tms = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms = float(tms.item())
+    value = world * w.model_tokens * args.steps / (ms / 1e3)
+
+    # ---- end to end through the same C-ABI call with HOST buffers ----
+    e2e = None
+    if not args.no_e2e:
+        names = ["Q", "K", "V"] + (["dO"] if w.backward else [])
+        host_in = {k: torch.empty(inp[k].shape, dtype=inp[k].dtype, pin_memory=True).copy_(inp[k]) for k in names}
+        outs = [O] + (list(grads) if w.backward else [])
+        host_out = [torch.empty(o.shape, dtype=o.dtype, pin_memory=True) for o in outs]
+        host_den = torch.empty(den.shape, dtype=den.dtype, pin_memory=True)
+        bi = sum(t.numel() * t.element_size() for t in host_in.values())
+        bo = sum(t.numel() * t.element_size() for t in host_out) + host_den.numel() * 4
+
+        def e2e_step():
+            for k in names:
+                inp[k].copy_(host_in[k], non_blocking=True)
+            step()
+            for o, ho in zip(outs, host_out):
+                ho.copy_(o, non_blocking=True)
+            host_den.copy_(den, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b_.record()
+        barrier()
+        t2 = torch.tensor([a.elapsed_time(b_)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * w.model_tokens * args.e2e_steps / (float(t2.item()) / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo, "steps": args.e2e_steps}
+        del host_in, host_out
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ----
+    pk = peaks()
+    agg = {}
+    for name, t in records:
+        a = agg.setdefault(name, [0, 0.0])
+        a[0] += 1; a[1] += t
+    total_kernel_ms = sum(v[1] for v in agg.values()) or 1.0
+    top = max(agg.items(), key=lambda kv: kv[1][1]) if agg else (None, [0, 0.0])
+    roof = None
+    if top[0] is not None:
+        name, (cnt, tot) = top
+        fl = kernel_flops_per_head_token(name, w)
+        tensor = name.startswith("tc_")
+        peak = pk["bf16_sustained"] if tensor else ALU_PEAK_TFLOPS
+        achieved = (fl * w.head_tokens / ((tot / cnt) / 1e3) / 1e12) if fl else None
+        roof = {"kernel": name, "bound": "tensor" if tensor else "alu", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "peak_source": (pk["source"] + " (sustained bf16)") if tensor else "derived: 148 SM x 128 FMA x 1.965 GHz",
+                "launches": cnt, "avg_ms": tot / cnt, "share_of_kernel_time": tot / total_kernel_ms}
+    kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / total_kernel_ms, 4)}
+               for k, v in sorted(agg.items(), key=lambda kv: -kv[1][1])}
+
+    # ---- CPU baseline: the oracle on a bounded sample ----
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        heads = list(range(args.cpu_heads))
+        data = host_head_inputs(w, heads)
+        secs = sum(oracle_step(w, data, i) for i in range(len(heads)))
+        cpu = {"value": (w.n * len(heads) / secs) / w.H, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": "%d (batch, head) slices of %s at full n=%d, %s; extrapolated linearly over heads"
+                         % (len(heads), w.name, w.n, "fwd+bwd" if w.backward else "fwd"),
+               "seconds": secs}
+
+    f_fwd, f_bwd = nominal_flops_per_head_token(w)
+    nominal_tflops = (f_fwd + f_bwd) * w.head_tokens * world * args.steps / (ms / 1e3) / 1e12
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
+                   "passes": "fwd+bwd" if w.backward else "fwd", "path": args.path,
+                   "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
+        "nominal_tflops": nominal_tflops,
+        "frac_bf16_peak": {"burst": nominal_tflops / world / pk["bf16_burst"],
+                           "sustained": nominal_tflops / world / pk["bf16_sustained"],
+                           "nominal_2250": nominal_tflops / world / 2250.0, "source": pk["source"]},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0], "roofline": roof, "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

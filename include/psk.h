@@ -1,0 +1,136 @@
+/*
+ * psk.h -- C ABI of the causal polynomial-sketch ("Polysketch") attention library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * What the calls compute (PolySketchFormer, arXiv 2310.01655), per (batch, head):
+ *   m(x)   = sqrt(1/r) * [(x G1) * (x G2)]              Section 2.2 / Algorithm 1, degree-2 level
+ *   phi'(x) = m(x) (x) m(x)   (r^2 features)            Algorithm 1, PolySketchNonNegative, p = 4
+ *   O      = D~^{-1} lt(phi'(Q) phi'(K)^T) V            Section 3
+ *   D~     = diag(1 + lt(phi'(Q) phi'(K)^T) 1)          Section 3 (the "1 +" is part of it)
+ * evaluated in time linear in n by the block lower-triangular multiply of
+ * Section 3.1 (diagonal blocks of b rows directly through (L R^T)^2, everything
+ * earlier through the prefix sum Z_l of per-block states H_l = phi'(K_l)^T [V_l | 1]).
+ * lt() keeps j <= i (diagonal included).  The paper prints no backward pass; the
+ * backward call returns the exact derivatives of the formulas above.
+ *
+ * Conventions
+ *   - Every pointer argument marked DEVICE is device memory owned by the caller; the
+ *     library allocates nothing and frees nothing.  Scratch space is the caller's
+ *     `workspace` (size from psk_workspace_bytes, 256-byte aligned).
+ *   - Tensors Q, K, V, O, dO, dQ, dK, dV are [B, H, n, h] with element strides
+ *     (stride_b, stride_h, stride_n) and a contiguous last dimension; all eight share
+ *     the strides in psk_shape.  G1, G2 are [g_heads, h, r] contiguous, g_heads = 1
+ *     (one pair for all heads) or H (one pair per head); the same pair sketches Q and K.
+ *   - Q and K are taken as already normalised (the paper applies LayerNorm first,
+ *     Section 2.1); dQ and dK are gradients with respect to those inputs.  No
+ *     gradient is produced for G1, G2 (random, untrained sketch).
+ *   - `dtype` is the storage type of Q, K, V, G1, G2, O and all gradients.  PSK_F32
+ *     computes in fp32 on the CUDA cores; PSK_BF16 computes on the tensor cores with
+ *     bf16 operands and fp32 accumulation.  `denom` is always fp32.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return
+ *     without synchronising.  Errors detectable on the host are returned before any
+ *     launch and leave the outputs untouched.  A device-side bounded wait that gives
+ *     up records a code in the workspace; psk_check() reads it.
+ *   - Supported: p = 4, h = 64, r in {16, 32, 64}, b a multiple of 128, n a multiple
+ *     of b (Section 3.1 assumes b = n / t).  Anything else: PSK_ERR_UNSUPPORTED or
+ *     PSK_ERR_SHAPE.
+ */
+#ifndef PSK_H_
+#define PSK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PSK_OK = 0,
+    PSK_ERR_INVALID_ARG = -1,   /* null pointer, bad enum value                      */
+    PSK_ERR_UNSUPPORTED = -2,   /* p != 4, h != 64, r not in {16,32,64}, bad path    */
+    PSK_ERR_SHAPE = -3,         /* n % b != 0, b % 128 != 0, non-positive extents    */
+    PSK_ERR_ALIGN = -4,         /* pointer or stride not 16-byte aligned             */
+    PSK_ERR_WORKSPACE = -5,     /* workspace missing, misaligned or too small        */
+    PSK_ERR_CUDA = -6,          /* a CUDA runtime call or launch failed              */
+    PSK_ERR_TIMEOUT = -7        /* a bounded device-side wait gave up (psk_check)    */
+} psk_status;
+
+typedef enum { PSK_F32 = 0, PSK_BF16 = 1 } psk_dtype;
+
+/* Which implementation runs.  PSK_PATH_AUTO picks by dtype (fp32 -> CUDA cores,
+ * bf16 -> tensor cores).  PSK_PATH_CUDA_CORES forces the fp32-arithmetic kernels for
+ * either storage type (used to cross-check the tensor-core path). */
+typedef enum { PSK_PATH_AUTO = 0, PSK_PATH_CUDA_CORES = 1, PSK_PATH_TENSOR_CORES = 2 } psk_path;
+
+typedef struct {
+    int32_t B, H, n, h, r, p, b;
+    int32_t dtype;              /* psk_dtype */
+    int64_t stride_b, stride_h, stride_n;   /* elements; last dimension contiguous */
+    int32_t g_heads;            /* 1 or H */
+    int32_t path;               /* psk_path */
+} psk_shape;
+
+/* Library version (major*100 + minor). */
+int psk_version(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* psk_status_string(int status);
+
+/* Bytes of caller-provided scratch the forward (for_backward = 0) or the backward
+ * (for_backward = 1) needs for this shape; 0 if the shape is invalid.  Section 3.1:
+ * the scratch holds the per-block states H_l / prefix sums Z_l and the half sketches. */
+size_t psk_workspace_bytes(const psk_shape* shape, int for_backward);
+
+/* Half sketch and, optionally, the self-tensored features (Algorithm 1).
+ *   X        DEVICE [B,H,n,h] storage dtype, strides from `shape`
+ *   G1, G2   DEVICE [g_heads,h,r] storage dtype
+ *   M_out    DEVICE [B,H,n,r] fp32 contiguous: m(x)
+ *   Phi_out  DEVICE [B,H,n,r*r] fp32 contiguous or NULL: phi'(x)[a*r+b] = m_a m_b
+ * (row-major Kronecker order of Section 1.2).  Phi_out is meant for tests on small
+ * shapes; the attention calls never materialise it in HBM. */
+int psk_sketch(const psk_shape* shape, const void* X, const void* G1, const void* G2,
+               float* M_out, float* Phi_out, void* stream);
+
+/* Causal Polysketch attention forward (Section 3 through Section 3.1).
+ *   Q, K, V  DEVICE inputs; O DEVICE output [B,H,n,h] storage dtype
+ *   denom    DEVICE [B,H,n] fp32 or NULL: d_i = 1 + sum_{j<=i} <phi'(q_i), phi'(k_j)>
+ *   workspace DEVICE scratch, >= psk_workspace_bytes(shape, 0), 256-byte aligned */
+int psk_causal_attn_fwd(const psk_shape* shape, const void* Q, const void* K, const void* V,
+                        const void* G1, const void* G2, void* O, float* denom,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward of psk_causal_attn_fwd: given dO = dL/dO, writes dQ, dK, dV (storage dtype).
+ * O and denom are the forward's outputs (both required).  Derived from Section 3's
+ * formula; evaluated with a forward prefix of key states and a reverse prefix of
+ * query states in the manner of Section 3.1.
+ *   workspace DEVICE scratch, >= psk_workspace_bytes(shape, 1) */
+int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, const void* V,
+                        const void* G1, const void* G2, const void* O, const float* denom,
+                        const void* dO, void* dQ, void* dK, void* dV,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, then reports PSK_ERR_TIMEOUT if a kernel of the last call that
+ * used `workspace` abandoned a bounded wait, PSK_ERR_CUDA if the stream is in error,
+ * else PSK_OK.  Never traps. */
+int psk_check(const void* workspace, void* stream);
+
+/* Number of kernel launches the last forward / backward call on this thread enqueued
+ * (for launch accounting in benchmarks). */
+int psk_last_launch_count(void);
+
+/* Measurement aid (no counterpart in the paper).  psk_profile_enable(1) makes every
+ * later kernel launch of the library be bracketed by a pair of CUDA events on the launch
+ * stream and discards earlier records; psk_profile_enable(0) stops recording and frees
+ * them.  psk_profile_count() is the number of launches recorded so far;
+ * psk_profile_get(i, name, cap, &ms) waits for launch i to finish and returns its kernel
+ * name (HOST buffer, NUL-terminated, truncated to cap) and device duration in ms.
+ * Process-wide state; not thread-safe. */
+int psk_profile_enable(int enable);
+int psk_profile_count(void);
+int psk_profile_get(int index, char* name, size_t name_cap, float* ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSK_H_ */

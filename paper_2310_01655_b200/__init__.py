@@ -1,0 +1,17 @@
+"""Causal polynomial-sketch (Polysketch) attention for B200: Python binding of libpsk.
+
+The binding only marshals arguments (pointers, shapes, strides, stream) into the
+C ABI declared in include/psk.h; every step of the computation runs in the library's
+CUDA kernels.  There is no CPU or PyTorch fallback: if libpsk.so is missing or no CUDA
+device is present the calls raise.
+"""
+from . import binding
+from .binding import (PskError, Shape, lib, library_path, sketch, causal_attn_fwd, causal_attn_bwd,
+                      workspace_bytes, check, last_launch_count, status_string,
+                      profile_enable, profile_records,
+                      PATH_AUTO, PATH_CUDA_CORES, PATH_TENSOR_CORES)
+
+__all__ = ["PskError", "Shape", "lib", "library_path", "sketch", "causal_attn_fwd", "causal_attn_bwd",
+           "workspace_bytes", "check", "last_launch_count", "status_string",
+           "profile_enable", "profile_records",
+           "PATH_AUTO", "PATH_CUDA_CORES", "PATH_TENSOR_CORES"]

@@ -1,0 +1,192 @@
+"""ctypes binding of libpsk.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_int, c_int32, c_int64, c_size_t, c_void_p, c_char_p, POINTER, Structure, byref
+
+import torch
+
+PATH_AUTO, PATH_CUDA_CORES, PATH_TENSOR_CORES = 0, 1, 2
+_DTYPES = {torch.float32: 0, torch.bfloat16: 1}
+_PKG = os.path.dirname(os.path.abspath(__file__))
+
+
+class PskError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, status_string(code), code))
+
+
+class Shape(Structure):
+    """Mirror of `psk_shape`."""
+    _fields_ = [("B", c_int32), ("H", c_int32), ("n", c_int32), ("h", c_int32), ("r", c_int32),
+                ("p", c_int32), ("b", c_int32), ("dtype", c_int32),
+                ("stride_b", c_int64), ("stride_h", c_int64), ("stride_n", c_int64),
+                ("g_heads", c_int32), ("path", c_int32)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return os.path.join(_PKG, "libpsk.so")
+
+
+def lib():
+    """Loads libpsk.so (built in-tree by `python -m paper_2310_01655_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError("libpsk.so is not built: run `python -m paper_2310_01655_b200.build` "
+                           "(there is no fallback implementation)")
+    L = ctypes.CDLL(path)
+    P = POINTER(Shape)
+    L.psk_version.restype = c_int
+    L.psk_status_string.restype = c_char_p
+    L.psk_status_string.argtypes = [c_int]
+    L.psk_workspace_bytes.restype = c_size_t
+    L.psk_workspace_bytes.argtypes = [P, c_int]
+    L.psk_sketch.restype = c_int
+    L.psk_sketch.argtypes = [P] + [c_void_p] * 6
+    L.psk_causal_attn_fwd.restype = c_int
+    L.psk_causal_attn_fwd.argtypes = [P] + [c_void_p] * 8 + [c_size_t, c_void_p]
+    L.psk_causal_attn_bwd.restype = c_int
+    L.psk_causal_attn_bwd.argtypes = [P] + [c_void_p] * 12 + [c_size_t, c_void_p]
+    L.psk_check.restype = c_int
+    L.psk_check.argtypes = [c_void_p, c_void_p]
+    L.psk_last_launch_count.restype = c_int
+    L.psk_profile_enable.restype = c_int
+    L.psk_profile_enable.argtypes = [c_int]
+    L.psk_profile_count.restype = c_int
+    L.psk_profile_get.restype = c_int
+    L.psk_profile_get.argtypes = [c_int, ctypes.c_char_p, c_size_t, POINTER(ctypes.c_float)]
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().psk_status_string(int(code)).decode()
+
+
+def _require_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise RuntimeError("psk: tensors must live on a CUDA device (no CPU path exists)")
+
+
+def _ptr(t):
+    return c_void_p(t.data_ptr()) if t is not None else c_void_p(0)
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, path: int = PATH_AUTO) -> Shape:
+    """Shape descriptor for a [B,H,n,h] tensor `x` (its strides are used for all eight tensors)."""
+    if x.dim() != 4 or x.stride(3) != 1:
+        raise ValueError("expected a [B,H,n,h] tensor with a contiguous last dimension")
+    if x.dtype not in _DTYPES:
+        raise ValueError("unsupported storage dtype %s" % x.dtype)
+    B, H, n, h = x.shape
+    g_heads = G1.shape[0] if G1.dim() == 3 else 1
+    return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path)
+
+
+def workspace_bytes(shape: Shape, for_backward: bool) -> int:
+    return int(lib().psk_workspace_bytes(byref(shape), 1 if for_backward else 0))
+
+
+def _workspace(shape, for_backward, workspace):
+    need = workspace_bytes(shape, for_backward)
+    if need == 0:
+        # let the library report the precise reason
+        return None, 0
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device="cuda")
+    return workspace, workspace.numel()
+
+
+def _same_layout(ref, *ts):
+    for t in ts:
+        if t is not None and (t.shape != ref.shape or t.stride() != ref.stride() or t.dtype != ref.dtype):
+            raise ValueError("all [B,H,n,h] tensors must share shape, strides and dtype")
+
+
+def sketch(X, G1, G2, r=None, b=128, want_phi=False, path=PATH_AUTO):
+    """psk_sketch: returns (M [B,H,n,r] fp32, Phi [B,H,n,r*r] fp32 or None)."""
+    _require_cuda(X, G1, G2)
+    r = G1.shape[-1] if r is None else r
+    shp = make_shape(X, G1, r, b, path=path)
+    B, H, n, _ = X.shape
+    M = torch.empty((B, H, n, r), dtype=torch.float32, device=X.device)
+    Phi = torch.empty((B, H, n, r * r), dtype=torch.float32, device=X.device) if want_phi else None
+    st = lib().psk_sketch(byref(shp), _ptr(X), _ptr(G1.contiguous()), _ptr(G2.contiguous()), _ptr(M), _ptr(Phi),
+                          _stream())
+    if st != 0:
+        raise PskError(st, "psk_sketch")
+    return M, Phi
+
+
+def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out=None, denom=None):
+    """psk_causal_attn_fwd: returns (O, denom)."""
+    _require_cuda(Q, K, V, G1, G2)
+    _same_layout(Q, K, V, out)
+    shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
+    O = torch.empty_like(Q) if out is None else out
+    B, H, n, _ = Q.shape
+    if denom is None:
+        denom = torch.empty((B, H, n), dtype=torch.float32, device=Q.device)
+    ws, nbytes = _workspace(shp, False, workspace)
+    st = lib().psk_causal_attn_fwd(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(G1), _ptr(G2), _ptr(O),
+                                   _ptr(denom), _ptr(ws), nbytes, _stream())
+    if st != 0:
+        raise PskError(st, "psk_causal_attn_fwd")
+    return O, denom
+
+
+def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, workspace=None, out=None):
+    """psk_causal_attn_bwd: returns (dQ, dK, dV)."""
+    _require_cuda(Q, K, V, G1, G2, O, denom, dO)
+    _same_layout(Q, K, V, O, dO)
+    shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
+    dQ, dK, dV = out if out is not None else (torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q))
+    _same_layout(Q, dQ, dK, dV)
+    ws, nbytes = _workspace(shp, True, workspace)
+    st = lib().psk_causal_attn_bwd(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(G1), _ptr(G2), _ptr(O),
+                                   _ptr(denom), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), nbytes,
+                                   _stream())
+    if st != 0:
+        raise PskError(st, "psk_causal_attn_bwd")
+    return dQ, dK, dV
+
+
+def check(workspace) -> int:
+    """psk_check: synchronises the current stream and returns the device-side status."""
+    return int(lib().psk_check(_ptr(workspace), _stream()))
+
+
+def last_launch_count() -> int:
+    return int(lib().psk_last_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    """psk_profile_enable: start (discarding old records) or stop per-kernel event timing."""
+    lib().psk_profile_enable(1 if on else 0)
+
+
+def profile_records():
+    """All launches recorded since profile_enable(True): list of (kernel name, ms)."""
+    L = lib()
+    out = []
+    buf = ctypes.create_string_buffer(64)
+    ms = ctypes.c_float()
+    for i in range(L.psk_profile_count()):
+        st = L.psk_profile_get(i, buf, 64, byref(ms))
+        if st != 0:
+            raise PskError(st, "psk_profile_get")
+        out.append((buf.value.decode(), float(ms.value)))
+    return out

@@ -1,0 +1,618 @@
+// CUDA-core path: causal Polysketch attention in fp32 arithmetic, the steps of
+// Section 3.1 as separate kernels (half sketch -> per-block states H_l -> prefix scan
+// Z_l -> output rows P_l + phi'(Q_l) Z_l -> division by D~).  Serves fp32 storage (the
+// tensor cores' tf32 rounding cannot hold 1e-4 through a degree-4 polynomial) and
+// cross-checks the tensor-core path on bf16 storage.
+#include "psk_internal.cuh"
+
+namespace psk {
+
+CcWorkspace cc_workspace(const Dims& d, bool backward) {
+    CcWorkspace w{};
+    const size_t rows = (size_t)d.BH() * d.n;
+    const size_t st = (size_t)d.BH() * d.t * d.r * d.r * 65 * sizeof(float);
+    size_t off = 0;
+    w.status = off; off += kStatusBytes;
+    w.Mq = off;  off += align_up(rows * d.r * sizeof(float));
+    w.Mk = off;  off += align_up(rows * d.r * sizeof(float));
+    w.Vt = off;  off += align_up(rows * 65 * sizeof(float));
+    w.Zst = off; off += align_up(st);
+    if (backward) {
+        w.E = off;   off += align_up(rows * 65 * sizeof(float));
+        w.Rst = off; off += align_up(st);
+        w.dMq = off; off += align_up(rows * d.r * sizeof(float));
+        w.dMk = off; off += align_up(rows * d.r * sizeof(float));
+    }
+    w.total = off;
+    return w;
+}
+
+namespace {
+
+constexpr int H64 = 64;     // head dimension (only value supported)
+constexpr int YC = 65;      // columns of [V | 1] and of E
+constexpr int YS = 68;      // padded shared-memory row stride for 65-column rows
+
+struct Slice {              // addressing of one [B,H,n,h] tensor
+    int H; int64_t sb, sh, sn;
+    __device__ int64_t row(int bh, int i) const {
+        return (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn;
+    }
+};
+
+// ---------------------------------------------------------------------------
+// Half sketch m(x) = (x G1)*(x G2)/sqrt(r)  (Algorithm 1, degree-2 level), 64 rows per CTA
+// ---------------------------------------------------------------------------
+template <typename T, int R>
+__global__ void __launch_bounds__(256)
+sketch_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const T* __restrict__ G2,
+              int g_heads, int n, float* __restrict__ M_out, float* __restrict__ Phi_out) {
+    extern __shared__ float smem[];
+    float* sG1 = smem;                  // [64][R]
+    float* sG2 = sG1 + H64 * R;         // [64][R]
+    float* sX = sG2 + H64 * R;          // [64][65]
+    float* sM = sX + 64 * 65;           // [64][R+1]
+    const int bh = blockIdx.y, i0 = blockIdx.x * 64, tid = threadIdx.x;
+    const int g = (g_heads == 1) ? 0 : (bh % sl.H);
+    for (int e = tid; e < H64 * R; e += 256) {
+        sG1[e] = ldf(G1 + (size_t)g * H64 * R + e);
+        sG2[e] = ldf(G2 + (size_t)g * H64 * R + e);
+    }
+    for (int e = tid; e < 64 * H64; e += 256) {
+        const int rr = e / H64, c = e % H64;
+        sX[rr * 65 + c] = ldf(X + sl.row(bh, i0 + rr) + c);
+    }
+    __syncthreads();
+    const float rs = rsqrtf((float)R);
+    const int c = tid % R;
+    for (int rr = tid / R; rr < 64; rr += 256 / R) {
+        float a1 = 0.f, a2 = 0.f;
+#pragma unroll 16
+        for (int t = 0; t < H64; ++t) {
+            const float x = sX[rr * 65 + t];
+            a1 = fmaf(x, sG1[t * R + c], a1);
+            a2 = fmaf(x, sG2[t * R + c], a2);
+        }
+        const float m = a1 * a2 * rs;
+        sM[rr * (R + 1) + c] = m;
+        M_out[((size_t)bh * n + i0 + rr) * R + c] = m;
+    }
+    if (Phi_out != nullptr) {           // phi'(x)[a*R+b] = m_a m_b (Section 1.2 ordering)
+        __syncthreads();
+        for (int e = tid; e < 64 * R * R; e += 256) {
+            const int rr = e / (R * R), f = e % (R * R);
+            Phi_out[((size_t)bh * n + i0 + rr) * R * R + f] =
+                sM[rr * (R + 1) + f / R] * sM[rr * (R + 1) + f % R];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Row preparation: mode 0 writes V~ = [V | 1]; mode 1 writes E = [dO/d | -(dO.O)/d]
+// One warp per row.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+rows_prep_kernel(Slice sl, int n, int total_rows, int mode, const T* __restrict__ V,
+                 const T* __restrict__ O, const float* __restrict__ denom,
+                 const T* __restrict__ dO, float* __restrict__ out) {
+    const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (row >= total_rows) return;
+    const int bh = row / n, i = row % n;
+    const int64_t base = sl.row(bh, i);
+    float* o = out + (size_t)row * YC;
+    if (mode == 0) {
+        o[lane] = ldf(V + base + lane);
+        o[lane + 32] = ldf(V + base + lane + 32);
+        if (lane == 0) o[64] = 1.f;
+    } else {
+        const float g0 = ldf(dO + base + lane), g1 = ldf(dO + base + lane + 32);
+        float dot = g0 * ldf(O + base + lane) + g1 * ldf(O + base + lane + 32);
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
+        const float inv = 1.f / denom[row];
+        o[lane] = g0 * inv;
+        o[lane + 32] = g1 * inv;
+        if (lane == 0) o[64] = -dot * inv;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Per-block state H_l = phi'(M_l)^T Y_l  (Section 3.1), M the half sketches of the
+// block's rows, Y its [b,65] right-hand side.  One thread per feature (a,b).
+// ---------------------------------------------------------------------------
+template <int R>
+__global__ void __launch_bounds__(128)
+state_kernel(const float* __restrict__ M, const float* __restrict__ Y, int n, int b, int t,
+             float* __restrict__ S) {
+    __shared__ float sM[32][R];
+    __shared__ __align__(16) float sY[32][YS];
+    const int tid = threadIdx.x, l = blockIdx.y, bh = blockIdx.z;
+    const int f = blockIdx.x * 128 + tid, fa = f / R, fb = f % R;
+    float acc[YC];
+#pragma unroll
+    for (int c = 0; c < YC; ++c) acc[c] = 0.f;
+    const size_t row0 = (size_t)bh * n + (size_t)l * b;
+    for (int j0 = 0; j0 < b; j0 += 32) {
+        __syncthreads();
+        for (int e = tid; e < 32 * R; e += 128) sM[e / R][e % R] = M[(row0 + j0) * R + e];
+        for (int e = tid; e < 32 * YC; e += 128) sY[e / YC][e % YC] = Y[(row0 + j0) * YC + e];
+        __syncthreads();
+        if (f < R * R) {
+#pragma unroll 4
+            for (int j = 0; j < 32; ++j) {
+                const float phi = sM[j][fa] * sM[j][fb];
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+                    const float4 y = *reinterpret_cast<const float4*>(&sY[j][c]);
+                    acc[c] = fmaf(phi, y.x, acc[c]);
+                    acc[c + 1] = fmaf(phi, y.y, acc[c + 1]);
+                    acc[c + 2] = fmaf(phi, y.z, acc[c + 2]);
+                    acc[c + 3] = fmaf(phi, y.w, acc[c + 3]);
+                }
+                acc[64] = fmaf(phi, sY[j][64], acc[64]);
+            }
+        }
+    }
+    if (f < R * R) {
+        float* o = S + (((size_t)bh * t + l) * R * R + f) * YC;
+#pragma unroll
+        for (int c = 0; c < YC; ++c) o[c] = acc[c];
+    }
+}
+
+// Exclusive prefix (reverse = 0: Z_l = sum_{j<l} H_j, Section 3.1) or exclusive suffix
+// (reverse = 1: sum_{j>l} H_j) over the t states of each head, in place, sequential in l.
+__global__ void __launch_bounds__(256)
+scan_kernel(float* __restrict__ S, size_t elems, int t, int reverse) {
+    const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= elems) return;
+    float* p = S + (size_t)blockIdx.y * t * elems + e;
+    float run = 0.f;
+    if (!reverse) {
+        for (int l = 0; l < t; ++l) { const float v = p[(size_t)l * elems]; p[(size_t)l * elems] = run; run += v; }
+    } else {
+        for (int l = t - 1; l >= 0; --l) { const float v = p[(size_t)l * elems]; p[(size_t)l * elems] = run; run += v; }
+    }
+}
+
+// acc[0..64] += coef * row[0..64]   (row in shared memory, 16-byte aligned, stride YS)
+__device__ __forceinline__ void axpy65(float (&acc)[YC], float coef, const float* row) {
+#pragma unroll
+    for (int c = 0; c < 64; c += 4) {
+        const float4 z = *reinterpret_cast<const float4*>(row + c);
+        acc[c] = fmaf(coef, z.x, acc[c]);
+        acc[c + 1] = fmaf(coef, z.y, acc[c + 1]);
+        acc[c + 2] = fmaf(coef, z.z, acc[c + 2]);
+        acc[c + 3] = fmaf(coef, z.w, acc[c + 3]);
+    }
+    acc[64] = fmaf(coef, row[64], acc[64]);
+}
+// row[0..64] . y[0..64]
+__device__ __forceinline__ float dot65(const float* row, const float (&y)[YC]) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int c = 0; c < 64; c += 4) {
+        const float4 z = *reinterpret_cast<const float4*>(row + c);
+        s0 = fmaf(z.x, y[c], s0);
+        s1 = fmaf(z.y, y[c + 1], s1);
+        s2 = fmaf(z.z, y[c + 2], s2);
+        s3 = fmaf(z.w, y[c + 3], s3);
+    }
+    return (s0 + s1) + (s2 + s3) + row[64] * y[64];
+}
+
+// Shared-memory carve-up of the three row kernels (one thread per row, 128 rows per CTA):
+//   sS   [R][YS]        slice a of the block's prefix/suffix state: rows (a, 0..R-1)
+//   sOwn [128][R+1]     this tile's own half sketches (runtime-indexed access by a)
+//   sOut [128][R+1]     per-row results indexed by a
+//   sM2  [32][R]        chunk of the other side's half sketches (diagonal tile)
+//   sY2  [32][YS]       chunk of the other side's 65-column rows (diagonal tile)
+template <int R> struct RowSmem {
+    static constexpr int S = 0;
+    static constexpr int Own = S + R * YS;
+    static constexpr int Out = Own + 128 * (R + 1);
+    static constexpr int M2 = Out + 128 * (R + 1);
+    static constexpr int Y2 = M2 + 32 * R;
+    static constexpr int total = Y2 + 32 * YS;
+    static constexpr size_t bytes = (size_t)total * sizeof(float);
+};
+
+// ---------------------------------------------------------------------------
+// Forward output rows (Section 3.1): row i of block l = P_l row + phi'(q_i)^T Z_l, with
+// P_l = lt((L R^T)^2) [V_l | 1]; then d_i = 1 + last column, O_i = first 64 / d_i.
+// ---------------------------------------------------------------------------
+template <typename T, int R>
+__global__ void __launch_bounds__(128)
+fwd_out_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
+               const float* __restrict__ Vt, const float* __restrict__ Z,
+               T* __restrict__ O, float* __restrict__ denom) {
+    extern __shared__ __align__(16) float smem[];
+    float* sS = smem + RowSmem<R>::S;
+    float* sOwn = smem + RowSmem<R>::Own;
+    float* sM2 = smem + RowSmem<R>::M2;
+    float* sY2 = smem + RowSmem<R>::Y2;
+    const int tid = threadIdx.x, tile = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
+    const int i_blk = tile * 128 + tid;                 // row within the block
+    const size_t blk0 = (size_t)bh * n + (size_t)l * b;  // first row of the block
+    const size_t row = blk0 + i_blk;
+    float mq[R], acc[YC];
+#pragma unroll
+    for (int c = 0; c < R; ++c) { mq[c] = Mq[row * R + c]; sOwn[tid * (R + 1) + c] = mq[c]; }
+#pragma unroll
+    for (int c = 0; c < YC; ++c) acc[c] = 0.f;
+    // earlier blocks through the prefix state
+    const float* Zl = Z + ((size_t)bh * t + l) * R * R * YC;
+    if (l > 0) {
+        for (int a = 0; a < R; ++a) {
+            __syncthreads();
+            for (int e = tid; e < R * YC; e += 128) sS[(e / YC) * YS + e % YC] = Zl[(size_t)a * R * YC + e];
+            __syncthreads();
+            const float ma = sOwn[tid * (R + 1) + a];
+#pragma unroll
+            for (int bb = 0; bb < R; ++bb) axpy65(acc, ma * mq[bb], sS + bb * YS);
+        }
+    }
+    // same block: j <= i through the b x b tile of squared half-sketch scores
+    const int jend = tile * 128 + 128;                  // keys needed by this row tile
+    const int warp_imax = tile * 128 + (tid | 31);
+    for (int j0 = 0; j0 < jend; j0 += 32) {
+        __syncthreads();
+        for (int e = tid; e < 32 * R; e += 128) sM2[e] = Mk[(blk0 + j0) * R + e];
+        for (int e = tid; e < 32 * YC; e += 128) sY2[(e / YC) * YS + e % YC] = Vt[(blk0 + j0) * YC + e];
+        __syncthreads();
+        if (j0 > warp_imax) continue;
+        for (int jj = 0; jj < 32; ++jj) {
+            if (j0 + jj > i_blk) break;
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
+            axpy65(acc, s * s, sY2 + jj * YS);
+        }
+    }
+    const float d = 1.f + acc[64];
+    const float inv = 1.f / d;
+    const int64_t o = sl.row(bh, l * b + i_blk);
+#pragma unroll
+    for (int c = 0; c < 64; ++c) stf(O + o + c, acc[c] * inv);
+    if (denom != nullptr) denom[row] = d;
+}
+
+// ---------------------------------------------------------------------------
+// Backward, query side.  d m(q_i) = 2 mat(Z_l E_i) m(q_i)  +  sum_{j<=i, same block}
+// 2 s_ij (E_i . v~_j) m(k_j).
+// ---------------------------------------------------------------------------
+template <int R>
+__global__ void __launch_bounds__(128)
+bwd_q_kernel(int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
+             const float* __restrict__ Vt, const float* __restrict__ E, const float* __restrict__ Z,
+             float* __restrict__ dMq) {
+    extern __shared__ __align__(16) float smem[];
+    float* sS = smem + RowSmem<R>::S;
+    float* sOut = smem + RowSmem<R>::Out;
+    float* sM2 = smem + RowSmem<R>::M2;
+    float* sY2 = smem + RowSmem<R>::Y2;
+    const int tid = threadIdx.x, tile = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
+    const int i_blk = tile * 128 + tid;
+    const size_t blk0 = (size_t)bh * n + (size_t)l * b;
+    const size_t row = blk0 + i_blk;
+    float mq[R], dm[R], e[YC];
+#pragma unroll
+    for (int c = 0; c < R; ++c) { mq[c] = Mq[row * R + c]; dm[c] = 0.f; sOut[tid * (R + 1) + c] = 0.f; }
+#pragma unroll
+    for (int c = 0; c < YC; ++c) e[c] = E[row * YC + c];
+    const float* Zl = Z + ((size_t)bh * t + l) * R * R * YC;
+    if (l > 0) {
+        for (int a = 0; a < R; ++a) {
+            __syncthreads();
+            for (int x = tid; x < R * YC; x += 128) sS[(x / YC) * YS + x % YC] = Zl[(size_t)a * R * YC + x];
+            __syncthreads();
+            float ta = 0.f;
+#pragma unroll
+            for (int bb = 0; bb < R; ++bb) ta = fmaf(dot65(sS + bb * YS, e), mq[bb], ta);
+            sOut[tid * (R + 1) + a] = 2.f * ta;
+        }
+    }
+    const int jend = tile * 128 + 128;
+    const int warp_imax = tile * 128 + (tid | 31);
+    for (int j0 = 0; j0 < jend; j0 += 32) {
+        __syncthreads();
+        for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mk[(blk0 + j0) * R + x];
+        for (int x = tid; x < 32 * YC; x += 128) sY2[(x / YC) * YS + x % YC] = Vt[(blk0 + j0) * YC + x];
+        __syncthreads();
+        if (j0 > warp_imax) continue;
+        for (int jj = 0; jj < 32; ++jj) {
+            if (j0 + jj > i_blk) break;
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
+            const float ds = 2.f * s * dot65(sY2 + jj * YS, e);
+#pragma unroll
+            for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[jj * R + c], dm[c]);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < R; ++c) dMq[row * R + c] = dm[c] + sOut[tid * (R + 1) + c];
+}
+
+// ---------------------------------------------------------------------------
+// Backward, key/value side.  With R_l the suffix state sum_{blocks>l} phi'(Q)^T E:
+//   d m(k_j) = 2 mat(R_l v~_j) m(k_j) + sum_{i>=j, same block} 2 s_ij (E_i . v~_j) m(q_i)
+//   dV_j     = (R_l^T phi'(k_j))[:h]  + sum_{i>=j, same block} s_ij^2 E_i[:h]
+// ---------------------------------------------------------------------------
+template <typename T, int R>
+__global__ void __launch_bounds__(128)
+bwd_k_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
+             const float* __restrict__ Vt, const float* __restrict__ E, const float* __restrict__ Rs,
+             float* __restrict__ dMk, T* __restrict__ dV) {
+    extern __shared__ __align__(16) float smem[];
+    float* sS = smem + RowSmem<R>::S;
+    float* sOwn = smem + RowSmem<R>::Own;
+    float* sOut = smem + RowSmem<R>::Out;
+    float* sM2 = smem + RowSmem<R>::M2;
+    float* sY2 = smem + RowSmem<R>::Y2;
+    const int tid = threadIdx.x, tile = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
+    const int j_blk = tile * 128 + tid;
+    const size_t blk0 = (size_t)bh * n + (size_t)l * b;
+    const size_t row = blk0 + j_blk;
+    float mk[R], dm[R], v[YC], dv[YC];
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+        mk[c] = Mk[row * R + c]; dm[c] = 0.f;
+        sOwn[tid * (R + 1) + c] = mk[c]; sOut[tid * (R + 1) + c] = 0.f;
+    }
+#pragma unroll
+    for (int c = 0; c < YC; ++c) { v[c] = Vt[row * YC + c]; dv[c] = 0.f; }
+    const float* Rl = Rs + ((size_t)bh * t + l) * R * R * YC;
+    if (l < t - 1) {
+        for (int a = 0; a < R; ++a) {
+            __syncthreads();
+            for (int x = tid; x < R * YC; x += 128) sS[(x / YC) * YS + x % YC] = Rl[(size_t)a * R * YC + x];
+            __syncthreads();
+            const float ma = sOwn[tid * (R + 1) + a];
+            float ta = 0.f;
+#pragma unroll
+            for (int bb = 0; bb < R; ++bb) {
+                ta = fmaf(dot65(sS + bb * YS, v), mk[bb], ta);
+                axpy65(dv, ma * mk[bb], sS + bb * YS);
+            }
+            sOut[tid * (R + 1) + a] = 2.f * ta;
+        }
+    }
+    // same block: queries i >= j
+    const int i_begin = tile * 128;                     // first query row any thread here needs
+    const int warp_jmin = tile * 128 + (tid & ~31);
+    for (int i0 = i_begin; i0 < b; i0 += 32) {
+        __syncthreads();
+        for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mq[(blk0 + i0) * R + x];
+        for (int x = tid; x < 32 * YC; x += 128) sY2[(x / YC) * YS + x % YC] = E[(blk0 + i0) * YC + x];
+        __syncthreads();
+        if (i0 + 31 < warp_jmin) continue;
+        for (int ii = 0; ii < 32; ++ii) {
+            if (i0 + ii < j_blk) continue;
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < R; ++c) s = fmaf(mk[c], sM2[ii * R + c], s);
+            const float ds = 2.f * s * dot65(sY2 + ii * YS, v);
+#pragma unroll
+            for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[ii * R + c], dm[c]);
+            axpy65(dv, s * s, sY2 + ii * YS);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < R; ++c) dMk[row * R + c] = dm[c] + sOut[tid * (R + 1) + c];
+    const int64_t o = sl.row(bh, l * b + j_blk);
+#pragma unroll
+    for (int c = 0; c < 64; ++c) stf(dV + o + c, dv[c]);
+}
+
+// ---------------------------------------------------------------------------
+// Chain rule through the half sketch: dX = ((dM*A2) G1^T + (dM*A1) G2^T)/sqrt(r),
+// A1 = X G1, A2 = X G2 recomputed.  64 rows per CTA.
+// ---------------------------------------------------------------------------
+template <typename T, int R>
+__global__ void __launch_bounds__(256)
+sketch_bwd_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const T* __restrict__ G2,
+                  int g_heads, int n, const float* __restrict__ dM, T* __restrict__ dX) {
+    extern __shared__ float smem[];
+    float* sG1 = smem;                      // [64][R+1]
+    float* sG2 = sG1 + H64 * (R + 1);       // [64][R+1]
+    float* sX = sG2 + H64 * (R + 1);        // [64][65]
+    float* sU1 = sX + 64 * 65;              // [64][R+1]
+    float* sU2 = sU1 + 64 * (R + 1);        // [64][R+1]
+    const int bh = blockIdx.y, i0 = blockIdx.x * 64, tid = threadIdx.x;
+    const int g = (g_heads == 1) ? 0 : (bh % sl.H);
+    for (int e = tid; e < H64 * R; e += 256) {
+        sG1[(e / R) * (R + 1) + e % R] = ldf(G1 + (size_t)g * H64 * R + e);
+        sG2[(e / R) * (R + 1) + e % R] = ldf(G2 + (size_t)g * H64 * R + e);
+    }
+    for (int e = tid; e < 64 * H64; e += 256) {
+        const int rr = e / H64, c = e % H64;
+        sX[rr * 65 + c] = ldf(X + sl.row(bh, i0 + rr) + c);
+    }
+    __syncthreads();
+    const float rs = rsqrtf((float)R);
+    {
+        const int c = tid % R;
+        for (int rr = tid / R; rr < 64; rr += 256 / R) {
+            float a1 = 0.f, a2 = 0.f;
+#pragma unroll 16
+            for (int t = 0; t < H64; ++t) {
+                const float x = sX[rr * 65 + t];
+                a1 = fmaf(x, sG1[t * (R + 1) + c], a1);
+                a2 = fmaf(x, sG2[t * (R + 1) + c], a2);
+            }
+            const float g_m = dM[((size_t)bh * n + i0 + rr) * R + c] * rs;
+            sU1[rr * (R + 1) + c] = g_m * a2;
+            sU2[rr * (R + 1) + c] = g_m * a1;
+        }
+    }
+    __syncthreads();
+    {
+        const int t = tid % 64;
+        for (int rr = tid / 64; rr < 64; rr += 4) {
+            float dx = 0.f;
+#pragma unroll 16
+            for (int c = 0; c < R; ++c) {
+                dx = fmaf(sU1[rr * (R + 1) + c], sG1[t * (R + 1) + c], dx);
+                dx = fmaf(sU2[rr * (R + 1) + c], sG2[t * (R + 1) + c], dx);
+            }
+            stf(dX + sl.row(bh, i0 + rr) + t, dx);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host-side launch helpers
+// ---------------------------------------------------------------------------
+#define PSK_TRY(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
+
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+template <typename T, int R>
+cudaError_t launch_sketch(const Dims& d, const T* X, const T* G1, const T* G2, float* M, float* Phi,
+                          cudaStream_t s, int* launches) {
+    const size_t smem = (size_t)(2 * H64 * R + 64 * 65 + 64 * (R + 1)) * sizeof(float);
+    PSK_TRY(allow_smem(sketch_kernel<T, R>, smem));
+    Slice sl{d.H, d.sb, d.sh, d.sn};
+    prof_begin("sketch_kernel", s);
+    sketch_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, X, G1, G2, d.g_heads, d.n, M, Phi);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <int R>
+cudaError_t launch_states(const Dims& d, const float* M, const float* Y, float* S, bool reverse,
+                          cudaStream_t s, int* launches) {
+    prof_begin("state_kernel", s);
+    state_kernel<R><<<dim3((R * R + 127) / 128, d.t, d.BH()), 128, 0, s>>>(M, Y, d.n, d.b, d.t, S);
+    prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    const size_t elems = (size_t)R * R * YC;
+    prof_begin("scan_kernel", s);
+    scan_kernel<<<dim3((unsigned)((elems + 255) / 256), d.BH()), 256, 0, s>>>(S, elems, d.t, reverse ? 1 : 0);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <typename T, int R>
+cudaError_t fwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T* G1, const T* G2,
+                     T* O, float* denom, char* ws, cudaStream_t s, int* launches) {
+    const CcWorkspace w = cc_workspace(d, false);
+    float* Mq = (float*)(ws + w.Mq); float* Mk = (float*)(ws + w.Mk);
+    float* Vt = (float*)(ws + w.Vt); float* Z = (float*)(ws + w.Zst);
+    Slice sl{d.H, d.sb, d.sh, d.sn};
+    const int rows = d.BH() * d.n;
+    PSK_TRY((launch_sketch<T, R>(d, Q, G1, G2, Mq, nullptr, s, launches)));
+    PSK_TRY((launch_sketch<T, R>(d, K, G1, G2, Mk, nullptr, s, launches)));
+    prof_begin("rows_prep_kernel", s);
+    rows_prep_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, 0, V, nullptr, nullptr, nullptr, Vt);
+    prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    PSK_TRY((launch_states<R>(d, Mk, Vt, Z, false, s, launches)));
+    PSK_TRY(allow_smem(fwd_out_kernel<T, R>, RowSmem<R>::bytes));
+    prof_begin("fwd_out_kernel", s);
+    fwd_out_kernel<T, R><<<dim3(d.b / 128, d.t, d.BH()), 128, RowSmem<R>::bytes, s>>>(
+        sl, d.n, d.b, d.t, Mq, Mk, Vt, Z, O, denom);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <typename T, int R>
+cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T* G1, const T* G2,
+                     const T* O, const float* denom, const T* dO, T* dQ, T* dK, T* dV,
+                     char* ws, cudaStream_t s, int* launches) {
+    const CcWorkspace w = cc_workspace(d, true);
+    float* Mq = (float*)(ws + w.Mq); float* Mk = (float*)(ws + w.Mk);
+    float* Vt = (float*)(ws + w.Vt); float* Z = (float*)(ws + w.Zst);
+    float* E = (float*)(ws + w.E); float* Rs = (float*)(ws + w.Rst);
+    float* dMq = (float*)(ws + w.dMq); float* dMk = (float*)(ws + w.dMk);
+    Slice sl{d.H, d.sb, d.sh, d.sn};
+    const int rows = d.BH() * d.n;
+    PSK_TRY((launch_sketch<T, R>(d, Q, G1, G2, Mq, nullptr, s, launches)));
+    PSK_TRY((launch_sketch<T, R>(d, K, G1, G2, Mk, nullptr, s, launches)));
+    prof_begin("rows_prep_kernel", s);
+    rows_prep_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, 0, V, nullptr, nullptr, nullptr, Vt);
+    prof_end(s);
+    prof_begin("rows_prep_kernel", s);
+    rows_prep_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, 1, nullptr, O, denom, dO, E);
+    prof_end(s);
+    *launches += 2;
+    PSK_TRY(cudaGetLastError());
+    PSK_TRY((launch_states<R>(d, Mk, Vt, Z, false, s, launches)));
+    PSK_TRY((launch_states<R>(d, Mq, E, Rs, true, s, launches)));
+    PSK_TRY(allow_smem(bwd_q_kernel<R>, RowSmem<R>::bytes));
+    PSK_TRY(allow_smem(bwd_k_kernel<T, R>, RowSmem<R>::bytes));
+    const dim3 grid(d.b / 128, d.t, d.BH());
+    prof_begin("bwd_q_kernel", s);
+    bwd_q_kernel<R><<<grid, 128, RowSmem<R>::bytes, s>>>(d.n, d.b, d.t, Mq, Mk, Vt, E, Z, dMq);
+    prof_end(s);
+    prof_begin("bwd_k_kernel", s);
+    bwd_k_kernel<T, R><<<grid, 128, RowSmem<R>::bytes, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Rs, dMk, dV);
+    prof_end(s);
+    *launches += 2;
+    PSK_TRY(cudaGetLastError());
+    const size_t smem = (size_t)(2 * H64 * (R + 1) + 64 * 65 + 2 * 64 * (R + 1)) * sizeof(float);
+    PSK_TRY(allow_smem(sketch_bwd_kernel<T, R>, smem));
+    prof_begin("sketch_bwd_kernel", s);
+    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dQ);
+    prof_end(s);
+    prof_begin("sketch_bwd_kernel", s);
+    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dK);
+    prof_end(s);
+    *launches += 2;
+    return cudaGetLastError();
+}
+
+#define PSK_DISPATCH(CALL_F32, CALL_BF16)                                   \
+    if (d.bf16) {                                                           \
+        typedef __nv_bfloat16 T;                                            \
+        switch (d.r) { case 16: { constexpr int R = 16; return CALL_BF16; } \
+                       case 32: { constexpr int R = 32; return CALL_BF16; } \
+                       case 64: { constexpr int R = 64; return CALL_BF16; } } \
+    } else {                                                                \
+        typedef float T;                                                    \
+        switch (d.r) { case 16: { constexpr int R = 16; return CALL_F32; }  \
+                       case 32: { constexpr int R = 32; return CALL_F32; }  \
+                       case 64: { constexpr int R = 64; return CALL_F32; } } \
+    }                                                                       \
+    return cudaErrorInvalidValue;
+
+}  // namespace
+
+cudaError_t cc_sketch(const Dims& d, const void* X, const void* G1, const void* G2,
+                      float* M_out, float* Phi_out, cudaStream_t s, int* launches) {
+#define C_ (launch_sketch<T, R>(d, (const T*)X, (const T*)G1, (const T*)G2, M_out, Phi_out, s, launches))
+    PSK_DISPATCH(C_, C_)
+#undef C_
+}
+
+cudaError_t cc_fwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, void* O, float* denom,
+                   char* ws, cudaStream_t s, int* launches) {
+#define C_ (fwd_impl<T, R>(d, (const T*)Q, (const T*)K, (const T*)V, (const T*)G1, (const T*)G2, \
+                           (T*)O, denom, ws, s, launches))
+    PSK_DISPATCH(C_, C_)
+#undef C_
+}
+
+cudaError_t cc_bwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, const void* O, const float* denom,
+                   const void* dO, void* dQ, void* dK, void* dV,
+                   char* ws, cudaStream_t s, int* launches) {
+#define C_ (bwd_impl<T, R>(d, (const T*)Q, (const T*)K, (const T*)V, (const T*)G1, (const T*)G2, \
+                           (const T*)O, denom, (const T*)dO, (T*)dQ, (T*)dK, (T*)dV, ws, s, launches))
+    PSK_DISPATCH(C_, C_)
+#undef C_
+}
+
+}  // namespace psk

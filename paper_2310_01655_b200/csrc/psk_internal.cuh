@@ -1,0 +1,66 @@
+// Internal declarations shared by the translation units of libpsk (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "psk.h"
+
+namespace psk {
+
+// Validated problem description handed to the launchers.
+struct Dims {
+    int B, H, n, h, r, b, t;          // t = n / b blocks per head (Section 3.1)
+    int64_t sb, sh, sn;               // element strides of the [B,H,n,h] tensors
+    int g_heads;                      // 1 or H
+    bool bf16;                        // storage type
+    int BH() const { return B * H; }
+};
+
+constexpr size_t kAlign = 256;
+constexpr size_t kStatusBytes = 256;  // first bytes of every workspace: device status word(s)
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Scratch layout of the CUDA-core path (all fp32).
+struct CcWorkspace {
+    size_t status, Mq, Mk, Vt, Zst, E, Rst, dMq, dMk, total;
+};
+CcWorkspace cc_workspace(const Dims& d, bool backward);
+
+// CUDA-core (fp32 arithmetic) launchers.  Each returns a cudaError_t from the launches
+// and adds the number of kernels it enqueued to *launches.
+cudaError_t cc_sketch(const Dims& d, const void* X, const void* G1, const void* G2,
+                      float* M_out, float* Phi_out, cudaStream_t s, int* launches);
+cudaError_t cc_fwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, void* O, float* denom,
+                   char* ws, cudaStream_t s, int* launches);
+cudaError_t cc_bwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, const void* O, const float* denom,
+                   const void* dO, void* dQ, void* dK, void* dV,
+                   char* ws, cudaStream_t s, int* launches);
+
+// Tensor-core (bf16 operands, fp32 accumulation) launchers.
+size_t tc_workspace_bytes(const Dims& d, bool backward);
+bool tc_supported(const Dims& d);
+cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, void* O, float* denom,
+                   char* ws, cudaStream_t s, int* launches);
+cudaError_t tc_bwd(const Dims& d, const void* Q, const void* K, const void* V,
+                   const void* G1, const void* G2, const void* O, const float* denom,
+                   const void* dO, void* dQ, void* dK, void* dV,
+                   char* ws, cudaStream_t s, int* launches);
+
+// Optional per-kernel timing (psk_profile_*): when enabled, each launch is bracketed by
+// CUDA events on its own stream; disabled, these are no-ops.
+void prof_begin(const char* name, cudaStream_t s);
+void prof_end(cudaStream_t s);
+
+__device__ __forceinline__ float ldf(const float* p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float* p, float v) { *p = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+}  // namespace psk
