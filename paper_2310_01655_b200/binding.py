@@ -116,6 +116,11 @@ def _same_layout(ref, *ts):
             raise ValueError("all [B,H,n,h] tensors must share shape, strides and dtype")
 
 
+def _empty_like(x):
+    """Uninitialised tensor with exactly x's shape AND strides (views included)."""
+    return torch.empty_strided(x.shape, x.stride(), dtype=x.dtype, device=x.device)
+
+
 def sketch(X, G1, G2, r=None, b=128, want_phi=False, path=PATH_AUTO):
     """psk_sketch: returns (M [B,H,n,r] fp32, Phi [B,H,n,r*r] fp32 or None)."""
     _require_cuda(X, G1, G2)
@@ -136,7 +141,7 @@ def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out
     _require_cuda(Q, K, V, G1, G2)
     _same_layout(Q, K, V, out)
     shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
-    O = torch.empty_like(Q) if out is None else out
+    O = _empty_like(Q) if out is None else out
     B, H, n, _ = Q.shape
     if denom is None:
         denom = torch.empty((B, H, n), dtype=torch.float32, device=Q.device)
@@ -153,7 +158,7 @@ def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, works
     _require_cuda(Q, K, V, G1, G2, O, denom, dO)
     _same_layout(Q, K, V, O, dO)
     shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
-    dQ, dK, dV = out if out is not None else (torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q))
+    dQ, dK, dV = out if out is not None else (_empty_like(Q), _empty_like(Q), _empty_like(Q))
     _same_layout(Q, dQ, dK, dV)
     ws, nbytes = _workspace(shp, True, workspace)
     st = lib().psk_causal_attn_bwd(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(G1), _ptr(G2), _ptr(O),
