@@ -110,6 +110,28 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
                         const void* dO, void* dQ, void* dK, void* dV,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* Forward pass for callers that must not allocate device memory (no counterpart in the
+ * paper: it computes exactly what psk_causal_attn_fwd computes).  Think of a plug-in that
+ * runs inside a host application which has already handed the whole GPU to its own
+ * memory pool, a real-time loop that may not call the allocator, or code that is not
+ * allowed to touch cudaMalloc at all: none of them can size and allocate a workspace.
+ * Here the scratch is a fixed array of psk_static_scratch_bytes() bytes (16 MiB) that
+ * lives inside the library image; every GPU that loads the library holds it until the
+ * process exits.  The caller passes inputs and outputs only.
+ *   - Always runs the CUDA-core (fp32 arithmetic) kernels, for either storage type.
+ *   - Shapes whose forward scratch (psk_workspace_bytes with path = PSK_PATH_CUDA_CORES)
+ *     exceeds the array are refused with PSK_ERR_WORKSPACE before any launch.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls on a device share the one array and it keeps the previous call's bytes;
+ *     the call zeroes the part that must start at zero.  Two calls that overlap on the
+ *     GPU (different streams, or different threads) race on it: serialise them.
+ * Arguments and error codes otherwise as psk_causal_attn_fwd. */
+size_t psk_static_scratch_bytes(void);
+int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void* K, const void* V,
+                               const void* G1, const void* G2, void* O, float* denom, void* stream);
+
 /* Synchronises `stream`, then reports PSK_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` abandoned a bounded wait, PSK_ERR_CUDA if the stream is in error,
  * else PSK_OK.  Never traps. */

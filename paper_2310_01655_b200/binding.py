@@ -55,6 +55,9 @@ def lib():
     L.psk_causal_attn_fwd.argtypes = [P] + [c_void_p] * 8 + [c_size_t, c_void_p]
     L.psk_causal_attn_bwd.restype = c_int
     L.psk_causal_attn_bwd.argtypes = [P] + [c_void_p] * 12 + [c_size_t, c_void_p]
+    L.psk_static_scratch_bytes.restype = c_size_t
+    L.psk_causal_attn_fwd_static.restype = c_int
+    L.psk_causal_attn_fwd_static.argtypes = [P] + [c_void_p] * 8
     L.psk_check.restype = c_int
     L.psk_check.argtypes = [c_void_p, c_void_p]
     L.psk_last_launch_count.restype = c_int
@@ -150,6 +153,29 @@ def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out
                                    _ptr(denom), _ptr(ws), nbytes, _stream())
     if st != 0:
         raise PskError(st, "psk_causal_attn_fwd")
+    return O, denom
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().psk_static_scratch_bytes())
+
+
+def causal_attn_fwd_static(Q, K, V, G1, G2, b, p=4, out=None, denom=None):
+    """psk_causal_attn_fwd_static: the forward for callers that cannot allocate device
+    memory.  The library uses its built-in 16 MiB scratch array, so no workspace is passed
+    and nothing is allocated by the call itself; `out` and `denom` must be supplied by such
+    a caller (they are created here only as a convenience when omitted)."""
+    _require_cuda(Q, K, V, G1, G2)
+    _same_layout(Q, K, V, out)
+    shp = make_shape(Q, G1, G1.shape[-1], b, p, PATH_CUDA_CORES)
+    O = _empty_like(Q) if out is None else out
+    B, H, n, _ = Q.shape
+    if denom is None:
+        denom = torch.empty((B, H, n), dtype=torch.float32, device=Q.device)
+    st = lib().psk_causal_attn_fwd_static(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(G1), _ptr(G2), _ptr(O),
+                                          _ptr(denom), _stream())
+    if st != 0:
+        raise PskError(st, "psk_causal_attn_fwd_static")
     return O, denom
 
 
