@@ -56,10 +56,10 @@ int make_dims(const psk_shape* sh, Dims* d) {
 }
 
 // 0 = CUDA cores, 1 = tensor cores, <0 = error
-int pick_path(const psk_shape* sh, const Dims& d) {
+int pick_path(const psk_shape* sh, const Dims& d, bool backward) {
     if (sh->path == PSK_PATH_CUDA_CORES) return 0;
-    if (sh->path == PSK_PATH_TENSOR_CORES) return (d.bf16 && tc_supported(d)) ? 1 : PSK_ERR_UNSUPPORTED;
-    return (d.bf16 && tc_supported(d)) ? 1 : 0;
+    if (sh->path == PSK_PATH_TENSOR_CORES) return (d.bf16 && tc_supported(d, backward)) ? 1 : PSK_ERR_UNSUPPORTED;
+    return (d.bf16 && tc_supported(d, backward)) ? 1 : 0;
 }
 
 }  // namespace
@@ -85,7 +85,7 @@ const char* psk_status_string(int status) {
 size_t psk_workspace_bytes(const psk_shape* shape, int for_backward) {
     Dims d;
     if (make_dims(shape, &d) != PSK_OK) return 0;
-    const int path = pick_path(shape, d);
+    const int path = pick_path(shape, d, for_backward != 0);
     if (path < 0) return 0;
     return path == 1 ? tc_workspace_bytes(d, for_backward != 0) : cc_workspace(d, for_backward != 0).total;
 }
@@ -114,7 +114,7 @@ int psk_causal_attn_fwd(const psk_shape* shape, const void* Q, const void* K, co
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(G1) || !aligned16(G2) ||
         !aligned16(O) || !aligned16(denom))
         return PSK_ERR_ALIGN;
-    const int path = pick_path(shape, d);
+    const int path = pick_path(shape, d, false);
     if (path < 0) return path;
     const size_t need = psk_workspace_bytes(shape, 0);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign))
@@ -141,7 +141,7 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
         !aligned16(O) || !aligned16(denom) || !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) ||
         !aligned16(dV))
         return PSK_ERR_ALIGN;
-    const int path = pick_path(shape, d);
+    const int path = pick_path(shape, d, true);
     if (path < 0) return path;
     const size_t need = psk_workspace_bytes(shape, 1);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign))

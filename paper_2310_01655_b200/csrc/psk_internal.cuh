@@ -44,7 +44,7 @@ cudaError_t cc_bwd(const Dims& d, const void* Q, const void* K, const void* V,
 
 // Tensor-core (bf16 operands, fp32 accumulation) launchers.
 size_t tc_workspace_bytes(const Dims& d, bool backward);
-bool tc_supported(const Dims& d);
+bool tc_supported(const Dims& d, bool backward);
 cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V,
                    const void* G1, const void* G2, void* O, float* denom,
                    char* ws, cudaStream_t s, int* launches);
