@@ -10,6 +10,7 @@
 // or as an MN-major B operand with K = 80 (contract over the 65 columns).
 #include "psk_internal.cuh"
 #include "tc_features.cuh"
+#include "tc_common.cuh"
 
 #include <mutex>
 #include <type_traits>
@@ -19,8 +20,6 @@ namespace psk {
 using namespace tc;
 typedef __nv_bfloat16 bf16;
 
-namespace {
-
 // ---------------------------------------------------------------------------
 // host: tensor maps
 // ---------------------------------------------------------------------------
@@ -28,7 +27,7 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeFn encoder() {
+static EncodeFn encoder() {
     static EncodeFn fn = nullptr;
     static std::once_flag once;
     std::call_once(once, [] {
@@ -42,7 +41,7 @@ EncodeFn encoder() {
 }
 
 // [B,H,n,64] bf16 tensor with element strides; box = 128 rows x 64 columns, 128-byte swizzle.
-bool map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t sb, int64_t sh, int64_t sn) {
+bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t sb, int64_t sh, int64_t sn) {
     EncodeFn enc = encoder();
     if (!enc) return false;
     cuuint64_t dims[4] = {64, (cuuint64_t)n, (cuuint64_t)H, (cuuint64_t)B};
@@ -53,7 +52,7 @@ bool map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t sb,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 // States S[nblk][80][FP] bf16; box = 80 rows x 64 features.
-bool map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
+bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
     EncodeFn enc = encoder();
     if (!enc) return false;
     cuuint64_t dims[3] = {(cuuint64_t)FP, 80, (cuuint64_t)nblk};
@@ -64,73 +63,7 @@ bool map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// ---------------------------------------------------------------------------
-// device helpers
-// ---------------------------------------------------------------------------
-template <int I, int N, typename Fn>
-__device__ __forceinline__ void static_for(Fn&& f) {
-    if constexpr (I < N) {
-        f(std::integral_constant<int, I>{});
-        static_for<I + 1, N>(f);
-    }
-}
-
-constexpr int kErrTma = 1, kErrMma = 2;
-
-__device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
-    return p + ((1024u - (smem_u32(p) & 1023u)) & 1023u);
-}
-
-// [G1 | G2]^T as a K-major, 128-byte-swizzled tile: row n (< 2R) holds sketch column n over the 64
-// head dimensions.  B operand of the sketch GEMM X [G1 | G2].
-template <int R>
-__device__ __forceinline__ void build_g_tile(uint8_t* sG, const bf16* G1, const bf16* G2, int tid) {
-    for (int e = tid; e < 2 * R * 64; e += 128) {
-        const int nn = e / 64, k = e % 64;
-        const bf16 v = (nn < R ? G1 : G2)[k * R + (nn % R)];
-        *reinterpret_cast<bf16*>(sG + swz128_offset(nn, k / 8) + (k % 8) * 2) = v;
-    }
-}
-
-// Sketch GEMM D[128 tokens x 2R] = X_tile [G1 | G2], 4 K steps of 16 over the head dimension.
-template <int R>
-__device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX, const uint8_t* sG) {
-    constexpr uint32_t idesc = idesc_bf16(128, 2 * R, false, false);
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-        umma_ss(d_tmem, smem_desc(smem_u32(sX) + k * 32, 0, 1024, kSwz128),
-                smem_desc(smem_u32(sG) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
-}
-
-// m[c] = A1[c] A2[c] / sqrt(R) from the sketch accumulator (this thread's lane).
-template <int R>
-__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R]) {
-    const float rs = rsqrtf((float)R);
-#pragma unroll
-    for (int c0 = 0; c0 < R; c0 += 16) {
-        uint32_t a1[16], a2[16];
-        tmem_ld16(lane_tmem + c0, a1);
-        tmem_ld16(lane_tmem + R + c0, a2);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) m[c0 + j] = __uint_as_float(a1[j]) * __uint_as_float(a2[j]) * rs;
-    }
-}
-
-// Half sketch rows as a K-major, un-swizzled operand: 8x8 core matrices, [k chunk][row/8][row%8][16 B]
-// (K-direction stride 2048 B, 8-row-group stride 128 B).
-template <int R>
-__device__ __forceinline__ void store_half_sketch_rows(uint8_t* dst, const float (&m)[R], int row) {
-#pragma unroll
-    for (int kc = 0; kc < R / 8; ++kc) {
-        uint4 v;
-        v.x = pack_bf16(m[kc * 8 + 0], m[kc * 8 + 1]);
-        v.y = pack_bf16(m[kc * 8 + 2], m[kc * 8 + 3]);
-        v.z = pack_bf16(m[kc * 8 + 4], m[kc * 8 + 5]);
-        v.w = pack_bf16(m[kc * 8 + 6], m[kc * 8 + 7]);
-        *reinterpret_cast<uint4*>(dst + kc * 2048 + (row / 8) * 128 + (row % 8) * 16) = v;
-    }
-}
+namespace {
 
 // ---------------------------------------------------------------------------
 // Per-block state  H_l = phi(X_l)^T [Y_l | y65]   (Section 3.1), feature tiles [T0, T0+TN)
@@ -511,26 +444,6 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 // ---------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------
-#define PSK_TRY(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
-
-template <typename Kern>
-cudaError_t set_smem(Kern k, size_t bytes) {
-    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
-
-struct TcWorkspace { size_t status, Z, Rst, total; };
-
-template <int R>
-TcWorkspace tc_ws(const Dims& d, bool backward) {
-    TcWorkspace w{};
-    const size_t st = (size_t)d.BH() * d.t * 80 * Feat<R>::FP * sizeof(bf16);
-    size_t off = 0;
-    w.status = off; off += kStatusBytes;
-    w.Z = off; off += align_up(st);
-    if (backward) { w.Rst = off; off += align_up(st); }
-    w.total = off;
-    return w;
-}
 
 // States of every block + scan.  X is sketched, Y is the right-hand side.
 template <int R, int T0, int TN>
@@ -575,8 +488,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     int* status = reinterpret_cast<int*>(ws + w.status);
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
     CUtensorMap mQ, mK, mV, mZ;
-    if (!map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
-        !map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
+    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
         return cudaErrorInvalidValue;
     PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, Z, false, status, s, launches)));
     constexpr size_t smem = OutSmem<R>::total + 1024;
@@ -593,7 +506,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 }  // namespace
 
 bool tc_supported(const Dims& d, bool backward) {
-    return d.bf16 && !backward && encoder() != nullptr;
+    (void)backward;
+    return d.bf16 && encoder() != nullptr;
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
@@ -614,9 +528,14 @@ cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V, c
     return cudaErrorInvalidValue;
 }
 
-cudaError_t tc_bwd(const Dims&, const void*, const void*, const void*, const void*, const void*, const void*,
-                   const float*, const void*, void*, void*, void*, char*, cudaStream_t, int*) {
-    return cudaErrorNotSupported;
+cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+                      const float* y65, bf16* S, bool reverse, int* status, cudaStream_t s, int* launches) {
+    switch (d.r) {
+        case 16: return launch_states<16>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
+        case 32: return launch_states<32>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
+        case 64: return launch_states<64>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace psk

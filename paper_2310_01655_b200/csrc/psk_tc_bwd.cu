@@ -1,0 +1,504 @@
+// Tensor-core backward of causal Polysketch attention.
+//
+// With g = dO, E_i = [g_i/d_i | -(g_i.O_i)/d_i], V~_j = [v_j | 1], s_ij = m(q_i).m(k_j):
+//   dL/dW_ij = E_i.V~_j (j <= i),  ds_ij = 2 s_ij dW_ij,
+//   dm(q_i) = sum_j ds_ij m(k_j),  dm(k_j) = sum_i ds_ij m(q_i),  dV_j = sum_i s_ij^2 E_i[:h].
+// Pairs in the same block of b rows go through 128 x 128 tiles; pairs in different blocks go
+// through the prefix state Z_l = sum_{blocks<l} phi(K)^T V~ (queries) and the suffix state
+// R_l = sum_{blocks>l} phi(Q)^T E (keys, values), in the manner of Section 3.1:
+//   d phi_w(q_i) = Z_l E_i,   d phi(k_j) = w * (R_l V~_j),   dV~_j = R_l^T phi_w(k_j),
+// and, because every feature is a product m_a m_b, dm = 2 * sum over features of
+// (d feature) * (the other factor)  (tc_features.cuh explains the weights w).
+// One kernel, two roles: QSIDE rows own (Q, E) and meet keys j <= i; key-side rows own (K, V)
+// and meet queries i >= j.  Thread = own row throughout.
+#include "tc_common.cuh"
+
+namespace psk {
+
+using namespace tc;
+
+namespace {
+
+// E = dO / d (bf16) and e65 = -(dO . O) / d (fp32), one warp per row.
+__global__ void __launch_bounds__(256)
+tc_bwd_prep_kernel(const bf16* __restrict__ O, const bf16* __restrict__ dO, const float* __restrict__ denom,
+                   int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn, bf16* __restrict__ E,
+                   float* __restrict__ e65) {
+    const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (row >= total_rows) return;
+    const int bh = row / n, i = row % n;
+    const int64_t base = (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn + 2 * lane;
+    const __nv_bfloat162 g2 = *reinterpret_cast<const __nv_bfloat162*>(dO + base);
+    const __nv_bfloat162 o2 = *reinterpret_cast<const __nv_bfloat162*>(O + base);
+    const float g0 = __low2float(g2), g1 = __high2float(g2);
+    float dot = g0 * __low2float(o2) + g1 * __high2float(o2);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
+    const float inv = 1.f / denom[row];
+    *reinterpret_cast<uint32_t*>(E + (size_t)row * 64 + 2 * lane) = pack_bf16(g0 * inv, g1 * inv);
+    if (lane == 0) e65[row] = -dot * inv;
+}
+
+constexpr int kStages = 3;
+constexpr uint32_t kBoxBytes = 80 * 128;
+
+struct BwdSmem {
+    // every tile: 128 rows x 128 B, 128-byte swizzle
+    static constexpr uint32_t Xown = 0, Yown = 16384, Xoth = 32768, Yoth = 49152, Mown = 65536, Moth = 81920;
+    static constexpr uint32_t G = 98304;                 // up to 128 rows
+    static constexpr uint32_t ExtA = G + 16384;          // [128 x 16] un-swizzled: column 0 = own 65th column
+    static constexpr uint32_t Eoth = ExtA + 4096;        // 128 floats: other side's 65th column
+    static constexpr uint32_t Box = ExtA + 4096 + 1024;  // state boxes
+    static constexpr uint32_t total = Box + kStages * ((kBoxBytes + 1023) / 1024 * 1024);
+};
+constexpr uint32_t kBoxStride = (kBoxBytes + 1023) / 1024 * 1024;
+
+// Half-sketch rows as a [128 rows x 128 B] swizzled tile, zero beyond R columns: K-major operand
+// of the score GEMM (K steps over R) and MN-major B operand (N = 64) of the dM GEMMs.
+template <int R>
+__device__ __forceinline__ void store_padded_rows(uint8_t* dst, const float (&m)[R], int row) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < R / 8) {
+            v.x = pack_bf16(m[(c % (R / 8)) * 8 + 0], m[(c % (R / 8)) * 8 + 1]);
+            v.y = pack_bf16(m[(c % (R / 8)) * 8 + 2], m[(c % (R / 8)) * 8 + 3]);
+            v.z = pack_bf16(m[(c % (R / 8)) * 8 + 4], m[(c % (R / 8)) * 8 + 5]);
+            v.w = pack_bf16(m[(c % (R / 8)) * 8 + 6], m[(c % (R / 8)) * 8 + 7]);
+        }
+        *reinterpret_cast<uint4*>(dst + swz128_offset(row, c)) = v;
+    }
+}
+
+// dm += (d feature) * (the other factor) for the 32 features F0 .. F0+31 held in x
+template <int R, int F0>
+__device__ __forceinline__ void untensor32(const uint32_t (&x)[32], const float (&m)[R], float (&dm)[R]) {
+    static_for<0, 32>([&](auto jc) {
+        constexpr int J = decltype(jc)::value;
+        constexpr int f = F0 + J;
+        if constexpr (f < Feat<R>::F) {
+            constexpr int A = Feat<R>::a(f), B = Feat<R>::b(f);
+            const float v = __uint_as_float(x[J]);
+            if constexpr (A != B) {
+                dm[A] = fmaf(v, m[B], dm[A]);
+                dm[B] = fmaf(v, m[A], dm[B]);
+            } else {
+                dm[A] = fmaf(v, m[A], dm[A]);
+            }
+        }
+    });
+}
+
+template <int R, bool QSIDE>
+__global__ void __launch_bounds__(128)
+tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
+                   const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
+                   const __grid_constant__ CUtensorMap mapS, const bf16* __restrict__ G1,
+                   const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
+                   const float* __restrict__ e65, bf16* __restrict__ dX, bf16* __restrict__ dV, int64_t sb,
+                   int64_t sh, int64_t sn, int* status) {
+    using F = Feat<R>;
+    using L = BwdSmem;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_phi[2], bar_box[kStages];
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
+    const int hi = bh % H, bi = bh / H;
+    const int g = g_heads == 1 ? 0 : hi;
+    const int row0 = l * b + tau * 128;
+    const int blk = bh * t + l;
+    const int ntiles = b / 128;
+    const bool has_state = QSIDE ? (l > 0) : (l < t - 1);
+
+    if (tid == 0) {
+        mbar_init(&bar_own, 1); mbar_init(&bar_oth, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
+        tma_prefetch_desc(&mapYoth); tma_prefetch_desc(&mapS);
+        mbar_expect_tx(&bar_own, 32768);
+        tma_load_4d(smem + L::Xown, &mapXown, 0, row0, hi, bi, &bar_own);
+        tma_load_4d(smem + L::Yown, &mapYown, 0, row0, hi, bi, &bar_own);
+        if (has_state) {
+            for (int c = 0; c < kStages && c < F::NC; ++c) {
+                mbar_expect_tx(&bar_box[c], kBoxBytes);
+                tma_load_3d(smem + L::Box + c * kBoxStride, &mapS, c * 64, 0, blk, &bar_box[c]);
+            }
+        }
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
+    // own 65th column (e_i for query rows, 1 for key rows) as the K extension of the d-phi GEMM
+    const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
+    {
+        uint8_t* ext = smem + L::ExtA;
+        *reinterpret_cast<uint4*>(ext + (tid / 8) * 128 + (tid % 8) * 16) =
+            make_uint4(pack_bf16(y65, 0.f), 0, 0, 0);
+        *reinterpret_cast<uint4*>(ext + 2048 + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tmem_slot;
+    const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
+    // tensor-memory columns.  Phase B (states) and phase C (tiles) reuse [0, 256).
+    constexpr uint32_t cS = 0, cDW = 128;                 // phase C: scores, dW; then packed dS / W
+    constexpr uint32_t cPhi = 0, cFA = 128;               // phase B: d-phi (2 x 64), feature staging (2 x 32)
+    constexpr uint32_t cSk = 256;                         // sketch accumulators (transient, <= 128)
+    constexpr uint32_t cdM = 384, cdV = 448;              // accumulators: dM (64), dV (64)
+    uint32_t mma_uses = 0;
+    bool ok = true;
+
+    // ---- phase A: half sketch of the own rows ----
+    ok = mbar_wait(&bar_own, 0, status, kErrTma);
+    if (tid == 0) {
+        tc_fence_after();
+        issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);
+        umma_commit(&bar_mma);
+    }
+    ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+    ++mma_uses;
+    tc_fence_after();
+    float m[R], dm[R];
+    read_half_sketch<R>(lane_tm + cSk, m);
+    store_padded_rows<R>(smem + L::Mown, m, tid);
+#pragma unroll
+    for (int c = 0; c < R; ++c) dm[c] = 0.f;
+    bool dv_started = false;
+
+    // ---- phase B: other blocks through the state ----
+    if (has_state) {
+        constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, true);
+        auto issue_dphi = [&](int c, int buf) {      // d-phi chunk c = [Yown | y65] x box(c), K = 64 + 16
+            const uint32_t box = smem_u32(smem + L::Box + (c % kStages) * kBoxStride);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
+                        smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc_phi, k > 0);
+            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
+                    smem_desc(box + 4 * 2048, 0, 1024, kSwz128), idesc_phi, 1);
+        };
+        ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
+        if (tid == 0) {
+            tc_fence_after();
+            issue_dphi(0, 0);
+            umma_commit(&bar_phi[0]);
+        }
+        static_for<0, F::NC>([&](auto cc) {
+            constexpr int C = decltype(cc)::value;
+            constexpr int buf = C & 1;
+            constexpr int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+            if constexpr (!QSIDE) {
+                // dV += phi_w(k) chunk (tensor memory) x box, contraction over the chunk's features
+                uint32_t pk[16];
+                gen_features<R, C * 64, true, 16>(m, pk);
+                tmem_st16(lane_tm + cFA + buf * 32, pk);
+                gen_features<R, C * 64 + 32, true, 16>(m, pk);
+                tmem_st16(lane_tm + cFA + buf * 32 + 16, pk);
+                tmem_st_wait();
+                tc_fence_before();
+                __syncthreads();
+                if (tid == 0) {
+                    tc_fence_after();
+                    constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
+                    const uint32_t box = smem_u32(smem + L::Box + (C % kStages) * kBoxStride);
+#pragma unroll
+                    for (int k = 0; k < ksteps; ++k)
+                        umma_ts(tm + cdV, tm + cFA + buf * 32 + k * 8, smem_desc(box + k * 32, 0, 1024, kSwz128), idesc,
+                                (C > 0 || k > 0) ? 1u : 0u);
+                }
+            }
+            if constexpr (C + 1 < F::NC) {
+                ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
+                if (tid == 0) {
+                    tc_fence_after();
+                    issue_dphi(C + 1, buf ^ 1);
+                    umma_commit(&bar_phi[buf ^ 1]);     // also covers this chunk's dV MMAs
+                }
+            } else if constexpr (!QSIDE) {
+                if (tid == 0) umma_commit(&bar_mma);    // last chunk's dV MMAs
+            }
+            ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+            tc_fence_after();
+            // box C-1 is free once d-phi(C) has completed (its commit also covered dV(C-1))
+            if constexpr (C >= 1 && C - 1 + kStages < F::NC) {
+                if (tid == 0) {
+                    constexpr int s2 = (C - 1) % kStages;
+                    mbar_expect_tx(&bar_box[s2], kBoxBytes);
+                    tma_load_3d(smem + L::Box + s2 * kBoxStride, &mapS, (C - 1 + kStages) * 64, 0, blk, &bar_box[s2]);
+                }
+            }
+            {
+                uint32_t x[32];
+                tmem_ld32(lane_tm + cPhi + buf * 64, x);
+                tmem_ld_wait();
+                untensor32<R, C * 64>(x, m, dm);
+                tmem_ld32(lane_tm + cPhi + buf * 64 + 32, x);
+                tmem_ld_wait();
+                untensor32<R, C * 64 + 32>(x, m, dm);
+            }
+            // every thread has read this d-phi buffer before chunk C+2 is issued into it
+            tc_fence_before();
+            __syncthreads();
+        });
+        if constexpr (!QSIDE) {
+            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
+            dv_started = true;
+        }
+#pragma unroll
+        for (int c = 0; c < R; ++c) dm[c] *= 2.f;
+        __syncthreads();
+        tc_fence_after();
+    }
+
+    // ---- phase C: same block, other-side tiles ----
+    const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
+    bool dm_started = false;
+    uint32_t oth_uses = 0;
+    float* e_oth = reinterpret_cast<float*>(smem + L::Eoth);
+    for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
+        const int orow0 = l * b + tp * 128;
+        if (tid == 0) {
+            mbar_expect_tx(&bar_oth, 32768);
+            tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0, hi, bi, &bar_oth);
+            tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0, hi, bi, &bar_oth);
+        }
+        if constexpr (!QSIDE) e_oth[tid] = e65[(size_t)bh * n + orow0 + tid];
+        ok = mbar_wait(&bar_oth, oth_uses & 1, status, kErrTma);
+        ++oth_uses;
+        if (tid == 0) {
+            tc_fence_after();
+            issue_sketch<R>(tm + cSk, smem + L::Xoth, smem + L::G);
+            umma_commit(&bar_mma);
+        }
+        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+        {
+            float mo[R];
+            read_half_sketch<R>(lane_tm + cSk, mo);
+            store_padded_rows<R>(smem + L::Moth, mo, tid);
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
+#pragma unroll
+            for (int k = 0; k < R / 16; ++k)      // scores: own rows x other rows over the sketch dimension
+                umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mown) + k * 32, 0, 1024, kSwz128),
+                        smem_desc(smem_u32(smem + L::Moth) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
+                umma_ss(tm + cDW, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
+                        smem_desc(smem_u32(smem + L::Yoth) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+            umma_commit(&bar_mma);
+        }
+        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+        const bool diag = (tp == tau);
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t sv[32], wv[32], pds[16], pw[16];
+            tmem_ld32(lane_tm + cS + c0, sv);
+            tmem_ld32(lane_tm + cDW + c0, wv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int col = c0 + j;
+                const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
+                const float s = keep ? __uint_as_float(sv[j]) : 0.f;
+                const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65 : e_oth[col]);
+                sv[j] = __float_as_uint(2.f * s * dw);
+                wv[j] = __float_as_uint(s * s);
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                pds[j] = pack_bf16(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1]));
+                pw[j] = pack_bf16(__uint_as_float(wv[2 * j]), __uint_as_float(wv[2 * j + 1]));
+            }
+            // the packed tiles overwrite columns whose fp32 contents have already been read
+            tmem_st16(lane_tm + cS + c0 / 2, pds);
+            if constexpr (!QSIDE) tmem_st16(lane_tm + cDW + c0 / 2, pw);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)           // dM_own += dS x M_other
+                umma_ts(tm + cdM, tm + cS + k * 8, smem_desc(smem_u32(smem + L::Moth) + k * 2048, 0, 1024, kSwz128),
+                        idesc, (dm_started || k > 0) ? 1u : 0u);
+            if constexpr (!QSIDE) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)       // dV += W x E_other
+                    umma_ts(tm + cdV, tm + cDW + k * 8,
+                            smem_desc(smem_u32(smem + L::Yoth) + k * 2048, 0, 1024, kSwz128), idesc,
+                            (dv_started || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&bar_mma);
+        }
+        dm_started = true;
+        dv_started = true;
+        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+    }
+
+    // ---- phase D: through the sketch, dX = ((dM*A2) G1^T + (dM*A1) G2^T) / sqrt(R) ----
+    if (ok) {
+        if (tid == 0) {
+            tc_fence_after();
+            issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);   // A1, A2 again
+            umma_commit(&bar_mma);
+        }
+        ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+    }
+    if (ok) {
+        const float rs = rsqrtf((float)R);
+        // dM total = state part (registers) + tile part (tensor memory), scaled by 1/sqrt(R)
+#pragma unroll
+        for (int c0 = 0; c0 < R; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(lane_tm + cdM + c0, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + __uint_as_float(v[j])) * rs;
+        }
+        // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cS)
+#pragma unroll
+        for (int c0 = 0; c0 < R; c0 += 16) {
+            uint32_t a1[16], a2[16], u1[8], u2[8];
+            tmem_ld16(lane_tm + cSk + c0, a1);
+            tmem_ld16(lane_tm + cSk + R + c0, a2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                u1[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a2[2 * j]),
+                                  dm[c0 + 2 * j + 1] * __uint_as_float(a2[2 * j + 1]));
+                u2[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a1[2 * j]),
+                                  dm[c0 + 2 * j + 1] * __uint_as_float(a1[2 * j + 1]));
+            }
+            tmem_st8(lane_tm + cS + c0 / 2, u1);
+            tmem_st8(lane_tm + cS + R / 2 + c0 / 2, u2);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+#pragma unroll
+            for (int k = 0; k < 2 * R / 16; ++k)    // contraction over the 2R sketch columns
+                umma_ts(tm + cDW, tm + cS + k * 8, smem_desc(smem_u32(smem + L::G) + k * 2048, 0, 1024, kSwz128), idesc,
+                        k > 0);
+            umma_commit(&bar_mma);
+        }
+        ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+    }
+    if (ok) {
+        const int64_t o = (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
+#pragma unroll
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(lane_tm + cDW + c0, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; j += 8)
+                *reinterpret_cast<uint4*>(dX + o + c0 + j) =
+                    make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+                               pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
+                               pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
+                               pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+        }
+        if constexpr (!QSIDE) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_tm + cdV + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; j += 8)
+                    *reinterpret_cast<uint4*>(dV + o + c0 + j) =
+                        make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+                                   pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
+                                   pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
+                                   pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
+template <int R>
+cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
+                     const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV, char* ws,
+                     cudaStream_t s, int* launches) {
+    const TcWorkspace w = tc_ws<R>(d, true);
+    int* status = reinterpret_cast<int*>(ws + w.status);
+    bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
+    bf16* Rs = reinterpret_cast<bf16*>(ws + w.Rst);
+    bf16* E = reinterpret_cast<bf16*>(ws + w.E);
+    float* e65 = reinterpret_cast<float*>(ws + w.e65);
+    const int rows = d.BH() * d.n;
+    prof_begin("tc_bwd_prep_kernel", s);
+    tc_bwd_prep_kernel<<<(rows + 7) / 8, 256, 0, s>>>((const bf16*)O, (const bf16*)dO, denom, d.H, d.n, rows, d.sb,
+                                                     d.sh, d.sn, E, e65);
+    prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    CUtensorMap mQ, mK, mV, mE, mZ, mR;
+    const int64_t nblk = (int64_t)d.BH() * d.t;
+    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_rows(&mE, E, d.B, d.H, d.n, (int64_t)d.H * d.n * 64, (int64_t)d.n * 64, 64) ||
+        !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk))
+        return cudaErrorInvalidValue;
+    const bf16* g1 = (const bf16*)G1;
+    const bf16* g2 = (const bf16*)G2;
+    PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, Z, false, status, s, launches));
+    PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, Rs, true, status, s, launches));
+    constexpr size_t smem = BwdSmem::total + 1024;
+    PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
+    PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
+    const dim3 grid(d.b / 128, d.t, d.BH());
+    prof_begin("tc_bwd_q_kernel", s);
+    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mE, mK, mV, mZ, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+                                                        (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
+    prof_end(s);
+    prof_begin("tc_bwd_k_kernel", s);
+    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mE, mR, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+                                                         (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
+    prof_end(s);
+    *launches += 2;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t tc_bwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
+                   const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV, char* ws,
+                   cudaStream_t s, int* launches) {
+    switch (d.r) {
+        case 16: return bwd_impl<16>(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, ws, s, launches);
+        case 32: return bwd_impl<32>(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, ws, s, launches);
+        case 64: return bwd_impl<64>(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, ws, s, launches);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace psk

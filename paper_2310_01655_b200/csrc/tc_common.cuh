@@ -1,0 +1,118 @@
+// Device helpers shared by the tensor-core kernels (forward and backward translation units).
+#pragma once
+
+#include "psk_internal.cuh"
+#include "tc_features.cuh"
+
+#include <type_traits>
+
+namespace psk {
+
+typedef __nv_bfloat16 bf16;
+
+// host: tensor maps (defined in psk_tc.cu)
+// [B,H,n,64] bf16 rows, box 128 rows x 64 columns, 128-byte swizzle
+bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t sb, int64_t sh, int64_t sn);
+// states S[nblk][80][FP] bf16, box 80 rows x 64 features
+bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
+// per-block states of every head + prefix (reverse = false) or suffix (reverse = true) scan
+cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+                      const float* y65, bf16* S, bool reverse, int* status, cudaStream_t s, int* launches);
+
+// Scratch layout of the tensor-core path.
+struct TcWorkspace { size_t status, Z, Rst, E, e65, total; };
+
+template <int R>
+inline TcWorkspace tc_ws(const Dims& d, bool backward) {
+    TcWorkspace w{};
+    const size_t st = (size_t)d.BH() * d.t * 80 * tc::Feat<R>::FP * sizeof(bf16);
+    const size_t rows = (size_t)d.BH() * d.n;
+    size_t off = 0;
+    w.status = off; off += kStatusBytes;
+    w.Z = off; off += align_up(st);
+    if (backward) {
+        w.Rst = off; off += align_up(st);
+        w.E = off; off += align_up(rows * 64 * sizeof(bf16));
+        w.e65 = off; off += align_up(rows * sizeof(float));
+    }
+    w.total = off;
+    return w;
+}
+
+#define PSK_TRY(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
+
+template <typename Kern>
+inline cudaError_t set_smem(Kern k, size_t bytes) {
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+namespace tc {
+
+template <int I, int N, typename Fn>
+__device__ __forceinline__ void static_for(Fn&& f) {
+    if constexpr (I < N) {
+        f(std::integral_constant<int, I>{});
+        static_for<I + 1, N>(f);
+    }
+}
+
+constexpr int kErrTma = 1, kErrMma = 2;
+
+__device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
+    return p + ((1024u - (smem_u32(p) & 1023u)) & 1023u);
+}
+
+// [G1 | G2]^T as a K-major, 128-byte-swizzled tile: row n (< 2R) holds sketch column n over the 64
+// head dimensions.  B operand of the sketch GEMM X [G1 | G2].
+template <int R>
+__device__ __forceinline__ void build_g_tile(uint8_t* sG, const bf16* G1, const bf16* G2, int tid) {
+    for (int e = tid; e < 2 * R * 64; e += 128) {
+        const int nn = e / 64, k = e % 64;
+        const bf16 v = (nn < R ? G1 : G2)[k * R + (nn % R)];
+        *reinterpret_cast<bf16*>(sG + swz128_offset(nn, k / 8) + (k % 8) * 2) = v;
+    }
+}
+
+// Sketch GEMM D[128 tokens x 2R] = X_tile [G1 | G2], 4 K steps of 16 over the head dimension.
+template <int R>
+__device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX, const uint8_t* sG) {
+    constexpr uint32_t idesc = idesc_bf16(128, 2 * R, false, false);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        umma_ss(d_tmem, smem_desc(smem_u32(sX) + k * 32, 0, 1024, kSwz128),
+                smem_desc(smem_u32(sG) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+}
+
+// m[c] = A1[c] A2[c] / sqrt(R) from the sketch accumulator (this thread's lane).
+template <int R>
+__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R]) {
+    const float rs = rsqrtf((float)R);
+#pragma unroll
+    for (int c0 = 0; c0 < R; c0 += 16) {
+        uint32_t a1[16], a2[16];
+        tmem_ld16(lane_tmem + c0, a1);
+        tmem_ld16(lane_tmem + R + c0, a2);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) m[c0 + j] = __uint_as_float(a1[j]) * __uint_as_float(a2[j]) * rs;
+    }
+}
+
+// Half sketch rows as a K-major, un-swizzled operand: 8x8 core matrices, [k chunk][row/8][row%8][16 B]
+// (K-direction stride 2048 B, 8-row-group stride 128 B).
+template <int R>
+__device__ __forceinline__ void store_half_sketch_rows(uint8_t* dst, const float (&m)[R], int row) {
+#pragma unroll
+    for (int kc = 0; kc < R / 8; ++kc) {
+        uint4 v;
+        v.x = pack_bf16(m[kc * 8 + 0], m[kc * 8 + 1]);
+        v.y = pack_bf16(m[kc * 8 + 2], m[kc * 8 + 3]);
+        v.z = pack_bf16(m[kc * 8 + 4], m[kc * 8 + 5]);
+        v.w = pack_bf16(m[kc * 8 + 6], m[kc * 8 + 7]);
+        *reinterpret_cast<uint4*>(dst + kc * 2048 + (row / 8) * 128 + (row % 8) * 16) = v;
+    }
+}
+
+
+}  // namespace tc
+}  // namespace psk
