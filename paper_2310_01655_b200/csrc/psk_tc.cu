@@ -83,13 +83,15 @@ template <int R, int T0, int TN>
 __global__ void __launch_bounds__(128)
 tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                 const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
-                const float* __restrict__ y65, bf16* __restrict__ S, int* status) {
+                const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode,
+                bf16* __restrict__ S, int* status) {
     using F = Feat<R>;
     using L = StateSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_load, bar_sketch, bar_a[2];
     __shared__ uint32_t tmem_slot;
+    __shared__ float cm[64];
     const int tid = threadIdx.x, warp = tid / 32, l = blockIdx.x, bh = blockIdx.y;
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
@@ -101,6 +103,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
+    if (cmean != nullptr && tid < 64) cm[tid] = cmean[(size_t)bh * 64 + tid];
     for (int e = tid; e < 16384 / 16; e += 128) reinterpret_cast<uint4*>(smem + L::Ext)[e] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     tc_fence_before();
@@ -175,14 +178,33 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             constexpr int I = decltype(ic)::value;
             const int f = (T0 + I) * 128 + tid;
             bf16* dst = S + blk * 80 * F::FP + f;
+            float last;                         // column 64 of this feature row
+            {
+                uint32_t v[16];
+                tmem_ld16(lane_tm + kAcc + 80 * I + 64, v);
+                tmem_ld_wait();
+                last = __uint_as_float(v[0]);
+            }
+            float corr = 0.f;
 #pragma unroll
-            for (int c0 = 0; c0 < 80; c0 += 16) {
+            for (int c0 = 0; c0 < 64; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld16(lane_tm + kAcc + 80 * I + c0, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) dst[(size_t)(c0 + j) * F::FP] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                for (int j = 0; j < 16; ++j) {
+                    float x = __uint_as_float(v[j]);
+                    // centred values without touching the operands (all in fp32):
+                    //   mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
+                    //   mode 2: last column becomes H[:, 64] - H[:, :64] c
+                    if (center_mode == 1) x = fmaf(-cm[c0 + j], last, x);
+                    if (center_mode == 2) corr = fmaf(cm[c0 + j], x, corr);
+                    dst[(size_t)(c0 + j) * F::FP] = __float2bfloat16_rn(x);
+                }
             }
+            dst[(size_t)64 * F::FP] = __float2bfloat16_rn(last - corr);
+#pragma unroll
+            for (int j = 1; j < 16; ++j) dst[(size_t)(64 + j) * F::FP] = __float2bfloat16_rn(0.f);
         });
     }
     tc_fence_before();
@@ -200,18 +222,29 @@ tc_scan_kernel(bf16* __restrict__ S, size_t elems8, int t, int reverse) {
     float run[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) run[j] = 0.f;
-    for (int s = 0; s < t; ++s) {
-        const int l = reverse ? (t - 1 - s) : s;
-        const uint4 v = p[(size_t)l * elems8];
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[4];
+    constexpr int U = 8;                       // loads in flight per thread
+    for (int s0 = 0; s0 < t; s0 += U) {
+        uint4 v[U];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            o[j] = pack_bf16(run[2 * j], run[2 * j + 1]);
-            run[2 * j] += __uint_as_float(w[j] << 16);
-            run[2 * j + 1] += __uint_as_float(w[j] & 0xFFFF0000u);
+        for (int u = 0; u < U; ++u) {
+            const int s = s0 + u;
+            if (s < t) v[u] = p[(size_t)(reverse ? (t - 1 - s) : s) * elems8];
         }
-        p[(size_t)l * elems8] = make_uint4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int s = s0 + u;
+            if (s < t) {
+                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    o[j] = pack_bf16(run[2 * j], run[2 * j + 1]);
+                    run[2 * j] += __uint_as_float(w[j] << 16);
+                    run[2 * j + 1] += __uint_as_float(w[j] & 0xFFFF0000u);
+                }
+                p[(size_t)(reverse ? (t - 1 - s) : s) * elems8] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
     }
 }
 
@@ -229,23 +262,30 @@ template <int R>
 struct OutSmem {
     static constexpr uint32_t Q = 0, K = 16384, V = 32768, G = 49152;
     static constexpr uint32_t Mq = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t Mk = Mq + 128 * R * 2;
-    static constexpr uint32_t Z = (Mk + 128 * R * 2 + 1023) / 1024 * 1024;
+    static constexpr uint32_t Mk = Mq + 128 * 3 * R * 2;      // split operands: 3R columns
+    static constexpr uint32_t Z = (Mk + 128 * 3 * R * 2 + 1023) / 1024 * 1024;
     static constexpr uint32_t total = Z + kZStages * kZStageBytes;
 };
 
-template <int R>
+// MODE 0: forward (writes O, denom).  MODE 1: the backward's recomputation of the row numerators
+// against centred prefix states; writes E = dO/d (bf16), e65 = -(dO.(O - c))/d and
+// e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32 accumulators rather than
+// from the rounded O the caller holds.
+template <int R, int MODE>
 __global__ void __launch_bounds__(128)
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
                   const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
-                  bf16* __restrict__ O, int64_t sb, int64_t sh, int64_t sn, float* __restrict__ denom, int* status) {
+                  const float* __restrict__ cmean, bf16* __restrict__ O, int64_t sb, int64_t sh, int64_t sn,
+                  float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
+                  float* __restrict__ e65, float* __restrict__ e65h, int* status) {
     using F = Feat<R>;
     using L = OutSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_q, bar_kv, bar_mma, bar_a[2], bar_z[kZStages];
     __shared__ uint32_t tmem_slot;
+    __shared__ float cm[64];
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
@@ -269,6 +309,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
+    if (MODE == 1 && tid < 64) cm[tid] = cmean[(size_t)bh * 64 + tid];
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -292,7 +333,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     tc_fence_after();
     float mq[R];
     read_half_sketch<R>(lane_tm + cSk, mq);
-    store_half_sketch_rows<R>(smem + L::Mq, mq, tid);
+    store_split_rows<R, true>(smem + L::Mq, mq, tid);
 
     // ---- earlier blocks: weighted features (tensor memory) x prefix state ----
     if (l > 0) {
@@ -355,7 +396,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         {
             float mk[R];
             read_half_sketch<R>(lane_tm + cSk, mk);
-            store_half_sketch_rows<R>(smem + L::Mk, mk, tid);
+            store_split_rows<R, false>(smem + L::Mk, mk, tid);
         }
         fence_proxy_async_smem();
         tc_fence_before();
@@ -364,7 +405,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tc_fence_after();
             constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
 #pragma unroll
-            for (int k = 0; k < R / 16; ++k)
+            for (int k = 0; k < 3 * R / 16; ++k)
                 umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mq) + k * 4096, 2048, 128, kSwzNone),
                         smem_desc(smem_u32(smem + L::Mk) + k * 4096, 2048, 128, kSwzNone), idesc, k > 0);
             umma_commit(&bar_mma);
@@ -423,22 +464,79 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tmem_ld_wait();
             d += __uint_as_float(v[0]);
         }
-        const float inv = 1.f / d;
-        bf16* o = O + (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
+        if constexpr (MODE == 0) {
+            const float inv = 1.f / d;
+            bf16* o = O + (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
 #pragma unroll
-        for (int c = 0; c < 64; c += 8) {
-            uint4 v;
-            v.x = pack_bf16(acc[c] * inv, acc[c + 1] * inv);
-            v.y = pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
-            v.z = pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv);
-            v.w = pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
-            *reinterpret_cast<uint4*>(o + c) = v;
+            for (int c = 0; c < 64; c += 8) {
+                uint4 v;
+                v.x = pack_bf16(acc[c] * inv, acc[c + 1] * inv);
+                v.y = pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
+                v.z = pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv);
+                v.w = pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
+                *reinterpret_cast<uint4*>(o + c) = v;
+            }
+            if (denom != nullptr) denom[(size_t)bh * n + row0 + tid] = d;
+        } else {
+            // acc = phi Z' + W V with Z' built from centred values and V raw:
+            // N' = acc - rowsum(W) c is the numerator of centred values, O - c = (N' - c) / d.
+            const size_t row = (size_t)bh * n + row0 + tid;
+            const float dd = denom[row];              // the forward's normaliser (fp32 input)
+            const float inv = 1.f / dd;
+            const bf16* gp = dO + (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
+            float dot = 0.f, ec = 0.f;
+#pragma unroll
+            for (int c = 0; c < 64; c += 8) {
+                const uint4 gv = *reinterpret_cast<const uint4*>(gp + c);
+                const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+                uint32_t ew[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
+                    const float c0 = cm[c + 2 * j], c1 = cm[c + 2 * j + 1];
+                    dot = fmaf(g0, acc[c + 2 * j] - (rowsum + 1.f) * c0, dot);
+                    dot = fmaf(g1, acc[c + 2 * j + 1] - (rowsum + 1.f) * c1, dot);
+                    ec = fmaf(g0 * inv, c0, ec);
+                    ec = fmaf(g1 * inv, c1, ec);
+                    ew[j] = pack_bf16(g0 * inv, g1 * inv);
+                }
+                *reinterpret_cast<uint4*>(E + row * 64 + c) = make_uint4(ew[0], ew[1], ew[2], ew[3]);
+            }
+            const float e = -dot * inv * inv;
+            e65[row] = e;
+            e65h[row] = e - ec;
         }
-        if (denom != nullptr) denom[(size_t)bh * n + row0 + tid] = d;
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tm, 512);
+}
+
+// Column means of V per head: cmean[bh][c] = (1/n) sum_i V[bh][i][c].  The kernels work with
+// v - cmean (and add cmean back times the row's weight sum): an exact identity that keeps the
+// bf16 states free of the common component of the values, which otherwise cancels only after
+// rounding in the backward.  One CTA per head, fixed summation order.
+__global__ void __launch_bounds__(256)
+tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh, int64_t sn,
+                float* __restrict__ cmean) {
+    __shared__ float part[8][64];
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid % 32, rg = tid / 32;
+    const bf16* base = V + (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + 2 * lane;
+    float s0 = 0.f, s1 = 0.f;
+    for (int i = rg; i < n; i += 8) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(base + (int64_t)i * sn);
+        s0 += __low2float(v);
+        s1 += __high2float(v);
+    }
+    part[rg][2 * lane] = s0;
+    part[rg][2 * lane + 1] = s1;
+    __syncthreads();
+    if (tid < 64) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) s += part[r][tid];
+        cmean[(size_t)bh * 64 + tid] = s / (float)n;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -448,12 +546,13 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 // States of every block + scan.  X is sketched, Y is the right-hand side.
 template <int R, int T0, int TN>
 cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1,
-                               const bf16* G2, const float* y65, bf16* S, int* status, cudaStream_t s, int* launches) {
+                               const bf16* G2, const float* y65, const float* cmean, int center_mode, bf16* S, int* status,
+                               cudaStream_t s, int* launches) {
     constexpr size_t smem = StateSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_state_kernel<R, T0, TN>, smem));
     prof_begin("tc_state_kernel", s);
     tc_state_kernel<R, T0, TN><<<dim3(d.t, d.BH()), 128, smem, s>>>(mX, mY, G1, G2, d.g_heads, d.H, d.n, d.b, d.t,
-                                                                   y65, S, status);
+                                                                   y65, cmean, center_mode, S, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -461,17 +560,18 @@ cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUten
 
 template <int R>
 cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
-                          const float* y65, bf16* S, bool reverse, int* status, cudaStream_t s, int* launches) {
+                          const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
+                          cudaStream_t s, int* launches) {
     if constexpr (R == 16) {
-        PSK_TRY((launch_state_group<16, 0, 2>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
+        PSK_TRY((launch_state_group<16, 0, 2>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
     } else if constexpr (R == 32) {
-        PSK_TRY((launch_state_group<32, 0, 5>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
+        PSK_TRY((launch_state_group<32, 0, 5>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
     } else {
-        PSK_TRY((launch_state_group<64, 0, 4>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 4, 4>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 8, 3>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 11, 3>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 14, 3>(d, mX, mY, G1, G2, y65, S, status, s, launches)));
+        PSK_TRY((launch_state_group<64, 0, 4>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_TRY((launch_state_group<64, 4, 4>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_TRY((launch_state_group<64, 8, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_TRY((launch_state_group<64, 11, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_TRY((launch_state_group<64, 14, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
     }
     const size_t elems8 = (size_t)80 * Feat<R>::FP / 8;
     prof_begin("tc_scan_kernel", s);
@@ -491,13 +591,14 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
         return cudaErrorInvalidValue;
-    PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, Z, false, status, s, launches)));
+    PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, nullptr, 0, Z, false, status, s,
+                              launches)));
     constexpr size_t smem = OutSmem<R>::total + 1024;
-    PSK_TRY(set_smem(tc_fwd_out_kernel<R>, smem));
+    PSK_TRY(set_smem(tc_fwd_out_kernel<R, 0>, smem));
     prof_begin("tc_fwd_out_kernel", s);
-    tc_fwd_out_kernel<R><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, (bf16*)O, d.sb, d.sh, d.sn,
-        denom, status);
+    tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
+        mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, nullptr, (bf16*)O, d.sb, d.sh, d.sn,
+        denom, nullptr, nullptr, nullptr, nullptr, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -528,12 +629,48 @@ cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V, c
     return cudaErrorInvalidValue;
 }
 
-cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
-                      const float* y65, bf16* S, bool reverse, int* status, cudaStream_t s, int* launches) {
+template <int R>
+static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+                                  const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean,
+                                  const float* denom, const bf16* dO, bf16* E, float* e65, float* e65h, int* status,
+                                  cudaStream_t s, int* launches) {
+    constexpr size_t smem = OutSmem<R>::total + 1024;
+    PSK_TRY(set_smem(tc_fwd_out_kernel<R, 1>, smem));
+    prof_begin("tc_bwd_recompute_kernel", s);
+    tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
+        mQ, mK, mV, mZ, G1, G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, nullptr, d.sb, d.sh, d.sn,
+        const_cast<float*>(denom), dO, E, e65, e65h, status);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+                         const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean, const float* denom,
+                         const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return launch_states<16>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
-        case 32: return launch_states<32>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
-        case 64: return launch_states<64>(d, mX, mY, G1, G2, y65, S, reverse, status, s, launches);
+        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches) {
+    prof_begin("tc_vmean_kernel", s);
+    tc_vmean_kernel<<<d.BH(), 256, 0, s>>>((const bf16*)V, d.H, d.n, d.sb, d.sh, d.sn, cmean);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+                      const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
+                          cudaStream_t s, int* launches) {
+    switch (d.r) {
+        case 16: return launch_states<16>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 32: return launch_states<32>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 64: return launch_states<64>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
     }
     return cudaErrorInvalidValue;
 }

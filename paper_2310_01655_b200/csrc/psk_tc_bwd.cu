@@ -19,56 +19,21 @@ using namespace tc;
 
 namespace {
 
-// E = dO / d (bf16) and e65 = -(dO . O) / d (fp32), one warp per row.
-__global__ void __launch_bounds__(256)
-tc_bwd_prep_kernel(const bf16* __restrict__ O, const bf16* __restrict__ dO, const float* __restrict__ denom,
-                   int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn, bf16* __restrict__ E,
-                   float* __restrict__ e65) {
-    const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
-    if (row >= total_rows) return;
-    const int bh = row / n, i = row % n;
-    const int64_t base = (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn + 2 * lane;
-    const __nv_bfloat162 g2 = *reinterpret_cast<const __nv_bfloat162*>(dO + base);
-    const __nv_bfloat162 o2 = *reinterpret_cast<const __nv_bfloat162*>(O + base);
-    const float g0 = __low2float(g2), g1 = __high2float(g2);
-    float dot = g0 * __low2float(o2) + g1 * __high2float(o2);
-#pragma unroll
-    for (int s = 16; s > 0; s >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, s);
-    const float inv = 1.f / denom[row];
-    *reinterpret_cast<uint32_t*>(E + (size_t)row * 64 + 2 * lane) = pack_bf16(g0 * inv, g1 * inv);
-    if (lane == 0) e65[row] = -dot * inv;
-}
-
 constexpr int kStages = 3;
 constexpr uint32_t kBoxBytes = 80 * 128;
 
+template <int R>
 struct BwdSmem {
     // every tile: 128 rows x 128 B, 128-byte swizzle
-    static constexpr uint32_t Xown = 0, Yown = 16384, Xoth = 32768, Yoth = 49152, Mown = 65536, Moth = 81920;
-    static constexpr uint32_t G = 98304;                 // up to 128 rows
+    static constexpr uint32_t kM = SplitTiles<R>::N * 16384;      // split half-sketch operand
+    static constexpr uint32_t Xown = 0, Yown = 16384, Xoth = 32768, Yoth = 49152, Mown = 65536, Moth = Mown + kM;
+    static constexpr uint32_t G = Moth + kM;             // up to 128 rows
     static constexpr uint32_t ExtA = G + 16384;          // [128 x 16] un-swizzled: column 0 = own 65th column
     static constexpr uint32_t Eoth = ExtA + 4096;        // 128 floats: other side's 65th column
     static constexpr uint32_t Box = ExtA + 4096 + 1024;  // state boxes
     static constexpr uint32_t total = Box + kStages * ((kBoxBytes + 1023) / 1024 * 1024);
 };
 constexpr uint32_t kBoxStride = (kBoxBytes + 1023) / 1024 * 1024;
-
-// Half-sketch rows as a [128 rows x 128 B] swizzled tile, zero beyond R columns: K-major operand
-// of the score GEMM (K steps over R) and MN-major B operand (N = 64) of the dM GEMMs.
-template <int R>
-__device__ __forceinline__ void store_padded_rows(uint8_t* dst, const float (&m)[R], int row) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < R / 8) {
-            v.x = pack_bf16(m[(c % (R / 8)) * 8 + 0], m[(c % (R / 8)) * 8 + 1]);
-            v.y = pack_bf16(m[(c % (R / 8)) * 8 + 2], m[(c % (R / 8)) * 8 + 3]);
-            v.z = pack_bf16(m[(c % (R / 8)) * 8 + 4], m[(c % (R / 8)) * 8 + 5]);
-            v.w = pack_bf16(m[(c % (R / 8)) * 8 + 6], m[(c % (R / 8)) * 8 + 7]);
-        }
-        *reinterpret_cast<uint4*>(dst + swz128_offset(row, c)) = v;
-    }
-}
 
 // dm += (d feature) * (the other factor) for the 32 features F0 .. F0+31 held in x
 template <int R, int F0>
@@ -95,10 +60,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
                    const __grid_constant__ CUtensorMap mapS, const bf16* __restrict__ G1,
                    const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
-                   const float* __restrict__ e65, bf16* __restrict__ dX, bf16* __restrict__ dV, int64_t sb,
-                   int64_t sh, int64_t sn, int* status) {
+                   const float* __restrict__ e65, const float* __restrict__ e65h, bf16* __restrict__ dX,
+                   bf16* __restrict__ dV, int64_t sb, int64_t sh, int64_t sn, int* status) {
     using F = Feat<R>;
-    using L = BwdSmem;
+    using L = BwdSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_phi[2], bar_box[kStages];
@@ -132,6 +97,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
     // own 65th column (e_i for query rows, 1 for key rows) as the K extension of the d-phi GEMM
     const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
+    // the same column as it enters the 128 x 128 tiles, where the values are not centred
+    const float y65h = QSIDE ? e65h[(size_t)bh * n + row0 + tid] : 1.f;
     {
         uint8_t* ext = smem + L::ExtA;
         *reinterpret_cast<uint4*>(ext + (tid / 8) * 128 + (tid % 8) * 16) =
@@ -164,10 +131,14 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     tc_fence_after();
     float m[R], dm[R];
     read_half_sketch<R>(lane_tm + cSk, m);
-    store_padded_rows<R>(smem + L::Mown, m, tid);
+    store_split_tiles<R, true>(smem + L::Mown, m, tid);
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
 
     // ---- phase B: other blocks through the state ----
     if (has_state) {
@@ -267,7 +238,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0, hi, bi, &bar_oth);
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0, hi, bi, &bar_oth);
         }
-        if constexpr (!QSIDE) e_oth[tid] = e65[(size_t)bh * n + orow0 + tid];
+        if constexpr (!QSIDE) e_oth[tid] = e65h[(size_t)bh * n + orow0 + tid];
         ok = mbar_wait(&bar_oth, oth_uses & 1, status, kErrTma);
         ++oth_uses;
         if (tid == 0) {
@@ -281,7 +252,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         {
             float mo[R];
             read_half_sketch<R>(lane_tm + cSk, mo);
-            store_padded_rows<R>(smem + L::Moth, mo, tid);
+            store_split_tiles<R, false>(smem + L::Moth, mo, tid);
         }
         fence_proxy_async_smem();
         tc_fence_before();
@@ -290,9 +261,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tc_fence_after();
             constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
 #pragma unroll
-            for (int k = 0; k < R / 16; ++k)      // scores: own rows x other rows over the sketch dimension
-                umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mown) + k * 32, 0, 1024, kSwz128),
-                        smem_desc(smem_u32(smem + L::Moth) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+            for (int k = 0; k < 3 * R / 16; ++k)  // scores over the 3R split columns (4 K steps per tile)
+                umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mown) + (k / 4) * 16384 + (k % 4) * 32, 0, 1024, kSwz128),
+                        smem_desc(smem_u32(smem + L::Moth) + (k / 4) * 16384 + (k % 4) * 32, 0, 1024, kSwz128), idesc,
+                        k > 0);
 #pragma unroll
             for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
                 umma_ss(tm + cDW, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
@@ -314,7 +286,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 const int col = c0 + j;
                 const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
                 const float s = keep ? __uint_as_float(sv[j]) : 0.f;
-                const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65 : e_oth[col]);
+                const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col]);
                 sv[j] = __float_as_uint(2.f * s * dw);
                 wv[j] = __float_as_uint(s * s);
             }
@@ -454,13 +426,9 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     bf16* Rs = reinterpret_cast<bf16*>(ws + w.Rst);
     bf16* E = reinterpret_cast<bf16*>(ws + w.E);
     float* e65 = reinterpret_cast<float*>(ws + w.e65);
-    const int rows = d.BH() * d.n;
-    prof_begin("tc_bwd_prep_kernel", s);
-    tc_bwd_prep_kernel<<<(rows + 7) / 8, 256, 0, s>>>((const bf16*)O, (const bf16*)dO, denom, d.H, d.n, rows, d.sb,
-                                                     d.sh, d.sn, E, e65);
-    prof_end(s);
-    ++*launches;
-    PSK_TRY(cudaGetLastError());
+    float* cmean = reinterpret_cast<float*>(ws + w.vmean);
+    float* e65h = reinterpret_cast<float*>(ws + w.e65h);
+    PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     CUtensorMap mQ, mK, mV, mE, mZ, mR;
     const int64_t nblk = (int64_t)d.BH() * d.t;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
@@ -470,19 +438,21 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         return cudaErrorInvalidValue;
     const bf16* g1 = (const bf16*)G1;
     const bf16* g2 = (const bf16*)G2;
-    PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, Z, false, status, s, launches));
-    PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, Rs, true, status, s, launches));
-    constexpr size_t smem = BwdSmem::total + 1024;
+    // prefix states of centred values; forward rows again in fp32 -> E, e65, e65h; suffix states
+    PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, cmean, 1, Z, false, status, s, launches));
+    PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, g1, g2, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
+    PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, cmean, 2, Rs, true, status, s, launches));
+    constexpr size_t smem = BwdSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
     prof_begin("tc_bwd_q_kernel", s);
     tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mE, mK, mV, mZ, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                        (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
+                                                        e65h, (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
     prof_end(s);
     prof_begin("tc_bwd_k_kernel", s);
     tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mE, mR, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                         (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
+                                                         e65h, (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
     prof_end(s);
     *launches += 2;
     return cudaGetLastError();

@@ -16,11 +16,20 @@ bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t 
 // states S[nblk][80][FP] bf16, box 80 rows x 64 features
 bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
 // per-block states of every head + prefix (reverse = false) or suffix (reverse = true) scan
+// center_mode 0: states as they are; 1: values centred by the per-head vector cmean
+// (columns < 64 become H[:, c] - cmean[c] H[:, 64]); 2: last column becomes H[:, 64] - H[:, :64] cmean.
 cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
-                      const float* y65, bf16* S, bool reverse, int* status, cudaStream_t s, int* launches);
+                      const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
+                      cudaStream_t s, int* launches);
+// the backward's recomputation of the forward rows: writes E, e65, e65h (see tc_fwd_out_kernel)
+cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+                         const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean, const float* denom,
+                         const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches);
+// cmean[bh][c] = mean over the n rows of V[bh][:, c]  (deterministic reduction)
+cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
 
 // Scratch layout of the tensor-core path.
-struct TcWorkspace { size_t status, Z, Rst, E, e65, total; };
+struct TcWorkspace { size_t status, vmean, Z, Rst, E, e65, e65h, total; };
 
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
@@ -29,11 +38,13 @@ inline TcWorkspace tc_ws(const Dims& d, bool backward) {
     const size_t rows = (size_t)d.BH() * d.n;
     size_t off = 0;
     w.status = off; off += kStatusBytes;
+    w.vmean = off; off += align_up((size_t)d.BH() * 64 * sizeof(float));
     w.Z = off; off += align_up(st);
     if (backward) {
         w.Rst = off; off += align_up(st);
         w.E = off; off += align_up(rows * 64 * sizeof(bf16));
         w.e65 = off; off += align_up(rows * sizeof(float));
+        w.e65h = off; off += align_up(rows * sizeof(float));
     }
     w.total = off;
     return w;
@@ -73,6 +84,23 @@ __device__ __forceinline__ void build_g_tile(uint8_t* sG, const bf16* G1, const 
     }
 }
 
+// Subtracts the per-head vector cm[0..63] (shared memory, fp32) from row `row` of a TMA-written
+// [128 rows x 64] bf16 tile in the 128-byte-swizzled layout.
+__device__ __forceinline__ void center_row(uint8_t* tile, const float* cm, int row) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint4* p = reinterpret_cast<uint4*>(tile + swz128_offset(row, c));
+        const uint4 v = *p;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            o[j] = pack_bf16(__uint_as_float(w[j] << 16) - cm[c * 8 + 2 * j],
+                             __uint_as_float(w[j] & 0xFFFF0000u) - cm[c * 8 + 2 * j + 1]);
+        *p = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 // Sketch GEMM D[128 tokens x 2R] = X_tile [G1 | G2], 4 K steps of 16 over the head dimension.
 template <int R>
 __device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX, const uint8_t* sG) {
@@ -98,21 +126,53 @@ __device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[
     }
 }
 
-// Half sketch rows as a K-major, un-swizzled operand: 8x8 core matrices, [k chunk][row/8][row%8][16 B]
-// (K-direction stride 2048 B, 8-row-group stride 128 B).
-template <int R>
-__device__ __forceinline__ void store_half_sketch_rows(uint8_t* dst, const float (&m)[R], int row) {
+// Split of an fp32 half-sketch entry into two bf16 terms, m = hi + lo (+ O(2^-17) |m|).  Scores
+// s = m(q).m(k) are formed as hi.hi + hi.lo + lo.hi by one GEMM over 3R columns, the own rows laid
+// out as [hi | hi | lo] and the other rows as [hi | lo | hi]; a score is a cancelling sum, so
+// rounding m to a single bf16 would cost several percent on rows with few keys.
+template <int R, bool OWN>
+__device__ __forceinline__ float split_col(const float (&m)[R], int col) {
+    const int sec = col / R, c = col % R;
+    const float hi = __bfloat162float(__float2bfloat16_rn(m[c]));
+    const bool want_lo = OWN ? (sec == 2) : (sec == 1);
+    return want_lo ? (m[c] - hi) : hi;
+}
+
+// Rows of the 3R-column split operand, K-major and un-swizzled: 8x8 core matrices,
+// [k chunk][row/8][row%8][16 B] (K-direction stride 2048 B, 8-row-group stride 128 B).
+template <int R, bool OWN>
+__device__ __forceinline__ void store_split_rows(uint8_t* dst, const float (&m)[R], int row) {
 #pragma unroll
-    for (int kc = 0; kc < R / 8; ++kc) {
+    for (int kc = 0; kc < 3 * R / 8; ++kc) {
         uint4 v;
-        v.x = pack_bf16(m[kc * 8 + 0], m[kc * 8 + 1]);
-        v.y = pack_bf16(m[kc * 8 + 2], m[kc * 8 + 3]);
-        v.z = pack_bf16(m[kc * 8 + 4], m[kc * 8 + 5]);
-        v.w = pack_bf16(m[kc * 8 + 6], m[kc * 8 + 7]);
+        v.x = pack_bf16(split_col<R, OWN>(m, kc * 8 + 0), split_col<R, OWN>(m, kc * 8 + 1));
+        v.y = pack_bf16(split_col<R, OWN>(m, kc * 8 + 2), split_col<R, OWN>(m, kc * 8 + 3));
+        v.z = pack_bf16(split_col<R, OWN>(m, kc * 8 + 4), split_col<R, OWN>(m, kc * 8 + 5));
+        v.w = pack_bf16(split_col<R, OWN>(m, kc * 8 + 6), split_col<R, OWN>(m, kc * 8 + 7));
         *reinterpret_cast<uint4*>(dst + kc * 2048 + (row / 8) * 128 + (row % 8) * 16) = v;
     }
 }
 
+// The same 3R columns as ceil(3R/64) tiles of [128 rows x 128 B] in the 128-byte-swizzled layout
+// (zero beyond 3R).  Tile 0 starts with the R `hi` columns, so it doubles as the MN-major B
+// operand (N = 64, columns >= R ignored by the reader) of the dM GEMMs.
+template <int R>
+struct SplitTiles { static constexpr int N = (3 * R + 63) / 64; };
+
+template <int R, bool OWN>
+__device__ __forceinline__ void store_split_tiles(uint8_t* dst, const float (&m)[R], int row) {
+#pragma unroll
+    for (int ch = 0; ch < SplitTiles<R>::N * 8; ++ch) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ch * 8 < 3 * R) {
+            v.x = pack_bf16(split_col<R, OWN>(m, ch * 8 + 0), split_col<R, OWN>(m, ch * 8 + 1));
+            v.y = pack_bf16(split_col<R, OWN>(m, ch * 8 + 2), split_col<R, OWN>(m, ch * 8 + 3));
+            v.z = pack_bf16(split_col<R, OWN>(m, ch * 8 + 4), split_col<R, OWN>(m, ch * 8 + 5));
+            v.w = pack_bf16(split_col<R, OWN>(m, ch * 8 + 6), split_col<R, OWN>(m, ch * 8 + 7));
+        }
+        *reinterpret_cast<uint4*>(dst + (ch / 8) * 16384 + swz128_offset(row, ch % 8)) = v;
+    }
+}
 
 }  // namespace tc
 }  // namespace psk
