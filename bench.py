@@ -53,6 +53,23 @@ def kernel_flops_per_head_token(name, w):
         "bwd_k_kernel": 4 * r * r * k + 3 * r * r + half * 2 * (2 * r + 2 * k),
         "sketch_bwd_kernel": 8 * h * r,
     }
+    # tensor-core path: MMA flops actually issued (symmetric features: F = r(r+1)/2, padded)
+    F = r * (r + 1) // 2
+    FK = (F + 15) // 16 * 16            # contraction extent over features
+    FP = (F + 127) // 128 * 128         # stored / accumulated feature rows
+    nt = b // 128
+    other = (nt + 1) / 2.0              # other-side 128-row tiles met per own tile, averaged
+    sk = 2 * h * 2 * r                  # one half-sketch GEMM
+    tile_fwd = sk + 2 * 128 * 3 * r + 2 * 128 * h
+    tile_bwd = sk + 2 * 128 * 3 * r + 2 * 128 * h + 2 * 128 * 64
+    table.update({
+        "tc_state_kernel": sk * (1 if r <= 32 else 5) + 2 * FP * 80,
+        "tc_fwd_out_kernel": sk + 2 * FK * 80 + other * tile_fwd,
+        "tc_bwd_recompute_kernel": sk + 2 * FK * 80 + other * tile_fwd,
+        "tc_bwd_q_kernel": 2 * sk + 2 * FK * 80 + other * tile_bwd + 2 * 2 * r * 64,
+        "tc_bwd_k_kernel": 2 * sk + 2 * FK * 80 + 2 * FK * 64 + other * (tile_bwd + 2 * 128 * 64) + 2 * 2 * r * 64,
+        "tc_scan_kernel": None, "tc_vmean_kernel": None,
+    })
     return table.get(name)
 
 
@@ -187,6 +204,8 @@ def main():
     ap.add_argument("--cpu-heads", type=int, default=3, help="head slices the CPU baseline leg times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-keep-states", action="store_true",
+                    help="let the backward rebuild the prefix states instead of reading the forward's")
     args = ap.parse_args()
 
     from paper_2310_01655_b200 import inputs as wl
@@ -224,11 +243,14 @@ def main():
     grads = tuple(torch.empty_like(Q) for _ in range(3)) if w.backward else None
     launches = [0]
 
+    # forward and backward of one step share the workspace: the backward reads the forward's states
+    flags = psk.FLAG_KEEP_STATES if (w.backward and not args.no_keep_states) else 0
+
     def step():
-        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den)
+        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den, flags)
         n = psk.last_launch_count()
         if w.backward:
-            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, path, ws, grads)
+            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, path, ws, grads, flags)
             n += psk.last_launch_count()
         launches[0] += n
 
@@ -348,6 +370,7 @@ def main():
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
                    "passes": "fwd+bwd" if w.backward else "fwd", "path": args.path,
+                   "keep_states": bool(flags),
                    "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
         "nominal_tflops": nominal_tflops,
         "frac_bf16_peak": {"burst": nominal_tflops / world / pk["bf16_burst"],

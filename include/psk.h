@@ -69,7 +69,17 @@ typedef struct {
     int64_t stride_b, stride_h, stride_n;   /* elements; last dimension contiguous */
     int32_t g_heads;            /* 1 or H */
     int32_t path;               /* psk_path */
+    int32_t flags;              /* bit set of psk_flags, 0 for none */
 } psk_shape;
+
+/* PSK_FLAG_KEEP_STATES (tensor-core path; ignored by the CUDA-core path): set on BOTH the
+ * forward and the backward call of one training step.  The forward then leaves the prefix
+ * states Z_l of Section 3.1 (and the per-head value means they are centred by) in its
+ * workspace, and the backward, given the SAME workspace memory (sized for the backward,
+ * psk_workspace_bytes(shape, 1), and not written in between) with the same shape and inputs,
+ * reads them instead of rebuilding them from K and V.  Without the flag each call is
+ * self-contained. */
+typedef enum { PSK_FLAG_KEEP_STATES = 1 } psk_flags;
 
 /* Library version (major*100 + minor). */
 int psk_version(void);

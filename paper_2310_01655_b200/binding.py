@@ -8,6 +8,7 @@ from ctypes import c_int, c_int32, c_int64, c_size_t, c_void_p, c_char_p, POINTE
 import torch
 
 PATH_AUTO, PATH_CUDA_CORES, PATH_TENSOR_CORES = 0, 1, 2
+FLAG_KEEP_STATES = 1
 _DTYPES = {torch.float32: 0, torch.bfloat16: 1}
 _PKG = os.path.dirname(os.path.abspath(__file__))
 
@@ -23,7 +24,7 @@ class Shape(Structure):
     _fields_ = [("B", c_int32), ("H", c_int32), ("n", c_int32), ("h", c_int32), ("r", c_int32),
                 ("p", c_int32), ("b", c_int32), ("dtype", c_int32),
                 ("stride_b", c_int64), ("stride_h", c_int64), ("stride_n", c_int64),
-                ("g_heads", c_int32), ("path", c_int32)]
+                ("g_heads", c_int32), ("path", c_int32), ("flags", c_int32)]
 
 
 _lib = None
@@ -88,7 +89,8 @@ def _stream():
     return c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, path: int = PATH_AUTO) -> Shape:
+def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, path: int = PATH_AUTO,
+               flags: int = 0) -> Shape:
     """Shape descriptor for a [B,H,n,h] tensor `x` (its strides are used for all eight tensors)."""
     if x.dim() != 4 or x.stride(3) != 1:
         raise ValueError("expected a [B,H,n,h] tensor with a contiguous last dimension")
@@ -96,7 +98,7 @@ def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, pa
         raise ValueError("unsupported storage dtype %s" % x.dtype)
     B, H, n, h = x.shape
     g_heads = G1.shape[0] if G1.dim() == 3 else 1
-    return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path)
+    return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path, flags)
 
 
 def workspace_bytes(shape: Shape, for_backward: bool) -> int:
@@ -139,11 +141,11 @@ def sketch(X, G1, G2, r=None, b=128, want_phi=False, path=PATH_AUTO):
     return M, Phi
 
 
-def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out=None, denom=None):
+def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out=None, denom=None, flags=0):
     """psk_causal_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, G1, G2)
     _same_layout(Q, K, V, out)
-    shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
+    shp = make_shape(Q, G1, G1.shape[-1], b, p, path, flags)
     O = _empty_like(Q) if out is None else out
     B, H, n, _ = Q.shape
     if denom is None:
@@ -179,11 +181,11 @@ def causal_attn_fwd_static(Q, K, V, G1, G2, b, p=4, out=None, denom=None):
     return O, denom
 
 
-def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, workspace=None, out=None):
+def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, workspace=None, out=None, flags=0):
     """psk_causal_attn_bwd: returns (dQ, dK, dV)."""
     _require_cuda(Q, K, V, G1, G2, O, denom, dO)
     _same_layout(Q, K, V, O, dO)
-    shp = make_shape(Q, G1, G1.shape[-1], b, p, path)
+    shp = make_shape(Q, G1, G1.shape[-1], b, p, path, flags)
     dQ, dK, dV = out if out is not None else (_empty_like(Q), _empty_like(Q), _empty_like(Q))
     _same_layout(Q, dQ, dK, dV)
     ws, nbytes = _workspace(shp, True, workspace)

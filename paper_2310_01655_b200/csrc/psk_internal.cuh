@@ -16,6 +16,7 @@ struct Dims {
     int64_t sb, sh, sn;               // element strides of the [B,H,n,h] tensors
     int g_heads;                      // 1 or H
     bool bf16;                        // storage type
+    bool keep_states;                 // PSK_FLAG_KEEP_STATES
     int BH() const { return B * H; }
 };
 

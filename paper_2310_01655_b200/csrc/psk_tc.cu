@@ -3,11 +3,15 @@
 // the r(r+1)/2 distinct features of the self-tensored sketch (tc_features.cuh) generated in
 // registers and handed to tcgen05.mma without ever touching HBM.
 //
-// State storage (HBM scratch): S[BH][t][80][FP] bf16, "transposed + extended": row c < 64 is
+// State storage (HBM scratch): S[BH][t][65][FP] bf16, "transposed + extended": row c < 64 is
 // column c of H_l / Z_l (features contiguous), row 64 is the normaliser column (the "| 1" of
-// [V | 1], or the last column of E in the backward), rows 65..79 are zero.  One TMA box of
+// [V | 1], or the last column of E in the backward).  TMA boxes ask for 80 rows; rows 65..79
+// lie outside the tensor and arrive as zeros.  One TMA box of
 // [80 rows x 64 features] serves as a K-major B operand with N = 80 (contract over features)
 // or as an MN-major B operand with K = 80 (contract over the 65 columns).
+#ifndef PSK_EXP
+#define PSK_EXP 0
+#endif
 #include "psk_internal.cuh"
 #include "tc_features.cuh"
 #include "tc_common.cuh"
@@ -51,12 +55,13 @@ bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t 
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// States S[nblk][80][FP] bf16; box = 80 rows x 64 features.
+// States S[nblk][65][FP] bf16; box = 80 rows x 64 features.
 bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
     EncodeFn enc = encoder();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)FP, 80, (cuuint64_t)nblk};
-    cuuint64_t strides[2] = {(cuuint64_t)FP * 2, (cuuint64_t)FP * 160};
+    // 65 rows are stored; the box asks for 80 and TMA fills rows 65..79 with zeros
+    cuuint64_t dims[3] = {(cuuint64_t)FP, 65, (cuuint64_t)nblk};
+    cuuint64_t strides[2] = {(cuuint64_t)FP * 2, (cuuint64_t)FP * 130};
     cuuint32_t box[3] = {64, 80, 1}, es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -66,186 +71,259 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
 namespace {
 
 // ---------------------------------------------------------------------------
-// Per-block state  H_l = phi(X_l)^T [Y_l | y65]   (Section 3.1), feature tiles [T0, T0+TN)
+// Prefix states of one head, sequentially along the sequence (Section 3.1, Z_l = sum_{j<l} H_j):
+//   S[l] = sum over blocks before l (after l when `reverse`) of phi(X_blk)^T [Y_blk | y65]
+// for feature tiles [T0, T0+TN).  The running sum never leaves tensor memory (fp32); at every
+// block boundary it is rounded to bf16 and written out, then the block's own contribution is
+// accumulated on top -- the per-block states H_l and the scan over them are fused away.
 //   X: tensor that is sketched (K for the forward state, Q for the backward's reverse state)
 //   Y: [V] or [E(:, :64)];  y65: last column (nullptr = all ones)
-// grid (t, BH), 128 threads: thread = token for the sketch and the feature generator,
-// thread = feature row for the epilogue.
+// grid (BH).  Warp roles:
+//   NWG generator warpgroups  thread = token: read the half sketches, write their feature tiles
+//                             (dealt round-robin) as MN-major A operands into shared memory;
+//   1 store warpgroup         thread = feature row: at block boundaries reads the accumulators,
+//                             centres, rounds and stores them;
+//   1 feeder warp             one thread issues every TMA load, sketch GEMM and state GEMM.
+// Stored layout S[blk][65][FP]: row c < 64 is column c of the state, row 64 the last column.
 // ---------------------------------------------------------------------------
-template <int R>
+template <int R, int NWG>
 struct StateSmem {
-    static constexpr uint32_t X = 0, Y = 16384, Ext = 32768, G = 49152;
+    static constexpr uint32_t X = 0;                     // 2 x 16 KB: rows to sketch
+    static constexpr uint32_t Y = 32768;                 // 2 x (16 KB values + 16 KB last-column chunk)
+    static constexpr uint32_t kYSlot = 32768;
+    static constexpr uint32_t G = Y + 2 * kYSlot;
     static constexpr uint32_t A0 = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t A1 = A0 + 32768, total = A1 + 32768;
+    static constexpr uint32_t Stage = A0 + NWG * 32768;   // [65][128] bf16: one accumulator tile on its way out
+    static constexpr uint32_t total = Stage + 17408;
 };
 
-template <int R, int T0, int TN>
-__global__ void __launch_bounds__(128)
+__device__ __forceinline__ void wg_barrier(int wg) {
+    asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
+}
+
+constexpr int kErrState = 3;
+
+template <int R, int T0, int TN, int NWG>
+__global__ void __launch_bounds__(128 * (NWG + 1) + 32)
 tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                 const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
-                const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode,
+                const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode, int reverse,
                 bf16* __restrict__ S, int* status) {
     using F = Feat<R>;
-    using L = StateSmem<R>;
+    using L = StateSmem<R, NWG>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_load, bar_sketch, bar_a[2];
+    __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread;
+    __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull, bar_accread[TN];
     __shared__ uint32_t tmem_slot;
     __shared__ float cm[64];
-    const int tid = threadIdx.x, warp = tid / 32, l = blockIdx.x, bh = blockIdx.y;
+    const int tid = threadIdx.x, wg = tid / 128, wt = tid % 128, warp = tid / 32;
+    const int bh = blockIdx.x;
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
+    const int tpb = b / 128, NJ = n / 128;               // token tiles per block / per head
+    constexpr int kThreads = 128 * (NWG + 1) + 32;
 
     if (tid == 0) {
-        mbar_init(&bar_load, 1); mbar_init(&bar_sketch, 1); mbar_init(&bar_a[0], 1); mbar_init(&bar_a[1], 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bar_fullx[i], 1); mbar_init(&bar_fully[i], 1); mbar_init(&bar_yfree[i], 1);
+            mbar_init(&bar_ext[i], 1);
+        }
+        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_accfull, 1);
+        for (int i = 0; i < NWG; ++i) { mbar_init(&bar_aready[i], 1); mbar_init(&bar_afree[i], 1); }
+        for (int i = 0; i < TN; ++i) mbar_init(&bar_accread[i], 4);
         mbar_fence_init();
         tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapY);
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
-    build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
-    if (cmean != nullptr && tid < 64) cm[tid] = cmean[(size_t)bh * 64 + tid];
-    for (int e = tid; e < 16384 / 16; e += 128) reinterpret_cast<uint4*>(smem + L::Ext)[e] = make_uint4(0, 0, 0, 0);
+    if (wg == 0) build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, wt);
+    if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
+    // last-column chunks of both slots: zero, and column 0 = 1 when the last column is all ones
+    for (int e = tid; e < 2 * 1024; e += kThreads) {
+        const int s = e / 1024, i = e % 1024;
+        reinterpret_cast<uint4*>(smem + L::Y + s * L::kYSlot + 16384)[i] = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    if (y65 == nullptr && tid < 128) {
+        *reinterpret_cast<bf16*>(smem + L::Y + 16384 + swz128_offset(tid, 0)) = __float2bfloat16_rn(1.f);
+        *reinterpret_cast<bf16*>(smem + L::Y + L::kYSlot + 16384 + swz128_offset(tid, 0)) = __float2bfloat16_rn(1.f);
+    }
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tm = tmem_slot;
-    const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
-    constexpr uint32_t kAcc = 2 * R;               // accumulators start after the sketch columns
-    constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
+    constexpr uint32_t kAcc = 2 * R;                      // accumulators start after the sketch columns
+    auto tile_of = [&](int j) { return reverse ? (NJ - 1 - j) : j; };
 
-    uint32_t a_use0 = 0, a_use1 = 0;
-    bool ok = true;
-    const int ntt = b / 128;
-    for (int tt = 0; tt < ntt && ok; ++tt) {
-        const int row0 = l * b + tt * 128;
-        if (tid == 0) {
-            mbar_expect_tx(&bar_load, 32768);
-            tma_load_4d(smem + L::X, &mapX, 0, row0, hi, bi, &bar_load);
-            tma_load_4d(smem + L::Y, &mapY, 0, row0, hi, bi, &bar_load);
-        }
-        {   // last column of this token's right-hand side row
-            const float y = y65 ? y65[(size_t)bh * n + row0 + tid] : 1.f;
-            *reinterpret_cast<bf16*>(smem + L::Ext + swz128_offset(tid, 0)) = __float2bfloat16_rn(y);
-        }
-        ok = mbar_wait(&bar_load, tt & 1, status, kErrTma);
-        if (tid == 0) {
+    if (wg == NWG + 1) {
+        // =============================== feeder ===============================
+        if (tid == 128 * (NWG + 1)) {
+            constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
+            bool ok = true;
+            auto load_x = [&](int j) {
+                mbar_expect_tx(&bar_fullx[j & 1], 16384);
+                tma_load_4d(smem + L::X + (j & 1) * 16384, &mapX, 0, tile_of(j) * 128, hi, bi, &bar_fullx[j & 1]);
+            };
+            auto load_y = [&](int j) {
+                mbar_expect_tx(&bar_fully[j & 1], 16384);
+                tma_load_4d(smem + L::Y + (j & 1) * L::kYSlot, &mapY, 0, tile_of(j) * 128, hi, bi, &bar_fully[j & 1]);
+            };
+            load_x(0);
+            if (NJ > 1) load_x(1);
+            load_y(0);
+            ok = mbar_wait(&bar_fullx[0], 0, status, kErrTma);
             tc_fence_after();
             issue_sketch<R>(tm, smem + L::X, smem + L::G);
-            umma_commit(&bar_sketch);
-        }
-        ok = ok && mbar_wait(&bar_sketch, tt & 1, status, kErrMma);
-        tc_fence_after();
-        float m[R];
-        read_half_sketch<R>(lane_tm, m);
-        static_for<0, TN>([&](auto ic) {
-            constexpr int I = decltype(ic)::value;
-            const int it = tt * TN + I, buf = it & 1;
-            const uint32_t used = buf ? a_use1 : a_use0;
-            if (used > 0) ok = ok && mbar_wait(&bar_a[buf], (used - 1) & 1, status, kErrMma);
-            uint8_t* sA = smem + (buf ? L::A1 : L::A0);
-            static_for<0, 16>([&](auto cc) {
-                constexpr int C = decltype(cc)::value;
-                uint32_t pk[4];
-                gen_features<R, (T0 + I) * 128 + C * 8, false, 4>(m, pk);
-                *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(tid, C % 8)) =
-                    make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            });
-            fence_proxy_async_smem();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
+            umma_commit(&bar_sk);
+            uint32_t a_cnt[NWG];
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_ss(tm + kAcc + 80 * I, smem_desc(smem_u32(sA) + k * 2048, 16384, 1024, kSwz128),
-                            smem_desc(smem_u32(smem + L::Y) + k * 2048, 16384, 1024, kSwz128), idesc_state,
-                            (tt > 0 || k > 0) ? 1u : 0u);
-                umma_commit(&bar_a[buf]);
-            }
-            if (buf) ++a_use1; else ++a_use0;
-        });
-        // the next token tile overwrites Y / Ext (and the sketch columns): drain the state MMAs
-        if (a_use0 > 0) ok = ok && mbar_wait(&bar_a[0], (a_use0 - 1) & 1, status, kErrMma);
-        if (a_use1 > 0) ok = ok && mbar_wait(&bar_a[1], (a_use1 - 1) & 1, status, kErrMma);
-        tc_fence_after();
-        __syncthreads();
-    }
-    // epilogue: lane = feature row; store transposed (+ extended) as bf16
-    if (ok) {
-        const size_t blk = (size_t)bh * t + l;
-        static_for<0, TN>([&](auto ic) {
-            constexpr int I = decltype(ic)::value;
-            const int f = (T0 + I) * 128 + tid;
-            bf16* dst = S + blk * 80 * F::FP + f;
-            float last;                         // column 64 of this feature row
-            {
-                uint32_t v[16];
-                tmem_ld16(lane_tm + kAcc + 80 * I + 64, v);
-                tmem_ld_wait();
-                last = __uint_as_float(v[0]);
-            }
-            float corr = 0.f;
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld16(lane_tm + kAcc + 80 * I + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float x = __uint_as_float(v[j]);
-                    // centred values without touching the operands (all in fp32):
-                    //   mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
-                    //   mode 2: last column becomes H[:, 64] - H[:, :64] c
-                    if (center_mode == 1) x = fmaf(-cm[c0 + j], last, x);
-                    if (center_mode == 2) corr = fmaf(cm[c0 + j], x, corr);
-                    dst[(size_t)(c0 + j) * F::FP] = __float2bfloat16_rn(x);
+            for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
+            for (int j = 0; j < NJ && ok; ++j) {
+                // sketch of the next token tile, as soon as this tile's half sketches are read out
+                if (j + 1 < NJ) {
+                    ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
+                    ok = ok && mbar_wait(&bar_fullx[(j + 1) & 1], ((j + 1) >> 1) & 1, status, kErrTma);
+                    tc_fence_after();
+                    issue_sketch<R>(tm, smem + L::X + ((j + 1) & 1) * 16384, smem + L::G);
+                    umma_commit(&bar_sk);
+                    if (j + 2 < NJ) load_x(j + 2);        // its slot: sketch j has completed (it was read)
+                    if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
+                    load_y(j + 1);
                 }
-            }
-            dst[(size_t)64 * F::FP] = __float2bfloat16_rn(last - corr);
+                ok = ok && mbar_wait(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
+                if (y65 != nullptr) ok = ok && mbar_wait(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
+                const bool boundary = (j % tpb == 0) && j > 0;
+                const uint32_t yb = smem_u32(smem + L::Y + (j & 1) * L::kYSlot);
+                static_for<0, TN>([&](auto ic) {
+                    constexpr int I = decltype(ic)::value;
+                    constexpr int w = I % NWG;
+                    // the store warpgroup has taken this accumulator's values for the boundary
+                    if (boundary) ok = ok && mbar_wait(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
+                    ok = ok && mbar_wait(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
+                    ++a_cnt[w];
+                    tc_fence_after();
+                    const uint32_t ab = smem_u32(smem + L::A0 + w * 32768);
 #pragma unroll
-            for (int j = 1; j < 16; ++j) dst[(size_t)(64 + j) * F::FP] = __float2bfloat16_rn(0.f);
-        });
+                    for (int k = 0; k < 8; ++k)
+                        umma_ss(tm + kAcc + 80 * I, smem_desc(ab + k * 2048, 16384, 1024, kSwz128),
+                                smem_desc(yb + k * 2048, 16384, 1024, kSwz128), idesc_state, (j > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&bar_afree[w]);
+                });
+                umma_commit(&bar_yfree[j & 1]);
+                if ((j + 1) % tpb == 0) umma_commit(&bar_accfull);
+            }
+            // drain: everything issued has completed before tensor memory is released
+            umma_commit(&bar_sk);
+            mbar_wait(&bar_sk, NJ & 1, status, kErrMma);
+        }
+    } else if (wg == NWG) {
+        // ============================ store warpgroup ============================
+        const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
+        bool ok = true;
+        for (int p = 0; p < t && ok; ++p) {
+            const int l = reverse ? (t - 1 - p) : p;
+            if (p > 0) {
+                ok = mbar_wait(&bar_accfull, (p - 1) & 1, status, kErrMma);
+                tc_fence_after();
+            }
+            static_for<0, TN>([&](auto ic) {
+                constexpr int I = decltype(ic)::value;
+                // centred values, in fp32, without touching the operands (the mode only selects
+                // coefficients):  mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
+                //                 mode 2: last column H[:, 64] - H[:, :64] c
+                bf16* stage = reinterpret_cast<bf16*>(smem + L::Stage);
+                float last = 0.f, corr = 0.f;
+                if (p > 0) {
+                    uint32_t v[16];
+                    tmem_ld16(lane_tm + kAcc + 80 * I + 64, v);
+                    tmem_ld_wait();
+                    last = __uint_as_float(v[0]);
+                }
+                const float k1 = center_mode == 1 ? -last : 0.f, k2 = center_mode == 2 ? 1.f : 0.f;
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 16) {
+                    uint32_t v[16];
+                    if (p > 0) {
+                        tmem_ld16(lane_tm + kAcc + 80 * I + c0, v);
+                        tmem_ld_wait();
+                        if (c0 == 48) {          // last read of this accumulator: hand it back
+                            tc_fence_before();
+                            if (wt % 32 == 0) mbar_arrive(&bar_accread[I]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) v[q] = 0u;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        const float x = fmaf(k1, cm[c0 + q], __uint_as_float(v[q]));
+                        corr = fmaf(k2 * cm[c0 + q], x, corr);
+#if PSK_EXP != 1
+                        stage[(c0 + q) * 128 + wt] = __float2bfloat16_rn(x);
+#endif
+                    }
+                }
+                stage[64 * 128 + wt] = __float2bfloat16_rn(last - corr);
+                wg_barrier(NWG);
+                // 65 rows of 256 contiguous bytes each: 16-byte stores
+                bf16* dst = S + ((size_t)bh * t + l) * 65 * F::FP + (size_t)(T0 + I) * 128;
+#if PSK_EXP != 2
+                for (int e = wt; e < 65 * 16; e += 128) {
+                    const int c = e / 16, ch = e % 16;
+                    *reinterpret_cast<uint4*>(dst + (size_t)c * F::FP + ch * 8) =
+                        *reinterpret_cast<const uint4*>(stage + c * 128 + ch * 8);
+                }
+#endif
+                wg_barrier(NWG);
+            });
+        }
+    } else {
+        // ============================= generators =============================
+        const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
+        uint8_t* sA = smem + L::A0 + wg * 32768;
+        uint32_t a_uses = 0;                              // times this warpgroup's buffer has been filled
+        bool ok = true;
+        for (int j = 0; j < NJ && ok; ++j) {
+            ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
+            tc_fence_after();
+            float m[R];
+            read_half_sketch<R>(lane_tm, m);
+            tc_fence_before();
+            wg_barrier(wg);
+            if (wt == 0) mbar_arrive(&bar_mread);
+            if (y65 != nullptr && wg == 0) {
+                // last-column chunk of this token tile; its slot is free once tile j-2's MMAs are done
+                if (j >= 2) ok = ok && mbar_wait(&bar_yfree[j & 1], ((j >> 1) - 1) & 1, status, kErrState);
+                const float y = y65[(size_t)bh * n + tile_of(j) * 128 + wt];
+                *reinterpret_cast<bf16*>(smem + L::Y + (j & 1) * L::kYSlot + 16384 + swz128_offset(wt, 0)) =
+                    __float2bfloat16_rn(y);
+                fence_proxy_async_smem();
+                wg_barrier(0);
+                if (wt == 0) mbar_arrive(&bar_ext[j & 1]);
+            }
+            static_for<0, TN>([&](auto ic) {
+                constexpr int I = decltype(ic)::value;
+                if (I % NWG == wg) {
+                    if (a_uses > 0) ok = ok && mbar_wait(&bar_afree[wg], (a_uses - 1) & 1, status, kErrMma);
+                    static_for<0, 16>([&](auto cc) {
+                        constexpr int C = decltype(cc)::value;
+                        uint32_t pk[4];
+                        gen_features<R, (T0 + I) * 128 + C * 8, false, 4>(m, pk);
+                        *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(wt, C % 8)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    });
+                    fence_proxy_async_smem();
+                    wg_barrier(wg);
+                    if (wt == 0) mbar_arrive(&bar_aready[wg]);
+                    ++a_uses;
+                }
+            });
+        }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tm, 512);
-}
-
-// Exclusive prefix (or suffix) over the t block states of each head, in place: fp32 running sum,
-// bf16 storage.  Each thread owns 8 consecutive elements.
-__global__ void __launch_bounds__(256)
-tc_scan_kernel(bf16* __restrict__ S, size_t elems8, int t, int reverse) {
-    const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
-    if (e >= elems8) return;
-    uint4* p = reinterpret_cast<uint4*>(S) + (size_t)blockIdx.y * t * elems8 + e;
-    float run[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) run[j] = 0.f;
-    constexpr int U = 8;                       // loads in flight per thread
-    for (int s0 = 0; s0 < t; s0 += U) {
-        uint4 v[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int s = s0 + u;
-            if (s < t) v[u] = p[(size_t)(reverse ? (t - 1 - s) : s) * elems8];
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int s = s0 + u;
-            if (s < t) {
-                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-                uint32_t o[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    o[j] = pack_bf16(run[2 * j], run[2 * j + 1]);
-                    run[2 * j] += __uint_as_float(w[j] << 16);
-                    run[2 * j + 1] += __uint_as_float(w[j] & 0xFFFF0000u);
-                }
-                p[(size_t)(reverse ? (t - 1 - s) : s) * elems8] = make_uint4(o[0], o[1], o[2], o[3]);
-            }
-        }
-    }
 }
 
 // ---------------------------------------------------------------------------
@@ -260,11 +338,15 @@ constexpr uint32_t kZStageBytes = 80 * 128;     // one [80 rows x 64 features] b
 
 template <int R>
 struct OutSmem {
-    static constexpr uint32_t Q = 0, K = 16384, V = 32768, G = 49152;
+    // The prefix-state stages (first phase) and the key/value tiles with the keys' split half
+    // sketches (second phase) share one region; small enough for two CTAs per SM when R <= 32.
+    static constexpr uint32_t Q = 0, G = 16384;
     static constexpr uint32_t Mq = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t Mk = Mq + 128 * 3 * R * 2;      // split operands: 3R columns
-    static constexpr uint32_t Z = (Mk + 128 * 3 * R * 2 + 1023) / 1024 * 1024;
-    static constexpr uint32_t total = Z + kZStages * kZStageBytes;
+    static constexpr uint32_t U = (Mq + 128 * 3 * R * 2 + 1023) / 1024 * 1024;   // split operand: 3R columns
+    static constexpr uint32_t Z = U;
+    static constexpr uint32_t K = U, V = U + 16384, Mk = U + 32768;
+    static constexpr uint32_t kPhase1 = kZStages * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2;
+    static constexpr uint32_t total = U + (kPhase1 > kPhase2 ? kPhase1 : kPhase2);
 };
 
 // MODE 0: forward (writes O, denom).  MODE 1: the backward's recomputation of the row numerators
@@ -272,7 +354,7 @@ struct OutSmem {
 // e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32 accumulators rather than
 // from the rounded O the caller holds.
 template <int R, int MODE>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 2)
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
                   const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
@@ -307,9 +389,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
         }
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
-    if (MODE == 1 && tid < 64) cm[tid] = cmean[(size_t)bh * 64 + tid];
+    if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -317,7 +399,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const uint32_t tm = tmem_slot;
     const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
     // tensor-memory columns
-    constexpr uint32_t cSk = 0, cS = 128, cW = 256, cA = 320, cO = 384;
+    // sketch accumulators, scores, packed weights and the feature staging buffers all live in
+    // [0, 128): each is consumed before the next is produced; the output accumulator follows
+    constexpr uint32_t cSk = 0, cS = 0, cW = 0, cA = 0, cO = 128;
     uint32_t mma_uses = 0;
     bool ok = true;
 
@@ -373,6 +457,16 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
             ++a_uses[buf];
         });
+    }
+
+    // the key/value tiles reuse the stages' memory and the sketch reuses the staging columns:
+    // every MMA of the first phase must have completed
+    if (l > 0) {
+        if (tid == 0) umma_commit(&bar_mma);
+        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+        __syncthreads();
     }
 
     // ---- same block: key tiles tp <= tau through squared half-sketch scores ----
@@ -458,13 +552,18 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(v[j]);
         }
+        float noff = 0.f;                   // normaliser part from earlier blocks
         if (l > 0) {
             uint32_t v[16];
             tmem_ld16(lane_tm + cO + 64, v);
             tmem_ld_wait();
-            d += __uint_as_float(v[0]);
+            noff = __uint_as_float(v[0]);
+            d += noff;
         }
         if constexpr (MODE == 0) {
+            // with centred prefix states (cmean given) the earlier blocks' numerator lacks c * noff
+#pragma unroll
+            for (int c = 0; c < 64; ++c) acc[c] = fmaf(cm[c], noff, acc[c]);
             const float inv = 1.f / d;
             bf16* o = O + (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
 #pragma unroll
@@ -509,7 +608,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 512);
+    if (warp == 0) tmem_dealloc(tm, 256);
 }
 
 // Column means of V per head: cmean[bh][c] = (1/n) sum_i V[bh][i][c].  The kernels work with
@@ -543,16 +642,16 @@ tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh
 // host launchers
 // ---------------------------------------------------------------------------
 
-// States of every block + scan.  X is sketched, Y is the right-hand side.
-template <int R, int T0, int TN>
+// Prefix (or suffix) states of every head.  X is sketched, Y is the right-hand side.
+template <int R, int T0, int TN, int NWG>
 cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1,
-                               const bf16* G2, const float* y65, const float* cmean, int center_mode, bf16* S, int* status,
-                               cudaStream_t s, int* launches) {
-    constexpr size_t smem = StateSmem<R>::total + 1024;
-    PSK_TRY(set_smem(tc_state_kernel<R, T0, TN>, smem));
+                               const bf16* G2, const float* y65, const float* cmean, int center_mode, bool reverse,
+                               bf16* S, int* status, cudaStream_t s, int* launches) {
+    constexpr size_t smem = StateSmem<R, NWG>::total + 1024;
+    PSK_TRY(set_smem(tc_state_kernel<R, T0, TN, NWG>, smem));
     prof_begin("tc_state_kernel", s);
-    tc_state_kernel<R, T0, TN><<<dim3(d.t, d.BH()), 128, smem, s>>>(mX, mY, G1, G2, d.g_heads, d.H, d.n, d.b, d.t,
-                                                                   y65, cmean, center_mode, S, status);
+    tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 32, smem, s>>>(
+        mX, mY, G1, G2, d.g_heads, d.H, d.n, d.b, d.t, y65, cmean, center_mode, reverse ? 1 : 0, S, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -562,23 +661,17 @@ template <int R>
 cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
                           const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
                           cudaStream_t s, int* launches) {
+#define PSK_SG(T0, TN, NWG) \
+    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, G1, G2, y65, cmean, center_mode, reverse, S, status, s, launches)))
     if constexpr (R == 16) {
-        PSK_TRY((launch_state_group<16, 0, 2>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_SG(0, 2, 2);
     } else if constexpr (R == 32) {
-        PSK_TRY((launch_state_group<32, 0, 5>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_SG(0, 5, 3);
     } else {
-        PSK_TRY((launch_state_group<64, 0, 4>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 4, 4>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 8, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 11, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
-        PSK_TRY((launch_state_group<64, 14, 3>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, status, s, launches)));
+        PSK_SG(0, 4, 3); PSK_SG(4, 4, 3); PSK_SG(8, 3, 3); PSK_SG(11, 3, 3); PSK_SG(14, 3, 3);
     }
-    const size_t elems8 = (size_t)80 * Feat<R>::FP / 8;
-    prof_begin("tc_scan_kernel", s);
-    tc_scan_kernel<<<dim3((unsigned)((elems8 + 255) / 256), d.BH()), 256, 0, s>>>(S, elems8, d.t, reverse ? 1 : 0);
-    prof_end(s);
-    ++*launches;
-    return cudaGetLastError();
+#undef PSK_SG
+    return cudaSuccess;
 }
 
 template <int R>
@@ -591,13 +684,16 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
         return cudaErrorInvalidValue;
-    PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, nullptr, 0, Z, false, status, s,
-                              launches)));
+    // keep_states: the backward will read these states, so they are built from centred values
+    float* cmean = d.keep_states ? reinterpret_cast<float*>(ws + w.vmean) : nullptr;
+    if (cmean != nullptr) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
+    PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, cmean, cmean ? 1 : 0, Z, false,
+                              status, s, launches)));
     constexpr size_t smem = OutSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_fwd_out_kernel<R, 0>, smem));
     prof_begin("tc_fwd_out_kernel", s);
     tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, nullptr, (bf16*)O, d.sb, d.sh, d.sn,
+        mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, (bf16*)O, d.sb, d.sh, d.sn,
         denom, nullptr, nullptr, nullptr, nullptr, status);
     prof_end(s);
     ++*launches;

@@ -428,7 +428,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     float* e65 = reinterpret_cast<float*>(ws + w.e65);
     float* cmean = reinterpret_cast<float*>(ws + w.vmean);
     float* e65h = reinterpret_cast<float*>(ws + w.e65h);
-    PSK_TRY(tc_vmean(d, V, cmean, s, launches));
+    if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     CUtensorMap mQ, mK, mV, mE, mZ, mR;
     const int64_t nblk = (int64_t)d.BH() * d.t;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
@@ -439,7 +439,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     const bf16* g1 = (const bf16*)G1;
     const bf16* g2 = (const bf16*)G2;
     // prefix states of centred values; forward rows again in fp32 -> E, e65, e65h; suffix states
-    PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, cmean, 1, Z, false, status, s, launches));
+    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, cmean, 1, Z, false, status, s, launches));
     PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, g1, g2, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
     PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, cmean, 2, Rs, true, status, s, launches));
     constexpr size_t smem = BwdSmem<R>::total + 1024;

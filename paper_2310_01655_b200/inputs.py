@@ -53,6 +53,9 @@ WORKLOADS = {
     "c2": Workload("c2", 32, 12, 32768, 64, 32, 4, 256, "bf16", True, 1002, 2002),
     "c3": Workload("c3", 32, 12, 32768, 64, 64, 4, 512, "bf16", True, 1003, 2003),
     "c4": Workload("c4", 8, 16, 131072, 64, 32, 4, 256, "bf16", True, 1004, 2004, True),
+    # profiling-sized slices of c2 / c3 (same n, r, b; 2 batch elements): a few GB on the device
+    "c2s": Workload("c2s", 2, 12, 32768, 64, 32, 4, 256, "bf16", True, 1002, 2002),
+    "c3s": Workload("c3s", 2, 12, 32768, 64, 64, 4, 512, "bf16", True, 1003, 2003),
 }
 
 

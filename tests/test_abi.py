@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(L):
 
 
 def good():
-    return Shape(1, 2, 512, 64, 32, 4, 256, 1, 2 * 512 * 64, 512 * 64, 64, 2, 0)
+    return Shape(1, 2, 512, 64, 32, 4, 256, 1, 2 * 512 * 64, 512 * 64, 64, 2, 0, 0)
 
 
 def test_status_strings(L):
@@ -60,7 +60,7 @@ def test_workspace_size_formula(L):
 @pytest.mark.parametrize("field,value,code", [
     ("p", 2, -2), ("p", 8, -2), ("h", 128, -2), ("r", 48, -2),
     ("b", 100, -3), ("n", 500, -3), ("B", 0, -3), ("g_heads", 3, -3),
-    ("dtype", 7, -1), ("path", 9, -1), ("stride_n", 66, -4),
+    ("dtype", 7, -1), ("path", 9, -1), ("flags", 6, -1), ("stride_n", 66, -4),
 ])
 def test_bad_shapes_are_rejected_before_any_launch(L, field, value, code):
     s = good()

@@ -30,11 +30,13 @@ def test_full_size_configuration(name):
     shp = psk.binding.make_shape(Q, G1, w.r, w.b)
     ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, w.backward)),
                      dtype=torch.uint8, device="cuda")
-    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, workspace=ws)
+    # as bench.py runs it: forward and backward share the workspace and the forward's states
+    flags = psk.FLAG_KEEP_STATES if w.backward else 0
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, workspace=ws, flags=flags)
     assert psk.check(ws) == 0
     grads = None
     if w.backward:
-        grads = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, inp["dO"], w.b, workspace=ws)
+        grads = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, inp["dO"], w.b, workspace=ws, flags=flags)
         assert psk.check(ws) == 0
     tol = TOL[w.dtype]
     for t in (O, den) + tuple(grads or ()):

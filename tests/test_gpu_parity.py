@@ -53,6 +53,26 @@ def test_forward_and_backward_small(r, b, n, dtype):
                     check(name, got[bi, hi], ref, TOL[dtype])
 
 
+@pytest.mark.parametrize("r,b,n,corr", [(32, 256, 1024, False), (16, 128, 512, True), (64, 512, 1024, True)])
+def test_backward_reading_the_forwards_states(r, b, n, corr):
+    # PSK_FLAG_KEEP_STATES: forward and backward share one workspace; the backward skips the
+    # prefix-state pass.  Values with a common mean direction exercise the centring.
+    w = wl.small_workload(B=1, H=2, n=n, r=r, b=b, dtype="bf16", seed=61 + r, correlated=corr)
+    inp = wl.make_inputs(w, "cuda")
+    args = (inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"])
+    shp = psk.binding.make_shape(inp["Q"], inp["G1"], r, b, flags=psk.FLAG_KEEP_STATES)
+    ws = torch.empty(psk.workspace_bytes(shp, True), dtype=torch.uint8, device="cuda")
+    O, den = psk.causal_attn_fwd(*args, b, workspace=ws, flags=psk.FLAG_KEEP_STATES)
+    dQ, dK, dV = psk.causal_attn_bwd(*args, O, den, inp["dO"], b, workspace=ws, flags=psk.FLAG_KEEP_STATES)
+    assert psk.check(ws) == 0
+    for hi in range(w.H):
+        O_ref, d_ref = oracle_forward(inp, 0, hi, b)
+        check("O", O[0, hi], O_ref, TOL["bf16"])
+        check("denom", den[0, hi], d_ref, TOL["bf16"])
+        for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), oracle_backward(inp, 0, hi, b)):
+            check(name, got[0, hi], ref, TOL["bf16"])
+
+
 def test_config0_full():
     w = wl.WORKLOADS["c0"]
     inp = wl.make_inputs(w, "cuda")
