@@ -287,8 +287,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         for (int j = 0; j < NJ && ok; ++j) {
             ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
             tc_fence_after();
-            float m[R];
-            read_half_sketch<R>(lane_tm, m);
+            PackedM<R> pm;
+            {
+                float m[R];
+                read_half_sketch<R>(lane_tm, m);
+                pack_half_sketch<R>(m, pm);
+            }
             tc_fence_before();
             wg_barrier(wg);
             if (wt == 0) mbar_arrive(&bar_mread);
@@ -309,7 +313,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     static_for<0, 16>([&](auto cc) {
                         constexpr int C = decltype(cc)::value;
                         uint32_t pk[4];
-                        gen_features<R, (T0 + I) * 128 + C * 8, false, 4>(m, pk);
+                        gen_features<R, (T0 + I) * 128 + C * 8, false, 4>(pm, pk);
                         *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(wt, C % 8)) =
                             make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     });
@@ -418,6 +422,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     float mq[R];
     read_half_sketch<R>(lane_tm + cSk, mq);
     store_split_rows<R, true>(smem + L::Mq, mq, tid);
+    PackedM<R> pmq;
+    pack_half_sketch<R>(mq, pmq);
 
     // ---- earlier blocks: weighted features (tensor memory) x prefix state ----
     if (l > 0) {
@@ -437,9 +443,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
             tc_fence_after();
             uint32_t pk[16];
-            gen_features<R, C * 64, true, 16>(mq, pk);
+            gen_features<R, C * 64, true, 16>(pmq, pk);
             tmem_st16(lane_tm + cA + buf * 32, pk);
-            gen_features<R, C * 64 + 32, true, 16>(mq, pk);
+            gen_features<R, C * 64 + 32, true, 16>(pmq, pk);
             tmem_st16(lane_tm + cA + buf * 32 + 16, pk);
             tmem_st_wait();
             ok = ok && mbar_wait(&bar_z[stage], (C / kZStages) & 1, status, kErrTma);

@@ -25,13 +25,16 @@ constexpr uint32_t kBoxBytes = 80 * 128;
 template <int R>
 struct BwdSmem {
     // every tile: 128 rows x 128 B, 128-byte swizzle
-    static constexpr uint32_t kM = SplitTiles<R>::N * 16384;      // split half-sketch operand
-    static constexpr uint32_t Xown = 0, Yown = 16384, Xoth = 32768, Yoth = 49152, Mown = 65536, Moth = Mown + kM;
-    static constexpr uint32_t G = Moth + kM;             // up to 128 rows
-    static constexpr uint32_t ExtA = G + 16384;          // [128 x 16] un-swizzled: column 0 = own 65th column
+    static constexpr uint32_t kM = HiLoTiles<R>::N * 16384;      // [hi | lo] half-sketch operand
+    static constexpr uint32_t Xown = 0, Yown = 16384;
+    static constexpr uint32_t G = 32768;
+    static constexpr uint32_t ExtA = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);   // [128 x 16] un-swizzled
     static constexpr uint32_t Eoth = ExtA + 4096;        // 128 floats: other side's 65th column
-    static constexpr uint32_t Box = ExtA + 4096 + 1024;  // state boxes
-    static constexpr uint32_t total = Box + kStages * ((kBoxBytes + 1023) / 1024 * 1024);
+    static constexpr uint32_t U = Eoth + 1024;           // phase B: state boxes; phase C: the tiles below
+    static constexpr uint32_t Box = U;
+    static constexpr uint32_t Xoth = U, Yoth = U + 16384, Moth = U + 32768, Mown = Moth + kM;
+    static constexpr uint32_t kPhaseB = kStages * ((kBoxBytes + 1023) / 1024 * 1024), kPhaseC = 32768 + 2 * kM;
+    static constexpr uint32_t total = U + (kPhaseB > kPhaseC ? kPhaseB : kPhaseC);
 };
 constexpr uint32_t kBoxStride = (kBoxBytes + 1023) / 1024 * 1024;
 
@@ -54,8 +57,25 @@ __device__ __forceinline__ void untensor32(const uint32_t (&x)[32], const float 
     });
 }
 
+// Score GEMM  own rows x 64 other rows over the split half sketches:
+//   hi.hi + lo.hi + hi.lo, the [hi | lo] columns of both operands addressed in place.
+template <int R>
+__device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint32_t own, uint32_t oth) {
+    constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
+    constexpr int offA[3] = {0, R, 0}, offB[3] = {0, 0, R};
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+#pragma unroll
+        for (int kk = 0; kk < R / 16; ++kk) {
+            const int ca = offA[g] + kk * 16, cb = offB[g] + kk * 16;
+            umma_ss(d_tmem, smem_desc(own + (ca / 64) * 16384 + (ca % 64) * 2, 0, 1024, kSwz128),
+                    smem_desc(oth + (cb / 64) * 16384 + (cb % 64) * 2, 0, 1024, kSwz128), idesc, (g > 0 || kk > 0) ? 1u : 0u);
+        }
+    }
+}
+
 template <int R, bool QSIDE>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, (R <= 32 ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
                    const __grid_constant__ CUtensorMap mapS, const bf16* __restrict__ G1,
@@ -66,7 +86,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     using L = BwdSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_phi[2], bar_box[kStages];
+    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_box[kStages];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
@@ -78,7 +98,6 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     if (tid == 0) {
         mbar_init(&bar_own, 1); mbar_init(&bar_oth, 1); mbar_init(&bar_mma, 1);
-        mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
         for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
         mbar_fence_init();
         tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
@@ -93,7 +112,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             }
         }
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
     // own 65th column (e_i for query rows, 1 for key rows) as the K extension of the d-phi GEMM
     const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
@@ -111,11 +130,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     tc_fence_after();
     const uint32_t tm = tmem_slot;
     const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
-    // tensor-memory columns.  Phase B (states) and phase C (tiles) reuse [0, 256).
-    constexpr uint32_t cS = 0, cDW = 128;                 // phase C: scores, dW; then packed dS / W
-    constexpr uint32_t cPhi = 0, cFA = 128;               // phase B: d-phi (2 x 64), feature staging (2 x 32)
-    constexpr uint32_t cSk = 256;                         // sketch accumulators (transient, <= 128)
-    constexpr uint32_t cdM = 384, cdV = 448;              // accumulators: dM (64), dV (64)
+    // tensor-memory columns (256): [0,128) is scratch, reused phase by phase; accumulators follow
+    constexpr uint32_t cS = 0, cDW = 64;                  // phase C: scores, dW (64 other rows); then packed dS / W
+    constexpr uint32_t cPhi = 0, cFA = 64;                // phase B: d-phi (64), feature staging (2 x 32)
+    constexpr uint32_t cSk = 0;                           // sketch accumulators (transient, <= 128)
+    constexpr uint32_t cdM = 128, cdV = 192;              // accumulators: dM (64), dV (64)
     uint32_t mma_uses = 0;
     bool ok = true;
 
@@ -131,102 +150,84 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     tc_fence_after();
     float m[R], dm[R];
     read_half_sketch<R>(lane_tm + cSk, m);
-    store_split_tiles<R, true>(smem + L::Mown, m, tid);
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
-    fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 
     // ---- phase B: other blocks through the state ----
     if (has_state) {
+        PackedM<R> pm;
+        if constexpr (!QSIDE) pack_half_sketch<R>(m, pm);
         constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, true);
-        auto issue_dphi = [&](int c, int buf) {      // d-phi chunk c = [Yown | y65] x box(c), K = 64 + 16
-            const uint32_t box = smem_u32(smem + L::Box + (c % kStages) * kBoxStride);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
-                        smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc_phi, k > 0);
-            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
-                    smem_desc(box + 4 * 2048, 0, 1024, kSwz128), idesc_phi, 1);
-        };
-        ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
-        if (tid == 0) {
-            tc_fence_after();
-            issue_dphi(0, 0);
-            umma_commit(&bar_phi[0]);
-        }
         static_for<0, F::NC>([&](auto cc) {
             constexpr int C = decltype(cc)::value;
-            constexpr int buf = C & 1;
+            constexpr int buf = C & 1, stage = C % kStages;
             constexpr int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
             if constexpr (!QSIDE) {
-                // dV += phi_w(k) chunk (tensor memory) x box, contraction over the chunk's features
+                // weighted features of this chunk -> tensor memory (A operand of the dV GEMM)
                 uint32_t pk[16];
-                gen_features<R, C * 64, true, 16>(m, pk);
+                gen_features<R, C * 64, true, 16>(pm, pk);
                 tmem_st16(lane_tm + cFA + buf * 32, pk);
-                gen_features<R, C * 64 + 32, true, 16>(m, pk);
+                gen_features<R, C * 64 + 32, true, 16>(pm, pk);
                 tmem_st16(lane_tm + cFA + buf * 32 + 16, pk);
                 tmem_st_wait();
-                tc_fence_before();
-                __syncthreads();
-                if (tid == 0) {
-                    tc_fence_after();
+            }
+            ok = ok && mbar_wait(&bar_box[stage], (C / kStages) & 1, status, kErrTma);
+            tc_fence_before();
+            __syncthreads();               // previous chunk's d-phi has been read by every thread
+            if (tid == 0) {
+                tc_fence_after();
+                const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
+                // d-phi chunk = [Yown | y65] x box, contraction over the 64 + 16 state columns
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
+                            smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc_phi, k > 0);
+                umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
+                        smem_desc(box + 4 * 2048, 0, 1024, kSwz128), idesc_phi, 1);
+                if constexpr (!QSIDE) {
+                    // dV += phi_w(k) chunk x box, contraction over the chunk's features
                     constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
-                    const uint32_t box = smem_u32(smem + L::Box + (C % kStages) * kBoxStride);
 #pragma unroll
                     for (int k = 0; k < ksteps; ++k)
                         umma_ts(tm + cdV, tm + cFA + buf * 32 + k * 8, smem_desc(box + k * 32, 0, 1024, kSwz128), idesc,
                                 (C > 0 || k > 0) ? 1u : 0u);
                 }
+                umma_commit(&bar_mma);
             }
-            if constexpr (C + 1 < F::NC) {
-                ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
-                if (tid == 0) {
-                    tc_fence_after();
-                    issue_dphi(C + 1, buf ^ 1);
-                    umma_commit(&bar_phi[buf ^ 1]);     // also covers this chunk's dV MMAs
-                }
-            } else if constexpr (!QSIDE) {
-                if (tid == 0) umma_commit(&bar_mma);    // last chunk's dV MMAs
-            }
-            ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
             tc_fence_after();
-            // box C-1 is free once d-phi(C) has completed (its commit also covered dV(C-1))
-            if constexpr (C >= 1 && C - 1 + kStages < F::NC) {
+            // this chunk's box is free: refill it
+            if constexpr (C + kStages < F::NC) {
                 if (tid == 0) {
-                    constexpr int s2 = (C - 1) % kStages;
-                    mbar_expect_tx(&bar_box[s2], kBoxBytes);
-                    tma_load_3d(smem + L::Box + s2 * kBoxStride, &mapS, (C - 1 + kStages) * 64, 0, blk, &bar_box[s2]);
+                    mbar_expect_tx(&bar_box[stage], kBoxBytes);
+                    tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, (C + kStages) * 64, 0, blk, &bar_box[stage]);
                 }
             }
             {
                 uint32_t x[32];
-                tmem_ld32(lane_tm + cPhi + buf * 64, x);
+                tmem_ld32(lane_tm + cPhi, x);
                 tmem_ld_wait();
                 untensor32<R, C * 64>(x, m, dm);
-                tmem_ld32(lane_tm + cPhi + buf * 64 + 32, x);
+                tmem_ld32(lane_tm + cPhi + 32, x);
                 tmem_ld_wait();
                 untensor32<R, C * 64 + 32>(x, m, dm);
             }
-            // every thread has read this d-phi buffer before chunk C+2 is issued into it
-            tc_fence_before();
-            __syncthreads();
         });
-        if constexpr (!QSIDE) {
-            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-            ++mma_uses;
-            dv_started = true;
-        }
+        if constexpr (!QSIDE) dv_started = true;
 #pragma unroll
         for (int c = 0; c < R; ++c) dm[c] *= 2.f;
-        __syncthreads();
+        tc_fence_before();
+        __syncthreads();                   // boxes and the scratch columns are dead: phase C reuses them
         tc_fence_after();
     }
 
-    // ---- phase C: same block, other-side tiles ----
+    // ---- phase C: same block, other-side tiles, 64 other rows at a time ----
+    store_hilo_tiles<R>(smem + L::Mown, m, tid);
     const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
     bool dm_started = false;
     uint32_t oth_uses = 0;
@@ -252,90 +253,79 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         {
             float mo[R];
             read_half_sketch<R>(lane_tm + cSk, mo);
-            store_split_tiles<R, false>(smem + L::Moth, mo, tid);
+            store_hilo_tiles<R>(smem + L::Moth, mo, tid);
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
-#pragma unroll
-            for (int k = 0; k < 3 * R / 16; ++k)  // scores over the 3R split columns (4 K steps per tile)
-                umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mown) + (k / 4) * 16384 + (k % 4) * 32, 0, 1024, kSwz128),
-                        smem_desc(smem_u32(smem + L::Moth) + (k / 4) * 16384 + (k % 4) * 32, 0, 1024, kSwz128), idesc,
-                        k > 0);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
-                umma_ss(tm + cDW, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
-                        smem_desc(smem_u32(smem + L::Yoth) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
-            umma_commit(&bar_mma);
-        }
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
         const bool diag = (tp == tau);
+        for (int hh = 0; hh < 2; ++hh) {
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
+                constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
 #pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t sv[32], wv[32], pds[16], pw[16];
-            tmem_ld32(lane_tm + cS + c0, sv);
-            tmem_ld32(lane_tm + cDW + c0, wv);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int col = c0 + j;
-                const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
-                const float s = keep ? __uint_as_float(sv[j]) : 0.f;
-                const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col]);
-                sv[j] = __float_as_uint(2.f * s * dw);
-                wv[j] = __float_as_uint(s * s);
+                for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
+                    umma_ss(tm + cDW, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
+                            smem_desc(smem_u32(smem + L::Yoth) + hh * 8192 + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+                umma_commit(&bar_mma);
             }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                pds[j] = pack_bf16(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1]));
-                pw[j] = pack_bf16(__uint_as_float(wv[2 * j]), __uint_as_float(wv[2 * j + 1]));
-            }
-            // the packed tiles overwrite columns whose fp32 contents have already been read
-            tmem_st16(lane_tm + cS + c0 / 2, pds);
-            if constexpr (!QSIDE) tmem_st16(lane_tm + cDW + c0 / 2, pw);
-        }
-        tmem_st_wait();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
             tc_fence_after();
-            constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)           // dM_own += dS x M_other
-                umma_ts(tm + cdM, tm + cS + k * 8, smem_desc(smem_u32(smem + L::Moth) + k * 2048, 0, 1024, kSwz128),
-                        idesc, (dm_started || k > 0) ? 1u : 0u);
-            if constexpr (!QSIDE) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t sv[32], wv[32], pds[16], pw[16];
+                tmem_ld32(lane_tm + cS + c0, sv);
+                tmem_ld32(lane_tm + cDW + c0, wv);
+                tmem_ld_wait();
 #pragma unroll
-                for (int k = 0; k < 8; ++k)       // dV += W x E_other
-                    umma_ts(tm + cdV, tm + cDW + k * 8,
-                            smem_desc(smem_u32(smem + L::Yoth) + k * 2048, 0, 1024, kSwz128), idesc,
-                            (dv_started || k > 0) ? 1u : 0u);
+                for (int j = 0; j < 32; ++j) {
+                    const int col = hh * 64 + c0 + j;
+                    const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
+                    const float s = keep ? __uint_as_float(sv[j]) : 0.f;
+                    const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col]);
+                    sv[j] = __float_as_uint(2.f * s * dw);
+                    wv[j] = __float_as_uint(s * s);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    pds[j] = pack_bf16(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1]));
+                    pw[j] = pack_bf16(__uint_as_float(wv[2 * j]), __uint_as_float(wv[2 * j + 1]));
+                }
+                // the packed tiles overwrite columns whose fp32 contents have already been read
+                tmem_st16(lane_tm + cS + c0 / 2, pds);
+                if constexpr (!QSIDE) tmem_st16(lane_tm + cDW + c0 / 2, pw);
             }
-            umma_commit(&bar_mma);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)           // dM_own += dS x M_other (its hi columns)
+                    umma_ts(tm + cdM, tm + cS + k * 8,
+                            smem_desc(smem_u32(smem + L::Moth) + hh * 8192 + k * 2048, 0, 1024, kSwz128), idesc,
+                            (dm_started || k > 0) ? 1u : 0u);
+                if constexpr (!QSIDE) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)       // dV += W x E_other
+                        umma_ts(tm + cdV, tm + cDW + k * 8,
+                                smem_desc(smem_u32(smem + L::Yoth) + hh * 8192 + k * 2048, 0, 1024, kSwz128), idesc,
+                                (dv_started || k > 0) ? 1u : 0u);
+                }
+                umma_commit(&bar_mma);
+            }
+            dm_started = true;
+            dv_started = true;
+            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
+            tc_fence_after();
         }
-        dm_started = true;
-        dv_started = true;
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
     }
 
     // ---- phase D: through the sketch, dX = ((dM*A2) G1^T + (dM*A1) G2^T) / sqrt(R) ----
-    if (ok) {
-        if (tid == 0) {
-            tc_fence_after();
-            issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);   // A1, A2 again
-            umma_commit(&bar_mma);
-        }
-        ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
-    }
     if (ok) {
         const float rs = rsqrtf((float)R);
         // dM total = state part (registers) + tile part (tensor memory), scaled by 1/sqrt(R)
@@ -347,7 +337,19 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
             for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + __uint_as_float(v[j])) * rs;
         }
-        // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cS)
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);   // A1, A2 again
+            umma_commit(&bar_mma);
+        }
+        ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+        ++mma_uses;
+        tc_fence_after();
+    }
+    if (ok) {
+        // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cdM)
 #pragma unroll
         for (int c0 = 0; c0 < R; c0 += 16) {
             uint32_t a1[16], a2[16], u1[8], u2[8];
@@ -361,8 +363,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 u2[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a1[2 * j]),
                                   dm[c0 + 2 * j + 1] * __uint_as_float(a1[2 * j + 1]));
             }
-            tmem_st8(lane_tm + cS + c0 / 2, u1);
-            tmem_st8(lane_tm + cS + R / 2 + c0 / 2, u2);
+            tmem_st8(lane_tm + cdM + c0 / 2, u1);
+            tmem_st8(lane_tm + cdM + R / 2 + c0 / 2, u2);
         }
         tmem_st_wait();
         tc_fence_before();
@@ -372,7 +374,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
             for (int k = 0; k < 2 * R / 16; ++k)    // contraction over the 2R sketch columns
-                umma_ts(tm + cDW, tm + cS + k * 8, smem_desc(smem_u32(smem + L::G) + k * 2048, 0, 1024, kSwz128), idesc,
+                umma_ts(tm + cS, tm + cdM + k * 8, smem_desc(smem_u32(smem + L::G) + k * 2048, 0, 1024, kSwz128), idesc,
                         k > 0);
             umma_commit(&bar_mma);
         }
@@ -385,7 +387,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
             uint32_t v[32];
-            tmem_ld32(lane_tm + cDW + c0, v);
+            tmem_ld32(lane_tm + cS + c0, v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; j += 8)
@@ -413,7 +415,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 512);
+    if (warp == 0) tmem_dealloc(tm, 256);
 }
 
 template <int R>

@@ -153,6 +153,32 @@ __device__ __forceinline__ void store_split_rows(uint8_t* dst, const float (&m)[
     }
 }
 
+// The split half sketch as [hi | lo] columns (2R of them) in ceil(2R/64) tiles of
+// [128 rows x 128 B], 128-byte-swizzled, zero beyond 2R.  Tile 0 starts with the R `hi` columns,
+// so it doubles as the MN-major B operand (N = 64, columns >= R ignored) of the dM GEMMs.
+template <int R>
+struct HiLoTiles { static constexpr int N = (2 * R + 63) / 64; };
+
+template <int R>
+__device__ __forceinline__ void store_hilo_tiles(uint8_t* dst, const float (&m)[R], int row) {
+#pragma unroll
+    for (int ch = 0; ch < HiLoTiles<R>::N * 8; ++ch) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ch * 8 < 2 * R) {
+            float x[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int col = ch * 8 + j, c = col % R;
+                const float hi = __bfloat162float(__float2bfloat16_rn(m[c]));
+                x[j] = col < R ? hi : (m[c] - hi);
+            }
+            v.x = pack_bf16(x[0], x[1]); v.y = pack_bf16(x[2], x[3]);
+            v.z = pack_bf16(x[4], x[5]); v.w = pack_bf16(x[6], x[7]);
+        }
+        *reinterpret_cast<uint4*>(dst + (ch / 8) * 16384 + swz128_offset(row, ch % 8)) = v;
+    }
+}
+
 // The same 3R columns as ceil(3R/64) tiles of [128 rows x 128 B] in the 128-byte-swizzled layout
 // (zero beyond 3R).  Tile 0 starts with the R `hi` columns, so it doubles as the MN-major B
 // operand (N = 64, columns >= R ignored by the reader) of the dM GEMMs.

@@ -45,34 +45,77 @@ struct Feat {
     }
 };
 
-// One feature from the half sketch held in registers; zero beyond F.
+// The half sketch of one row as packed bf16 pairs, the generator's working set:
+//   e[k] = (m[2k], m[2k+1])   even-aligned pairs,   o[k] = (m[2k+1], m[2k+2])   odd-aligned pairs.
+// Consecutive features mostly share `a` and step `b` by one, so a pair of features is one
+// packed multiply  (m_a, m_a) * (m_b, m_b+1); the product is rounded to bf16 once more, which
+// the tolerance budget covers (relative 2^-9 each, independent across features).
+template <int R>
+struct PackedM {
+    uint32_t e[R / 2], o[R / 2];
+};
+
+template <int R>
+__device__ __forceinline__ void pack_half_sketch(const float (&m)[R], PackedM<R>& pm) {
+#pragma unroll
+    for (int k = 0; k < R / 2; ++k) {
+        pm.e[k] = pack_bf16(m[2 * k], m[2 * k + 1]);
+        pm.o[k] = pack_bf16(m[2 * k + 1], (2 * k + 2 < R) ? m[2 * k + 2] : 0.f);
+    }
+}
+
+__device__ __forceinline__ uint32_t hmul2_bf16(uint32_t x, uint32_t y) {
+    uint32_t r;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+    return r;
+}
+
+// (m_i, m_j) as a packed pair, from the even-aligned registers
+template <int R, int I, int J>
+__device__ __forceinline__ uint32_t pair_of(const PackedM<R>& pm) {
+    constexpr uint32_t sel = (uint32_t)((I % 2) ? 0x32 : 0x10) | ((uint32_t)((J % 2) ? 0x76 : 0x54) << 8);
+    return __byte_perm(pm.e[I / 2], pm.e[J / 2], sel);
+}
+
+// bf16x2 (feature F0, feature F0 + 1); F0 even.  WEIGHTED doubles the a < b features (exact).
 template <int R, int F0, bool WEIGHTED>
-__device__ __forceinline__ float feat_value(const float (&m)[R]) {
+__device__ __forceinline__ uint32_t feat_pair(const PackedM<R>& pm) {
     if constexpr (F0 >= Feat<R>::F) {
-        return 0.f;
+        return 0u;
     } else {
-        constexpr int A = Feat<R>::a(F0), B = Feat<R>::b(F0);
-        const float v = m[A] * m[B];
-        return (WEIGHTED && A != B) ? 2.f * v : v;
+        static_assert(Feat<R>::F % 2 == 0 && F0 % 2 == 0, "features are generated in pairs");
+        constexpr int A1 = Feat<R>::a(F0), B1 = Feat<R>::b(F0), A2 = Feat<R>::a(F0 + 1), B2 = Feat<R>::b(F0 + 1);
+        constexpr uint32_t kOne = 0x3F80u, kTwo = 0x4000u;       // bf16 1.0, 2.0
+        constexpr uint32_t w = ((WEIGHTED && A1 != B1) ? kTwo : kOne) | (((WEIGHTED && A2 != B2) ? kTwo : kOne) << 16);
+        uint32_t x, y;
+        if constexpr (A1 == A2 && B2 == B1 + 1) {
+            x = pair_of<R, A1, A1>(pm);                           // (m_a, m_a): shared by the whole run
+            y = (B1 % 2 == 0) ? pm.e[B1 / 2] : pm.o[B1 / 2];
+        } else {
+            x = pair_of<R, A1, A2>(pm);
+            y = pair_of<R, B1, B2>(pm);
+        }
+        if constexpr (w != (kOne | (kOne << 16))) x = hmul2_bf16(x, w);   // per run, not per pair
+        return hmul2_bf16(x, y);
     }
 }
 
 template <int R, int F0, bool WEIGHTED, int J, int N>
 struct FeatPack {
-    static __device__ __forceinline__ void run(const float (&m)[R], uint32_t (&out)[N]) {
-        out[J] = pack_bf16(feat_value<R, F0 + 2 * J, WEIGHTED>(m), feat_value<R, F0 + 2 * J + 1, WEIGHTED>(m));
-        FeatPack<R, F0, WEIGHTED, J + 1, N>::run(m, out);
+    static __device__ __forceinline__ void run(const PackedM<R>& pm, uint32_t (&out)[N]) {
+        out[J] = feat_pair<R, F0 + 2 * J, WEIGHTED>(pm);
+        FeatPack<R, F0, WEIGHTED, J + 1, N>::run(pm, out);
     }
 };
 template <int R, int F0, bool WEIGHTED, int N>
 struct FeatPack<R, F0, WEIGHTED, N, N> {
-    static __device__ __forceinline__ void run(const float (&)[R], uint32_t (&)[N]) {}
+    static __device__ __forceinline__ void run(const PackedM<R>&, uint32_t (&)[N]) {}
 };
 
 // out[j] = bf16x2(feature F0+2j, feature F0+2j+1), j < N  (2N consecutive features)
 template <int R, int F0, bool WEIGHTED, int N>
-__device__ __forceinline__ void gen_features(const float (&m)[R], uint32_t (&out)[N]) {
-    FeatPack<R, F0, WEIGHTED, 0, N>::run(m, out);
+__device__ __forceinline__ void gen_features(const PackedM<R>& pm, uint32_t (&out)[N]) {
+    FeatPack<R, F0, WEIGHTED, 0, N>::run(pm, out);
 }
 
 }  // namespace tc
