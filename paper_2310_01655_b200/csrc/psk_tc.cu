@@ -3,12 +3,12 @@
 // the r(r+1)/2 distinct features of the self-tensored sketch (tc_features.cuh) generated in
 // registers and handed to tcgen05.mma without ever touching HBM.
 //
-// State storage (HBM scratch): S[BH][t][65][FP] bf16, "transposed + extended": row c < 64 is
-// column c of H_l / Z_l (features contiguous), row 64 is the normaliser column (the "| 1" of
-// [V | 1], or the last column of E in the backward).  TMA boxes ask for 80 rows; rows 65..79
-// lie outside the tensor and arrive as zeros.  One TMA box of
-// [80 rows x 64 features] serves as a K-major B operand with N = 80 (contract over features)
-// or as an MN-major B operand with K = 80 (contract over the 65 columns).
+// State storage (HBM scratch): S[BH][t][FP][80] bf16, one 160-byte row per feature: the 64
+// columns of H_l / Z_l, then the normaliser column (the "| 1" of [V | 1], or the last column of E
+// in the backward), then zeros.  A stage of a consumer is two TMA boxes of [64 features x 128 B]:
+// columns 0..63 and columns 64..79 (+ zero fill).  Together they are an MN-major B operand with
+// N = 80 (contract over features) or a K-major B operand with K = 64 + 16 (contract over the
+// state's columns).
 #ifndef PSK_EXP
 #define PSK_EXP 0
 #endif
@@ -55,14 +55,15 @@ bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t 
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// States S[nblk][65][FP] bf16; box = 80 rows x 64 features.
+// States S[nblk][FP][80] bf16 (feature-major rows: 64 state columns, the last column, 15 zeros).
+// Box = 64 features x 64 columns; a second box at column 64 brings the last column (columns
+// beyond 80 lie outside the tensor and arrive as zeros).
 bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
     EncodeFn enc = encoder();
     if (!enc) return false;
-    // 65 rows are stored; the box asks for 80 and TMA fills rows 65..79 with zeros
-    cuuint64_t dims[3] = {(cuuint64_t)FP, 65, (cuuint64_t)nblk};
-    cuuint64_t strides[2] = {(cuuint64_t)FP * 2, (cuuint64_t)FP * 130};
-    cuuint32_t box[3] = {64, 80, 1}, es[3] = {1, 1, 1};
+    cuuint64_t dims[3] = {80, (cuuint64_t)FP, (cuuint64_t)nblk};
+    cuuint64_t strides[2] = {160, (cuuint64_t)FP * 160};
+    cuuint32_t box[3] = {64, 64, 1}, es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -84,7 +85,7 @@ namespace {
 //   1 store warpgroup         thread = feature row: at block boundaries reads the accumulators,
 //                             centres, rounds and stores them;
 //   1 feeder warp             one thread issues every TMA load, sketch GEMM and state GEMM.
-// Stored layout S[blk][65][FP]: row c < 64 is column c of the state, row 64 the last column.
+// Stored layout S[blk][FP][80]: one row per feature, 64 state columns, the last column, zeros.
 // ---------------------------------------------------------------------------
 template <int R, int NWG>
 struct StateSmem {
@@ -93,8 +94,7 @@ struct StateSmem {
     static constexpr uint32_t kYSlot = 32768;
     static constexpr uint32_t G = Y + 2 * kYSlot;
     static constexpr uint32_t A0 = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t Stage = A0 + NWG * 32768;   // [65][128] bf16: one accumulator tile on its way out
-    static constexpr uint32_t total = Stage + 17408;
+    static constexpr uint32_t total = A0 + NWG * 32768;
 };
 
 __device__ __forceinline__ void wg_barrier(int wg) {
@@ -232,7 +232,6 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 // centred values, in fp32, without touching the operands (the mode only selects
                 // coefficients):  mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
                 //                 mode 2: last column H[:, 64] - H[:, :64] c
-                bf16* stage = reinterpret_cast<bf16*>(smem + L::Stage);
                 float last = 0.f, corr = 0.f;
                 if (p > 0) {
                     uint32_t v[16];
@@ -241,6 +240,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     last = __uint_as_float(v[0]);
                 }
                 const float k1 = center_mode == 1 ? -last : 0.f, k2 = center_mode == 2 ? 1.f : 0.f;
+                // this thread's feature row: 80 bf16 = ten 16-byte stores
+                uint4* dst = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + wt) * 80);
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 16) {
                     uint32_t v[16];
@@ -255,27 +256,20 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
 #pragma unroll
                         for (int q = 0; q < 16; ++q) v[q] = 0u;
                     }
+                    uint32_t pk[8];
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        const float x = fmaf(k1, cm[c0 + q], __uint_as_float(v[q]));
-                        corr = fmaf(k2 * cm[c0 + q], x, corr);
-#if PSK_EXP != 1
-                        stage[(c0 + q) * 128 + wt] = __float2bfloat16_rn(x);
-#endif
+                    for (int q = 0; q < 16; q += 2) {
+                        const float x0 = fmaf(k1, cm[c0 + q], __uint_as_float(v[q]));
+                        const float x1 = fmaf(k1, cm[c0 + q + 1], __uint_as_float(v[q + 1]));
+                        corr = fmaf(k2 * cm[c0 + q], x0, corr);
+                        corr = fmaf(k2 * cm[c0 + q + 1], x1, corr);
+                        pk[q / 2] = pack_bf16(x0, x1);
                     }
+                    dst[c0 / 8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    dst[c0 / 8 + 1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
-                stage[64 * 128 + wt] = __float2bfloat16_rn(last - corr);
-                wg_barrier(NWG);
-                // 65 rows of 256 contiguous bytes each: 16-byte stores
-                bf16* dst = S + ((size_t)bh * t + l) * 65 * F::FP + (size_t)(T0 + I) * 128;
-#if PSK_EXP != 2
-                for (int e = wt; e < 65 * 16; e += 128) {
-                    const int c = e / 16, ch = e % 16;
-                    *reinterpret_cast<uint4*>(dst + (size_t)c * F::FP + ch * 8) =
-                        *reinterpret_cast<const uint4*>(stage + c * 128 + ch * 8);
-                }
-#endif
-                wg_barrier(NWG);
+                dst[8] = make_uint4(pack_bf16(last - corr, 0.f), 0, 0, 0);
+                dst[9] = make_uint4(0, 0, 0, 0);
             });
         }
     } else {
@@ -337,8 +331,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
 //   d = 1 + rowsum(diagonal weights) + N[:, 64];  O = N[:, :64] / d
 // grid (b/128, t, BH), 128 threads (thread = query row).
 // ---------------------------------------------------------------------------
-constexpr int kZStages = 4;
-constexpr uint32_t kZStageBytes = 80 * 128;     // one [80 rows x 64 features] box
+constexpr int kZStages = 3;
+constexpr uint32_t kZStageBytes = 16384;        // two [64 features x 128 B] boxes: columns 0..63, 64..79
 
 template <int R>
 struct OutSmem {
@@ -389,7 +383,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         if (l > 0) {
             for (int c = 0; c < kZStages && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_z[c], kZStageBytes);
-                tma_load_3d(smem + L::Z + c * kZStageBytes, &mapZ, c * 64, 0, blk, &bar_z[c]);
+                tma_load_3d(smem + L::Z + c * kZStageBytes, &mapZ, 0, c * 64, blk, &bar_z[c]);
+                tma_load_3d(smem + L::Z + c * kZStageBytes + 8192, &mapZ, 64, c * 64, blk, &bar_z[c]);
             }
         }
     }
@@ -438,7 +433,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 if (tid == 0 && C - 2 + kZStages < F::NC) {
                     constexpr int s2 = (C - 2 + 2 * kZStages) % kZStages;
                     mbar_expect_tx(&bar_z[s2], kZStageBytes);
-                    tma_load_3d(smem + L::Z + s2 * kZStageBytes, &mapZ, (C - 2 + kZStages) * 64, 0, blk, &bar_z[s2]);
+                    tma_load_3d(smem + L::Z + s2 * kZStageBytes, &mapZ, 0, (C - 2 + kZStages) * 64, blk, &bar_z[s2]);
+                    tma_load_3d(smem + L::Z + s2 * kZStageBytes + 8192, &mapZ, 64, (C - 2 + kZStages) * 64, blk,
+                                &bar_z[s2]);
                 }
             }
             tc_fence_after();
@@ -453,11 +450,13 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
-                constexpr uint32_t idesc = idesc_bf16(128, 80, false, false);
+                // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step,
+                // the second 64-column group (columns 64..79) 8192 B further on
+                constexpr uint32_t idesc = idesc_bf16(128, 80, false, true);
                 const uint32_t zb = smem_u32(smem + L::Z + stage * kZStageBytes);
 #pragma unroll
                 for (int k = 0; k < ksteps; ++k)
-                    umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, smem_desc(zb + k * 32, 0, 1024, kSwz128), idesc,
+                    umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, smem_desc(zb + k * 2048, 8192, 1024, kSwz128), idesc,
                             (C > 0 || k > 0) ? 1u : 0u);
                 umma_commit(&bar_a[buf]);
             }

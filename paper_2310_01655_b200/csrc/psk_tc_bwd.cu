@@ -20,7 +20,7 @@ using namespace tc;
 namespace {
 
 constexpr int kStages = 3;
-constexpr uint32_t kBoxBytes = 80 * 128;
+constexpr uint32_t kBoxBytes = 16384;      // two [64 features x 128 B] boxes: state columns 0..63, 64..79
 
 template <int R>
 struct BwdSmem {
@@ -108,7 +108,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         if (has_state) {
             for (int c = 0; c < kStages && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_box[c], kBoxBytes);
-                tma_load_3d(smem + L::Box + c * kBoxStride, &mapS, c * 64, 0, blk, &bar_box[c]);
+                tma_load_3d(smem + L::Box + c * kBoxStride, &mapS, 0, c * 64, blk, &bar_box[c]);
+                tma_load_3d(smem + L::Box + c * kBoxStride + 8192, &mapS, 64, c * 64, blk, &bar_box[c]);
             }
         }
     }
@@ -161,7 +162,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     if (has_state) {
         PackedM<R> pm;
         if constexpr (!QSIDE) pack_half_sketch<R>(m, pm);
-        constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, true);
+        constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, false);
         static_for<0, F::NC>([&](auto cc) {
             constexpr int C = decltype(cc)::value;
             constexpr int buf = C & 1, stage = C % kStages;
@@ -181,19 +182,20 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             if (tid == 0) {
                 tc_fence_after();
                 const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
-                // d-phi chunk = [Yown | y65] x box, contraction over the 64 + 16 state columns
+                // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
+                // contraction over the 64 state columns, then the last column (second box)
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
-                            smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc_phi, k > 0);
+                            smem_desc(box + k * 32, 0, 1024, kSwz128), idesc_phi, k > 0);
                 umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
-                        smem_desc(box + 4 * 2048, 0, 1024, kSwz128), idesc_phi, 1);
+                        smem_desc(box + 8192, 0, 1024, kSwz128), idesc_phi, 1);
                 if constexpr (!QSIDE) {
-                    // dV += phi_w(k) chunk x box, contraction over the chunk's features
-                    constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
+                    // dV += phi_w(k) chunk x box (MN-major B: 16 features per K step)
+                    constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
                     for (int k = 0; k < ksteps; ++k)
-                        umma_ts(tm + cdV, tm + cFA + buf * 32 + k * 8, smem_desc(box + k * 32, 0, 1024, kSwz128), idesc,
+                        umma_ts(tm + cdV, tm + cFA + buf * 32 + k * 8, smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc,
                                 (C > 0 || k > 0) ? 1u : 0u);
                 }
                 umma_commit(&bar_mma);
@@ -205,7 +207,9 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             if constexpr (C + kStages < F::NC) {
                 if (tid == 0) {
                     mbar_expect_tx(&bar_box[stage], kBoxBytes);
-                    tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, (C + kStages) * 64, 0, blk, &bar_box[stage]);
+                    tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
+                    tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk,
+                                &bar_box[stage]);
                 }
             }
             {

@@ -34,7 +34,7 @@ struct TcWorkspace { size_t status, vmean, Z, Rst, E, e65, e65h, total; };
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
     TcWorkspace w{};
-    const size_t st = (size_t)d.BH() * d.t * 65 * tc::Feat<R>::FP * sizeof(bf16);
+    const size_t st = (size_t)d.BH() * d.t * tc::Feat<R>::FP * 80 * sizeof(bf16);
     const size_t rows = (size_t)d.BH() * d.n;
     size_t off = 0;
     w.status = off; off += kStatusBytes;
