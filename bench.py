@@ -68,7 +68,7 @@ def kernel_flops_per_head_token(name, w):
         "tc_bwd_recompute_kernel": sk + 2 * FK * 80 + other * tile_fwd,
         "tc_bwd_q_kernel": 2 * sk + 2 * FK * 80 + other * tile_bwd + 2 * 2 * r * 64,
         "tc_bwd_k_kernel": 2 * sk + 2 * FK * 80 + 2 * FK * 64 + other * (tile_bwd + 2 * 128 * 64) + 2 * 2 * r * 64,
-        "tc_scan_kernel": None, "tc_vmean_kernel": None,
+        "tc_vmean_kernel": None, "tc_bwd_prep_kernel": None,
     })
     return table.get(name)
 
@@ -235,16 +235,15 @@ def main():
     wr = wl.Workload(**dict(w.asdict(), data_seed=w.data_seed + 7919 * rank))
     inp = wl.make_inputs(wr, "cuda", with_dO=True)
     Q, K, V, dO, G1, G2 = (inp[k] for k in ("Q", "K", "V", "dO", "G1", "G2"))
-    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path)
+    # forward and backward of one step share the workspace: the backward reads the forward's states
+    flags = psk.FLAG_KEEP_STATES if (w.backward and not args.no_keep_states) else 0
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path, flags)
     ws_bytes = max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True) if w.backward else 0)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     O = torch.empty_like(Q)
     den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
     grads = tuple(torch.empty_like(Q) for _ in range(3)) if w.backward else None
     launches = [0]
-
-    # forward and backward of one step share the workspace: the backward reads the forward's states
-    flags = psk.FLAG_KEEP_STATES if (w.backward and not args.no_keep_states) else 0
 
     def step():
         psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den, flags)

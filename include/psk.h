@@ -73,12 +73,13 @@ typedef struct {
 } psk_shape;
 
 /* PSK_FLAG_KEEP_STATES (tensor-core path; ignored by the CUDA-core path): set on BOTH the
- * forward and the backward call of one training step.  The forward then leaves the prefix
- * states Z_l of Section 3.1 (and the per-head value means they are centred by) in its
- * workspace, and the backward, given the SAME workspace memory (sized for the backward,
- * psk_workspace_bytes(shape, 1), and not written in between) with the same shape and inputs,
- * reads them instead of rebuilding them from K and V.  Without the flag each call is
- * self-contained. */
+ * forward and the backward call of one training step.  The forward then leaves in its
+ * workspace the prefix states Z_l of Section 3.1, the per-head value means c they are centred
+ * by, and O - c at higher relative precision than the rounded O; the backward, given the SAME
+ * workspace memory (not written in between) with the same shape and inputs, reads them instead
+ * of rebuilding the states from K and V and recomputing the forward rows.  With the flag set
+ * psk_workspace_bytes() returns the backward's size for both calls.  Without the flag each
+ * call is self-contained. */
 typedef enum { PSK_FLAG_KEEP_STATES = 1 } psk_flags;
 
 /* Library version (major*100 + minor). */

@@ -179,7 +179,15 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             uint32_t a_cnt[NWG];
 #pragma unroll
             for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
+#if PSK_EXP == 9
+            long long* trace = reinterpret_cast<long long*>(status) + 2;
+            int tr = 0;
+#define TRF() do { if (bh == 0 && (j == 8 || j == 9) && tr < 30) trace[tr++] = clock64(); } while (0)
+#else
+#define TRF() do {} while (0)
+#endif
             for (int j = 0; j < NJ && ok; ++j) {
+                TRF();
                 // sketch of the next token tile, as soon as this tile's half sketches are read out
                 if (j + 1 < NJ) {
                     ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
@@ -199,8 +207,11 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     constexpr int I = decltype(ic)::value;
                     constexpr int w = I % NWG;
                     // the store warpgroup has taken this accumulator's values for the boundary
+                    TRF();
                     if (boundary) ok = ok && mbar_wait(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
+                    TRF();
                     ok = ok && mbar_wait(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
+                    TRF();
                     ++a_cnt[w];
                     tc_fence_after();
                     const uint32_t ab = smem_u32(smem + L::A0 + w * 32768);
@@ -358,7 +369,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                   const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
                   const float* __restrict__ cmean, bf16* __restrict__ O, int64_t sb, int64_t sh, int64_t sn,
                   float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
-                  float* __restrict__ e65, float* __restrict__ e65h, int* status) {
+                  float* __restrict__ e65, float* __restrict__ e65h, float* __restrict__ Oc, int* status) {
     using F = Feat<R>;
     using L = OutSmem<R>;
     extern __shared__ uint8_t smem_raw[];
@@ -523,8 +534,12 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
                 w0 = (diag && c0 + j > tid) ? 0.f : w0 * w0;
                 w1 = (diag && c0 + j + 1 > tid) ? 0.f : w1 * w1;
-                rowsum += w0 + w1;
-                pk[j / 2] = pack_bf16(w0, w1);
+                // the normaliser sums the weights as the value GEMM will see them (rounded to bf16):
+                // where one key dominates a row, v_j - O_i = v_j / d_i only holds if numerator and
+                // denominator use the same numbers
+                const uint32_t p2 = pack_bf16(w0, w1);
+                rowsum += __uint_as_float(p2 << 16) + __uint_as_float(p2 & 0xFFFF0000u);
+                pk[j / 2] = p2;
             }
             tmem_st16(lane_tm + cW + c0 / 2, pk);
         }
@@ -581,6 +596,16 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 *reinterpret_cast<uint4*>(o + c) = v;
             }
             if (denom != nullptr) denom[(size_t)bh * n + row0 + tid] = d;
+            if (Oc != nullptr) {
+                // kept for the backward: O - c in fp32.  (The rounded O cannot supply it: where the
+                // values share a common component, or one key dominates a row, |O - c| and
+                // |v - O| are far below |O|.)
+                float4* oc = reinterpret_cast<float4*>(Oc + ((size_t)bh * n + row0 + tid) * 64);
+#pragma unroll
+                for (int c = 0; c < 64; c += 4)
+                    oc[c / 4] = make_float4(acc[c] * inv - cm[c], acc[c + 1] * inv - cm[c + 1],
+                                            acc[c + 2] * inv - cm[c + 2], acc[c + 3] * inv - cm[c + 3]);
+            }
         } else {
             // acc = phi Z' + W V with Z' built from centred values and V raw:
             // N' = acc - rowsum(W) c is the numerator of centred values, O - c = (N' - c) / d.
@@ -620,26 +645,31 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 // v - cmean (and add cmean back times the row's weight sum): an exact identity that keeps the
 // bf16 states free of the common component of the values, which otherwise cancels only after
 // rounding in the backward.  One CTA per head, fixed summation order.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh, int64_t sn,
                 float* __restrict__ cmean) {
-    __shared__ float part[8][64];
-    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid % 32, rg = tid / 32;
-    const bf16* base = V + (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + 2 * lane;
-    float s0 = 0.f, s1 = 0.f;
-    for (int i = rg; i < n; i += 8) {
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(base + (int64_t)i * sn);
-        s0 += __low2float(v);
-        s1 += __high2float(v);
+    __shared__ float part[128][65];
+    const int bh = blockIdx.x, tid = threadIdx.x, ch = tid % 8, rg = tid / 8;   // 8 threads x 16 B per row
+    const bf16* base = V + (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + 8 * ch;
+    float s[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[j] = 0.f;
+    for (int i = rg; i < n; i += 128) {
+        const uint4 v = *reinterpret_cast<const uint4*>(base + (int64_t)i * sn);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            s[2 * j] += __uint_as_float(w[j] << 16);
+            s[2 * j + 1] += __uint_as_float(w[j] & 0xFFFF0000u);
+        }
     }
-    part[rg][2 * lane] = s0;
-    part[rg][2 * lane + 1] = s1;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) part[rg][8 * ch + j] = s[j];
     __syncthreads();
     if (tid < 64) {
-        float s = 0.f;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) s += part[r][tid];
-        cmean[(size_t)bh * 64 + tid] = s / (float)n;
+        float acc = 0.f;
+        for (int r = 0; r < 128; ++r) acc += part[r][tid];
+        cmean[(size_t)bh * 64 + tid] = acc / (float)n;
     }
 }
 
@@ -682,9 +712,10 @@ cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMa
 template <int R>
 cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
                      void* O, float* denom, char* ws, cudaStream_t s, int* launches) {
-    const TcWorkspace w = tc_ws<R>(d, false);
+    const TcWorkspace w = tc_ws<R>(d, d.keep_states);
     int* status = reinterpret_cast<int*>(ws + w.status);
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
+    float* Oc = d.keep_states ? reinterpret_cast<float*>(ws + w.Oc) : nullptr;
     CUtensorMap mQ, mK, mV, mZ;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
@@ -699,7 +730,7 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     prof_begin("tc_fwd_out_kernel", s);
     tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
         mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, (bf16*)O, d.sb, d.sh, d.sn,
-        denom, nullptr, nullptr, nullptr, nullptr, status);
+        denom, nullptr, nullptr, nullptr, nullptr, Oc, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -713,6 +744,7 @@ bool tc_supported(const Dims& d, bool backward) {
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
+    backward = backward || d.keep_states;       // kept states: the forward writes into the backward's layout
     switch (d.r) {
         case 16: return tc_ws<16>(d, backward).total;
         case 32: return tc_ws<32>(d, backward).total;
@@ -740,7 +772,7 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
     prof_begin("tc_bwd_recompute_kernel", s);
     tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
         mQ, mK, mV, mZ, G1, G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, nullptr, d.sb, d.sh, d.sn,
-        const_cast<float*>(denom), dO, E, e65, e65h, status);
+        const_cast<float*>(denom), dO, E, e65, e65h, nullptr, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -759,7 +791,7 @@ cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap
 
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches) {
     prof_begin("tc_vmean_kernel", s);
-    tc_vmean_kernel<<<d.BH(), 256, 0, s>>>((const bf16*)V, d.H, d.n, d.sb, d.sh, d.sn, cmean);
+    tc_vmean_kernel<<<d.BH(), 1024, 0, s>>>((const bf16*)V, d.H, d.n, d.sb, d.sh, d.sn, cmean);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();

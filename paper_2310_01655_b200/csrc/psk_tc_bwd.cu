@@ -19,6 +19,47 @@ using namespace tc;
 
 namespace {
 
+// With kept states the forward left Oc = O - c (fp32).  Eight lanes x 8 columns per row (four
+// rows per warp):  E = dO / d (bf16, for the suffix states),  e65 = -(dO . Oc) / d,  e65h = e65 - E . c
+__global__ void __launch_bounds__(256)
+tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom, const float* __restrict__ cmean,
+                   const float* __restrict__ Oc, int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn,
+                   bf16* __restrict__ E, float* __restrict__ e65, float* __restrict__ e65h) {
+    const int row = blockIdx.x * 32 + threadIdx.x / 8, ch = threadIdx.x % 8;
+    if (row >= total_rows) return;                 // total_rows is a multiple of 128: whole warps leave together
+    const int bh = row / n, i = row % n;
+    const int64_t base = (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn + 8 * ch;
+    const uint4 gv = *reinterpret_cast<const uint4*>(dO + base);
+    const float4 o0 = *reinterpret_cast<const float4*>(Oc + (size_t)row * 64 + 8 * ch);
+    const float4 o1 = *reinterpret_cast<const float4*>(Oc + (size_t)row * 64 + 8 * ch + 4);
+    const float ov[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+    const float inv = 1.f / denom[row];
+    const float* c = cmean + (size_t)bh * 64 + 8 * ch;
+    float dot = 0.f, ec = 0.f;
+    uint32_t ew[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
+        dot = fmaf(g0, ov[2 * j], dot);
+        dot = fmaf(g1, ov[2 * j + 1], dot);
+        ec = fmaf(g0 * inv, c[2 * j], ec);
+        ec = fmaf(g1 * inv, c[2 * j + 1], ec);
+        ew[j] = pack_bf16(g0 * inv, g1 * inv);
+    }
+#pragma unroll
+    for (int s = 4; s > 0; s >>= 1) {
+        dot += __shfl_xor_sync(0xffffffffu, dot, s);
+        ec += __shfl_xor_sync(0xffffffffu, ec, s);
+    }
+    *reinterpret_cast<uint4*>(E + (size_t)row * 64 + 8 * ch) = make_uint4(ew[0], ew[1], ew[2], ew[3]);
+    if (ch == 0) {
+        const float e = -dot * inv;
+        e65[row] = e;
+        e65h[row] = e - ec;
+    }
+}
+
 constexpr int kStages = 3;
 constexpr uint32_t kBoxBytes = 16384;      // two [64 features x 128 B] boxes: state columns 0..63, 64..79
 
@@ -80,8 +121,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
                    const __grid_constant__ CUtensorMap mapS, const bf16* __restrict__ G1,
                    const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
-                   const float* __restrict__ e65, const float* __restrict__ e65h, bf16* __restrict__ dX,
-                   bf16* __restrict__ dV, int64_t sb, int64_t sh, int64_t sn, int* status) {
+                   const float* __restrict__ e65, const float* __restrict__ e65h, const float* __restrict__ denom,
+                   bf16* __restrict__ dX, bf16* __restrict__ dV, int64_t sb, int64_t sh, int64_t sn, int* status) {
     using F = Feat<R>;
     using L = BwdSmem<R>;
     extern __shared__ uint8_t smem_raw[];
@@ -115,10 +156,14 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
     build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
-    // own 65th column (e_i for query rows, 1 for key rows) as the K extension of the d-phi GEMM
-    const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
-    // the same column as it enters the 128 x 128 tiles, where the values are not centred
-    const float y65h = QSIDE ? e65h[(size_t)bh * n + row0 + tid] : 1.f;
+    // Query rows work on the raw dO rows g_i (exact bf16 inputs) and apply 1/d_i in fp32 afterwards:
+    // dL/dW_ij = (g_i . v_j - g_i . O_i) / d_i cancels heavily when one key dominates a row, and a
+    // rounded g_i / d_i would not survive it.  y65 = -(g_i . (O_i - c)) pairs with the centred
+    // states, y65h = -(g_i . O_i) with the raw values of the 128 x 128 tiles.  Key rows: 1.
+    const float d_own = QSIDE ? denom[(size_t)bh * n + row0 + tid] : 1.f;
+    const float inv_own = 1.f / d_own;
+    const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] * d_own : 1.f;
+    const float y65h = QSIDE ? e65h[(size_t)bh * n + row0 + tid] * d_own : 1.f;
     {
         uint8_t* ext = smem + L::ExtA;
         *reinterpret_cast<uint4*>(ext + (tid / 8) * 128 + (tid % 8) * 16) =
@@ -224,7 +269,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         });
         if constexpr (!QSIDE) dv_started = true;
 #pragma unroll
-        for (int c = 0; c < R; ++c) dm[c] *= 2.f;
+        for (int c = 0; c < R; ++c) dm[c] *= 2.f * inv_own;
         tc_fence_before();
         __syncthreads();                   // boxes and the scratch columns are dead: phase C reuses them
         tc_fence_after();
@@ -235,7 +280,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
     bool dm_started = false;
     uint32_t oth_uses = 0;
-    float* e_oth = reinterpret_cast<float*>(smem + L::Eoth);
+    float* e_oth = reinterpret_cast<float*>(smem + L::Eoth);       // other rows: -(g . O), 1/d
+    float* inv_oth = e_oth + 128;
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
         if (tid == 0) {
@@ -243,7 +289,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0, hi, bi, &bar_oth);
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0, hi, bi, &bar_oth);
         }
-        if constexpr (!QSIDE) e_oth[tid] = e65h[(size_t)bh * n + orow0 + tid];
+        if constexpr (!QSIDE) {
+            const float dd = denom[(size_t)bh * n + orow0 + tid];
+            e_oth[tid] = e65h[(size_t)bh * n + orow0 + tid] * dd;
+            inv_oth[tid] = 1.f / dd;
+        }
         ok = mbar_wait(&bar_oth, oth_uses & 1, status, kErrTma);
         ++oth_uses;
         if (tid == 0) {
@@ -288,9 +338,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                     const int col = hh * 64 + c0 + j;
                     const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
                     const float s = keep ? __uint_as_float(sv[j]) : 0.f;
-                    const float dw = __uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col]);
+                    const float inv = QSIDE ? inv_own : inv_oth[col];
+                    const float dw = (__uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col])) * inv;
                     sv[j] = __float_as_uint(2.f * s * dw);
-                    wv[j] = __float_as_uint(s * s);
+                    wv[j] = __float_as_uint(s * s * inv);       // weight times 1/d_i: the value side sees g_i / d_i
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -435,30 +486,42 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     float* cmean = reinterpret_cast<float*>(ws + w.vmean);
     float* e65h = reinterpret_cast<float*>(ws + w.e65h);
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
-    CUtensorMap mQ, mK, mV, mE, mZ, mR;
+    CUtensorMap mQ, mK, mV, mE, mG, mZ, mR;
     const int64_t nblk = (int64_t)d.BH() * d.t;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mE, E, d.B, d.H, d.n, (int64_t)d.H * d.n * 64, (int64_t)d.n * 64, 64) ||
+        !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk))
         return cudaErrorInvalidValue;
     const bf16* g1 = (const bf16*)G1;
     const bf16* g2 = (const bf16*)G2;
     // prefix states of centred values; forward rows again in fp32 -> E, e65, e65h; suffix states
     if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, cmean, 1, Z, false, status, s, launches));
-    PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, g1, g2, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
+    if (d.keep_states) {
+        const int rows = d.BH() * d.n;
+        prof_begin("tc_bwd_prep_kernel", s);
+        tc_bwd_prep_kernel<<<(rows + 31) / 32, 256, 0, s>>>((const bf16*)dO, denom, cmean,
+                                                           reinterpret_cast<const float*>(ws + w.Oc), d.H, d.n, rows, d.sb,
+                                                           d.sh, d.sn, E, e65, e65h);
+        prof_end(s);
+        ++*launches;
+        PSK_TRY(cudaGetLastError());
+    } else {
+        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, g1, g2, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
+    }
     PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, cmean, 2, Rs, true, status, s, launches));
     constexpr size_t smem = BwdSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
     prof_begin("tc_bwd_q_kernel", s);
-    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mE, mK, mV, mZ, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                        e65h, (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
+    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+                                                        e65h, denom, (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
     prof_end(s);
     prof_begin("tc_bwd_k_kernel", s);
-    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mE, mR, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                         e65h, (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
+    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+                                                         e65h, denom, (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
     prof_end(s);
     *launches += 2;
     return cudaGetLastError();

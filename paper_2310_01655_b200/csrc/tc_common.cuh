@@ -29,7 +29,7 @@ cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
 
 // Scratch layout of the tensor-core path.
-struct TcWorkspace { size_t status, vmean, Z, Rst, E, e65, e65h, total; };
+struct TcWorkspace { size_t status, vmean, Z, Rst, E, e65, e65h, Oc, total; };
 
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
@@ -45,6 +45,7 @@ inline TcWorkspace tc_ws(const Dims& d, bool backward) {
         w.E = off; off += align_up(rows * 64 * sizeof(bf16));
         w.e65 = off; off += align_up(rows * sizeof(float));
         w.e65h = off; off += align_up(rows * sizeof(float));
+        if (d.keep_states) { w.Oc = off; off += align_up(rows * 64 * sizeof(float)); }   // forward's O - c, fp32
     }
     w.total = off;
     return w;

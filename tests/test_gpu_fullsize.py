@@ -27,11 +27,11 @@ def test_full_size_configuration(name):
     w = wl.WORKLOADS[name]
     inp = wl.make_inputs(w, "cuda")
     Q, K, V, G1, G2 = (inp[k] for k in ("Q", "K", "V", "G1", "G2"))
-    shp = psk.binding.make_shape(Q, G1, w.r, w.b)
-    ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, w.backward)),
-                     dtype=torch.uint8, device="cuda")
     # as bench.py runs it: forward and backward share the workspace and the forward's states
     flags = psk.FLAG_KEEP_STATES if w.backward else 0
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, flags=flags)
+    ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, w.backward)),
+                     dtype=torch.uint8, device="cuda")
     O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, workspace=ws, flags=flags)
     assert psk.check(ws) == 0
     grads = None
