@@ -217,8 +217,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     const uint32_t ab = smem_u32(smem + L::A0 + w * 32768);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        umma_ss(tm + kAcc + 80 * I, smem_desc(ab + k * 2048, 16384, 1024, kSwz128),
-                                smem_desc(yb + k * 2048, 16384, 1024, kSwz128), idesc_state, (j > 0 || k > 0) ? 1u : 0u);
+                        umma_ss(tm + kAcc + 80 * I, desc_off(smem_desc(ab, 16384, 1024, kSwz128), k * 2048),
+                                desc_off(smem_desc(yb, 16384, 1024, kSwz128), k * 2048), idesc_state, (j > 0 || k > 0) ? 1u : 0u);
                     umma_commit(&bar_afree[w]);
                 });
                 umma_commit(&bar_yfree[j & 1]);
@@ -467,7 +467,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 const uint32_t zb = smem_u32(smem + L::Z + stage * kZStageBytes);
 #pragma unroll
                 for (int k = 0; k < ksteps; ++k)
-                    umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, smem_desc(zb + k * 2048, 8192, 1024, kSwz128), idesc,
+                    umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, desc_off(smem_desc(zb, 8192, 1024, kSwz128), k * 2048), idesc,
                             (C > 0 || k > 0) ? 1u : 0u);
                 umma_commit(&bar_a[buf]);
             }
@@ -516,8 +516,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
 #pragma unroll
             for (int k = 0; k < 3 * R / 16; ++k)
-                umma_ss(tm + cS, smem_desc(smem_u32(smem + L::Mq) + k * 4096, 2048, 128, kSwzNone),
-                        smem_desc(smem_u32(smem + L::Mk) + k * 4096, 2048, 128, kSwzNone), idesc, k > 0);
+                umma_ss(tm + cS, desc_off(smem_desc(smem_u32(smem + L::Mq), 2048, 128, kSwzNone), k * 4096),
+                        desc_off(smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone), k * 4096), idesc, k > 0);
             umma_commit(&bar_mma);
         }
         ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
@@ -551,7 +551,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                umma_ts(tm + cO, tm + cW + k * 8, smem_desc(smem_u32(smem + L::V) + k * 2048, 0, 1024, kSwz128), idesc,
+                umma_ts(tm + cO, tm + cW + k * 8, desc_off(smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128), k * 2048), idesc,
                         (l > 0 || tp > 0 || k > 0) ? 1u : 0u);
             umma_commit(&bar_mma);
         }

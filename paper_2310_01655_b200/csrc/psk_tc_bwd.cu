@@ -11,6 +11,9 @@
 // (d feature) * (the other factor)  (tc_features.cuh explains the weights w).
 // One kernel, two roles: QSIDE rows own (Q, E) and meet keys j <= i; key-side rows own (K, V)
 // and meet queries i >= j.  Thread = own row throughout.
+#ifndef PSK_EXP
+#define PSK_EXP 0
+#endif
 #include "tc_common.cuh"
 
 namespace psk {
@@ -109,8 +112,8 @@ __device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint32_t own, uint
 #pragma unroll
         for (int kk = 0; kk < R / 16; ++kk) {
             const int ca = offA[g] + kk * 16, cb = offB[g] + kk * 16;
-            umma_ss(d_tmem, smem_desc(own + (ca / 64) * 16384 + (ca % 64) * 2, 0, 1024, kSwz128),
-                    smem_desc(oth + (cb / 64) * 16384 + (cb % 64) * 2, 0, 1024, kSwz128), idesc, (g > 0 || kk > 0) ? 1u : 0u);
+            umma_ss(d_tmem, desc_off(smem_desc(own, 0, 1024, kSwz128), (ca / 64) * 16384 + (ca % 64) * 2),
+                    desc_off(smem_desc(oth, 0, 1024, kSwz128), (cb / 64) * 16384 + (cb % 64) * 2), idesc, (g > 0 || kk > 0) ? 1u : 0u);
         }
     }
 }
@@ -127,7 +130,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     using L = BwdSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_box[kStages];
+    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_phi[2], bar_box[kStages];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
@@ -135,10 +138,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const int row0 = l * b + tau * 128;
     const int blk = bh * t + l;
     const int ntiles = b / 128;
-    const bool has_state = QSIDE ? (l > 0) : (l < t - 1);
+    const bool has_state = (PSK_EXP == 11) ? false : (QSIDE ? (l > 0) : (l < t - 1));
 
     if (tid == 0) {
         mbar_init(&bar_own, 1); mbar_init(&bar_oth, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
         for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
         mbar_fence_init();
         tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
@@ -178,7 +182,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
     // tensor-memory columns (256): [0,128) is scratch, reused phase by phase; accumulators follow
     constexpr uint32_t cS = 0, cDW = 64;                  // phase C: scores, dW (64 other rows); then packed dS / W
-    constexpr uint32_t cPhi = 0, cFA = 64;                // phase B: d-phi (64), feature staging (2 x 32)
+    constexpr uint32_t cPhi = 0;                          // phase B: d-phi, 2 x 64
     constexpr uint32_t cSk = 0;                           // sketch accumulators (transient, <= 128)
     constexpr uint32_t cdM = 128, cdV = 192;              // accumulators: dM (64), dV (64)
     uint32_t mma_uses = 0;
@@ -208,47 +212,67 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         PackedM<R> pm;
         if constexpr (!QSIDE) pack_half_sketch<R>(m, pm);
         constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, false);
-        static_for<0, F::NC>([&](auto cc) {
+        // Software pipeline over the 64-feature chunks: while the MMAs of chunk C run, the threads
+        // generate chunk C+1's features; while those of chunk C+1 run, they un-tensor chunk C.
+        // d-phi is double-buffered in [0,128); during this phase the feature staging buffers sit
+        // in the dM accumulator's columns, which only phase C uses.
+        constexpr uint32_t cFB = cdM;
+        auto stage_features = [&](auto cc) {      // weighted features of chunk C -> tensor memory
+            constexpr int C = decltype(cc)::value;
+            uint32_t pk[16];
+            gen_features<R, C * 64, true, 16>(pm, pk);
+            tmem_st16(lane_tm + cFB + (C & 1) * 32, pk);
+            gen_features<R, C * 64 + 32, true, 16>(pm, pk);
+            tmem_st16(lane_tm + cFB + (C & 1) * 32 + 16, pk);
+            tmem_st_wait();
+        };
+        auto issue_chunk = [&](auto cc) {         // one thread: the chunk's MMAs, then commit
             constexpr int C = decltype(cc)::value;
             constexpr int buf = C & 1, stage = C % kStages;
             constexpr int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+            const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
+            // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
+            // contraction over the 64 state columns, then the last column (second box)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_ss(tm + cPhi + buf * 64, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32),
+                        desc_off(smem_desc(box, 0, 1024, kSwz128), k * 32), idesc_phi, k > 0);
+            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
+                    desc_off(smem_desc(box, 0, 1024, kSwz128), 8192), idesc_phi, 1);
             if constexpr (!QSIDE) {
-                // weighted features of this chunk -> tensor memory (A operand of the dV GEMM)
-                uint32_t pk[16];
-                gen_features<R, C * 64, true, 16>(pm, pk);
-                tmem_st16(lane_tm + cFA + buf * 32, pk);
-                gen_features<R, C * 64 + 32, true, 16>(pm, pk);
-                tmem_st16(lane_tm + cFA + buf * 32 + 16, pk);
-                tmem_st_wait();
-            }
-            ok = ok && mbar_wait(&bar_box[stage], (C / kStages) & 1, status, kErrTma);
-            tc_fence_before();
-            __syncthreads();               // previous chunk's d-phi has been read by every thread
-            if (tid == 0) {
-                tc_fence_after();
-                const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
-                // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
-                // contraction over the 64 state columns, then the last column (second box)
+                // dV += phi_w(k) chunk x box (MN-major B: 16 features per K step)
+                constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
-                            smem_desc(box + k * 32, 0, 1024, kSwz128), idesc_phi, k > 0);
-                umma_ss(tm + cPhi, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
-                        smem_desc(box + 8192, 0, 1024, kSwz128), idesc_phi, 1);
-                if constexpr (!QSIDE) {
-                    // dV += phi_w(k) chunk x box (MN-major B: 16 features per K step)
-                    constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
-#pragma unroll
-                    for (int k = 0; k < ksteps; ++k)
-                        umma_ts(tm + cdV, tm + cFA + buf * 32 + k * 8, smem_desc(box + k * 2048, 0, 1024, kSwz128), idesc,
-                                (C > 0 || k > 0) ? 1u : 0u);
-                }
-                umma_commit(&bar_mma);
+                for (int k = 0; k < ksteps; ++k)
+                    umma_ts(tm + cdV, tm + cFB + buf * 32 + k * 8, desc_off(smem_desc(box, 0, 1024, kSwz128), k * 2048), idesc,
+                            (C > 0 || k > 0) ? 1u : 0u);
             }
-            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-            ++mma_uses;
+            umma_commit(&bar_phi[buf]);
+        };
+        if constexpr (!QSIDE) stage_features(std::integral_constant<int, 0>{});
+        ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
             tc_fence_after();
-            // this chunk's box is free: refill it
+            issue_chunk(std::integral_constant<int, 0>{});
+        }
+        static_for<0, F::NC>([&](auto cc) {
+            constexpr int C = decltype(cc)::value;
+            constexpr int buf = C & 1, stage = C % kStages;
+            if constexpr (C + 1 < F::NC) {
+                if constexpr (!QSIDE) stage_features(std::integral_constant<int, C + 1>{});
+                ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
+                tc_fence_before();
+                __syncthreads();           // chunk C-1's d-phi has been read by every thread
+                if (tid == 0) {
+                    tc_fence_after();
+                    issue_chunk(std::integral_constant<int, C + 1>{});
+                }
+            }
+            ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+            tc_fence_after();
+            // chunk C's box is free (its MMAs have completed): refill it
             if constexpr (C + kStages < F::NC) {
                 if (tid == 0) {
                     mbar_expect_tx(&bar_box[stage], kBoxBytes);
@@ -259,10 +283,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             }
             {
                 uint32_t x[32];
-                tmem_ld32(lane_tm + cPhi, x);
+                tmem_ld32(lane_tm + cPhi + buf * 64, x);
                 tmem_ld_wait();
                 untensor32<R, C * 64>(x, m, dm);
-                tmem_ld32(lane_tm + cPhi + 32, x);
+                tmem_ld32(lane_tm + cPhi + buf * 64 + 32, x);
                 tmem_ld_wait();
                 untensor32<R, C * 64 + 32>(x, m, dm);
             }
@@ -277,11 +301,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     // ---- phase C: same block, other-side tiles, 64 other rows at a time ----
     store_hilo_tiles<R>(smem + L::Mown, m, tid);
-    const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
+    const int tp_begin = QSIDE ? 0 : tau, tp_end = (PSK_EXP == 12) ? tp_begin : (QSIDE ? tau + 1 : ntiles);
     bool dm_started = false;
     uint32_t oth_uses = 0;
-    float* e_oth = reinterpret_cast<float*>(smem + L::Eoth);       // other rows: -(g . O), 1/d
-    float* inv_oth = e_oth + 128;
+    float2* oth_col = reinterpret_cast<float2*>(smem + L::Eoth);   // other rows: (1/d, -(g . O)/d)
+    const float y65h_inv = y65h * inv_own;
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
         if (tid == 0) {
@@ -290,9 +314,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0, hi, bi, &bar_oth);
         }
         if constexpr (!QSIDE) {
-            const float dd = denom[(size_t)bh * n + orow0 + tid];
-            e_oth[tid] = e65h[(size_t)bh * n + orow0 + tid] * dd;
-            inv_oth[tid] = 1.f / dd;
+            // e65h is already -(g . O) / d
+            oth_col[tid] = make_float2(1.f / denom[(size_t)bh * n + orow0 + tid], e65h[(size_t)bh * n + orow0 + tid]);
         }
         ok = mbar_wait(&bar_oth, oth_uses & 1, status, kErrTma);
         ++oth_uses;
@@ -320,38 +343,49 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
-                    umma_ss(tm + cDW, smem_desc(smem_u32(smem + L::Yown) + k * 32, 0, 1024, kSwz128),
-                            smem_desc(smem_u32(smem + L::Yoth) + hh * 8192 + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+                    umma_ss(tm + cDW, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32),
+                            desc_off(smem_desc(smem_u32(smem + L::Yoth) + hh * 8192, 0, 1024, kSwz128), k * 32), idesc, k > 0);
                 umma_commit(&bar_mma);
             }
             ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
             ++mma_uses;
             tc_fence_after();
+            // dW = (own . other + y) / d_i,  ds = 2 s dW,  W / d_i = s^2 / d_i, masked on the diagonal
+            // tile; packed to bf16 over columns whose fp32 contents have already been read
+            auto tile_math = [&](auto diag_c) {
+                constexpr bool DIAG = decltype(diag_c)::value;
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t sv[32], wv[32], pds[16], pw[16];
-                tmem_ld32(lane_tm + cS + c0, sv);
-                tmem_ld32(lane_tm + cDW + c0, wv);
-                tmem_ld_wait();
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t sv[32], wv[32], pds[16], pw[16];
+                    tmem_ld32(lane_tm + cS + c0, sv);
+                    tmem_ld32(lane_tm + cDW + c0, wv);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int col = hh * 64 + c0 + j;
-                    const bool keep = !diag || (QSIDE ? (col <= tid) : (col >= tid));
-                    const float s = keep ? __uint_as_float(sv[j]) : 0.f;
-                    const float inv = QSIDE ? inv_own : inv_oth[col];
-                    const float dw = (__uint_as_float(wv[j]) + (QSIDE ? y65h : e_oth[col])) * inv;
-                    sv[j] = __float_as_uint(2.f * s * dw);
-                    wv[j] = __float_as_uint(s * s * inv);       // weight times 1/d_i: the value side sees g_i / d_i
+                    for (int j = 0; j < 32; ++j) {
+                        const int col = hh * 64 + c0 + j;
+                        float s = __uint_as_float(sv[j]);
+                        if constexpr (DIAG) s = (QSIDE ? (col <= tid) : (col >= tid)) ? s : 0.f;
+                        float inv, yinv;
+                        if constexpr (QSIDE) {
+                            inv = inv_own; yinv = y65h_inv;
+                        } else {
+                            const float2 o = oth_col[col];
+                            inv = o.x; yinv = o.y;
+                        }
+                        const float dw = fmaf(__uint_as_float(wv[j]), inv, yinv);
+                        sv[j] = __float_as_uint((s + s) * dw);
+                        wv[j] = __float_as_uint(s * (s * inv));     // weight / d_i: the value side sees g_i / d_i
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        pds[j] = pack_bf16(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1]));
+                        pw[j] = pack_bf16(__uint_as_float(wv[2 * j]), __uint_as_float(wv[2 * j + 1]));
+                    }
+                    tmem_st16(lane_tm + cS + c0 / 2, pds);
+                    if constexpr (!QSIDE) tmem_st16(lane_tm + cDW + c0 / 2, pw);
                 }
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    pds[j] = pack_bf16(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1]));
-                    pw[j] = pack_bf16(__uint_as_float(wv[2 * j]), __uint_as_float(wv[2 * j + 1]));
-                }
-                // the packed tiles overwrite columns whose fp32 contents have already been read
-                tmem_st16(lane_tm + cS + c0 / 2, pds);
-                if constexpr (!QSIDE) tmem_st16(lane_tm + cDW + c0 / 2, pw);
-            }
+            };
+            if (diag) tile_math(std::true_type{}); else tile_math(std::false_type{});
             tmem_st_wait();
             tc_fence_before();
             __syncthreads();
@@ -361,13 +395,13 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
                 for (int k = 0; k < 4; ++k)           // dM_own += dS x M_other (its hi columns)
                     umma_ts(tm + cdM, tm + cS + k * 8,
-                            smem_desc(smem_u32(smem + L::Moth) + hh * 8192 + k * 2048, 0, 1024, kSwz128), idesc,
+                            desc_off(smem_desc(smem_u32(smem + L::Moth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
                             (dm_started || k > 0) ? 1u : 0u);
                 if constexpr (!QSIDE) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)       // dV += W x E_other
                         umma_ts(tm + cdV, tm + cDW + k * 8,
-                                smem_desc(smem_u32(smem + L::Yoth) + hh * 8192 + k * 2048, 0, 1024, kSwz128), idesc,
+                                desc_off(smem_desc(smem_u32(smem + L::Yoth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
                                 (dv_started || k > 0) ? 1u : 0u);
                 }
                 umma_commit(&bar_mma);
@@ -429,7 +463,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
             for (int k = 0; k < 2 * R / 16; ++k)    // contraction over the 2R sketch columns
-                umma_ts(tm + cS, tm + cdM + k * 8, smem_desc(smem_u32(smem + L::G) + k * 2048, 0, 1024, kSwz128), idesc,
+                umma_ts(tm + cS, tm + cdM + k * 8, desc_off(smem_desc(smem_u32(smem + L::G), 0, 1024, kSwz128), k * 2048), idesc,
                         k > 0);
             umma_commit(&bar_mma);
         }

@@ -108,8 +108,8 @@ __device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX,
     constexpr uint32_t idesc = idesc_bf16(128, 2 * R, false, false);
 #pragma unroll
     for (int k = 0; k < 4; ++k)
-        umma_ss(d_tmem, smem_desc(smem_u32(sX) + k * 32, 0, 1024, kSwz128),
-                smem_desc(smem_u32(sG) + k * 32, 0, 1024, kSwz128), idesc, k > 0);
+        umma_ss(d_tmem, desc_off(smem_desc(smem_u32(sX), 0, 1024, kSwz128), k * 32),
+                desc_off(smem_desc(smem_u32(sG), 0, 1024, kSwz128), k * 32), idesc, k > 0);
 }
 
 // m[c] = A1[c] A2[c] / sqrt(R) from the sketch accumulator (this thread's lane).

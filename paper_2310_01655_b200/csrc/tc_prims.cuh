@@ -127,6 +127,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
            | ((uint64_t)layout << 61);
 }
 constexpr uint32_t kSwz128 = 2, kSwzNone = 0;
+// The descriptor of the same operand `bytes` further on (bytes a multiple of 16): one 64-bit add,
+// so that a loop over K steps does not rebuild descriptors.
+__device__ __forceinline__ uint64_t desc_off(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
 
 // D[tmem] (+)= A[smem] * B[smem]; one elected thread issues.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
