@@ -196,8 +196,6 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     issue_sketch<R>(tm, smem + L::X + ((j + 1) & 1) * 16384, smem + L::G);
                     umma_commit(&bar_sk);
                     if (j + 2 < NJ) load_x(j + 2);        // its slot: sketch j has completed (it was read)
-                    if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
-                    load_y(j + 1);
                 }
                 ok = ok && mbar_wait(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
                 if (y65 != nullptr) ok = ok && mbar_wait(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
@@ -220,6 +218,14 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                         umma_ss(tm + kAcc + 80 * I, desc_off(smem_desc(ab, 16384, 1024, kSwz128), k * 2048),
                                 desc_off(smem_desc(yb, 16384, 1024, kSwz128), k * 2048), idesc_state, (j > 0 || k > 0) ? 1u : 0u);
                     umma_commit(&bar_afree[w]);
+                    if constexpr (I == 0) {
+                        // values of the next token tile: their slot held tile j-1, whose MMAs were
+                        // issued a whole tile ago (waiting for them here costs nothing)
+                        if (j + 1 < NJ) {
+                            if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
+                            load_y(j + 1);
+                        }
+                    }
                 });
                 umma_commit(&bar_yfree[j & 1]);
                 if ((j + 1) % tpb == 0) umma_commit(&bar_accfull);
