@@ -201,7 +201,7 @@ def main():
     ap.add_argument("--impl", default="psk", choices=["psk", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "cuda_cores", "tensor_cores"])
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-heads", type=int, default=3, help="head slices the CPU baseline leg times")
+    ap.add_argument("--cpu-heads", type=int, default=12, help="head slices the CPU baseline leg times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-keep-states", action="store_true",
@@ -215,24 +215,20 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
     import paper_2310_01655_b200 as psk
+    from paper_2310_01655_b200 import dist_util as du
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = du.env_rank()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the library")
     torch.cuda.set_device(local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    du.init("nccl", torch.device("cuda", local))
     psk.lib()
     path = {"auto": psk.PATH_AUTO, "cuda_cores": psk.PATH_CUDA_CORES, "tensor_cores": psk.PATH_TENSOR_CORES}[args.path]
 
     # every rank holds its own batch of the workload (independent (batch, head) problems:
     # no data-path collective), seeded differently per rank
-    wr = wl.Workload(**dict(w.asdict(), data_seed=w.data_seed + 7919 * rank))
+    wr = wl.Workload(**dict(w.asdict(), data_seed=du.rank_seed(w.data_seed, rank)))
     inp = wl.make_inputs(wr, "cuda", with_dO=True)
     Q, K, V, dO, G1, G2 = (inp[k] for k in ("Q", "K", "V", "dO", "G1", "G2"))
     # forward and backward of one step share the workspace: the backward reads the forward's states
@@ -254,8 +250,7 @@ def main():
         launches[0] += n
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        du.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -283,11 +278,8 @@ def main():
     psk.profile_enable(False)
     if psk.check(ws) != 0:
         raise RuntimeError("device-side error during the timed region")
-    tms = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    ms = float(tms.item())
-    value = world * w.model_tokens * args.steps / (ms / 1e3)
+    ms = du.max_over_ranks(ms, "cuda")
+    value = du.aggregate_throughput(w.model_tokens, args.steps, ms, world)
 
     # ---- end to end through the same C-ABI call with HOST buffers ----
     e2e = None
@@ -316,16 +308,13 @@ def main():
             e2e_step()
         b_.record()
         barrier()
-        t2 = torch.tensor([a.elapsed_time(b_)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * w.model_tokens * args.e2e_steps / (float(t2.item()) / 1e3), "unit": UNIT,
+        t2 = du.max_over_ranks(a.elapsed_time(b_), "cuda")
+        e2e = {"value": du.aggregate_throughput(w.model_tokens, args.e2e_steps, t2, world), "unit": UNIT,
                "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo, "steps": args.e2e_steps}
         del host_in, host_out
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        du.shutdown()
         return
 
     # ---- roofline of the dominant kernel ----
@@ -388,8 +377,7 @@ def main():
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    du.shutdown()
 
 
 if __name__ == "__main__":

@@ -32,6 +32,7 @@ def test_sketch_matches_oracle(r, dtype):
 @pytest.mark.parametrize("r,b,n,dtype", [
     (16, 128, 384, "f32"), (32, 256, 768, "f32"), (64, 128, 256, "f32"), (32, 128, 128, "f32"),
     (32, 256, 1024, "bf16"), (64, 512, 1024, "bf16"), (16, 128, 640, "bf16"),
+    (32, 128, 128, "bf16"), (32, 256, 256, "bf16"), (64, 512, 512, "bf16"),      # a single block: no prefix state at all
 ])
 def test_forward_and_backward_small(r, b, n, dtype):
     w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype=dtype, seed=3 * r + b)
@@ -53,7 +54,8 @@ def test_forward_and_backward_small(r, b, n, dtype):
                     check(name, got[bi, hi], ref, TOL[dtype])
 
 
-@pytest.mark.parametrize("r,b,n,corr", [(32, 256, 1024, False), (16, 128, 512, True), (64, 512, 1024, True)])
+@pytest.mark.parametrize("r,b,n,corr", [(32, 256, 1024, False), (16, 128, 512, True), (64, 512, 1024, True),
+                                        (32, 256, 256, True)])
 def test_backward_reading_the_forwards_states(r, b, n, corr):
     # PSK_FLAG_KEEP_STATES: forward and backward share one workspace; the backward skips the
     # prefix-state pass.  Values with a common mean direction exercise the centring.
