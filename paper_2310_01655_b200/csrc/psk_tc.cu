@@ -9,9 +9,6 @@
 // columns 0..63 and columns 64..79 (+ zero fill).  Together they are an MN-major B operand with
 // N = 80 (contract over features) or a K-major B operand with K = 64 + 16 (contract over the
 // state's columns).
-#ifndef PSK_EXP
-#define PSK_EXP 0
-#endif
 #include "psk_internal.cuh"
 #include "tc_features.cuh"
 #include "tc_common.cuh"
@@ -179,15 +176,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             uint32_t a_cnt[NWG];
 #pragma unroll
             for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
-#if PSK_EXP == 9
-            long long* trace = reinterpret_cast<long long*>(status) + 2;
-            int tr = 0;
-#define TRF() do { if (bh == 0 && (j == 8 || j == 9) && tr < 30) trace[tr++] = clock64(); } while (0)
-#else
-#define TRF() do {} while (0)
-#endif
             for (int j = 0; j < NJ && ok; ++j) {
-                TRF();
                 // sketch of the next token tile, as soon as this tile's half sketches are read out
                 if (j + 1 < NJ) {
                     ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
@@ -205,11 +194,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     constexpr int I = decltype(ic)::value;
                     constexpr int w = I % NWG;
                     // the store warpgroup has taken this accumulator's values for the boundary
-                    TRF();
                     if (boundary) ok = ok && mbar_wait(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
-                    TRF();
                     ok = ok && mbar_wait(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
-                    TRF();
                     ++a_cnt[w];
                     tc_fence_after();
                     const uint32_t ab = smem_u32(smem + L::A0 + w * 32768);

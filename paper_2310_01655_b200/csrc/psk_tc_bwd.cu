@@ -11,9 +11,6 @@
 // (d feature) * (the other factor)  (tc_features.cuh explains the weights w).
 // One kernel, two roles: QSIDE rows own (Q, E) and meet keys j <= i; key-side rows own (K, V)
 // and meet queries i >= j.  Thread = own row throughout.
-#ifndef PSK_EXP
-#define PSK_EXP 0
-#endif
 #include "tc_common.cuh"
 
 namespace psk {
@@ -138,7 +135,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const int row0 = l * b + tau * 128;
     const int blk = bh * t + l;
     const int ntiles = b / 128;
-    const bool has_state = (PSK_EXP == 11) ? false : (QSIDE ? (l > 0) : (l < t - 1));
+    const bool has_state = QSIDE ? (l > 0) : (l < t - 1);
 
     if (tid == 0) {
         mbar_init(&bar_own, 1); mbar_init(&bar_oth, 1); mbar_init(&bar_mma, 1);
@@ -301,7 +298,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     // ---- phase C: same block, other-side tiles, 64 other rows at a time ----
     store_hilo_tiles<R>(smem + L::Mown, m, tid);
-    const int tp_begin = QSIDE ? 0 : tau, tp_end = (PSK_EXP == 12) ? tp_begin : (QSIDE ? tau + 1 : ntiles);
+    const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
     bool dm_started = false;
     uint32_t oth_uses = 0;
     float2* oth_col = reinterpret_cast<float2*>(smem + L::Eoth);   // other rows: (1/d, -(g . O)/d)

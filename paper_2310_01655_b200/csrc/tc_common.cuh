@@ -85,23 +85,6 @@ __device__ __forceinline__ void build_g_tile(uint8_t* sG, const bf16* G1, const 
     }
 }
 
-// Subtracts the per-head vector cm[0..63] (shared memory, fp32) from row `row` of a TMA-written
-// [128 rows x 64] bf16 tile in the 128-byte-swizzled layout.
-__device__ __forceinline__ void center_row(uint8_t* tile, const float* cm, int row) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint4* p = reinterpret_cast<uint4*>(tile + swz128_offset(row, c));
-        const uint4 v = *p;
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            o[j] = pack_bf16(__uint_as_float(w[j] << 16) - cm[c * 8 + 2 * j],
-                             __uint_as_float(w[j] & 0xFFFF0000u) - cm[c * 8 + 2 * j + 1]);
-        *p = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-}
-
 // Sketch GEMM D[128 tokens x 2R] = X_tile [G1 | G2], 4 K steps of 16 over the head dimension.
 template <int R>
 __device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX, const uint8_t* sG) {
@@ -175,27 +158,6 @@ __device__ __forceinline__ void store_hilo_tiles(uint8_t* dst, const float (&m)[
             }
             v.x = pack_bf16(x[0], x[1]); v.y = pack_bf16(x[2], x[3]);
             v.z = pack_bf16(x[4], x[5]); v.w = pack_bf16(x[6], x[7]);
-        }
-        *reinterpret_cast<uint4*>(dst + (ch / 8) * 16384 + swz128_offset(row, ch % 8)) = v;
-    }
-}
-
-// The same 3R columns as ceil(3R/64) tiles of [128 rows x 128 B] in the 128-byte-swizzled layout
-// (zero beyond 3R).  Tile 0 starts with the R `hi` columns, so it doubles as the MN-major B
-// operand (N = 64, columns >= R ignored by the reader) of the dM GEMMs.
-template <int R>
-struct SplitTiles { static constexpr int N = (3 * R + 63) / 64; };
-
-template <int R, bool OWN>
-__device__ __forceinline__ void store_split_tiles(uint8_t* dst, const float (&m)[R], int row) {
-#pragma unroll
-    for (int ch = 0; ch < SplitTiles<R>::N * 8; ++ch) {
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (ch * 8 < 3 * R) {
-            v.x = pack_bf16(split_col<R, OWN>(m, ch * 8 + 0), split_col<R, OWN>(m, ch * 8 + 1));
-            v.y = pack_bf16(split_col<R, OWN>(m, ch * 8 + 2), split_col<R, OWN>(m, ch * 8 + 3));
-            v.z = pack_bf16(split_col<R, OWN>(m, ch * 8 + 4), split_col<R, OWN>(m, ch * 8 + 5));
-            v.w = pack_bf16(split_col<R, OWN>(m, ch * 8 + 6), split_col<R, OWN>(m, ch * 8 + 7));
         }
         *reinterpret_cast<uint4*>(dst + (ch / 8) * 16384 + swz128_offset(row, ch % 8)) = v;
     }
