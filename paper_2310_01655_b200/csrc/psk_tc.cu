@@ -479,6 +479,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
     // ---- same block: key tiles tp <= tau through squared half-sketch scores ----
     float rowsum = 0.f;
+#pragma unroll 1
     for (int tp = 0; tp <= tau && ok; ++tp) {
         if (tid == 0) {
             // previous users of sK / sV / cW (sketch, P) have completed: bar_mma was waited on below

@@ -303,6 +303,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     uint32_t oth_uses = 0;
     float2* oth_col = reinterpret_cast<float2*>(smem + L::Eoth);   // other rows: (1/d, -(g . O)/d)
     const float y65h_inv = y65h * inv_own;
+#pragma unroll 1
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
         if (tid == 0) {
@@ -330,6 +331,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             store_hilo_tiles<R>(smem + L::Moth, mo, tid);
         }
         const bool diag = (tp == tau);
+#pragma unroll 1
         for (int hh = 0; hh < 2; ++hh) {
             fence_proxy_async_smem();
             tc_fence_before();

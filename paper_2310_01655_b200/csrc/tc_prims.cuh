@@ -33,16 +33,19 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // A waiting thread is suspended by the hardware for up to this long per poll instead of spinning:
 // spinning warps take issue slots from the warps that do the work.
 constexpr uint32_t kSuspendHintNs = 20000;
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
+        : "r"(bar_addr), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    return mbar_try_wait_addr(smem_u32(bar), parity);
 }
 // Bounded wait: gives up after kSpinLimit polls, records `code` in *status (global) and
 // returns false; the caller then leaves its loop, so a lost signal cannot hang the GPU.
@@ -58,13 +61,19 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code) {
-    if (mbar_test(bar, parity)) return true;       // already complete: no suspension round trip
+// The bounded spin is one out-of-line copy: waits are everywhere in straight-line kernel code, and
+// instruction fetch is what those kernels run out of first.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, int* status, int code) {
+#pragma unroll 1
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_addr(bar_addr, parity)) return true;
     }
     if (status != nullptr) atomicCAS(status, 0, code);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code) {
+    if (mbar_test(bar, parity)) return true;       // already complete: no suspension round trip
+    return mbar_wait_slow(smem_u32(bar), parity, status, code);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
