@@ -103,7 +103,7 @@ constexpr int kErrState = 3;
 template <int R, int T0, int TN, int NWG>
 __global__ void __launch_bounds__(128 * (NWG + 1) + 32)
 tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
-                const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
+                const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                 const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode, int reverse,
                 bf16* __restrict__ S, int* status) {
     using F = Feat<R>;
@@ -133,7 +133,6 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapY);
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
-    if (wg == 0) build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, wt);
     if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
     // last-column chunks of both slots: zero, and column 0 = 1 when the last column is all ones
     for (int e = tid; e < 2 * 1024; e += kThreads) {
@@ -159,7 +158,9 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
             bool ok = true;
             auto load_x = [&](int j) {
-                mbar_expect_tx(&bar_fullx[j & 1], 16384);
+                // the first tile's barrier also covers the sketch matrices' image
+                mbar_expect_tx(&bar_fullx[j & 1], 16384 + (j == 0 ? GImage<R>::bytes : 0u));
+                if (j == 0) bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_fullx[0]);
                 tma_load_4d(smem + L::X + (j & 1) * 16384, &mapX, 0, tile_of(j) * 128, hi, bi, &bar_fullx[j & 1]);
             };
             auto load_y = [&](int j) {
@@ -358,7 +359,7 @@ template <int R, int MODE>
 __global__ void __launch_bounds__(128, 2)
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
-                  const bf16* __restrict__ G1, const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
+                  const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                   const float* __restrict__ cmean, bf16* __restrict__ O, int64_t sb, int64_t sh, int64_t sn,
                   float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
                   float* __restrict__ e65, float* __restrict__ e65h, float* __restrict__ Oc, int* status) {
@@ -381,8 +382,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         for (int s = 0; s < kZStages; ++s) mbar_init(&bar_z[s], 1);
         mbar_fence_init();
         tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV); tma_prefetch_desc(&mapZ);
-        mbar_expect_tx(&bar_q, 16384);
+        mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
         tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
+        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
         if (l > 0) {
             for (int c = 0; c < kZStages && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_z[c], kZStageBytes);
@@ -392,7 +394,6 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         }
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
-    build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
     if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
     fence_proxy_async_smem();
     tc_fence_before();
@@ -666,31 +667,44 @@ tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh
     }
 }
 
+// Image of [G1 | G2]^T (set g of the sketch matrices, each [64 x r] row-major) in the layout the
+// sketch GEMM reads from shared memory: row nn < 2r = sketch column, 64 head dimensions, swizzled.
+__global__ void __launch_bounds__(128)
+tc_gimage_kernel(const bf16* __restrict__ G1, const bf16* __restrict__ G2, int r, uint8_t* __restrict__ gimg) {
+    const int g = blockIdx.x;
+    uint8_t* img = gimg + (size_t)g * 2 * r * 128;
+    for (int e = threadIdx.x; e < 2 * r * 64; e += 128) {
+        const int nn = e / 64, k = e % 64;
+        const bf16 v = (nn < r ? G1 : G2)[(size_t)g * 64 * r + k * r + (nn % r)];
+        *reinterpret_cast<bf16*>(img + swz128_offset(nn, k / 8) + (k % 8) * 2) = v;
+    }
+}
+
 // ---------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------
 
 // Prefix (or suffix) states of every head.  X is sketched, Y is the right-hand side.
 template <int R, int T0, int TN, int NWG>
-cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1,
-                               const bf16* G2, const float* y65, const float* cmean, int center_mode, bool reverse,
+cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
+                               const float* y65, const float* cmean, int center_mode, bool reverse,
                                bf16* S, int* status, cudaStream_t s, int* launches) {
     constexpr size_t smem = StateSmem<R, NWG>::total + 1024;
     PSK_TRY(set_smem(tc_state_kernel<R, T0, TN, NWG>, smem));
     prof_begin("tc_state_kernel", s);
     tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 32, smem, s>>>(
-        mX, mY, G1, G2, d.g_heads, d.H, d.n, d.b, d.t, y65, cmean, center_mode, reverse ? 1 : 0, S, status);
+        mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, y65, cmean, center_mode, reverse ? 1 : 0, S, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
 }
 
 template <int R>
-cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
                           const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
                           cudaStream_t s, int* launches) {
 #define PSK_SG(T0, TN, NWG) \
-    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, G1, G2, y65, cmean, center_mode, reverse, S, status, s, launches)))
+    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, gimg, y65, cmean, center_mode, reverse, S, status, s, launches)))
     if constexpr (R == 16) {
         PSK_SG(0, 2, 2);
     } else if constexpr (R == 32) {
@@ -716,13 +730,15 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     // keep_states: the backward will read these states, so they are built from centred values
     float* cmean = d.keep_states ? reinterpret_cast<float*>(ws + w.vmean) : nullptr;
     if (cmean != nullptr) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
-    PSK_TRY((launch_states<R>(d, mK, mV, (const bf16*)G1, (const bf16*)G2, nullptr, cmean, cmean ? 1 : 0, Z, false,
+    uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
+    PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
+    PSK_TRY((launch_states<R>(d, mK, mV, gimg, nullptr, cmean, cmean ? 1 : 0, Z, false,
                               status, s, launches)));
     constexpr size_t smem = OutSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_fwd_out_kernel<R, 0>, smem));
     prof_begin("tc_fwd_out_kernel", s);
     tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, (const bf16*)G1, (const bf16*)G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, (bf16*)O, d.sb, d.sh, d.sn,
+        mQ, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, (bf16*)O, d.sb, d.sh, d.sn,
         denom, nullptr, nullptr, nullptr, nullptr, Oc, status);
     prof_end(s);
     ++*launches;
@@ -757,14 +773,14 @@ cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V, c
 
 template <int R>
 static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
-                                  const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean,
+                                  const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean,
                                   const float* denom, const bf16* dO, bf16* E, float* e65, float* e65h, int* status,
                                   cudaStream_t s, int* launches) {
     constexpr size_t smem = OutSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_fwd_out_kernel<R, 1>, smem));
     prof_begin("tc_bwd_recompute_kernel", s);
     tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, G1, G2, d.g_heads, d.H, d.n, d.b, d.t, cmean, nullptr, d.sb, d.sh, d.sn,
+        mQ, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, nullptr, d.sb, d.sh, d.sn,
         const_cast<float*>(denom), dO, E, e65, e65h, nullptr, status);
     prof_end(s);
     ++*launches;
@@ -772,14 +788,22 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
 }
 
 cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
-                         const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean, const float* denom,
+                         const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
                          const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
-        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
-        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, G1, G2, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
     }
     return cudaErrorInvalidValue;
+}
+
+cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gimg, cudaStream_t s, int* launches) {
+    prof_begin("tc_gimage_kernel", s);
+    tc_gimage_kernel<<<d.g_heads, 128, 0, s>>>((const bf16*)G1, (const bf16*)G2, d.r, gimg);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
 }
 
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches) {
@@ -790,13 +814,13 @@ cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s,
     return cudaGetLastError();
 }
 
-cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
                       const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
                           cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return launch_states<16>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
-        case 32: return launch_states<32>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
-        case 64: return launch_states<64>(d, mX, mY, G1, G2, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 16: return launch_states<16>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 32: return launch_states<32>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 64: return launch_states<64>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
     }
     return cudaErrorInvalidValue;
 }

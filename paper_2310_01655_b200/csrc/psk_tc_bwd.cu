@@ -119,8 +119,8 @@ template <int R, bool QSIDE>
 __global__ void __launch_bounds__(128, (R <= 32 ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
-                   const __grid_constant__ CUtensorMap mapS, const bf16* __restrict__ G1,
-                   const bf16* __restrict__ G2, int g_heads, int H, int n, int b, int t,
+                   const __grid_constant__ CUtensorMap mapS, const uint8_t* __restrict__ gimg,
+                   int g_heads, int H, int n, int b, int t,
                    const float* __restrict__ e65, const float* __restrict__ e65h, const float* __restrict__ denom,
                    bf16* __restrict__ dX, bf16* __restrict__ dV, int64_t sb, int64_t sh, int64_t sn, int* status) {
     using F = Feat<R>;
@@ -144,7 +144,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         mbar_fence_init();
         tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
         tma_prefetch_desc(&mapYoth); tma_prefetch_desc(&mapS);
-        mbar_expect_tx(&bar_own, 32768);
+        mbar_expect_tx(&bar_own, 32768 + GImage<R>::bytes);
+        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_own);
         tma_load_4d(smem + L::Xown, &mapXown, 0, row0, hi, bi, &bar_own);
         tma_load_4d(smem + L::Yown, &mapYown, 0, row0, hi, bi, &bar_own);
         if (has_state) {
@@ -156,7 +157,6 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         }
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
-    build_g_tile<R>(smem + L::G, G1 + (size_t)g * 64 * R, G2 + (size_t)g * 64 * R, tid);
     // Query rows work on the raw dO rows g_i (exact bf16 inputs) and apply 1/d_i in fp32 afterwards:
     // dL/dW_ij = (g_i . v_j - g_i . O_i) / d_i cancels heavily when one key dominates a row, and a
     // rounded g_i / d_i would not survive it.  y65 = -(g_i . (O_i - c)) pairs with the centred
@@ -527,10 +527,10 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk))
         return cudaErrorInvalidValue;
-    const bf16* g1 = (const bf16*)G1;
-    const bf16* g2 = (const bf16*)G2;
+    uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
+    PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
     // prefix states of centred values; forward rows again in fp32 -> E, e65, e65h; suffix states
-    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, g1, g2, nullptr, cmean, 1, Z, false, status, s, launches));
+    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, cmean, 1, Z, false, status, s, launches));
     if (d.keep_states) {
         const int rows = d.BH() * d.n;
         prof_begin("tc_bwd_prep_kernel", s);
@@ -541,19 +541,19 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         ++*launches;
         PSK_TRY(cudaGetLastError());
     } else {
-        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, g1, g2, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
+        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
     }
-    PSK_TRY(tc_states(d, mQ, mE, g1, g2, e65, cmean, 2, Rs, true, status, s, launches));
+    PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
     constexpr size_t smem = BwdSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
     prof_begin("tc_bwd_q_kernel", s);
-    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, e65,
                                                         e65h, denom, (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
     prof_end(s);
     prof_begin("tc_bwd_k_kernel", s);
-    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, g1, g2, d.g_heads, d.H, d.n, d.b, d.t, e65,
+    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, gimg, d.g_heads, d.H, d.n, d.b, d.t, e65,
                                                          e65h, denom, (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
     prof_end(s);
     *launches += 2;

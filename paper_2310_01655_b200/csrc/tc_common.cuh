@@ -18,18 +18,21 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
 // per-block states of every head + prefix (reverse = false) or suffix (reverse = true) scan
 // center_mode 0: states as they are; 1: values centred by the per-head vector cmean
 // (columns < 64 become H[:, c] - cmean[c] H[:, 64]); 2: last column becomes H[:, 64] - H[:, :64] cmean.
-cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const bf16* G1, const bf16* G2,
+cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
                       const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
                       cudaStream_t s, int* launches);
 // the backward's recomputation of the forward rows: writes E, e65, e65h (see tc_fwd_out_kernel)
 cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
-                         const CUtensorMap& mZ, const bf16* G1, const bf16* G2, const float* cmean, const float* denom,
+                         const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
                          const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches);
+// gimg[g] = [G1 | G2]^T of sketch-matrix set g as the shared-memory image of the sketch GEMM's B operand
+// (2r rows x 128 B, K-major, 128-byte swizzle): the kernels fetch it with one bulk copy
+cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gimg, cudaStream_t s, int* launches);
 // cmean[bh][c] = mean over the n rows of V[bh][:, c]  (deterministic reduction)
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
 
 // Scratch layout of the tensor-core path.
-struct TcWorkspace { size_t status, vmean, Z, Rst, E, e65, e65h, Oc, total; };
+struct TcWorkspace { size_t status, vmean, gimg, Z, Rst, E, e65, e65h, Oc, total; };
 
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
@@ -39,6 +42,7 @@ inline TcWorkspace tc_ws(const Dims& d, bool backward) {
     size_t off = 0;
     w.status = off; off += kStatusBytes;
     w.vmean = off; off += align_up((size_t)d.BH() * 64 * sizeof(float));
+    w.gimg = off; off += align_up((size_t)d.g_heads * 2 * R * 128);
     w.Z = off; off += align_up(st);
     if (backward) {
         w.Rst = off; off += align_up(st);
@@ -75,15 +79,10 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
 }
 
 // [G1 | G2]^T as a K-major, 128-byte-swizzled tile: row n (< 2R) holds sketch column n over the 64
-// head dimensions.  B operand of the sketch GEMM X [G1 | G2].
+// head dimensions.  B operand of the sketch GEMM X [G1 | G2]; built once per call by
+// tc_gimage_kernel, then copied into shared memory as it is.
 template <int R>
-__device__ __forceinline__ void build_g_tile(uint8_t* sG, const bf16* G1, const bf16* G2, int tid) {
-    for (int e = tid; e < 2 * R * 64; e += 128) {
-        const int nn = e / 64, k = e % 64;
-        const bf16 v = (nn < R ? G1 : G2)[k * R + (nn % R)];
-        *reinterpret_cast<bf16*>(sG + swz128_offset(nn, k / 8) + (k % 8) * 2) = v;
-    }
-}
+struct GImage { static constexpr uint32_t bytes = 2 * R * 128; };
 
 // Sketch GEMM D[128 tokens x 2R] = X_tile [G1 | G2], 4 K steps of 16 over the head dimension.
 template <int R>
