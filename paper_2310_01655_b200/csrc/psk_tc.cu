@@ -66,6 +66,18 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [rows, 64] fp32, contiguous; box = 128 rows x 32 columns (128 B), 128-byte swizzle.
+bool tc_map_f32rows(CUtensorMap* m, const void* base, int64_t rows) {
+    EncodeFn enc = encoder();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {64, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {32, 128}, es[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 namespace {
 
 // ---------------------------------------------------------------------------
@@ -331,43 +343,56 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
 // ---------------------------------------------------------------------------
 // Forward output rows (Section 3.1): for a 128-row tile of block l,
 //   N = phi_w(Q) Z_l  (tensor memory A operand x TMA-fed Z chunks, N = 80: column 64 = normaliser)
-//     + sum over key tiles of the same block  lt((M_q M_k^T)^2) V
-//   d = 1 + rowsum(diagonal weights) + N[:, 64];  O = N[:, :64] / d
-// grid (b/128, t, BH), 128 threads (thread = query row).
+//     + sum over key tiles of the same block  lt((M_q M_k^T)^2) [V | 1]
+//   d = 1 + normaliser;  O = N[:, :64] / d
+// grid (b/128, t, BH), 160 threads.  Warps 0-3: thread = query row (half sketches, features,
+// weights, epilogue).  Warp 4: one thread issues every TMA load and every MMA; the two sides meet
+// only at mbarriers, so the rows never wait for an issue sequence and the tensor pipe runs ahead.
 // ---------------------------------------------------------------------------
-constexpr int kZStages = 3;
+constexpr int kZStages = 4;                     // three in the shared region + the query tile's buffer
 constexpr uint32_t kZStageBytes = 16384;        // two [64 features x 128 B] boxes: columns 0..63, 64..79
+constexpr int kFeatBufs = 4;                    // feature staging buffers in tensor memory, 32 columns each
 
 template <int R>
 struct OutSmem {
-    // The prefix-state stages (first phase) and the key/value tiles with the keys' split half
-    // sketches (second phase) share one region; small enough for two CTAs per SM when R <= 32.
+    // The prefix-state stages (first phase), the key/value tiles with the keys' split half
+    // sketches (second phase) and the output staging tiles (epilogue) share one region; small
+    // enough for two CTAs per SM when R <= 32.
     static constexpr uint32_t Q = 0, G = 16384;
-    static constexpr uint32_t Mq = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
+    static constexpr uint32_t Ones = G + GImage<R>::bytes;           // 4 KB of bf16 1.0: B operand of the row sums
+    static constexpr uint32_t Mq = Ones + 4096;
     static constexpr uint32_t U = (Mq + 128 * 3 * R * 2 + 1023) / 1024 * 1024;   // split operand: 3R columns
     static constexpr uint32_t Z = U;
     static constexpr uint32_t K = U, V = U + 16384, Mk = U + 32768;
-    static constexpr uint32_t kPhase1 = kZStages * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2;
-    static constexpr uint32_t total = U + (kPhase1 > kPhase2 ? kPhase1 : kPhase2);
+    static constexpr uint32_t So = U, Soc = U + 16384;               // O tile (bf16), two fp32 half tiles
+    static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2, kEpi = 49152;
+    static constexpr uint32_t kMax12 = kPhase1 > kPhase2 ? kPhase1 : kPhase2;
+    static constexpr uint32_t total = U + (kMax12 > kEpi ? kMax12 : kEpi);
+    // stage s of the prefix-state ring; the last one is the query tile's buffer, dead after the sketch
+    __device__ static uint32_t zstage(int s) { return s < kZStages - 1 ? Z + s * kZStageBytes : Q; }
 };
 
-// MODE 0: forward (writes O, denom).  MODE 1: the backward's recomputation of the row numerators
-// against centred prefix states; writes E = dO/d (bf16), e65 = -(dO.(O - c))/d and
-// e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32 accumulators rather than
-// from the rounded O the caller holds.
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// MODE 0: forward (writes O, denom, optionally O - c in fp32).  MODE 1: the backward's
+// recomputation of the row numerators against centred prefix states; writes E = dO/d (bf16),
+// e65 = -(dO.(O - c))/d and e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32
+// accumulators rather than from the rounded O the caller holds.
 template <int R, int MODE>
-__global__ void __launch_bounds__(128, 2)
+__global__ void __launch_bounds__(160, (R <= 32 ? 2 : 1))
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
+                  const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapOc,
                   const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
-                  const float* __restrict__ cmean, bf16* __restrict__ O, int64_t sb, int64_t sh, int64_t sn,
+                  const float* __restrict__ cmean, int64_t sb, int64_t sh, int64_t sn,
                   float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
-                  float* __restrict__ e65, float* __restrict__ e65h, float* __restrict__ Oc, int* status) {
+                  float* __restrict__ e65, float* __restrict__ e65h, int keep_oc, int* status) {
     using F = Feat<R>;
     using L = OutSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_q, bar_kv, bar_mma, bar_a[2], bar_z[kZStages];
+    __shared__ uint64_t bar_q, bar_kv, bar_sk, bar_mk, bar_s, bar_p, bar_pv;
+    __shared__ uint64_t bar_z[kZStages], bar_feat[kFeatBufs], bar_a[kFeatBufs];
     __shared__ uint32_t tmem_slot;
     __shared__ float cm[64];
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
@@ -377,187 +402,194 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const int blk = bh * t + l;
 
     if (tid == 0) {
-        mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_mma, 1);
-        mbar_init(&bar_a[0], 1); mbar_init(&bar_a[1], 1);
+        mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_sk, 1); mbar_init(&bar_s, 1); mbar_init(&bar_pv, 1);
+        mbar_init(&bar_mk, 128); mbar_init(&bar_p, 128);
         for (int s = 0; s < kZStages; ++s) mbar_init(&bar_z[s], 1);
+        for (int s = 0; s < kFeatBufs; ++s) { mbar_init(&bar_feat[s], 128); mbar_init(&bar_a[s], 1); }
         mbar_fence_init();
         tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV); tma_prefetch_desc(&mapZ);
         mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
         tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
         bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
         if (l > 0) {
-            for (int c = 0; c < kZStages && c < F::NC; ++c) {
+            for (int c = 0; c < kZStages - 1 && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_z[c], kZStageBytes);
-                tma_load_3d(smem + L::Z + c * kZStageBytes, &mapZ, 0, c * 64, blk, &bar_z[c]);
-                tma_load_3d(smem + L::Z + c * kZStageBytes + 8192, &mapZ, 64, c * 64, blk, &bar_z[c]);
+                tma_load_3d(smem + L::zstage(c), &mapZ, 0, c * 64, blk, &bar_z[c]);
+                tma_load_3d(smem + L::zstage(c) + 8192, &mapZ, 64, c * 64, blk, &bar_z[c]);
             }
         }
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    if (warp == 4) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    for (int e = tid; e < 256; e += 160)
+        reinterpret_cast<uint4*>(smem + L::Ones)[e] = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
     if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tm = tmem_slot;
-    const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
-    // tensor-memory columns
-    // sketch accumulators, scores, packed weights and the feature staging buffers all live in
-    // [0, 128): each is consumed before the next is produced; the output accumulator follows
-    constexpr uint32_t cSk = 0, cS = 0, cW = 0, cA = 0, cO = 128;
-    uint32_t mma_uses = 0;
+    // tensor-memory columns: sketch accumulators, feature staging buffers, scores and packed
+    // weights all live in [0, 128), each consumed before the next is produced; then the output
+    // accumulator (64 + the prefix normaliser's 16) and the same-block row sums (16)
+    constexpr uint32_t cSk = 0, cS = 0, cW = 0, cA = 0, cO = 128, cN = cO + 80;
     bool ok = true;
 
-    // ---- half sketch of the query rows ----
-    ok = mbar_wait(&bar_q, 0, status, kErrTma);
-    if (tid == 0) {
-        tc_fence_after();
-        issue_sketch<R>(tm + cSk, smem + L::Q, smem + L::G);
-        umma_commit(&bar_mma);
-    }
-    ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-    ++mma_uses;
-    tc_fence_after();
-    float mq[R];
-    read_half_sketch<R>(lane_tm + cSk, mq);
-    store_split_rows<R, true>(smem + L::Mq, mq, tid);
-    PackedM<R> pmq;
-    pack_half_sketch<R>(mq, pmq);
-
-    // ---- earlier blocks: weighted features (tensor memory) x prefix state ----
-    if (l > 0) {
-        uint32_t a_uses[2] = {0, 0};
-        static_for<0, F::NC>([&](auto cc) {
-            constexpr int C = decltype(cc)::value;
-            constexpr int buf = C & 1, stage = C % kZStages;
-            constexpr int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
-            if (a_uses[buf] > 0) {
-                ok = ok && mbar_wait(&bar_a[buf], (a_uses[buf] - 1) & 1, status, kErrMma);
-                // chunk C-2 is done with its stage: refill it with chunk C-2+kZStages
-                if (tid == 0 && C - 2 + kZStages < F::NC) {
-                    constexpr int s2 = (C - 2 + 2 * kZStages) % kZStages;
-                    mbar_expect_tx(&bar_z[s2], kZStageBytes);
-                    tma_load_3d(smem + L::Z + s2 * kZStageBytes, &mapZ, 0, (C - 2 + kZStages) * 64, blk, &bar_z[s2]);
-                    tma_load_3d(smem + L::Z + s2 * kZStageBytes + 8192, &mapZ, 64, (C - 2 + kZStages) * 64, blk,
-                                &bar_z[s2]);
-                }
-            }
+    if (warp == 4) {
+        // ================================ issuer ================================
+        if (tid == 128) {
+            ok = mbar_spin(&bar_q, 0, status, kErrTma);
             tc_fence_after();
-            uint32_t pk[16];
-            gen_features<R, C * 64, true, 16>(pmq, pk);
-            tmem_st16(lane_tm + cA + buf * 32, pk);
-            gen_features<R, C * 64 + 32, true, 16>(pmq, pk);
-            tmem_st16(lane_tm + cA + buf * 32 + 16, pk);
-            tmem_st_wait();
-            ok = ok && mbar_wait(&bar_z[stage], (C / kZStages) & 1, status, kErrTma);
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
+            issue_sketch<R>(tm + cSk, smem + L::Q, smem + L::G);
+            umma_commit(&bar_sk);
+            if (l > 0 && kZStages - 1 < F::NC) {
+                // the query tile has been consumed: its buffer becomes the ring's last stage
+                ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);
+                mbar_expect_tx(&bar_z[kZStages - 1], kZStageBytes);
+                tma_load_3d(smem + L::zstage(kZStages - 1), &mapZ, 0, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
+                tma_load_3d(smem + L::zstage(kZStages - 1) + 8192, &mapZ, 64, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
+            }
+            if (l > 0) {
+                // earlier blocks: weighted features (tensor memory) x prefix state chunks.
                 // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step,
                 // the second 64-column group (columns 64..79) 8192 B further on
                 constexpr uint32_t idesc = idesc_bf16(128, 80, false, true);
-                const uint32_t zb = smem_u32(smem + L::Z + stage * kZStageBytes);
-#pragma unroll
-                for (int k = 0; k < ksteps; ++k)
-                    umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, desc_off(smem_desc(zb, 8192, 1024, kSwz128), k * 2048), idesc,
-                            (C > 0 || k > 0) ? 1u : 0u);
-                umma_commit(&bar_a[buf]);
-            }
-            ++a_uses[buf];
-        });
-    }
-
-    // the key/value tiles reuse the stages' memory and the sketch reuses the staging columns:
-    // every MMA of the first phase must have completed
-    if (l > 0) {
-        if (tid == 0) umma_commit(&bar_mma);
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
-        __syncthreads();
-    }
-
-    // ---- same block: key tiles tp <= tau through squared half-sketch scores ----
-    float rowsum = 0.f;
 #pragma unroll 1
-    for (int tp = 0; tp <= tau && ok; ++tp) {
-        if (tid == 0) {
-            // previous users of sK / sV / cW (sketch, P) have completed: bar_mma was waited on below
-            mbar_expect_tx(&bar_kv, 32768);
-            tma_load_4d(smem + L::K, &mapK, 0, l * b + tp * 128, hi, bi, &bar_kv);
-            tma_load_4d(smem + L::V, &mapV, 0, l * b + tp * 128, hi, bi, &bar_kv);
-        }
-        ok = mbar_wait(&bar_kv, tp & 1, status, kErrTma);
-        if (tid == 0) {
-            tc_fence_after();
-            issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
-            umma_commit(&bar_mma);
-        }
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
-        {
-            float mk[R];
-            read_half_sketch<R>(lane_tm + cSk, mk);
-            store_split_rows<R, false>(smem + L::Mk, mk, tid);
-        }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
-#pragma unroll
-            for (int k = 0; k < 3 * R / 16; ++k)
-                umma_ss(tm + cS, desc_off(smem_desc(smem_u32(smem + L::Mq), 2048, 128, kSwzNone), k * 4096),
-                        desc_off(smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone), k * 4096), idesc, k > 0);
-            umma_commit(&bar_mma);
-        }
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
-        const bool diag = (tp == tau);
-#pragma unroll
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t v[32], pk[16];
-            tmem_ld32(lane_tm + cS + c0, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
-                w0 = (diag && c0 + j > tid) ? 0.f : w0 * w0;
-                w1 = (diag && c0 + j + 1 > tid) ? 0.f : w1 * w1;
-                // the normaliser sums the weights as the value GEMM will see them (rounded to bf16):
-                // where one key dominates a row, v_j - O_i = v_j / d_i only holds if numerator and
-                // denominator use the same numbers
-                const uint32_t p2 = pack_bf16(w0, w1);
-                rowsum += __uint_as_float(p2 << 16) + __uint_as_float(p2 & 0xFFFF0000u);
-                pk[j / 2] = p2;
+                for (int C = 0; C < F::NC && ok; ++C) {
+                    const int buf = C % kFeatBufs, stage = C % kZStages;
+                    ok = mbar_spin(&bar_z[stage], (C / kZStages) & 1, status, kErrTma);
+                    ok = ok && mbar_spin(&bar_feat[buf], (C / kFeatBufs) & 1, status, kErrMma);
+                    tc_fence_after();
+                    const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+                    const uint64_t zd = smem_desc(smem_u32(smem + L::zstage(stage)), 8192, 1024, kSwz128);
+#pragma unroll 1
+                    for (int k = 0; k < ksteps; ++k)
+                        umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&bar_a[buf]);
+                    // chunk C-1 is done with its stage: refill it with chunk C-1+kZStages
+                    if (C >= 1 && C - 1 + kZStages < F::NC) {
+                        const int pc = C - 1, ps = pc % kZStages;
+                        ok = ok && mbar_spin(&bar_a[pc % kFeatBufs], (pc / kFeatBufs) & 1, status, kErrMma);
+                        mbar_expect_tx(&bar_z[ps], kZStageBytes);
+                        tma_load_3d(smem + L::zstage(ps), &mapZ, 0, (pc + kZStages) * 64, blk, &bar_z[ps]);
+                        tma_load_3d(smem + L::zstage(ps) + 8192, &mapZ, 64, (pc + kZStages) * 64, blk, &bar_z[ps]);
+                    }
+                }
+                // the key/value tiles reuse the stages' memory and the sketch reuses the staging
+                // columns: every MMA of the first phase must have completed
+                ok = ok && mbar_spin(&bar_a[(F::NC - 1) % kFeatBufs], ((F::NC - 1) / kFeatBufs) & 1, status, kErrMma);
             }
-            tmem_st16(lane_tm + cW + c0 / 2, pk);
+            // same block: key tiles tp <= tau through squared half-sketch scores
+#pragma unroll 1
+            for (int tp = 0; tp <= tau && ok; ++tp) {
+                if (tp > 0) ok = mbar_spin(&bar_pv, (tp - 1) & 1, status, kErrMma);   // K, V, Mk, weights are free
+                mbar_expect_tx(&bar_kv, 32768);
+                tma_load_4d(smem + L::K, &mapK, 0, l * b + tp * 128, hi, bi, &bar_kv);
+                tma_load_4d(smem + L::V, &mapV, 0, l * b + tp * 128, hi, bi, &bar_kv);
+                ok = ok && mbar_spin(&bar_kv, tp & 1, status, kErrTma);
+                tc_fence_after();
+                issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
+                umma_commit(&bar_sk);
+                ok = ok && mbar_spin(&bar_mk, tp & 1, status, kErrMma);
+                tc_fence_after();
+                {
+                    constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
+                    const uint64_t qd = smem_desc(smem_u32(smem + L::Mq), 2048, 128, kSwzNone);
+                    const uint64_t kd = smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone);
+#pragma unroll 1
+                    for (int k = 0; k < 3 * R / 16; ++k)
+                        umma_ss(tm + cS, desc_off(qd, k * 4096), desc_off(kd, k * 4096), idesc, k > 0);
+                    umma_commit(&bar_s);
+                }
+                ok = ok && mbar_spin(&bar_p, tp & 1, status, kErrMma);
+                tc_fence_after();
+                {
+                    // numerator += W V; row sums += W 1 (the weights exactly as the value GEMM sees them)
+                    constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+                    constexpr uint32_t idesc1 = idesc_bf16(128, 16, false, false);
+                    const uint64_t vd = smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128);
+                    const uint64_t od = smem_desc(smem_u32(smem + L::Ones), 256, 128, kSwzNone);
+#pragma unroll 1
+                    for (int k = 0; k < 8; ++k) {
+                        umma_ts(tm + cO, tm + cW + k * 8, desc_off(vd, k * 2048), idesc, (l > 0 || tp > 0 || k > 0) ? 1u : 0u);
+                        umma_ts(tm + cN, tm + cW + k * 8, desc_off(od, k * 512), idesc1, (tp > 0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&bar_pv);
+                }
+            }
         }
-        tmem_st_wait();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                umma_ts(tm + cO, tm + cW + k * 8, desc_off(smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128), k * 2048), idesc,
-                        (l > 0 || tp > 0 || k > 0) ? 1u : 0u);
-            umma_commit(&bar_mma);
-        }
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
+    } else {
+        // ================================= rows =================================
+        const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
+        ok = mbar_wait(&bar_sk, 0, status, kErrMma);
         tc_fence_after();
-    }
+        float mq[R];
+        read_half_sketch<R>(lane_tm + cSk, mq);
+        store_split_rows<R, true>(smem + L::Mq, mq, tid);
+        PackedM<R> pmq;
+        pack_half_sketch<R>(mq, pmq);
 
-    // ---- epilogue ----
-    if (ok) {
+        if (l > 0) {
+            static_for<0, F::NC>([&](auto cc) {
+                constexpr int C = decltype(cc)::value;
+                constexpr int buf = C % kFeatBufs;
+                if constexpr (C >= kFeatBufs) {       // the MMAs that read this buffer's previous contents
+                    ok = ok && mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
+                    tc_fence_after();
+                }
+                uint32_t pk[16];
+                gen_features<R, C * 64, true, 16>(pmq, pk);
+                tmem_st16(lane_tm + cA + buf * 32, pk);
+                gen_features<R, C * 64 + 32, true, 16>(pmq, pk);
+                tmem_st16(lane_tm + cA + buf * 32 + 16, pk);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&bar_feat[buf]);
+            });
+        }
+
+#pragma unroll 1
+        for (int tp = 0; tp <= tau && ok; ++tp) {
+            ok = mbar_wait(&bar_sk, (tp + 1) & 1, status, kErrMma);
+            tc_fence_after();
+            {
+                float mk[R];
+                read_half_sketch<R>(lane_tm + cSk, mk);
+                store_split_rows<R, false>(smem + L::Mk, mk, tid);
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(&bar_mk);
+            ok = ok && mbar_wait(&bar_s, tp & 1, status, kErrMma);
+            tc_fence_after();
+            // weights = squared scores (lower triangle on the diagonal tile), packed to bf16 over
+            // columns whose fp32 contents have already been read
+            auto weights = [&](auto diag_c) {
+                constexpr bool DIAG = decltype(diag_c)::value;
+#pragma unroll
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    uint32_t v[32], pk[16];
+                    tmem_ld32(lane_tm + cS + c0, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
+                        w0 = (DIAG && c0 + j > tid) ? 0.f : w0 * w0;
+                        w1 = (DIAG && c0 + j + 1 > tid) ? 0.f : w1 * w1;
+                        pk[j / 2] = pack_bf16(w0, w1);
+                    }
+                    tmem_st16(lane_tm + cW + c0 / 2, pk);
+                }
+            };
+            if (tp == tau) weights(std::true_type{}); else weights(std::false_type{});
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&bar_p);
+        }
+        ok = ok && mbar_wait(&bar_pv, tau & 1, status, kErrMma);
+        tc_fence_after();
+
+        // ---- epilogue ----
         float acc[64];
-        float d = 1.f + rowsum;
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
             uint32_t v[32];
@@ -566,41 +598,58 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(v[j]);
         }
-        float noff = 0.f;                   // normaliser part from earlier blocks
-        if (l > 0) {
+        float noff = 0.f, rowsum;             // normaliser parts: earlier blocks, same block
+        {
             uint32_t v[16];
-            tmem_ld16(lane_tm + cO + 64, v);
+            if (l > 0) {
+                tmem_ld16(lane_tm + cO + 64, v);
+                tmem_ld_wait();
+                noff = __uint_as_float(v[0]);
+            }
+            tmem_ld16(lane_tm + cN, v);
             tmem_ld_wait();
-            noff = __uint_as_float(v[0]);
-            d += noff;
+            rowsum = __uint_as_float(v[0]);
         }
         if constexpr (MODE == 0) {
+            const float d = 1.f + rowsum + noff;
             // with centred prefix states (cmean given) the earlier blocks' numerator lacks c * noff
 #pragma unroll
             for (int c = 0; c < 64; ++c) acc[c] = fmaf(cm[c], noff, acc[c]);
             const float inv = 1.f / d;
-            bf16* o = O + (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
+            // rows go out through shared memory and tiled stores: a thread-per-row store pattern
+            // would keep the load/store unit busy for thousands of cycles
 #pragma unroll
-            for (int c = 0; c < 64; c += 8) {
+            for (int c = 0; c < 8; ++c) {
                 uint4 v;
-                v.x = pack_bf16(acc[c] * inv, acc[c + 1] * inv);
-                v.y = pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
-                v.z = pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv);
-                v.w = pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
-                *reinterpret_cast<uint4*>(o + c) = v;
+                v.x = pack_bf16(acc[8 * c] * inv, acc[8 * c + 1] * inv);
+                v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                *reinterpret_cast<uint4*>(smem + L::So + swz128_offset(tid, c)) = v;
             }
-            if (denom != nullptr) denom[(size_t)bh * n + row0 + tid] = d;
-            if (Oc != nullptr) {
+            if (keep_oc) {
                 // kept for the backward: O - c in fp32.  (The rounded O cannot supply it: where the
                 // values share a common component, or one key dominates a row, |O - c| and
                 // |v - O| are far below |O|.)
-                float4* oc = reinterpret_cast<float4*>(Oc + ((size_t)bh * n + row0 + tid) * 64);
 #pragma unroll
-                for (int c = 0; c < 64; c += 4)
-                    oc[c / 4] = make_float4(acc[c] * inv - cm[c], acc[c + 1] * inv - cm[c + 1],
-                                            acc[c + 2] * inv - cm[c + 2], acc[c + 3] * inv - cm[c + 3]);
+                for (int c = 0; c < 16; ++c)
+                    *reinterpret_cast<float4*>(smem + L::Soc + (c / 8) * 16384 + swz128_offset(tid, c % 8)) =
+                        make_float4(acc[4 * c] * inv - cm[4 * c], acc[4 * c + 1] * inv - cm[4 * c + 1],
+                                    acc[4 * c + 2] * inv - cm[4 * c + 2], acc[4 * c + 3] * inv - cm[4 * c + 3]);
             }
-        } else {
+            if (denom != nullptr && ok) denom[(size_t)bh * n + row0 + tid] = d;
+            fence_proxy_async_smem();
+            consumer_barrier();
+            if (tid == 0 && ok) {
+                tma_store_4d(&mapO, smem + L::So, 0, row0, hi, bi);
+                if (keep_oc) {
+                    tma_store_2d(&mapOc, smem + L::Soc, 0, bh * n + row0);
+                    tma_store_2d(&mapOc, smem + L::Soc + 16384, 32, bh * n + row0);
+                }
+                bulk_commit();
+                bulk_wait_read();
+            }
+        } else if (ok) {
             // acc = phi Z' + W V with Z' built from centred values and V raw:
             // N' = acc - rowsum(W) c is the numerator of centred values, O - c = (N' - c) / d.
             const size_t row = (size_t)bh * n + row0 + tid;
@@ -632,7 +681,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 256);
+    if (warp == 4) tmem_dealloc(tm, 256);
 }
 
 // Column means of V per head: cmean[bh][c] = (1/n) sum_i V[bh][i][c].  The kernels work with
@@ -723,10 +772,16 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     int* status = reinterpret_cast<int*>(ws + w.status);
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
     float* Oc = d.keep_states ? reinterpret_cast<float*>(ws + w.Oc) : nullptr;
-    CUtensorMap mQ, mK, mV, mZ;
+    CUtensorMap mQ, mK, mV, mZ, mO, mOc;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
-        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t))
+        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t) ||
+        !tc_map_rows(&mO, O, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
+    if (Oc != nullptr) {
+        if (!tc_map_f32rows(&mOc, Oc, (int64_t)d.BH() * d.n)) return cudaErrorInvalidValue;
+    } else {
+        mOc = mO;       // never used
+    }
     // keep_states: the backward will read these states, so they are built from centred values
     float* cmean = d.keep_states ? reinterpret_cast<float*>(ws + w.vmean) : nullptr;
     if (cmean != nullptr) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
@@ -737,9 +792,9 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     constexpr size_t smem = OutSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_fwd_out_kernel<R, 0>, smem));
     prof_begin("tc_fwd_out_kernel", s);
-    tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, (bf16*)O, d.sb, d.sh, d.sn,
-        denom, nullptr, nullptr, nullptr, nullptr, Oc, status);
+    tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+        denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -779,9 +834,9 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
     constexpr size_t smem = OutSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_fwd_out_kernel<R, 1>, smem));
     prof_begin("tc_bwd_recompute_kernel", s);
-    tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 128, smem, s>>>(
-        mQ, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, nullptr, d.sb, d.sh, d.sn,
-        const_cast<float*>(denom), dO, E, e65, e65h, nullptr, status);
+    tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+        const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();

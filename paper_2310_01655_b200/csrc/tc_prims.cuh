@@ -71,6 +71,26 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t p
     if (status != nullptr) atomicCAS(status, 0, code);
     return false;
 }
+// Bounded wait by polling only (no suspension): for a lone issuing thread, whose wake-up latency
+// is on the critical path of everything it feeds and whose polling costs no one else issue slots.
+static __device__ __noinline__ bool mbar_spin_slow(uint32_t bar_addr, uint32_t parity, int* status, int code) {
+#pragma unroll 1
+    for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.b32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    if (status != nullptr) atomicCAS(status, 0, code);
+    return false;
+}
+__device__ __forceinline__ bool mbar_spin(uint64_t* bar, uint32_t parity, int* status, int code) {
+    if (mbar_test(bar, parity)) return true;
+    return mbar_spin_slow(smem_u32(bar), parity, status, code);
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code) {
     if (mbar_test(bar, parity)) return true;       // already complete: no suspension round trip
     return mbar_wait_slow(smem_u32(bar), parity, status, code);
@@ -113,6 +133,20 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, int
           "r"(c3)
         : "memory");
 }
+
+// Tiled stores shared -> global (bulk async-group completion).  The issuing thread commits the
+// group and waits until the copies have READ their shared-memory source before it is reused.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, const void* src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------
 // Tensor memory
