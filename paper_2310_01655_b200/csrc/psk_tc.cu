@@ -256,6 +256,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     last = __uint_as_float(v[0]);
                 }
                 const float k1 = center_mode == 1 ? -last : 0.f, k2 = center_mode == 2 ? 1.f : 0.f;
+                // the row's pair weight (tc_features.cuh) goes into the stored state; 0 on padding rows
+                const float wgt = F::weight((T0 + I) * 128 + wt);
                 // this thread's feature row: 80 bf16 = ten 16-byte stores
                 uint4* dst = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + wt) * 80);
 #pragma unroll
@@ -279,12 +281,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                         const float x1 = fmaf(k1, cm[c0 + q + 1], __uint_as_float(v[q + 1]));
                         corr = fmaf(k2 * cm[c0 + q], x0, corr);
                         corr = fmaf(k2 * cm[c0 + q + 1], x1, corr);
-                        pk[q / 2] = pack_bf16(x0, x1);
+                        pk[q / 2] = pack_bf16(x0 * wgt, x1 * wgt);
                     }
                     dst[c0 / 8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     dst[c0 / 8 + 1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
-                dst[8] = make_uint4(pack_bf16(last - corr, 0.f), 0, 0, 0);
+                dst[8] = make_uint4(pack_bf16((last - corr) * wgt, 0.f), 0, 0, 0);
                 dst[9] = make_uint4(0, 0, 0, 0);
             });
         }
@@ -298,10 +300,11 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
             tc_fence_after();
             PackedM<R> pm;
+            CircGen<R> gen;
             {
                 float m[R];
                 read_half_sketch<R>(lane_tm, m);
-                pack_half_sketch<R>(m, pm);
+                if constexpr (F::kCirc) gen.init(m); else pack_half_sketch<R>(m, pm);
             }
             tc_fence_before();
             wg_barrier(wg);
@@ -316,23 +319,48 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 wg_barrier(0);
                 if (wt == 0) mbar_arrive(&bar_ext[j & 1]);
             }
-            static_for<0, TN>([&](auto ic) {
-                constexpr int I = decltype(ic)::value;
-                if (I % NWG == wg) {
+            if constexpr (F::kCirc) {
+                // this warpgroup's tiles wg, wg + NWG, ...: the same loop body on a rotated copy of m
+                static_assert(T0 == 0, "circulant order: one launch covers every tile");
+                constexpr int kTileSteps = 128 / (2 * R);
+                for (int i = 0; i < wg; ++i) gen.template skip<kTileSteps>();
+#pragma unroll 1
+                for (int I = wg; I < TN && ok; I += NWG) {
                     if (a_uses > 0) ok = ok && mbar_wait(&bar_afree[wg], (a_uses - 1) & 1, status, kErrMma);
-                    static_for<0, 16>([&](auto cc) {
-                        constexpr int C = decltype(cc)::value;
-                        uint32_t pk[4];
-                        gen_features<R, (T0 + I) * 128 + C * 8, false, 4>(pm, pk);
-                        *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(wt, C % 8)) =
-                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    });
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t pk[32];
+                        gen.chunk(pk);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            *reinterpret_cast<uint4*>(sA + half * 16384 + swz128_offset(wt, c)) =
+                                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
                     fence_proxy_async_smem();
                     wg_barrier(wg);
                     if (wt == 0) mbar_arrive(&bar_aready[wg]);
                     ++a_uses;
+                    gen.template skip<(NWG - 1) * kTileSteps>();
                 }
-            });
+            } else {
+                static_for<0, TN>([&](auto ic) {
+                    constexpr int I = decltype(ic)::value;
+                    if (I % NWG == wg) {
+                        if (a_uses > 0) ok = ok && mbar_wait(&bar_afree[wg], (a_uses - 1) & 1, status, kErrMma);
+                        static_for<0, 16>([&](auto cc) {
+                            constexpr int C = decltype(cc)::value;
+                            uint32_t pk[4];
+                            gen_features<R, (T0 + I) * 128 + C * 8, 4>(pm, pk);
+                            *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(wt, C % 8)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        });
+                        fence_proxy_async_smem();
+                        wg_barrier(wg);
+                        if (wt == 0) mbar_arrive(&bar_aready[wg]);
+                        ++a_uses;
+                    }
+                });
+            }
         }
     }
     tc_fence_before();
@@ -525,26 +553,45 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         float mq[R];
         read_half_sketch<R>(lane_tm + cSk, mq);
         store_split_rows<R, true>(smem + L::Mq, mq, tid);
-        PackedM<R> pmq;
-        pack_half_sketch<R>(mq, pmq);
 
         if (l > 0) {
-            static_for<0, F::NC>([&](auto cc) {
-                constexpr int C = decltype(cc)::value;
-                constexpr int buf = C % kFeatBufs;
-                if constexpr (C >= kFeatBufs) {       // the MMAs that read this buffer's previous contents
-                    ok = ok && mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
-                    tc_fence_after();
+            if constexpr (F::kCirc) {
+                CircGen<R> gen;
+                gen.init(mq);
+#pragma unroll 1
+                for (int C = 0; C < F::NC && ok; ++C) {
+                    const int buf = C % kFeatBufs;
+                    if (C >= kFeatBufs) {             // the MMAs that read this buffer's previous contents
+                        ok = mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
+                        tc_fence_after();
+                    }
+                    uint32_t pk[32];
+                    gen.chunk(pk);
+                    tmem_st32(lane_tm + cA + buf * 32, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    mbar_arrive(&bar_feat[buf]);
                 }
-                uint32_t pk[16];
-                gen_features<R, C * 64, true, 16>(pmq, pk);
-                tmem_st16(lane_tm + cA + buf * 32, pk);
-                gen_features<R, C * 64 + 32, true, 16>(pmq, pk);
-                tmem_st16(lane_tm + cA + buf * 32 + 16, pk);
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&bar_feat[buf]);
-            });
+            } else {
+                PackedM<R> pmq;
+                pack_half_sketch<R>(mq, pmq);
+                static_for<0, F::NC>([&](auto cc) {
+                    constexpr int C = decltype(cc)::value;
+                    constexpr int buf = C % kFeatBufs;
+                    if constexpr (C >= kFeatBufs) {
+                        ok = ok && mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
+                        tc_fence_after();
+                    }
+                    uint32_t pk[16];
+                    gen_features<R, C * 64, 16>(pmq, pk);
+                    tmem_st16(lane_tm + cA + buf * 32, pk);
+                    gen_features<R, C * 64 + 32, 16>(pmq, pk);
+                    tmem_st16(lane_tm + cA + buf * 32 + 16, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    mbar_arrive(&bar_feat[buf]);
+                });
+            }
         }
 
 #pragma unroll 1

@@ -87,13 +87,9 @@ __device__ __forceinline__ void untensor32(const uint32_t (&x)[32], const float 
         constexpr int f = F0 + J;
         if constexpr (f < Feat<R>::F) {
             constexpr int A = Feat<R>::a(f), B = Feat<R>::b(f);
-            const float v = __uint_as_float(x[J]);
-            if constexpr (A != B) {
-                dm[A] = fmaf(v, m[B], dm[A]);
-                dm[B] = fmaf(v, m[A], dm[B]);
-            } else {
-                dm[A] = fmaf(v, m[A], dm[A]);
-            }
+            const float v = __uint_as_float(x[J]);        // weighted by the state row it came through
+            dm[A] = fmaf(v, m[B], dm[A]);
+            dm[B] = fmaf(v, m[A], dm[B]);
         }
     });
 }
@@ -206,91 +202,143 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     // ---- phase B: other blocks through the state ----
     if (has_state) {
-        PackedM<R> pm;
-        if constexpr (!QSIDE) pack_half_sketch<R>(m, pm);
         constexpr uint32_t idesc_phi = idesc_bf16(128, 64, false, false);
         // Software pipeline over the 64-feature chunks: while the MMAs of chunk C run, the threads
         // generate chunk C+1's features; while those of chunk C+1 run, they un-tensor chunk C.
         // d-phi is double-buffered in [0,128); during this phase the feature staging buffers sit
         // in the dM accumulator's columns, which only phase C uses.
         constexpr uint32_t cFB = cdM;
-        auto stage_features = [&](auto cc) {      // weighted features of chunk C -> tensor memory
-            constexpr int C = decltype(cc)::value;
-            uint32_t pk[16];
-            gen_features<R, C * 64, true, 16>(pm, pk);
-            tmem_st16(lane_tm + cFB + (C & 1) * 32, pk);
-            gen_features<R, C * 64 + 32, true, 16>(pm, pk);
-            tmem_st16(lane_tm + cFB + (C & 1) * 32 + 16, pk);
-            tmem_st_wait();
-        };
-        auto issue_chunk = [&](auto cc) {         // one thread: the chunk's MMAs, then commit
-            constexpr int C = decltype(cc)::value;
-            constexpr int buf = C & 1, stage = C % kStages;
-            constexpr int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+        auto issue_chunk = [&](int C) {           // one thread: the chunk's MMAs, then commit
+            const int buf = C & 1, stage = C % kStages;
+            const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
             const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
+            const uint64_t yd = smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128);
+            const uint64_t bd = smem_desc(box, 0, 1024, kSwz128);
             // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
             // contraction over the 64 state columns, then the last column (second box)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                umma_ss(tm + cPhi + buf * 64, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32),
-                        desc_off(smem_desc(box, 0, 1024, kSwz128), k * 32), idesc_phi, k > 0);
-            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone),
-                    desc_off(smem_desc(box, 0, 1024, kSwz128), 8192), idesc_phi, 1);
+                umma_ss(tm + cPhi + buf * 64, desc_off(yd, k * 32), desc_off(bd, k * 32), idesc_phi, k > 0);
+            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone), desc_off(bd, 8192),
+                    idesc_phi, 1);
             if constexpr (!QSIDE) {
-                // dV += phi_w(k) chunk x box (MN-major B: 16 features per K step)
+                // dV += phi(k) chunk x box (MN-major B: 16 features per K step)
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
-#pragma unroll
+#pragma unroll 1
                 for (int k = 0; k < ksteps; ++k)
-                    umma_ts(tm + cdV, tm + cFB + buf * 32 + k * 8, desc_off(smem_desc(box, 0, 1024, kSwz128), k * 2048), idesc,
-                            (C > 0 || k > 0) ? 1u : 0u);
+                    umma_ts(tm + cdV, tm + cFB + buf * 32 + k * 8, desc_off(bd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
             }
             umma_commit(&bar_phi[buf]);
         };
-        if constexpr (!QSIDE) stage_features(std::integral_constant<int, 0>{});
-        ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            issue_chunk(std::integral_constant<int, 0>{});
-        }
-        static_for<0, F::NC>([&](auto cc) {
-            constexpr int C = decltype(cc)::value;
-            constexpr int buf = C & 1, stage = C % kStages;
-            if constexpr (C + 1 < F::NC) {
-                if constexpr (!QSIDE) stage_features(std::integral_constant<int, C + 1>{});
-                ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
-                tc_fence_before();
-                __syncthreads();           // chunk C-1's d-phi has been read by every thread
-                if (tid == 0) {
-                    tc_fence_after();
-                    issue_chunk(std::integral_constant<int, C + 1>{});
-                }
+        auto refill = [&](int C) {                // chunk C's box is free: load chunk C + kStages into it
+            const int stage = C % kStages;
+            mbar_expect_tx(&bar_box[stage], kBoxBytes);
+            tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
+            tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk, &bar_box[stage]);
+        };
+        if constexpr (F::kCirc) {
+            // every chunk is the same code on rotated copies of m: a loop
+            CircGen<R> gen;
+            CircUntensor<R> ut;
+            if constexpr (!QSIDE) gen.init(m);
+            ut.init(m);
+            auto stage_features = [&](int C) {    // features of the next chunk -> tensor memory
+                uint32_t pk[32];
+                gen.chunk(pk);
+                tmem_st32(lane_tm + cFB + (C & 1) * 32, pk);
+                tmem_st_wait();
+            };
+            if constexpr (!QSIDE) stage_features(0);
+            ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                issue_chunk(0);
             }
-            ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
-            tc_fence_after();
-            // chunk C's box is free (its MMAs have completed): refill it
-            if constexpr (C + kStages < F::NC) {
-                if (tid == 0) {
-                    mbar_expect_tx(&bar_box[stage], kBoxBytes);
-                    tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
-                    tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk,
-                                &bar_box[stage]);
+#pragma unroll 1
+            for (int C = 0; C < F::NC && ok; ++C) {
+                const int buf = C & 1;
+                if (C + 1 < F::NC) {
+                    if constexpr (!QSIDE) stage_features(C + 1);
+                    ok = mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
+                    tc_fence_before();
+                    __syncthreads();           // chunk C-1's d-phi has been read by every thread
+                    if (tid == 0) {
+                        tc_fence_after();
+                        issue_chunk(C + 1);
+                    }
                 }
-            }
-            {
+                ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+                tc_fence_after();
+                if (C + kStages < F::NC && tid == 0) refill(C);
                 uint32_t x[32];
-                tmem_ld32(lane_tm + cPhi + buf * 64, x);
-                tmem_ld_wait();
-                untensor32<R, C * 64>(x, m, dm);
-                tmem_ld32(lane_tm + cPhi + buf * 64 + 32, x);
-                tmem_ld_wait();
-                untensor32<R, C * 64 + 32>(x, m, dm);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    tmem_ld32(lane_tm + cPhi + buf * 64 + h * 32, x);
+                    tmem_ld_wait();
+                    if constexpr (R == 32) {
+                        if (h == 0) ut.even(x, m, dm); else { ut.odd(x, m, dm); ut.advance(); }
+                    } else {
+                        ut.even(x, m, dm);
+                        ut.odd(x + 16, m, dm);
+                        ut.advance();
+                    }
+                }
             }
-        });
+            ut.template finish<F::NC * 64 / (2 * R)>(dm);
+        } else {
+            PackedM<R> pm;
+            if constexpr (!QSIDE) pack_half_sketch<R>(m, pm);
+            auto stage_features = [&](auto cc) {
+                constexpr int C = decltype(cc)::value;
+                uint32_t pk[16];
+                gen_features<R, C * 64, 16>(pm, pk);
+                tmem_st16(lane_tm + cFB + (C & 1) * 32, pk);
+                gen_features<R, C * 64 + 32, 16>(pm, pk);
+                tmem_st16(lane_tm + cFB + (C & 1) * 32 + 16, pk);
+                tmem_st_wait();
+            };
+            if constexpr (!QSIDE) stage_features(std::integral_constant<int, 0>{});
+            ok = ok && mbar_wait(&bar_box[0], 0, status, kErrTma);
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                issue_chunk(0);
+            }
+            static_for<0, F::NC>([&](auto cc) {
+                constexpr int C = decltype(cc)::value;
+                constexpr int buf = C & 1;
+                if constexpr (C + 1 < F::NC) {
+                    if constexpr (!QSIDE) stage_features(std::integral_constant<int, C + 1>{});
+                    ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
+                    tc_fence_before();
+                    __syncthreads();           // chunk C-1's d-phi has been read by every thread
+                    if (tid == 0) {
+                        tc_fence_after();
+                        issue_chunk(C + 1);
+                    }
+                }
+                ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+                tc_fence_after();
+                if constexpr (C + kStages < F::NC) {
+                    if (tid == 0) refill(C);
+                }
+                {
+                    uint32_t x[32];
+                    tmem_ld32(lane_tm + cPhi + buf * 64, x);
+                    tmem_ld_wait();
+                    untensor32<R, C * 64>(x, m, dm);
+                    tmem_ld32(lane_tm + cPhi + buf * 64 + 32, x);
+                    tmem_ld_wait();
+                    untensor32<R, C * 64 + 32>(x, m, dm);
+                }
+            });
+        }
         if constexpr (!QSIDE) dv_started = true;
 #pragma unroll
-        for (int c = 0; c < R; ++c) dm[c] *= 2.f * inv_own;
+        for (int c = 0; c < R; ++c) dm[c] *= inv_own;
         tc_fence_before();
         __syncthreads();                   // boxes and the scratch columns are dead: phase C reuses them
         tc_fence_after();
