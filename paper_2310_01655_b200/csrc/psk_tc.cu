@@ -379,7 +379,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
 // ---------------------------------------------------------------------------
 constexpr int kZStages = 4;                     // three in the shared region + the query tile's buffer
 constexpr uint32_t kZStageBytes = 16384;        // two [64 features x 128 B] boxes: columns 0..63, 64..79
-constexpr int kFeatBufs = 4;                    // feature staging buffers in tensor memory, 32 columns each
+constexpr int kFeatBufs = kZStages;             // feature staging buffers in tensor memory, 32 columns each:
+                                                // chunk C uses buffer and stage C % 4, both freed by its MMAs
 
 template <int R>
 struct OutSmem {
@@ -481,32 +482,41 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step,
                 // the second 64-column group (columns 64..79) 8192 B further on
                 constexpr uint32_t idesc = idesc_bf16(128, 80, false, true);
+                // Everything the loop needs is in registers before it waits: between "features
+                // staged" and "MMAs issued" lie the four MMA instructions and nothing else.  (The
+                // stages are refilled by the rows' side, which learns first that a buffer is free.)
+                uint64_t zd[kZStages];
+#pragma unroll
+                for (int s = 0; s < kZStages; ++s) zd[s] = smem_desc(smem_u32(smem + L::zstage(s)), 8192, 1024, kSwz128);
 #pragma unroll 1
-                for (int C = 0; C < F::NC && ok; ++C) {
-                    const int buf = C % kFeatBufs, stage = C % kZStages;
-                    ok = mbar_spin(&bar_z[stage], (C / kZStages) & 1, status, kErrTma);
-                    ok = ok && mbar_spin(&bar_feat[buf], (C / kFeatBufs) & 1, status, kErrMma);
-                    tc_fence_after();
-                    const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
-                    const uint64_t zd = smem_desc(smem_u32(smem + L::zstage(stage)), 8192, 1024, kSwz128);
-#pragma unroll 1
-                    for (int k = 0; k < ksteps; ++k)
-                        umma_ts(tm + cO, tm + cA + buf * 32 + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&bar_a[buf]);
-                    // chunk C-1 is done with its stage: refill it with chunk C-1+kZStages
-                    if (C >= 1 && C - 1 + kZStages < F::NC) {
-                        const int pc = C - 1, ps = pc % kZStages;
-                        ok = ok && mbar_spin(&bar_a[pc % kFeatBufs], (pc / kFeatBufs) & 1, status, kErrMma);
-                        mbar_expect_tx(&bar_z[ps], kZStageBytes);
-                        tma_load_3d(smem + L::zstage(ps), &mapZ, 0, (pc + kZStages) * 64, blk, &bar_z[ps]);
-                        tma_load_3d(smem + L::zstage(ps) + 8192, &mapZ, 64, (pc + kZStages) * 64, blk, &bar_z[ps]);
+                for (int C0 = 0; C0 < F::NC && ok; C0 += kZStages) {
+#pragma unroll
+                    for (int s = 0; s < kZStages; ++s) {
+                        const int C = C0 + s;
+                        if (C < F::NC && ok) {
+                            const uint32_t par = (C0 / kZStages) & 1;
+                            const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+                            ok = mbar_spin(&bar_z[s], par, status, kErrTma);
+                            ok = ok && mbar_spin(&bar_feat[s], par, status, kErrMma);
+                            tc_fence_after();
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                if (k < ksteps)
+                                    umma_ts(tm + cO, tm + cA + s * 32 + k * 8, desc_off(zd[s], k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
+                            umma_commit(&bar_a[s]);
+                        }
                     }
                 }
                 // the key/value tiles reuse the stages' memory and the sketch reuses the staging
                 // columns: every MMA of the first phase must have completed
                 ok = ok && mbar_spin(&bar_a[(F::NC - 1) % kFeatBufs], ((F::NC - 1) / kFeatBufs) & 1, status, kErrMma);
             }
-            // same block: key tiles tp <= tau through squared half-sketch scores
+            // same block: key tiles tp <= tau through squared half-sketch scores; descriptors and
+            // addresses are loop invariants, so every issue sequence below is MMA instructions only
+            const uint64_t qd = smem_desc(smem_u32(smem + L::Mq), 2048, 128, kSwzNone);
+            const uint64_t kd = smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone);
+            const uint64_t vd = smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128);
+            const uint64_t od = smem_desc(smem_u32(smem + L::Ones), 256, 128, kSwzNone);
 #pragma unroll 1
             for (int tp = 0; tp <= tau && ok; ++tp) {
                 if (tp > 0) ok = mbar_spin(&bar_pv, (tp - 1) & 1, status, kErrMma);   // K, V, Mk, weights are free
@@ -521,9 +531,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 tc_fence_after();
                 {
                     constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
-                    const uint64_t qd = smem_desc(smem_u32(smem + L::Mq), 2048, 128, kSwzNone);
-                    const uint64_t kd = smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone);
-#pragma unroll 1
+#pragma unroll
                     for (int k = 0; k < 3 * R / 16; ++k)
                         umma_ss(tm + cS, desc_off(qd, k * 4096), desc_off(kd, k * 4096), idesc, k > 0);
                     umma_commit(&bar_s);
@@ -534,12 +542,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     // numerator += W V; row sums += W 1 (the weights exactly as the value GEMM sees them)
                     constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
                     constexpr uint32_t idesc1 = idesc_bf16(128, 16, false, false);
-                    const uint64_t vd = smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128);
-                    const uint64_t od = smem_desc(smem_u32(smem + L::Ones), 256, 128, kSwzNone);
-#pragma unroll 1
+                    const uint32_t acc0 = (l > 0 || tp > 0) ? 1u : 0u, acc1 = tp > 0 ? 1u : 0u;
+#pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        umma_ts(tm + cO, tm + cW + k * 8, desc_off(vd, k * 2048), idesc, (l > 0 || tp > 0 || k > 0) ? 1u : 0u);
-                        umma_ts(tm + cN, tm + cW + k * 8, desc_off(od, k * 512), idesc1, (tp > 0 || k > 0) ? 1u : 0u);
+                        umma_ts(tm + cO, tm + cW + k * 8, desc_off(vd, k * 2048), idesc, k > 0 ? 1u : acc0);
+                        umma_ts(tm + cN, tm + cW + k * 8, desc_off(od, k * 512), idesc1, k > 0 ? 1u : acc1);
                     }
                     umma_commit(&bar_pv);
                 }
@@ -564,6 +571,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     if (C >= kFeatBufs) {             // the MMAs that read this buffer's previous contents
                         ok = mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
                         tc_fence_after();
+                        if (tid == 0) {               // ... and this stage's: refill it with chunk C's rows
+                            mbar_expect_tx(&bar_z[buf], kZStageBytes);
+                            tma_load_3d(smem + L::zstage(buf), &mapZ, 0, C * 64, blk, &bar_z[buf]);
+                            tma_load_3d(smem + L::zstage(buf) + 8192, &mapZ, 64, C * 64, blk, &bar_z[buf]);
+                        }
                     }
                     uint32_t pk[32];
                     gen.chunk(pk);
@@ -581,6 +593,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     if constexpr (C >= kFeatBufs) {
                         ok = ok && mbar_wait(&bar_a[buf], (C / kFeatBufs - 1) & 1, status, kErrMma);
                         tc_fence_after();
+                        if (tid == 0) {
+                            mbar_expect_tx(&bar_z[buf], kZStageBytes);
+                            tma_load_3d(smem + L::zstage(buf), &mapZ, 0, C * 64, blk, &bar_z[buf]);
+                            tma_load_3d(smem + L::zstage(buf) + 8192, &mapZ, 64, C * 64, blk, &bar_z[buf]);
+                        }
                     }
                     uint32_t pk[16];
                     gen_features<R, C * 64, 16>(pmq, pk);
