@@ -401,7 +401,6 @@ struct OutSmem {
     __device__ static uint32_t zstage(int s) { return s < kZStages - 1 ? Z + s * kZStageBytes : Q; }
 };
 
-__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // MODE 0: forward (writes O, denom, optionally O - c in fp32).  MODE 1: the backward's
 // recomputation of the row numerators against centred prefix states; writes E = dO/d (bf16),
@@ -420,7 +419,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     using L = OutSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_q, bar_kv, bar_sk, bar_mk, bar_s, bar_p, bar_pv;
+    __shared__ uint64_t bar_q, bar_kv, bar_sk, bar_go, bar_mk, bar_s, bar_p, bar_pv;
     __shared__ uint64_t bar_z[kZStages], bar_feat[kFeatBufs], bar_a[kFeatBufs];
     __shared__ uint32_t tmem_slot;
     __shared__ float cm[64];
@@ -432,7 +431,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
     if (tid == 0) {
         mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_sk, 1); mbar_init(&bar_s, 1); mbar_init(&bar_pv, 1);
-        mbar_init(&bar_mk, 128); mbar_init(&bar_p, 128);
+        mbar_init(&bar_mk, 128); mbar_init(&bar_p, 128); mbar_init(&bar_go, 128);
         for (int s = 0; s < kZStages; ++s) mbar_init(&bar_z[s], 1);
         for (int s = 0; s < kFeatBufs; ++s) { mbar_init(&bar_feat[s], 128); mbar_init(&bar_a[s], 1); }
         mbar_fence_init();
@@ -517,6 +516,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             const uint64_t kd = smem_desc(smem_u32(smem + L::Mk), 2048, 128, kSwzNone);
             const uint64_t vd = smem_desc(smem_u32(smem + L::V), 0, 1024, kSwz128);
             const uint64_t od = smem_desc(smem_u32(smem + L::Ones), 256, 128, kSwzNone);
+            // every row has read the query sketch (the first key sketch overwrites its columns, and
+            // bar_sk must not complete a second time before its slowest waiter has seen the first)
+            ok = ok && mbar_spin(&bar_go, 0, status, kErrMma);
 #pragma unroll 1
             for (int tp = 0; tp <= tau && ok; ++tp) {
                 if (tp > 0) ok = mbar_spin(&bar_pv, (tp - 1) & 1, status, kErrMma);   // K, V, Mk, weights are free
@@ -560,6 +562,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         float mq[R];
         read_half_sketch<R>(lane_tm + cSk, mq);
         store_split_rows<R, true>(smem + L::Mq, mq, tid);
+        tc_fence_before();
+        mbar_arrive(&bar_go);
 
         if (l > 0) {
             if constexpr (F::kCirc) {

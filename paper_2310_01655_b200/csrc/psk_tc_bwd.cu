@@ -60,7 +60,7 @@ tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom,
     }
 }
 
-constexpr int kStages = 3;
+constexpr int kStages = 4;
 constexpr uint32_t kBoxBytes = 16384;      // two [64 features x 128 B] boxes: state columns 0..63, 64..79
 
 template <int R>
@@ -69,15 +69,28 @@ struct BwdSmem {
     static constexpr uint32_t kM = HiLoTiles<R>::N * 16384;      // [hi | lo] half-sketch operand
     static constexpr uint32_t Xown = 0, Yown = 16384;
     static constexpr uint32_t G = 32768;
-    static constexpr uint32_t ExtA = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);   // [128 x 16] un-swizzled
-    static constexpr uint32_t Eoth = ExtA + 4096;        // 128 floats: other side's 65th column
-    static constexpr uint32_t U = Eoth + 1024;           // phase B: state boxes; phase C: the tiles below
-    static constexpr uint32_t Box = U;
-    static constexpr uint32_t Xoth = U, Yoth = U + 16384, Moth = U + 32768, Mown = Moth + kM;
-    static constexpr uint32_t kPhaseB = kStages * ((kBoxBytes + 1023) / 1024 * 1024), kPhaseC = 32768 + 2 * kM;
-    static constexpr uint32_t total = U + (kPhaseB > kPhaseC ? kPhaseB : kPhaseC);
+    static constexpr uint32_t ExtA = G + GImage<R>::bytes;       // [128 x 16] un-swizzled
+    static constexpr uint32_t Eoth = ExtA + 4096;        // 128 x (1/d, e65h) of the other side's rows
+    static constexpr uint32_t U = Eoth + 1024;
+    static constexpr uint32_t Box = U;                   // phase B: kStages state boxes
+    static constexpr int NC = Feat<R>::NC;
+    // Phase C tiles.  r <= 32 (two CTAs per SM): they reuse the boxes' memory, each tile in the
+    // stage that the last chunks free first, so the first other-side tile is fetched while the
+    // last chunks are still being processed.  r = 64 (one CTA per SM): memory of their own.
+    static constexpr bool kAlias = (R <= 32);
+    static constexpr int sX = NC >= 4 ? (NC - 4) % 4 : 3, sY = NC >= 4 ? (NC - 3) % 4 : 0;
+    static constexpr int sMo = NC >= 4 ? (NC - 2) % 4 : 1, sMn = NC >= 4 ? (NC - 1) % 4 : 2;
+    static constexpr uint32_t C0 = U + kStages * kBoxBytes;
+    static constexpr uint32_t Xoth = kAlias ? U + sX * kBoxBytes : C0;
+    static constexpr uint32_t Yoth = kAlias ? U + sY * kBoxBytes : C0 + 16384;
+    static constexpr uint32_t Moth = kAlias ? U + sMo * kBoxBytes : C0 + 32768;
+    static constexpr uint32_t Mown = kAlias ? U + sMn * kBoxBytes : C0 + 32768 + kM;
+    static_assert(!kAlias || kM == kBoxBytes, "aliased layout: one tile per stage");
+    static constexpr uint32_t total = kAlias ? C0 : C0 + 32768 + 2 * kM;
+    // output staging (epilogue): dX, dV tiles
+    static constexpr uint32_t Sx = U, Sv = U + 16384;
 };
-constexpr uint32_t kBoxStride = (kBoxBytes + 1023) / 1024 * 1024;
+constexpr uint32_t kBoxStride = kBoxBytes;
 
 // dm += (d feature) * (the other factor) for the 32 features F0 .. F0+31 held in x
 template <int R, int F0>
@@ -115,15 +128,16 @@ template <int R, bool QSIDE>
 __global__ void __launch_bounds__(128, (R <= 32 ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
-                   const __grid_constant__ CUtensorMap mapS, const uint8_t* __restrict__ gimg,
+                   const __grid_constant__ CUtensorMap mapS, const __grid_constant__ CUtensorMap mapDX,
+                   const __grid_constant__ CUtensorMap mapDV, const uint8_t* __restrict__ gimg,
                    int g_heads, int H, int n, int b, int t,
                    const float* __restrict__ e65, const float* __restrict__ e65h, const float* __restrict__ denom,
-                   bf16* __restrict__ dX, bf16* __restrict__ dV, int64_t sb, int64_t sh, int64_t sn, int* status) {
+                   int* status) {
     using F = Feat<R>;
     using L = BwdSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_own, bar_oth, bar_mma, bar_phi[2], bar_box[kStages];
+    __shared__ uint64_t bar_own, bar_xoth, bar_yoth, bar_mma, bar_phi[2], bar_box[kStages];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
@@ -134,7 +148,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const bool has_state = QSIDE ? (l > 0) : (l < t - 1);
 
     if (tid == 0) {
-        mbar_init(&bar_own, 1); mbar_init(&bar_oth, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_own, 1); mbar_init(&bar_xoth, 1); mbar_init(&bar_yoth, 1); mbar_init(&bar_mma, 1);
         mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
         for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
         mbar_fence_init();
@@ -150,6 +164,16 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 tma_load_3d(smem + L::Box + c * kBoxStride, &mapS, 0, c * 64, blk, &bar_box[c]);
                 tma_load_3d(smem + L::Box + c * kBoxStride + 8192, &mapS, 64, c * 64, blk, &bar_box[c]);
             }
+        }
+        // first other-side tile: at once where its memory is free from the start
+        const int orow_first = l * b + (QSIDE ? 0 : tau) * 128;
+        if (!has_state || !L::kAlias || F::NC < kStages) {
+            mbar_expect_tx(&bar_xoth, 16384);
+            tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow_first, hi, bi, &bar_xoth);
+        }
+        if (!has_state || !L::kAlias) {
+            mbar_expect_tx(&bar_yoth, 16384);
+            tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow_first, hi, bi, &bar_yoth);
         }
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
@@ -208,33 +232,48 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         // d-phi is double-buffered in [0,128); during this phase the feature staging buffers sit
         // in the dM accumulator's columns, which only phase C uses.
         constexpr uint32_t cFB = cdM;
+        // descriptors are loop invariants: an issue sequence is its MMA instructions and little else
+        const uint64_t yd = smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128);
+        const uint64_t ed = smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone);
+        const uint64_t bd0 = smem_desc(smem_u32(smem + L::Box), 0, 1024, kSwz128);
         auto issue_chunk = [&](int C) {           // one thread: the chunk's MMAs, then commit
             const int buf = C & 1, stage = C % kStages;
             const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
-            const uint32_t box = smem_u32(smem + L::Box + stage * kBoxStride);
-            const uint64_t yd = smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128);
-            const uint64_t bd = smem_desc(box, 0, 1024, kSwz128);
+            const uint64_t bd = desc_off(bd0, stage * kBoxStride);
+            const uint32_t dphi = tm + cPhi + buf * 64;
             // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
             // contraction over the 64 state columns, then the last column (second box)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_ss(tm + cPhi + buf * 64, desc_off(yd, k * 32), desc_off(bd, k * 32), idesc_phi, k > 0);
-            umma_ss(tm + cPhi + buf * 64, smem_desc(smem_u32(smem + L::ExtA), 2048, 128, kSwzNone), desc_off(bd, 8192),
-                    idesc_phi, 1);
+            for (int k = 0; k < 4; ++k) umma_ss(dphi, desc_off(yd, k * 32), desc_off(bd, k * 32), idesc_phi, k > 0);
+            umma_ss(dphi, ed, desc_off(bd, 8192), idesc_phi, 1);
             if constexpr (!QSIDE) {
                 // dV += phi(k) chunk x box (MN-major B: 16 features per K step)
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
-#pragma unroll 1
-                for (int k = 0; k < ksteps; ++k)
-                    umma_ts(tm + cdV, tm + cFB + buf * 32 + k * 8, desc_off(bd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
+                const uint32_t fb = tm + cFB + buf * 32;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (k < ksteps) umma_ts(tm + cdV, fb + k * 8, desc_off(bd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
             }
             umma_commit(&bar_phi[buf]);
         };
-        auto refill = [&](int C) {                // chunk C's box is free: load chunk C + kStages into it
-            const int stage = C % kStages;
-            mbar_expect_tx(&bar_box[stage], kBoxBytes);
-            tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
-            tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk, &bar_box[stage]);
+        auto refill = [&](int C) {                // tid 0: chunk C's box is free
+            if (C + kStages < F::NC) {
+                const int stage = C % kStages;
+                mbar_expect_tx(&bar_box[stage], kBoxBytes);
+                tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
+                tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk, &bar_box[stage]);
+            } else if (L::kAlias) {
+                // the last chunks free the stages that the first other-side tile goes into
+                const int orow_first = l * b + (QSIDE ? 0 : tau) * 128;
+                if (F::NC >= kStages && C == F::NC - 4) {
+                    mbar_expect_tx(&bar_xoth, 16384);
+                    tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow_first, hi, bi, &bar_xoth);
+                }
+                if (C == (F::NC >= kStages ? F::NC - 3 : 0)) {
+                    mbar_expect_tx(&bar_yoth, 16384);
+                    tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow_first, hi, bi, &bar_yoth);
+                }
+            }
         };
         if constexpr (F::kCirc) {
             // every chunk is the same code on rotated copies of m: a loop
@@ -271,7 +310,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 }
                 ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
                 tc_fence_after();
-                if (C + kStages < F::NC && tid == 0) refill(C);
+                if (tid == 0) refill(C);
                 uint32_t x[32];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -322,9 +361,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 }
                 ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
                 tc_fence_after();
-                if constexpr (C + kStages < F::NC) {
-                    if (tid == 0) refill(C);
-                }
+                if (tid == 0) refill(C);
                 {
                     uint32_t x[32];
                     tmem_ld32(lane_tm + cPhi + buf * 64, x);
@@ -354,17 +391,13 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll 1
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
-        if (tid == 0) {
-            mbar_expect_tx(&bar_oth, 32768);
-            tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0, hi, bi, &bar_oth);
-            tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0, hi, bi, &bar_oth);
-        }
+        // (this tile's rows were requested ahead: by the prologue, by phase B's last chunks, or
+        // by the previous tile as soon as its own copies had been consumed)
         if constexpr (!QSIDE) {
             // e65h is already -(g . O) / d
             oth_col[tid] = make_float2(1.f / denom[(size_t)bh * n + orow0 + tid], e65h[(size_t)bh * n + orow0 + tid]);
         }
-        ok = mbar_wait(&bar_oth, oth_uses & 1, status, kErrTma);
-        ++oth_uses;
+        ok = mbar_wait(&bar_xoth, oth_uses & 1, status, kErrTma);
         if (tid == 0) {
             tc_fence_after();
             issue_sketch<R>(tm + cSk, smem + L::Xoth, smem + L::G);
@@ -373,6 +406,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
         ++mma_uses;
         tc_fence_after();
+        ok = ok && mbar_wait(&bar_yoth, oth_uses & 1, status, kErrTma);
+        ++oth_uses;
         {
             float mo[R];
             read_half_sketch<R>(lane_tm + cSk, mo);
@@ -386,6 +421,13 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
+                // The X tile has been consumed, and every thread is past its wait for it (a
+                // barrier must not complete twice before its slowest waiter has looked): next
+                // tile's rows.
+                if (hh == 0 && tp + 1 < tp_end) {
+                    mbar_expect_tx(&bar_xoth, 16384);
+                    tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
+                }
                 issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
 #pragma unroll
@@ -459,6 +501,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             ++mma_uses;
             tc_fence_after();
         }
+        if (tid == 0 && tp + 1 < tp_end) {        // every MMA that read the Y tile has completed
+            mbar_expect_tx(&bar_yoth, 16384);
+            tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0 + 128, hi, bi, &bar_yoth);
+        }
     }
 
     // ---- phase D: through the sketch, dX = ((dM*A2) G1^T + (dM*A1) G2^T) / sqrt(R) ----
@@ -518,8 +564,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         ++mma_uses;
         tc_fence_after();
     }
+    // rows go out through shared memory and tiled stores (every MMA has completed: the other-side
+    // tiles' memory is free); a thread-per-row store pattern would keep the load/store unit busy
+    // for thousands of cycles
     if (ok) {
-        const int64_t o = (int64_t)bi * sb + (int64_t)hi * sh + (int64_t)(row0 + tid) * sn;
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
             uint32_t v[32];
@@ -527,7 +575,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; j += 8)
-                *reinterpret_cast<uint4*>(dX + o + c0 + j) =
+                *reinterpret_cast<uint4*>(smem + L::Sx + swz128_offset(tid, (c0 + j) / 8)) =
                     make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
                                pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
                                pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
@@ -541,13 +589,22 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; j += 8)
-                    *reinterpret_cast<uint4*>(dV + o + c0 + j) =
+                    *reinterpret_cast<uint4*>(smem + L::Sv + swz128_offset(tid, (c0 + j) / 8)) =
                         make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
                                    pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
                                    pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
                                    pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
             }
         }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && ok) {
+        tma_store_4d(&mapDX, smem + L::Sx, 0, row0, hi, bi);
+        if constexpr (!QSIDE) tma_store_4d(&mapDV, smem + L::Sv, 0, row0, hi, bi);
+        bulk_commit();
+        bulk_wait_read();
     }
     tc_fence_before();
     __syncthreads();
@@ -567,13 +624,15 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     float* cmean = reinterpret_cast<float*>(ws + w.vmean);
     float* e65h = reinterpret_cast<float*>(ws + w.e65h);
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
-    CUtensorMap mQ, mK, mV, mE, mG, mZ, mR;
+    CUtensorMap mQ, mK, mV, mE, mG, mZ, mR, mdQ, mdK, mdV;
     const int64_t nblk = (int64_t)d.BH() * d.t;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mE, E, d.B, d.H, d.n, (int64_t)d.H * d.n * 64, (int64_t)d.n * 64, 64) ||
         !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
-        !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk))
+        !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk) ||
+        !tc_map_rows(&mdQ, dQ, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mdK, dK, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_rows(&mdV, dV, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
@@ -597,12 +656,12 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
     prof_begin("tc_bwd_q_kernel", s);
-    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                        e65h, denom, (bf16*)dQ, nullptr, d.sb, d.sh, d.sn, status);
+    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n, d.b, d.t,
+                                                        e65, e65h, denom, status);
     prof_end(s);
     prof_begin("tc_bwd_k_kernel", s);
-    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, gimg, d.g_heads, d.H, d.n, d.b, d.t, e65,
-                                                         e65h, denom, (bf16*)dK, (bf16*)dV, d.sb, d.sh, d.sn, status);
+    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n, d.b, d.t,
+                                                         e65, e65h, denom, status);
     prof_end(s);
     *launches += 2;
     return cudaGetLastError();

@@ -74,6 +74,10 @@ __device__ __forceinline__ void static_for(Fn&& f) {
 
 constexpr int kErrTma = 1, kErrMma = 2;
 
+// barrier among the 128 row threads (warps 0-3) of a kernel whose fifth warp issues the MMAs;
+// only where every row thread is certain to arrive (never inside a loop a failed wait can leave)
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
     return p + ((1024u - (smem_u32(p) & 1023u)) & 1023u);
 }
