@@ -484,27 +484,22 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 // Everything the loop needs is in registers before it waits: between "features
                 // staged" and "MMAs issued" lie the four MMA instructions and nothing else.  (The
                 // stages are refilled by the rows' side, which learns first that a buffer is free.)
-                uint64_t zd[kZStages];
-#pragma unroll
-                for (int s = 0; s < kZStages; ++s) zd[s] = smem_desc(smem_u32(smem + L::zstage(s)), 8192, 1024, kSwz128);
+                const uint64_t zd0 = smem_desc(smem_u32(smem + L::Z), 8192, 1024, kSwz128);
+                const uint64_t zdq = smem_desc(smem_u32(smem + L::Q), 8192, 1024, kSwz128);
 #pragma unroll 1
-                for (int C0 = 0; C0 < F::NC && ok; C0 += kZStages) {
+                for (int C = 0; C < F::NC && ok; ++C) {
+                    const int s = C % kZStages;
+                    const uint32_t par = (C / kZStages) & 1;
+                    const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+                    const uint64_t zd = s == kZStages - 1 ? zdq : desc_off(zd0, s * kZStageBytes);
+                    const uint32_t at = tm + cA + s * 32;
+                    ok = mbar_spin(&bar_z[s], par, status, kErrTma);
+                    ok = ok && mbar_spin(&bar_feat[s], par, status, kErrMma);
+                    tc_fence_after();
 #pragma unroll
-                    for (int s = 0; s < kZStages; ++s) {
-                        const int C = C0 + s;
-                        if (C < F::NC && ok) {
-                            const uint32_t par = (C0 / kZStages) & 1;
-                            const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
-                            ok = mbar_spin(&bar_z[s], par, status, kErrTma);
-                            ok = ok && mbar_spin(&bar_feat[s], par, status, kErrMma);
-                            tc_fence_after();
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                if (k < ksteps)
-                                    umma_ts(tm + cO, tm + cA + s * 32 + k * 8, desc_off(zd[s], k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
-                            umma_commit(&bar_a[s]);
-                        }
-                    }
+                    for (int k = 0; k < 4; ++k)
+                        if (k < ksteps) umma_ts(tm + cO, at + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&bar_a[s]);
                 }
                 // the key/value tiles reuse the stages' memory and the sketch reuses the staging
                 // columns: every MMA of the first phase must have completed
@@ -631,24 +626,27 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tc_fence_after();
             // weights = squared scores (lower triangle on the diagonal tile), packed to bf16 over
             // columns whose fp32 contents have already been read
-            auto weights = [&](auto diag_c) {
-                constexpr bool DIAG = decltype(diag_c)::value;
+            // (one loop over the four 32-key groups.  On the diagonal tile a warp's rows
+            // 32 w .. 32 w + 31 see group g < w whole, group g > w not at all, and only group
+            // g == w through the triangular mask: the mask code runs for one group in four.)
+            const int gdiag = (tp == tau) ? warp : 4;
+#pragma unroll 1
+            for (int gq = 0; gq < 4; ++gq) {
+                uint32_t v[32], pk[16];
+                tmem_ld32(lane_tm + cS + gq * 32, v);
+                tmem_ld_wait();
+                if (gq >= gdiag) {
+                    const int lim = gq > gdiag ? -1 : (tid & 31);       // keep keys j <= lim of this group
 #pragma unroll
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t v[32], pk[16];
-                    tmem_ld32(lane_tm + cS + c0, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
-                        w0 = (DIAG && c0 + j > tid) ? 0.f : w0 * w0;
-                        w1 = (DIAG && c0 + j + 1 > tid) ? 0.f : w1 * w1;
-                        pk[j / 2] = pack_bf16(w0, w1);
-                    }
-                    tmem_st16(lane_tm + cW + c0 / 2, pk);
+                    for (int j = 0; j < 32; ++j) v[j] = j > lim ? 0u : v[j];
                 }
-            };
-            if (tp == tau) weights(std::true_type{}); else weights(std::false_type{});
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
+                    pk[j / 2] = pack_bf16(w0 * w0, w1 * w1);
+                }
+                tmem_st16(lane_tm + cW + gq * 16, pk);
+            }
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&bar_p);
