@@ -103,7 +103,9 @@ struct StateSmem {
     static constexpr uint32_t kYSlot = 32768;
     static constexpr uint32_t G = Y + 2 * kYSlot;
     static constexpr uint32_t A0 = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t total = A0 + NWG * 32768;
+    static constexpr uint32_t St = A0 + NWG * 32768;     // one state tile on its way out: 128 rows x 160 B
+    static constexpr bool kStaged = St + 128 * 160 + 2048 <= 232448;     // where it fits (r <= 32)
+    static constexpr uint32_t total = St + (kStaged ? 128 * 160 : 0);
 };
 
 __device__ __forceinline__ void wg_barrier(int wg) {
@@ -125,7 +127,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread;
     __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull, bar_accread[TN];
     __shared__ uint32_t tmem_slot;
-    __shared__ float cm[64];
+    __shared__ __align__(16) float cm[64];
     const int tid = threadIdx.x, wg = tid / 128, wt = tid % 128, warp = tid / 32;
     const int bh = blockIdx.x;
     const int hi = bh % H, bi = bh / H;
@@ -189,6 +191,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             uint32_t a_cnt[NWG];
 #pragma unroll
             for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
+            // This one thread feeds the tensor pipe for the whole CTA: whatever it executes between
+            // two MMAs is time the pipe idles.  Descriptors are built once, here.
+            uint64_t ad[NWG];
+#pragma unroll
+            for (int i = 0; i < NWG; ++i) ad[i] = smem_desc(smem_u32(smem + L::A0 + i * 32768), 16384, 1024, kSwz128);
+            const uint64_t yd0 = smem_desc(smem_u32(smem + L::Y), 16384, 1024, kSwz128);
             for (int j = 0; j < NJ && ok; ++j) {
                 // sketch of the next token tile, as soon as this tile's half sketches are read out
                 if (j + 1 < NJ) {
@@ -202,20 +210,19 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 ok = ok && mbar_wait(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
                 if (y65 != nullptr) ok = ok && mbar_wait(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
                 const bool boundary = (j % tpb == 0) && j > 0;
-                const uint32_t yb = smem_u32(smem + L::Y + (j & 1) * L::kYSlot);
+                const uint64_t yd = desc_off(yd0, (j & 1) * L::kYSlot);
+                const uint32_t acc0 = j > 0 ? 1u : 0u;
                 static_for<0, TN>([&](auto ic) {
                     constexpr int I = decltype(ic)::value;
                     constexpr int w = I % NWG;
                     // the store warpgroup has taken this accumulator's values for the boundary
-                    if (boundary) ok = ok && mbar_wait(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
-                    ok = ok && mbar_wait(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
+                    if (boundary) ok = ok && mbar_spin(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
+                    ok = ok && mbar_spin(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
                     ++a_cnt[w];
                     tc_fence_after();
-                    const uint32_t ab = smem_u32(smem + L::A0 + w * 32768);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        umma_ss(tm + kAcc + 80 * I, desc_off(smem_desc(ab, 16384, 1024, kSwz128), k * 2048),
-                                desc_off(smem_desc(yb, 16384, 1024, kSwz128), k * 2048), idesc_state, (j > 0 || k > 0) ? 1u : 0u);
+                        umma_ss(tm + kAcc + 80 * I, desc_off(ad[w], k * 2048), desc_off(yd, k * 2048), idesc_state, k > 0 ? 1u : acc0);
                     umma_commit(&bar_afree[w]);
                     if constexpr (I == 0) {
                         // values of the next token tile: their slot held tile j-1, whose MMAs were
@@ -235,7 +242,13 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         }
     } else if (wg == NWG) {
         // ============================ store warpgroup ============================
+        // Tiles leave through shared memory: a warp's 32 rows of 160 B are one contiguous 5 KB
+        // piece of the state array, which the warp writes out in ten 512-byte rows of lanes.
+        // (Rows stored by their threads directly would be 10 scattered 16-byte stores each: the L1
+        // data path, which the MMA operands and the generators' tiles also go through, is this
+        // kernel's busiest unit.)
         const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
+        uint8_t* stage = smem + L::St;
         bool ok = true;
         for (int p = 0; p < t && ok; ++p) {
             const int l = reverse ? (t - 1 - p) : p;
@@ -258,8 +271,10 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 const float k1 = center_mode == 1 ? -last : 0.f, k2 = center_mode == 2 ? 1.f : 0.f;
                 // the row's pair weight (tc_features.cuh) goes into the stored state; 0 on padding rows
                 const float wgt = F::weight((T0 + I) * 128 + wt);
-                // this thread's feature row: 80 bf16 = ten 16-byte stores
-                uint4* dst = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + wt) * 80);
+                // this thread's feature row: 80 bf16 = ten 16-byte pieces of the staging tile
+                if constexpr (L::kStaged) __syncwarp();       // the previous tile has been read back
+                uint4* const grow = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + wt) * 80);
+                uint4* dst = L::kStaged ? reinterpret_cast<uint4*>(stage + wt * 160) : grow;
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 16) {
                     uint32_t v[16];
@@ -275,12 +290,18 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                         for (int q = 0; q < 16; ++q) v[q] = 0u;
                     }
                     uint32_t pk[8];
+                    float cv[16];
+#pragma unroll
+                    for (int q = 0; q < 16; q += 4) {
+                        const float4 c4 = *reinterpret_cast<const float4*>(&cm[c0 + q]);
+                        cv[q] = c4.x; cv[q + 1] = c4.y; cv[q + 2] = c4.z; cv[q + 3] = c4.w;
+                    }
 #pragma unroll
                     for (int q = 0; q < 16; q += 2) {
-                        const float x0 = fmaf(k1, cm[c0 + q], __uint_as_float(v[q]));
-                        const float x1 = fmaf(k1, cm[c0 + q + 1], __uint_as_float(v[q + 1]));
-                        corr = fmaf(k2 * cm[c0 + q], x0, corr);
-                        corr = fmaf(k2 * cm[c0 + q + 1], x1, corr);
+                        const float x0 = fmaf(k1, cv[q], __uint_as_float(v[q]));
+                        const float x1 = fmaf(k1, cv[q + 1], __uint_as_float(v[q + 1]));
+                        corr = fmaf(k2 * cv[q], x0, corr);
+                        corr = fmaf(k2 * cv[q + 1], x1, corr);
                         pk[q / 2] = pack_bf16(x0 * wgt, x1 * wgt);
                     }
                     dst[c0 / 8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -288,6 +309,14 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 }
                 dst[8] = make_uint4(pack_bf16((last - corr) * wgt, 0.f), 0, 0, 0);
                 dst[9] = make_uint4(0, 0, 0, 0);
+                if constexpr (L::kStaged) {
+                    __syncwarp();
+                    const int w32 = wt & ~31, lane = wt & 31;
+                    const uint4* src = reinterpret_cast<const uint4*>(stage + w32 * 160);
+                    uint4* out = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + w32) * 80);
+#pragma unroll
+                    for (int i = 0; i < 10; ++i) out[i * 32 + lane] = src[i * 32 + lane];
+                }
             });
         }
     } else {

@@ -145,6 +145,11 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, const void* s
                  ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
                  : "memory");
 }
+// untiled bulk copy shared -> global (16-byte aligned addresses, size a multiple of 16 bytes)
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(reinterpret_cast<uint64_t>(dst)), "r"(smem_u32(src)), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
@@ -190,7 +195,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
 constexpr uint32_t kSwz128 = 2, kSwzNone = 0;
 // The descriptor of the same operand `bytes` further on (bytes a multiple of 16): one 64-bit add,
 // so that a loop over K steps does not rebuild descriptors.
-__device__ __forceinline__ uint64_t desc_off(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
+__device__ __forceinline__ uint64_t desc_off(uint64_t desc, uint32_t bytes) {
+    // The address field (bits 0-13, 16-byte units) never carries: every operand lies inside the
+    // CTA's shared memory.  A 32-bit add on the low word is one instruction for the issuing thread,
+    // whose instruction count per MMA bounds the tensor pipe's utilisation.
+    const uint32_t lo = (uint32_t)desc + (bytes >> 4);
+    return (desc & 0xFFFFFFFF00000000ull) | (uint64_t)lo;
+}
 
 // D[tmem] (+)= A[smem] * B[smem]; one elected thread issues.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
