@@ -393,6 +393,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         const int orow0 = l * b + tp * 128;
         // (this tile's rows were requested ahead: by the prologue, by phase B's last chunks, or
         // by the previous tile as soon as its own copies had been consumed)
+        // Every thread is past its wait for the previous tile's last MMAs before the next commit
+        // can complete the same barrier again: a waiter that looks after two completions sees
+        // the barrier back in the phase it started from.
+        __syncthreads();
         if constexpr (!QSIDE) {
             // e65h is already -(g . O) / d
             oth_col[tid] = make_float2(1.f / denom[(size_t)bh * n + orow0 + tid], e65h[(size_t)bh * n + orow0 + tid]);
