@@ -115,7 +115,7 @@ __device__ __forceinline__ void wg_barrier(int wg) {
 constexpr int kErrState = 3;
 
 template <int R, int T0, int TN, int NWG>
-__global__ void __launch_bounds__(128 * (NWG + 1) + 32)
+__global__ void __launch_bounds__(128 * (NWG + 1) + 64)
 tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                 const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                 const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode, int reverse,
@@ -124,7 +124,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     using L = StateSmem<R, NWG>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread;
+    __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread, bar_drain[2];
     __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull, bar_accread[TN];
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(16) float cm[64];
@@ -133,14 +133,14 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
     const int tpb = b / 128, NJ = n / 128;               // token tiles per block / per head
-    constexpr int kThreads = 128 * (NWG + 1) + 32;
+    constexpr int kThreads = 128 * (NWG + 1) + 64;
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bar_fullx[i], 1); mbar_init(&bar_fully[i], 1); mbar_init(&bar_yfree[i], 1);
             mbar_init(&bar_ext[i], 1);
         }
-        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_accfull, 1);
+        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_accfull, 1); mbar_init(&bar_drain[0], 1); mbar_init(&bar_drain[1], 1);
         for (int i = 0; i < NWG; ++i) { mbar_init(&bar_aready[i], 1); mbar_init(&bar_afree[i], 1); }
         for (int i = 0; i < TN; ++i) mbar_init(&bar_accread[i], 4);
         mbar_fence_init();
@@ -167,9 +167,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     auto tile_of = [&](int j) { return reverse ? (NJ - 1 - j) : j; };
 
     if (wg == NWG + 1) {
-        // =============================== feeder ===============================
+        // =============================== feeders ===============================
+        // Two issuing threads in two warps.  The first loads the tiles and issues the sketch
+        // GEMMs, the second issues the state GEMMs: between two of its MMAs lies as little as
+        // possible (each satisfied wait, commit or TMA issue costs a single thread about a
+        // hundred cycles, during which the tensor pipe would idle).
         if (tid == 128 * (NWG + 1)) {
-            constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
             bool ok = true;
             auto load_x = [&](int j) {
                 // the first tile's barrier also covers the sketch matrices' image
@@ -188,27 +191,36 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             tc_fence_after();
             issue_sketch<R>(tm, smem + L::X, smem + L::G);
             umma_commit(&bar_sk);
+            for (int j = 0; j + 1 < NJ && ok; ++j) {
+                // sketch of the next token tile, as soon as this tile's half sketches are read out
+                ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
+                ok = ok && mbar_wait(&bar_fullx[(j + 1) & 1], ((j + 1) >> 1) & 1, status, kErrTma);
+                tc_fence_after();
+                issue_sketch<R>(tm, smem + L::X + ((j + 1) & 1) * 16384, smem + L::G);
+                umma_commit(&bar_sk);
+                if (j + 2 < NJ) load_x(j + 2);            // its slot: sketch j has completed (it was read)
+                // values of the next token tile: their slot held tile j-1
+                if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
+                load_y(j + 1);
+            }
+            // drain: every sketch GEMM has completed before tensor memory is released.  (A barrier
+            // of its own: completing bar_sk once more, right behind the last sketch, could flip it
+            // twice before a generator thread has looked.)
+            umma_commit(&bar_drain[0]);
+            mbar_wait(&bar_drain[0], 0, status, kErrMma);
+        } else if (tid == 128 * (NWG + 1) + 32) {
+            constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
+            bool ok = true;
             uint32_t a_cnt[NWG];
 #pragma unroll
             for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
-            // This one thread feeds the tensor pipe for the whole CTA: whatever it executes between
-            // two MMAs is time the pipe idles.  Descriptors are built once, here.
             uint64_t ad[NWG];
 #pragma unroll
             for (int i = 0; i < NWG; ++i) ad[i] = smem_desc(smem_u32(smem + L::A0 + i * 32768), 16384, 1024, kSwz128);
             const uint64_t yd0 = smem_desc(smem_u32(smem + L::Y), 16384, 1024, kSwz128);
             for (int j = 0; j < NJ && ok; ++j) {
-                // sketch of the next token tile, as soon as this tile's half sketches are read out
-                if (j + 1 < NJ) {
-                    ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
-                    ok = ok && mbar_wait(&bar_fullx[(j + 1) & 1], ((j + 1) >> 1) & 1, status, kErrTma);
-                    tc_fence_after();
-                    issue_sketch<R>(tm, smem + L::X + ((j + 1) & 1) * 16384, smem + L::G);
-                    umma_commit(&bar_sk);
-                    if (j + 2 < NJ) load_x(j + 2);        // its slot: sketch j has completed (it was read)
-                }
-                ok = ok && mbar_wait(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
-                if (y65 != nullptr) ok = ok && mbar_wait(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
+                ok = mbar_spin(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
+                if (y65 != nullptr) ok = ok && mbar_spin(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
                 const bool boundary = (j % tpb == 0) && j > 0;
                 const uint64_t yd = desc_off(yd0, (j & 1) * L::kYSlot);
                 const uint32_t acc0 = j > 0 ? 1u : 0u;
@@ -224,21 +236,13 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     for (int k = 0; k < 8; ++k)
                         umma_ss(tm + kAcc + 80 * I, desc_off(ad[w], k * 2048), desc_off(yd, k * 2048), idesc_state, k > 0 ? 1u : acc0);
                     umma_commit(&bar_afree[w]);
-                    if constexpr (I == 0) {
-                        // values of the next token tile: their slot held tile j-1, whose MMAs were
-                        // issued a whole tile ago (waiting for them here costs nothing)
-                        if (j + 1 < NJ) {
-                            if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
-                            load_y(j + 1);
-                        }
-                    }
                 });
                 umma_commit(&bar_yfree[j & 1]);
                 if ((j + 1) % tpb == 0) umma_commit(&bar_accfull);
             }
-            // drain: everything issued has completed before tensor memory is released
-            umma_commit(&bar_sk);
-            mbar_wait(&bar_sk, NJ & 1, status, kErrMma);
+            // drain: every state GEMM has completed before tensor memory is released
+            umma_commit(&bar_drain[1]);
+            mbar_wait(&bar_drain[1], 0, status, kErrMma);
         }
     } else if (wg == NWG) {
         // ============================ store warpgroup ============================
@@ -836,7 +840,7 @@ cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUten
     constexpr size_t smem = StateSmem<R, NWG>::total + 1024;
     PSK_TRY(set_smem(tc_state_kernel<R, T0, TN, NWG>, smem));
     prof_begin("tc_state_kernel", s);
-    tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 32, smem, s>>>(
+    tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 64, smem, s>>>(
         mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, y65, cmean, center_mode, reverse ? 1 : 0, S, status);
     prof_end(s);
     ++*launches;
