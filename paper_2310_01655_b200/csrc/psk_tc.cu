@@ -125,7 +125,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread, bar_drain[2];
-    __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull, bar_accread[TN];
+    __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull[TN], bar_accread[TN];
     __shared__ uint32_t tmem_slot;
     __shared__ __align__(16) float cm[64];
     const int tid = threadIdx.x, wg = tid / 128, wt = tid % 128, warp = tid / 32;
@@ -140,9 +140,9 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             mbar_init(&bar_fullx[i], 1); mbar_init(&bar_fully[i], 1); mbar_init(&bar_yfree[i], 1);
             mbar_init(&bar_ext[i], 1);
         }
-        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_accfull, 1); mbar_init(&bar_drain[0], 1); mbar_init(&bar_drain[1], 1);
+        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_drain[0], 1); mbar_init(&bar_drain[1], 1);
         for (int i = 0; i < NWG; ++i) { mbar_init(&bar_aready[i], 1); mbar_init(&bar_afree[i], 1); }
-        for (int i = 0; i < TN; ++i) mbar_init(&bar_accread[i], 4);
+        for (int i = 0; i < TN; ++i) { mbar_init(&bar_accread[i], 4); mbar_init(&bar_accfull[i], 1); }
         mbar_fence_init();
         tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapY);
     }
@@ -236,9 +236,11 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                     for (int k = 0; k < 8; ++k)
                         umma_ss(tm + kAcc + 80 * I, desc_off(ad[w], k * 2048), desc_off(yd, k * 2048), idesc_state, k > 0 ? 1u : acc0);
                     umma_commit(&bar_afree[w]);
+                    // last token tile of a block: this accumulator is complete, and the store
+                    // warpgroup may take it while the remaining tiles are still being issued
+                    if ((j + 1) % tpb == 0) umma_commit(&bar_accfull[I]);
                 });
                 umma_commit(&bar_yfree[j & 1]);
-                if ((j + 1) % tpb == 0) umma_commit(&bar_accfull);
             }
             // drain: every state GEMM has completed before tensor memory is released
             umma_commit(&bar_drain[1]);
@@ -256,12 +258,12 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         bool ok = true;
         for (int p = 0; p < t && ok; ++p) {
             const int l = reverse ? (t - 1 - p) : p;
-            if (p > 0) {
-                ok = mbar_wait(&bar_accfull, (p - 1) & 1, status, kErrMma);
-                tc_fence_after();
-            }
             static_for<0, TN>([&](auto ic) {
                 constexpr int I = decltype(ic)::value;
+                if (p > 0) {
+                    ok = ok && mbar_wait(&bar_accfull[I], (p - 1) & 1, status, kErrMma);
+                    tc_fence_after();
+                }
                 // centred values, in fp32, without touching the operands (the mode only selects
                 // coefficients):  mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
                 //                 mode 2: last column H[:, 64] - H[:, :64] c
