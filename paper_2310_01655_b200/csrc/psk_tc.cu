@@ -427,7 +427,13 @@ struct OutSmem {
     static constexpr uint32_t Mq = Ones + 4096;
     static constexpr uint32_t U = (Mq + 128 * 3 * R * 2 + 1023) / 1024 * 1024;   // split operand: 3R columns
     static constexpr uint32_t Z = U;
-    static constexpr uint32_t K = U, V = U + 16384, Mk = U + 32768;
+    // key tile in ring stage 1, value tile in the query tile's buffer (ring stage 3), split key
+    // sketches over stage 2: the stages the last chunks free first, so the first key/value tile is
+    // fetched while the last chunks are still being multiplied
+    static constexpr uint32_t K = U + 16384, V = Q, Mk = U + 32768;
+    static constexpr int kStageK = 1, kStageV = kZStages - 1;
+    // last chunk that uses ring stage s (-1: none)
+    __host__ __device__ static constexpr int last_chunk(int nc, int s) { return nc > s ? s + (nc - 1 - s) / kZStages * kZStages : -1; }
     static constexpr uint32_t So = U, Soc = U + 16384;               // O tile (bf16), two fp32 half tiles
     static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2, kEpi = 49152;
     static constexpr uint32_t kMax12 = kPhase1 > kPhase2 ? kPhase1 : kPhase2;
@@ -536,8 +542,17 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         if (k < ksteps) umma_ts(tm + cO, at + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
                     umma_commit(&bar_a[s]);
                 }
-                // the key/value tiles reuse the stages' memory and the sketch reuses the staging
-                // columns: every MMA of the first phase must have completed
+                // first key/value tile of the same block, each into its stage as soon as the last
+                // chunk that used it has been multiplied
+                constexpr int cK = L::last_chunk(F::NC, L::kStageK), cV = L::last_chunk(F::NC, L::kStageV);
+                mbar_expect_tx(&bar_kv, 32768);
+                if (cK >= 0) ok = ok && mbar_spin(&bar_a[L::kStageK], (cK / kZStages) & 1, status, kErrMma);
+                tma_load_4d(smem + L::K, &mapK, 0, l * b, hi, bi, &bar_kv);
+                if (cV >= 0) ok = ok && mbar_spin(&bar_a[L::kStageV], (cV / kZStages) & 1, status, kErrMma);
+                else ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);     // no chunk used it: the query sketch did
+                tma_load_4d(smem + L::V, &mapV, 0, l * b, hi, bi, &bar_kv);
+                // the sketch reuses the staging columns and the split key sketches the remaining
+                // stage: every MMA of the first phase must have completed
                 ok = ok && mbar_spin(&bar_a[(F::NC - 1) % kFeatBufs], ((F::NC - 1) / kFeatBufs) & 1, status, kErrMma);
             }
             // same block: key tiles tp <= tau through squared half-sketch scores; descriptors and
@@ -552,9 +567,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll 1
             for (int tp = 0; tp <= tau && ok; ++tp) {
                 if (tp > 0) ok = mbar_spin(&bar_pv, (tp - 1) & 1, status, kErrMma);   // K, V, Mk, weights are free
-                mbar_expect_tx(&bar_kv, 32768);
-                tma_load_4d(smem + L::K, &mapK, 0, l * b + tp * 128, hi, bi, &bar_kv);
-                tma_load_4d(smem + L::V, &mapV, 0, l * b + tp * 128, hi, bi, &bar_kv);
+                if (tp > 0 || l == 0) {       // (block l > 0: the first tile was requested above)
+                    mbar_expect_tx(&bar_kv, 32768);
+                    tma_load_4d(smem + L::K, &mapK, 0, l * b + tp * 128, hi, bi, &bar_kv);
+                    tma_load_4d(smem + L::V, &mapV, 0, l * b + tp * 128, hi, bi, &bar_kv);
+                }
                 ok = ok && mbar_spin(&bar_kv, tp & 1, status, kErrTma);
                 tc_fence_after();
                 issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
