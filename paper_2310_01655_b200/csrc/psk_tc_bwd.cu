@@ -310,7 +310,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 }
                 ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
                 tc_fence_after();
-                if (tid == 0) refill(C);
+                if (tid == 32) refill(C);          // (warp 0 issues the MMAs; the loads go out from warp 1)
                 uint32_t x[32];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -361,7 +361,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 }
                 ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
                 tc_fence_after();
-                if (tid == 0) refill(C);
+                if (tid == 32) refill(C);          // (warp 0 issues the MMAs; the loads go out from warp 1)
                 {
                     uint32_t x[32];
                     tmem_ld32(lane_tm + cPhi + buf * 64, x);
