@@ -202,6 +202,13 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     constexpr uint32_t cPhi = 0;                          // phase B: d-phi, 2 x 64
     constexpr uint32_t cSk = 0;                           // sketch accumulators (transient, <= 128)
     constexpr uint32_t cdM = 128, cdV = 192;              // accumulators: dM (64), dV (64)
+    // r <= 32: the own rows' 64 Y columns also sit in tensor memory (bf16 pairs, 32 columns behind
+    // the r <= 32 columns dM needs), as the A operand of every GEMM that multiplies them.  An MMA
+    // whose operands both come from shared memory moves 6 KB through the 128 B/clk shared-memory
+    // path, which takes as long as its arithmetic and shares that path with everything else.
+    constexpr bool kTsA = (R <= 32);
+    constexpr uint32_t cYA = cdM + 32;
+    constexpr int kNdM = kTsA ? R : 64;                   // columns the dM GEMM writes
     uint32_t mma_uses = 0;
     bool ok = true;
 
@@ -220,6 +227,16 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
+    if constexpr (kTsA) {
+        uint32_t ya[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4*>(smem + L::Yown + swz128_offset(tid, c));
+            ya[4 * c] = v.x; ya[4 * c + 1] = v.y; ya[4 * c + 2] = v.z; ya[4 * c + 3] = v.w;
+        }
+        tmem_st32(lane_tm + cYA, ya);
+        tmem_st_wait();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -244,12 +261,15 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             // d-phi chunk = [Yown | y65] x box^T: the box's feature rows are a K-major B operand,
             // contraction over the 64 state columns, then the last column (second box)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) umma_ss(dphi, desc_off(yd, k * 32), desc_off(bd, k * 32), idesc_phi, k > 0);
+            for (int k = 0; k < 4; ++k) {
+                if constexpr (kTsA) umma_ts(dphi, tm + cYA + k * 8, desc_off(bd, k * 32), idesc_phi, k > 0);
+                else umma_ss(dphi, desc_off(yd, k * 32), desc_off(bd, k * 32), idesc_phi, k > 0);
+            }
             umma_ss(dphi, ed, desc_off(bd, 8192), idesc_phi, 1);
             if constexpr (!QSIDE) {
                 // dV += phi(k) chunk x box (MN-major B: 16 features per K step)
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
-                const uint32_t fb = tm + cFB + buf * 32;
+                const uint32_t fb = tm + cFB + (kTsA ? 0 : buf * 32);   // r <= 32: one staging buffer
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     if (k < ksteps) umma_ts(tm + cdV, fb + k * 8, desc_off(bd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
@@ -284,7 +304,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             auto stage_features = [&](int C) {    // features of the next chunk -> tensor memory
                 uint32_t pk[32];
                 gen.chunk(pk);
-                tmem_st32(lane_tm + cFB + (C & 1) * 32, pk);
+                (void)C;
+                tmem_st32(lane_tm + cFB, pk);          // one buffer: its previous reader (chunk C-1's MMAs) is done
                 tmem_st_wait();
             };
             if constexpr (!QSIDE) stage_features(0);
@@ -298,9 +319,16 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll 1
             for (int C = 0; C < F::NC && ok; ++C) {
                 const int buf = C & 1;
+                // Key side: chunk C's MMAs read the one staging buffer, so they must have completed
+                // before chunk C+1's features go in; query side: chunk C+1 is issued first and runs
+                // behind chunk C.
+                if constexpr (!QSIDE) {
+                    ok = mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+                    tc_fence_after();
+                }
                 if (C + 1 < F::NC) {
                     if constexpr (!QSIDE) stage_features(C + 1);
-                    ok = mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
+                    ok = ok && mbar_wait(&bar_box[(C + 1) % kStages], ((C + 1) / kStages) & 1, status, kErrTma);
                     tc_fence_before();
                     __syncthreads();           // chunk C-1's d-phi has been read by every thread
                     if (tid == 0) {
@@ -308,8 +336,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                         issue_chunk(C + 1);
                     }
                 }
-                ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
-                tc_fence_after();
+                if constexpr (QSIDE) {
+                    ok = ok && mbar_wait(&bar_phi[buf], (C / 2) & 1, status, kErrMma);
+                    tc_fence_after();
+                }
                 if (tid == 32) refill(C);          // (warp 0 issues the MMAs; the loads go out from warp 1)
                 uint32_t x[32];
 #pragma unroll
@@ -435,9 +465,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)           // dW without its 65th-column term
-                    umma_ss(tm + cDW, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32),
-                            desc_off(smem_desc(smem_u32(smem + L::Yoth) + hh * 8192, 0, 1024, kSwz128), k * 32), idesc, k > 0);
+                for (int k = 0; k < 4; ++k) {         // dW without its 65th-column term
+                    const uint64_t yod = desc_off(smem_desc(smem_u32(smem + L::Yoth) + hh * 8192, 0, 1024, kSwz128), k * 32);
+                    if constexpr (kTsA) umma_ts(tm + cDW, tm + cYA + k * 8, yod, idesc, k > 0);
+                    else umma_ss(tm + cDW, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32), yod, idesc, k > 0);
+                }
                 umma_commit(&bar_mma);
             }
             ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
@@ -485,10 +517,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             if (tid == 0) {
                 tc_fence_after();
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+                constexpr uint32_t idesc_dm = idesc_bf16(128, kNdM, false, true);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)           // dM_own += dS x M_other (its hi columns)
                     umma_ts(tm + cdM, tm + cS + k * 8,
-                            desc_off(smem_desc(smem_u32(smem + L::Moth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
+                            desc_off(smem_desc(smem_u32(smem + L::Moth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc_dm,
                             (dm_started || k > 0) ? 1u : 0u);
                 if constexpr (!QSIDE) {
 #pragma unroll
