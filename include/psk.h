@@ -163,6 +163,17 @@ int psk_profile_enable(int enable);
 int psk_profile_count(void);
 int psk_profile_get(int index, char* name, size_t name_cap, float* ms);
 
+/* Diagnostic, host only (no GPU needed): the feature order of the tensor-core path.
+ * Section 2.2's self-tensored sketch phi'(x) = m (x) m has one distinct entry per unordered pair
+ * {a, b} of half-sketch coordinates; the tensor-core kernels store one feature per pair (some
+ * pairs twice, some padding rows) and weight the rows of their states so that every pair {a, b}
+ * carries total weight 2 for a != b and 1 for a == b.  For r in {16, 32, 64} this writes, for
+ * stored feature f < count, a[f], b[f] (feature f is m_a m_b) and w[f] (the weight of state row
+ * f; 0 for padding) into HOST arrays of capacity `cap` each and returns the number of stored
+ * features; PSK_ERR_UNSUPPORTED for another r, PSK_ERR_INVALID_ARG for a null pointer,
+ * PSK_ERR_WORKSPACE if cap is too small. */
+int psk_feature_table(int r, int* a, int* b, float* w, int cap);
+
 #ifdef __cplusplus
 }
 #endif

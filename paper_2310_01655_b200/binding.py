@@ -65,6 +65,8 @@ def lib():
     L.psk_profile_enable.restype = c_int
     L.psk_profile_enable.argtypes = [c_int]
     L.psk_profile_count.restype = c_int
+    L.psk_feature_table.restype = c_int
+    L.psk_feature_table.argtypes = [c_int, c_void_p, c_void_p, c_void_p, c_int]
     L.psk_profile_get.restype = c_int
     L.psk_profile_get.argtypes = [c_int, ctypes.c_char_p, c_size_t, POINTER(ctypes.c_float)]
     _lib = L
@@ -223,3 +225,16 @@ def profile_records():
             raise PskError(st, "psk_profile_get")
         out.append((buf.value.decode(), float(ms.value)))
     return out
+
+
+def feature_table(r: int):
+    """psk_feature_table: (a, b, w) numpy arrays of the tensor-core path's stored features (host only)."""
+    import numpy as np
+    cap = 4096
+    a = np.zeros(cap, dtype=np.int32)
+    b = np.zeros(cap, dtype=np.int32)
+    w = np.zeros(cap, dtype=np.float32)
+    n = lib().psk_feature_table(int(r), a.ctypes.data, b.ctypes.data, w.ctypes.data, cap)
+    if n < 0:
+        raise PskError(n, "psk_feature_table")
+    return a[:n].copy(), b[:n].copy(), w[:n].copy()

@@ -1,5 +1,6 @@
 // C ABI of libpsk: argument validation and dispatch.  See include/psk.h for the contract.
 #include "psk_internal.cuh"
+#include "tc_features.cuh"
 
 #include <string.h>
 #include <string>
@@ -187,3 +188,33 @@ int psk_profile_get(int index, char* name, size_t name_cap, float* ms) {
 }
 
 }  // extern "C"
+
+namespace {
+template <int R>
+int feature_table(int* a, int* b, float* w, int cap) {
+    using F = psk::tc::Feat<R>;
+    if (cap < F::F) return PSK_ERR_WORKSPACE;
+    for (int f = 0; f < F::F; ++f) {
+        if (F::kCirc) {
+            const int s = 2 * (f / (2 * R)) + ((f / R) & 1);
+            a[f] = f % R;
+            b[f] = (a[f] + s) % R;
+        } else {
+            a[f] = F::a(f);
+            b[f] = F::b(f);
+        }
+        w[f] = F::weight(f);
+    }
+    return F::F;
+}
+}  // namespace
+
+extern "C" int psk_feature_table(int r, int* a, int* b, float* w, int cap) {
+    if (!a || !b || !w) return PSK_ERR_INVALID_ARG;
+    switch (r) {
+        case 16: return feature_table<16>(a, b, w, cap);
+        case 32: return feature_table<32>(a, b, w, cap);
+        case 64: return feature_table<64>(a, b, w, cap);
+    }
+    return PSK_ERR_UNSUPPORTED;
+}
