@@ -181,16 +181,12 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     // dL/dW_ij = (g_i . v_j - g_i . O_i) / d_i cancels heavily when one key dominates a row, and a
     // rounded g_i / d_i would not survive it.  y65 = -(g_i . (O_i - c)) pairs with the centred
     // states, y65h = -(g_i . O_i) with the raw values of the 128 x 128 tiles.  Key rows: 1.
-    const float d_own = QSIDE ? denom[(size_t)bh * n + row0 + tid] : 1.f;
-    const float inv_own = 1.f / d_own;
-    const float y65 = QSIDE ? e65[(size_t)bh * n + row0 + tid] * d_own : 1.f;
-    const float y65h = QSIDE ? e65h[(size_t)bh * n + row0 + tid] * d_own : 1.f;
-    {
-        uint8_t* ext = smem + L::ExtA;
-        *reinterpret_cast<uint4*>(ext + (tid / 8) * 128 + (tid % 8) * 16) =
-            make_uint4(pack_bf16(y65, 0.f), 0, 0, 0);
-        *reinterpret_cast<uint4*>(ext + 2048 + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(0, 0, 0, 0);
-    }
+    // (The three row scalars come from HBM.  They are requested here and first used after the half
+    // sketch has been read, a few thousand cycles later: the arithmetic on them stays below.)
+    const float d_raw = QSIDE ? denom[(size_t)bh * n + row0 + tid] : 1.f;
+    const float e65_raw = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
+    const float e65h_raw = QSIDE ? e65h[(size_t)bh * n + row0 + tid] : 1.f;
+    *reinterpret_cast<uint4*>(smem + L::ExtA + 2048 + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -227,6 +223,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
+    const float d_own = d_raw, inv_own = 1.f / d_own;
+    const float y65 = QSIDE ? e65_raw * d_own : 1.f, y65h = QSIDE ? e65h_raw * d_own : 1.f;
+    // the 65th column of the A operand [Y_own | y65]: first read by phase B's MMAs, after the barrier below
+    *reinterpret_cast<uint4*>(smem + L::ExtA + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(pack_bf16(y65, 0.f), 0, 0, 0);
+    fence_proxy_async_smem();
     if constexpr (kTsA) {
         uint32_t ya[32];
 #pragma unroll
