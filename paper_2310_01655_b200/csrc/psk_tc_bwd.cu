@@ -186,6 +186,12 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const float d_raw = QSIDE ? denom[(size_t)bh * n + row0 + tid] : 1.f;
     const float e65_raw = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
     const float e65h_raw = QSIDE ? e65h[(size_t)bh * n + row0 + tid] : 1.f;
+    // key side: the scalars of the first query tile it will meet (thread = that tile's row tid)
+    float od_raw = 1.f, oe_raw = 0.f;
+    if constexpr (!QSIDE) {
+        od_raw = denom[(size_t)bh * n + l * b + tau * 128 + tid];
+        oe_raw = e65h[(size_t)bh * n + l * b + tau * 128 + tid];
+    }
     *reinterpret_cast<uint4*>(smem + L::ExtA + 2048 + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     tc_fence_before();
@@ -429,8 +435,13 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         // the barrier back in the phase it started from.
         __syncthreads();
         if constexpr (!QSIDE) {
-            // e65h is already -(g . O) / d
-            oth_col[tid] = make_float2(1.f / denom[(size_t)bh * n + orow0 + tid], e65h[(size_t)bh * n + orow0 + tid]);
+            // e65h is already -(g . O) / d.  These two were requested a tile (or a phase) ago; the
+            // next tile's are requested now.
+            oth_col[tid] = make_float2(1.f / od_raw, oe_raw);
+            if (tp + 1 < tp_end) {
+                od_raw = denom[(size_t)bh * n + orow0 + 128 + tid];
+                oe_raw = e65h[(size_t)bh * n + orow0 + 128 + tid];
+            }
         }
         ok = mbar_wait(&bar_xoth, oth_uses & 1, status, kErrTma);
         if (tid == 0) {
