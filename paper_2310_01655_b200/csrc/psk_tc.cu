@@ -331,6 +331,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         uint8_t* sA = smem + L::A0 + wg * 32768;
         uint32_t a_uses = 0;                              // times this warpgroup's buffer has been filled
         bool ok = true;
+        // last-column entry of this thread's token, requested one token tile ahead of its use
+        float y_next = (y65 != nullptr && wg == 0) ? y65[(size_t)bh * n + tile_of(0) * 128 + wt] : 0.f;
         for (int j = 0; j < NJ && ok; ++j) {
             ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
             tc_fence_after();
@@ -347,7 +349,8 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             if (y65 != nullptr && wg == 0) {
                 // last-column chunk of this token tile; its slot is free once tile j-2's MMAs are done
                 if (j >= 2) ok = ok && mbar_wait(&bar_yfree[j & 1], ((j >> 1) - 1) & 1, status, kErrState);
-                const float y = y65[(size_t)bh * n + tile_of(j) * 128 + wt];
+                const float y = y_next;
+                if (j + 1 < NJ) y_next = y65[(size_t)bh * n + tile_of(j + 1) * 128 + wt];
                 *reinterpret_cast<bf16*>(smem + L::Y + (j & 1) * L::kYSlot + 16384 + swz128_offset(wt, 0)) =
                     __float2bfloat16_rn(y);
                 fence_proxy_async_smem();
