@@ -699,20 +699,24 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     } else {
         PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
     }
-    PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
     constexpr size_t smem = BwdSmem<R>::total + 1024;
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
     PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
+    // query side first: it needs only the prefix states, and the row scalars just written are
+    // still in L2; the suffix states (5 GB through L2) come after it
     prof_begin("tc_bwd_q_kernel", s);
     tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n, d.b, d.t,
                                                         e65, e65h, denom, status);
     prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
     prof_begin("tc_bwd_k_kernel", s);
     tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n, d.b, d.t,
                                                          e65, e65h, denom, status);
     prof_end(s);
-    *launches += 2;
+    ++*launches;
     return cudaGetLastError();
 }
 
