@@ -16,12 +16,16 @@ Notation (paper -> here)
   lt(.)                        keep the lower triangle INCLUDING the diagonal (Section 1.2)
   D~ = diag(1 + lt(..) 1)      row normaliser of Section 3 (the "1 +" is part of it)
   H_l, Z_l, P_l                per-block state, exclusive prefix, diagonal block (Section 3.1)
+  P_l = lt((Q_l K_l^T)^p) X_l  exact polynomial weights inside a block (Section 3.2)
 
 Pins (tests/test_oracle_*.py): exact-feature case against looped (q.k)^4
 attention, hand-worked rational example, G = I closed form, Monte-Carlo mean and
 closed-form variance of the sketch, V = 1 closed form, n = 1 closed form,
 causality, block-size invariance, lt-multiply against a dense triangle, central
-finite differences for every gradient, dV against the explicit weight matrix.
+finite differences for every gradient, dV against the explicit weight matrix;
+for the local-exact variant (Section 3.2): one block = exact polynomial
+attention, exact features = no dependence on the block size, looped definition,
+block algorithm against the masked definition, finite differences.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -149,13 +153,36 @@ def lt_multiply_blocked(A, B, C, b, diag_block=None):
     return out
 
 
+def same_block(n, b):
+    """Boolean n x n matrix: tokens i and j lie in the same block of b rows (Section 3.1's B_l)."""
+    blk = np.arange(n) // b
+    return blk[:, None] == blk[None, :]
+
+
+def causal_weights_local_exact(Q, K, G1, G2, b, p=4):
+    """Section 3.2 as a definition: the weight of (i, j), j <= i, is the exact polynomial
+    weight <q_i, k_j>^p when i and j share a block of b rows, and the Polysketch weight
+    (m(q_i) . m(k_j))^2 otherwise."""
+    Q, K = _f64(Q), _f64(K)
+    s = half_sketch(Q, G1, G2) @ half_sketch(K, G1, G2).T
+    return lt(np.where(same_block(Q.shape[0], b), (Q @ K.T) ** p, s * s))
+
+
+def causal_polysketch_local_exact_attention(Q, K, V, G1, G2, b):
+    """Section 3 with the weights of Section 3.2; returns (O, d), d including its "1 +"."""
+    W = causal_weights_local_exact(Q, K, G1, G2, b)
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
 def causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal="LR"):
     """Causal Polysketch attention in time linear in n (Section 3.1).
 
     A = phi'(Q), B = phi'(K), C = [V | 1_n]; the last output column is the
     normaliser without its "1 +".  diagonal="phi" forms the diagonal blocks from
     the r^2-dimensional features, diagonal="LR" from (L R^T)^2 with L, R the
-    b x r half sketches of the block.
+    b x r half sketches of the block, diagonal="exact" from the block's own
+    queries and keys, lt((Q_l K_l^T)^4) (Section 3.2, p = 4).
     """
     V = _f64(V)
     n, h = V.shape
@@ -167,6 +194,11 @@ def causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal="LR"):
         def diag_block(l):
             L, R = Mq[l * b:(l + 1) * b], Mk[l * b:(l + 1) * b]
             return lt((L @ R.T) ** 2)
+    elif diagonal == "exact":
+        Qf, Kf = _f64(Q), _f64(K)
+
+        def diag_block(l):
+            return lt((Qf[l * b:(l + 1) * b] @ Kf[l * b:(l + 1) * b].T) ** 4)
     else:
         raise ValueError(diagonal)
     N = lt_multiply_blocked(self_tensor(Mq), self_tensor(Mk), C, b, diag_block)
@@ -216,8 +248,36 @@ def causal_polysketch_attention_backward(Q, K, V, G1, G2, dO):
     return (_sketch_backward(Q, G1, G2, dMq), _sketch_backward(K, G1, G2, dMk), dV)
 
 
-def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b):
+def causal_polysketch_local_exact_attention_backward(Q, K, V, G1, G2, dO, b):
+    """Gradients (dQ, dK, dV) of sum(dO * O) for the weights of Section 3.2, through the
+    quadratic definition.  Same-block pairs: W_ij = x_ij^4 with x_ij = q_i . k_j, so
+    dL/dx_ij = 4 x_ij^3 dL/dW_ij reaches Q and K directly; other pairs go through the half
+    sketches as in causal_polysketch_attention_backward."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, h = V.shape
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    same = same_block(n, b)
+    s = Mq @ Mk.T
+    x = Q @ K.T
+    W = lt(np.where(same, x ** 4, s * s))
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = lt(E @ Vt.T)
+    dV = W.T @ E[:, :h]
+    ds = np.where(same, 0.0, 2.0 * s * dW)
+    dx = np.where(same, 4.0 * x ** 3 * dW, 0.0)
+    dQ = _sketch_backward(Q, G1, G2, ds @ Mk) + dx @ K
+    dK = _sketch_backward(K, G1, G2, ds.T @ Mq) + dx.T @ Q
+    return dQ, dK, dV
+
+
+def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b, diagonal="LR"):
     """Same gradients in time linear in n, in the style of Section 3.1.
+
+    diagonal="exact": the same-block pairs carry the weights of Section 3.2,
+    (q_i . k_j)^4, whose gradient 4 (q_i . k_j)^3 dW_ij reaches Q and K directly.
 
     Forward sweep carries Z_l = sum_{blocks < l} phi'(K)^T V~ (the forward's
     own prefix); reverse sweep carries R_l = sum_{blocks > l} phi'(Q)^T E.
@@ -234,7 +294,13 @@ def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b):
     G1 = _f64(G1)
     r = G1.shape[1]
     Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
-    O, d = causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal="LR")
+    if diagonal not in ("LR", "exact"):
+        raise ValueError(diagonal)
+    exact = diagonal == "exact"
+    Qf, Kf = _f64(Q), _f64(K)
+    dQl = np.zeros_like(Qf)
+    dKl = np.zeros_like(Kf)
+    O, d = causal_polysketch_attention_blocked(Q, K, V, G1, G2, b, diagonal=diagonal)
     E = _backward_rows(O, d, dO)
     Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
     PhiQ, PhiK = self_tensor(Mq), self_tensor(Mk)
@@ -250,12 +316,19 @@ def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b):
     Z = np.zeros((r * r, h + 1), dtype=F64)
     for l in range(t):
         rows = slice(l * b, (l + 1) * b)
-        s = Mq[rows] @ Mk[rows].T
-        W = lt(s * s)
         dW = lt(E[rows] @ Vt[rows].T)
-        ds = 2.0 * s * dW
-        dMq[rows] += ds @ Mk[rows]
-        dMk[rows] += ds.T @ Mq[rows]
+        if exact:
+            x = Qf[rows] @ Kf[rows].T
+            W = lt(x ** 4)
+            dx = 4.0 * x ** 3 * dW
+            dQl[rows] += dx @ Kf[rows]
+            dKl[rows] += dx.T @ Qf[rows]
+        else:
+            s = Mq[rows] @ Mk[rows].T
+            W = lt(s * s)
+            ds = 2.0 * s * dW
+            dMq[rows] += ds @ Mk[rows]
+            dMk[rows] += ds.T @ Mq[rows]
         dVt[rows] += W.T @ E[rows]
         dMq[rows] += untensor(E[rows] @ Z.T, Mq[rows])
         Z = Z + PhiK[rows].T @ Vt[rows]
@@ -266,7 +339,7 @@ def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b):
         dMk[rows] += untensor(Vt[rows] @ R.T, Mk[rows])
         dVt[rows] += PhiK[rows] @ R
         R = R + PhiQ[rows].T @ E[rows]
-    return (_sketch_backward(Q, G1, G2, dMq), _sketch_backward(K, G1, G2, dMk), dVt[:, :h])
+    return (_sketch_backward(Q, G1, G2, dMq) + dQl, _sketch_backward(K, G1, G2, dMk) + dKl, dVt[:, :h])
 
 
 # ---------------------------------------------------------------------------
