@@ -79,8 +79,17 @@ typedef struct {
  * workspace memory (not written in between) with the same shape and inputs, reads them instead
  * of rebuilding the states from K and V and recomputing the forward rows.  With the flag set
  * psk_workspace_bytes() returns the backward's size for both calls.  Without the flag each
- * call is self-contained. */
-typedef enum { PSK_FLAG_KEEP_STATES = 1 } psk_flags;
+ * call is self-contained.
+ *
+ * PSK_FLAG_LOCAL_EXACT: "applying exact attention locally" (Section 3.2).  Pairs (i, j) of the
+ * same block of b rows get the exact polynomial weight (q_i . k_j)^4 instead of the sketched
+ * (m(q_i) . m(k_j))^2, i.e. P_l = lt((Q_l K_l^T)^4) [V_l | 1]; pairs in different blocks are
+ * unchanged.  The result now depends on b (more exact pairs with larger blocks; b = n is exact
+ * degree-4 polynomial attention).  Set it on the forward and on the backward call alike; the
+ * backward sends the same-block part of dQ, dK straight to Q and K instead of through the
+ * sketch.  Served by the CUDA-core kernels (fp32 arithmetic) for both storage types:
+ * PSK_PATH_AUTO selects them, PSK_PATH_TENSOR_CORES with this flag is PSK_ERR_UNSUPPORTED. */
+typedef enum { PSK_FLAG_KEEP_STATES = 1, PSK_FLAG_LOCAL_EXACT = 2 } psk_flags;
 
 /* Library version (major*100 + minor). */
 int psk_version(void);

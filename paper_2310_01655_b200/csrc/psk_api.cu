@@ -38,7 +38,7 @@ int make_dims(const psk_shape* sh, Dims* d) {
     if (sh == nullptr) return PSK_ERR_INVALID_ARG;
     if (sh->dtype != PSK_F32 && sh->dtype != PSK_BF16) return PSK_ERR_INVALID_ARG;
     if (sh->path < PSK_PATH_AUTO || sh->path > PSK_PATH_TENSOR_CORES) return PSK_ERR_INVALID_ARG;
-    if (sh->flags & ~(int32_t)PSK_FLAG_KEEP_STATES) return PSK_ERR_INVALID_ARG;
+    if (sh->flags & ~(int32_t)(PSK_FLAG_KEEP_STATES | PSK_FLAG_LOCAL_EXACT)) return PSK_ERR_INVALID_ARG;
     if (sh->B <= 0 || sh->H <= 0 || sh->n <= 0 || sh->b <= 0) return PSK_ERR_SHAPE;
     if (sh->p != 4 || sh->h != 64) return PSK_ERR_UNSUPPORTED;
     if (sh->r != 16 && sh->r != 32 && sh->r != 64) return PSK_ERR_UNSUPPORTED;
@@ -55,6 +55,7 @@ int make_dims(const psk_shape* sh, Dims* d) {
     d->g_heads = sh->g_heads;
     d->bf16 = sh->dtype == PSK_BF16;
     d->keep_states = (sh->flags & PSK_FLAG_KEEP_STATES) != 0;
+    d->local = (sh->flags & PSK_FLAG_LOCAL_EXACT) != 0;
     return PSK_OK;
 }
 

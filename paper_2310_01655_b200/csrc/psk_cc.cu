@@ -22,6 +22,10 @@ CcWorkspace cc_workspace(const Dims& d, bool backward) {
         w.Rst = off; off += align_up(st);
         w.dMq = off; off += align_up(rows * d.r * sizeof(float));
         w.dMk = off; off += align_up(rows * d.r * sizeof(float));
+        if (d.local) {     // gradients that reach Q and K directly, through the exact same-block weights
+            w.dXq = off; off += align_up(rows * 64 * sizeof(float));
+            w.dXk = off; off += align_up(rows * 64 * sizeof(float));
+        }
     }
     w.total = off;
     return w;
@@ -208,6 +212,9 @@ __device__ __forceinline__ float dot65(const float* row, const float (&y)[YC]) {
 //   sOut [128][R+1]     per-row results indexed by a
 //   sM2  [32][R]        chunk of the other side's half sketches (diagonal tile)
 //   sY2  [32][YS]       chunk of the other side's 65-column rows (diagonal tile)
+// and, with exact same-block weights (Section 3.2):
+//   sXo  [128][65]      this tile's own raw rows (q or k), each read by its own thread only
+//   sX2  [32][64]       chunk of the other side's raw rows
 template <int R> struct RowSmem {
     static constexpr int S = 0;
     static constexpr int Own = S + R * YS;
@@ -216,16 +223,30 @@ template <int R> struct RowSmem {
     static constexpr int Y2 = M2 + 32 * R;
     static constexpr int total = Y2 + 32 * YS;
     static constexpr size_t bytes = (size_t)total * sizeof(float);
+    static constexpr int Xo = total;
+    static constexpr int X2 = Xo + 128 * 65;
+    static constexpr size_t bytes_local = (size_t)(X2 + 32 * 64) * sizeof(float);
 };
+
+// <own raw row (shared memory, stride 65), row jj of the other side's chunk>
+__device__ __forceinline__ float dot64_raw(const float* own, const float* other) {
+    float s = 0.f;
+#pragma unroll
+    for (int c = 0; c < 64; ++c) s = fmaf(own[c], other[c], s);
+    return s;
+}
 
 // ---------------------------------------------------------------------------
 // Forward output rows (Section 3.1): row i of block l = P_l row + phi'(q_i)^T Z_l, with
 // P_l = lt((L R^T)^2) [V_l | 1]; then d_i = 1 + last column, O_i = first 64 / d_i.
+// LOCAL: P_l = lt((Q_l K_l^T)^4) [V_l | 1] instead, from the block's raw queries and keys
+// (Section 3.2).
 // ---------------------------------------------------------------------------
-template <typename T, int R>
+template <typename T, int R, bool LOCAL>
 __global__ void __launch_bounds__(128)
 fwd_out_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
                const float* __restrict__ Vt, const float* __restrict__ Z,
+               const T* __restrict__ Qraw, const T* __restrict__ Kraw,
                T* __restrict__ O, float* __restrict__ denom) {
     extern __shared__ __align__(16) float smem[];
     float* sS = smem + RowSmem<R>::S;
@@ -241,6 +262,12 @@ fwd_out_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, cons
     for (int c = 0; c < R; ++c) { mq[c] = Mq[row * R + c]; sOwn[tid * (R + 1) + c] = mq[c]; }
 #pragma unroll
     for (int c = 0; c < YC; ++c) acc[c] = 0.f;
+    float* sXo = smem + RowSmem<R>::Xo + tid * 65;
+    float* sX2 = smem + RowSmem<R>::X2;
+    if constexpr (LOCAL) {
+        const int64_t o = sl.row(bh, l * b + i_blk);
+        for (int c = 0; c < 64; ++c) sXo[c] = ldf(Qraw + o + c);
+    }
     // earlier blocks through the prefix state
     const float* Zl = Z + ((size_t)bh * t + l) * R * R * YC;
     if (l > 0) {
@@ -258,15 +285,24 @@ fwd_out_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, cons
     const int warp_imax = tile * 128 + (tid | 31);
     for (int j0 = 0; j0 < jend; j0 += 32) {
         __syncthreads();
-        for (int e = tid; e < 32 * R; e += 128) sM2[e] = Mk[(blk0 + j0) * R + e];
+        if constexpr (LOCAL) {
+            for (int e = tid; e < 32 * 64; e += 128) sX2[e] = ldf(Kraw + sl.row(bh, l * b + j0 + e / 64) + e % 64);
+        } else {
+            for (int e = tid; e < 32 * R; e += 128) sM2[e] = Mk[(blk0 + j0) * R + e];
+        }
         for (int e = tid; e < 32 * YC; e += 128) sY2[(e / YC) * YS + e % YC] = Vt[(blk0 + j0) * YC + e];
         __syncthreads();
         if (j0 > warp_imax) continue;
         for (int jj = 0; jj < 32; ++jj) {
             if (j0 + jj > i_blk) break;
             float s = 0.f;
+            if constexpr (LOCAL) {
+                const float x = dot64_raw(sXo, sX2 + jj * 64);
+                s = x * x;                                  // weight s^2 = (q . k)^4
+            } else {
 #pragma unroll
-            for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
+                for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
+            }
             axpy65(acc, s * s, sY2 + jj * YS);
         }
     }
@@ -281,12 +317,15 @@ fwd_out_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, cons
 // ---------------------------------------------------------------------------
 // Backward, query side.  d m(q_i) = 2 mat(Z_l E_i) m(q_i)  +  sum_{j<=i, same block}
 // 2 s_ij (E_i . v~_j) m(k_j).
+// LOCAL (Section 3.2): the same-block pairs carry W_ij = x_ij^4, x_ij = q_i . k_j, whose gradient
+// reaches q_i directly:  dXl_i = sum_{j<=i, same block} 4 x_ij^3 (E_i . v~_j) k_j.
 // ---------------------------------------------------------------------------
-template <int R>
+template <typename T, int R, bool LOCAL>
 __global__ void __launch_bounds__(128)
-bwd_q_kernel(int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
+bwd_q_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
              const float* __restrict__ Vt, const float* __restrict__ E, const float* __restrict__ Z,
-             float* __restrict__ dMq) {
+             const T* __restrict__ Qraw, const T* __restrict__ Kraw,
+             float* __restrict__ dMq, float* __restrict__ dXl) {
     extern __shared__ __align__(16) float smem[];
     float* sS = smem + RowSmem<R>::S;
     float* sOut = smem + RowSmem<R>::Out;
@@ -315,36 +354,63 @@ bwd_q_kernel(int n, int b, int t, const float* __restrict__ Mq, const float* __r
     }
     const int jend = tile * 128 + 128;
     const int warp_imax = tile * 128 + (tid | 31);
+    float* sXo = smem + RowSmem<R>::Xo + tid * 65;
+    float* sX2 = smem + RowSmem<R>::X2;
+    float dxl[LOCAL ? 64 : 1];
+    if constexpr (LOCAL) {
+        const int64_t o = sl.row(bh, l * b + i_blk);
+        for (int c = 0; c < 64; ++c) sXo[c] = ldf(Qraw + o + c);
+#pragma unroll
+        for (int c = 0; c < 64; ++c) dxl[c] = 0.f;
+    }
     for (int j0 = 0; j0 < jend; j0 += 32) {
         __syncthreads();
-        for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mk[(blk0 + j0) * R + x];
+        if constexpr (LOCAL) {
+            for (int x = tid; x < 32 * 64; x += 128) sX2[x] = ldf(Kraw + sl.row(bh, l * b + j0 + x / 64) + x % 64);
+        } else {
+            for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mk[(blk0 + j0) * R + x];
+        }
         for (int x = tid; x < 32 * YC; x += 128) sY2[(x / YC) * YS + x % YC] = Vt[(blk0 + j0) * YC + x];
         __syncthreads();
         if (j0 > warp_imax) continue;
         for (int jj = 0; jj < 32; ++jj) {
             if (j0 + jj > i_blk) break;
-            float s = 0.f;
+            if constexpr (LOCAL) {
+                const float x = dot64_raw(sXo, sX2 + jj * 64);
+                const float dx = 4.f * x * x * x * dot65(sY2 + jj * YS, e);
 #pragma unroll
-            for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
-            const float ds = 2.f * s * dot65(sY2 + jj * YS, e);
+                for (int c = 0; c < 64; ++c) dxl[c] = fmaf(dx, sX2[jj * 64 + c], dxl[c]);
+            } else {
+                float s = 0.f;
 #pragma unroll
-            for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[jj * R + c], dm[c]);
+                for (int c = 0; c < R; ++c) s = fmaf(mq[c], sM2[jj * R + c], s);
+                const float ds = 2.f * s * dot65(sY2 + jj * YS, e);
+#pragma unroll
+                for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[jj * R + c], dm[c]);
+            }
         }
     }
 #pragma unroll
     for (int c = 0; c < R; ++c) dMq[row * R + c] = dm[c] + sOut[tid * (R + 1) + c];
+    if constexpr (LOCAL) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) dXl[row * 64 + c] = dxl[c];
+    }
 }
 
 // ---------------------------------------------------------------------------
 // Backward, key/value side.  With R_l the suffix state sum_{blocks>l} phi'(Q)^T E:
 //   d m(k_j) = 2 mat(R_l v~_j) m(k_j) + sum_{i>=j, same block} 2 s_ij (E_i . v~_j) m(q_i)
 //   dV_j     = (R_l^T phi'(k_j))[:h]  + sum_{i>=j, same block} s_ij^2 E_i[:h]
+// LOCAL (Section 3.2): same-block weights x_ij^4, x_ij = q_i . k_j:
+//   dXl_j = sum_{i>=j, same block} 4 x_ij^3 (E_i . v~_j) q_i,   dV_j += sum x_ij^4 E_i[:h]
 // ---------------------------------------------------------------------------
-template <typename T, int R>
+template <typename T, int R, bool LOCAL>
 __global__ void __launch_bounds__(128)
 bwd_k_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const float* __restrict__ Mk,
              const float* __restrict__ Vt, const float* __restrict__ E, const float* __restrict__ Rs,
-             float* __restrict__ dMk, T* __restrict__ dV) {
+             const T* __restrict__ Qraw, const T* __restrict__ Kraw,
+             float* __restrict__ dMk, float* __restrict__ dXl, T* __restrict__ dV) {
     extern __shared__ __align__(16) float smem[];
     float* sS = smem + RowSmem<R>::S;
     float* sOwn = smem + RowSmem<R>::Own;
@@ -382,25 +448,51 @@ bwd_k_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const 
     // same block: queries i >= j
     const int i_begin = tile * 128;                     // first query row any thread here needs
     const int warp_jmin = tile * 128 + (tid & ~31);
+    float* sXo = smem + RowSmem<R>::Xo + tid * 65;
+    float* sX2 = smem + RowSmem<R>::X2;
+    float dxl[LOCAL ? 64 : 1];
+    if constexpr (LOCAL) {
+        const int64_t o = sl.row(bh, l * b + j_blk);
+        for (int c = 0; c < 64; ++c) sXo[c] = ldf(Kraw + o + c);
+#pragma unroll
+        for (int c = 0; c < 64; ++c) dxl[c] = 0.f;
+    }
     for (int i0 = i_begin; i0 < b; i0 += 32) {
         __syncthreads();
-        for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mq[(blk0 + i0) * R + x];
+        if constexpr (LOCAL) {
+            for (int x = tid; x < 32 * 64; x += 128) sX2[x] = ldf(Qraw + sl.row(bh, l * b + i0 + x / 64) + x % 64);
+        } else {
+            for (int x = tid; x < 32 * R; x += 128) sM2[x] = Mq[(blk0 + i0) * R + x];
+        }
         for (int x = tid; x < 32 * YC; x += 128) sY2[(x / YC) * YS + x % YC] = E[(blk0 + i0) * YC + x];
         __syncthreads();
         if (i0 + 31 < warp_jmin) continue;
         for (int ii = 0; ii < 32; ++ii) {
             if (i0 + ii < j_blk) continue;
-            float s = 0.f;
+            if constexpr (LOCAL) {
+                const float x = dot64_raw(sXo, sX2 + ii * 64);
+                const float x2 = x * x;
+                const float dx = 4.f * x2 * x * dot65(sY2 + ii * YS, v);
 #pragma unroll
-            for (int c = 0; c < R; ++c) s = fmaf(mk[c], sM2[ii * R + c], s);
-            const float ds = 2.f * s * dot65(sY2 + ii * YS, v);
+                for (int c = 0; c < 64; ++c) dxl[c] = fmaf(dx, sX2[ii * 64 + c], dxl[c]);
+                axpy65(dv, x2 * x2, sY2 + ii * YS);
+            } else {
+                float s = 0.f;
 #pragma unroll
-            for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[ii * R + c], dm[c]);
-            axpy65(dv, s * s, sY2 + ii * YS);
+                for (int c = 0; c < R; ++c) s = fmaf(mk[c], sM2[ii * R + c], s);
+                const float ds = 2.f * s * dot65(sY2 + ii * YS, v);
+#pragma unroll
+                for (int c = 0; c < R; ++c) dm[c] = fmaf(ds, sM2[ii * R + c], dm[c]);
+                axpy65(dv, s * s, sY2 + ii * YS);
+            }
         }
     }
 #pragma unroll
     for (int c = 0; c < R; ++c) dMk[row * R + c] = dm[c] + sOut[tid * (R + 1) + c];
+    if constexpr (LOCAL) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) dXl[row * 64 + c] = dxl[c];
+    }
     const int64_t o = sl.row(bh, l * b + j_blk);
 #pragma unroll
     for (int c = 0; c < 64; ++c) stf(dV + o + c, dv[c]);
@@ -408,12 +500,14 @@ bwd_k_kernel(Slice sl, int n, int b, int t, const float* __restrict__ Mq, const 
 
 // ---------------------------------------------------------------------------
 // Chain rule through the half sketch: dX = ((dM*A2) G1^T + (dM*A1) G2^T)/sqrt(r),
-// A1 = X G1, A2 = X G2 recomputed.  64 rows per CTA.
+// A1 = X G1, A2 = X G2 recomputed.  64 rows per CTA.  `add` (optional, [rows][64]): gradient
+// that reached X without passing through the sketch, added before the result is rounded.
 // ---------------------------------------------------------------------------
 template <typename T, int R>
 __global__ void __launch_bounds__(256)
 sketch_bwd_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const T* __restrict__ G2,
-                  int g_heads, int n, const float* __restrict__ dM, T* __restrict__ dX) {
+                  int g_heads, int n, const float* __restrict__ dM, const float* __restrict__ add,
+                  T* __restrict__ dX) {
     extern __shared__ float smem[];
     float* sG1 = smem;                      // [64][R+1]
     float* sG2 = sG1 + H64 * (R + 1);       // [64][R+1]
@@ -451,7 +545,7 @@ sketch_bwd_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, c
     {
         const int t = tid % 64;
         for (int rr = tid / 64; rr < 64; rr += 4) {
-            float dx = 0.f;
+            float dx = add != nullptr ? add[((size_t)bh * n + i0 + rr) * 64 + t] : 0.f;
 #pragma unroll 16
             for (int c = 0; c < R; ++c) {
                 dx = fmaf(sU1[rr * (R + 1) + c], sG1[t * (R + 1) + c], dx);
@@ -518,10 +612,16 @@ cudaError_t fwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     ++*launches;
     PSK_TRY(cudaGetLastError());
     PSK_TRY((launch_states<R>(d, Mk, Vt, Z, false, s, launches)));
-    PSK_TRY(allow_smem(fwd_out_kernel<T, R>, RowSmem<R>::bytes));
     prof_begin("fwd_out_kernel", s);
-    fwd_out_kernel<T, R><<<dim3(d.b / 128, d.t, d.BH()), 128, RowSmem<R>::bytes, s>>>(
-        sl, d.n, d.b, d.t, Mq, Mk, Vt, Z, O, denom);
+    if (d.local) {
+        PSK_TRY((allow_smem(fwd_out_kernel<T, R, true>, RowSmem<R>::bytes_local)));
+        fwd_out_kernel<T, R, true><<<dim3(d.b / 128, d.t, d.BH()), 128, RowSmem<R>::bytes_local, s>>>(
+            sl, d.n, d.b, d.t, Mq, Mk, Vt, Z, Q, K, O, denom);
+    } else {
+        PSK_TRY((allow_smem(fwd_out_kernel<T, R, false>, RowSmem<R>::bytes)));
+        fwd_out_kernel<T, R, false><<<dim3(d.b / 128, d.t, d.BH()), 128, RowSmem<R>::bytes, s>>>(
+            sl, d.n, d.b, d.t, Mq, Mk, Vt, Z, Q, K, O, denom);
+    }
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -550,24 +650,37 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     PSK_TRY(cudaGetLastError());
     PSK_TRY((launch_states<R>(d, Mk, Vt, Z, false, s, launches)));
     PSK_TRY((launch_states<R>(d, Mq, E, Rs, true, s, launches)));
-    PSK_TRY(allow_smem(bwd_q_kernel<R>, RowSmem<R>::bytes));
-    PSK_TRY(allow_smem(bwd_k_kernel<T, R>, RowSmem<R>::bytes));
     const dim3 grid(d.b / 128, d.t, d.BH());
-    prof_begin("bwd_q_kernel", s);
-    bwd_q_kernel<R><<<grid, 128, RowSmem<R>::bytes, s>>>(d.n, d.b, d.t, Mq, Mk, Vt, E, Z, dMq);
-    prof_end(s);
-    prof_begin("bwd_k_kernel", s);
-    bwd_k_kernel<T, R><<<grid, 128, RowSmem<R>::bytes, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Rs, dMk, dV);
-    prof_end(s);
+    float* dXq = d.local ? (float*)(ws + w.dXq) : nullptr;
+    float* dXk = d.local ? (float*)(ws + w.dXk) : nullptr;
+    if (d.local) {
+        PSK_TRY((allow_smem(bwd_q_kernel<T, R, true>, RowSmem<R>::bytes_local)));
+        PSK_TRY((allow_smem(bwd_k_kernel<T, R, true>, RowSmem<R>::bytes_local)));
+        prof_begin("bwd_q_kernel", s);
+        bwd_q_kernel<T, R, true><<<grid, 128, RowSmem<R>::bytes_local, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Z, Q, K, dMq, dXq);
+        prof_end(s);
+        prof_begin("bwd_k_kernel", s);
+        bwd_k_kernel<T, R, true><<<grid, 128, RowSmem<R>::bytes_local, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Rs, Q, K, dMk, dXk, dV);
+        prof_end(s);
+    } else {
+        PSK_TRY((allow_smem(bwd_q_kernel<T, R, false>, RowSmem<R>::bytes)));
+        PSK_TRY((allow_smem(bwd_k_kernel<T, R, false>, RowSmem<R>::bytes)));
+        prof_begin("bwd_q_kernel", s);
+        bwd_q_kernel<T, R, false><<<grid, 128, RowSmem<R>::bytes, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Z, Q, K, dMq, nullptr);
+        prof_end(s);
+        prof_begin("bwd_k_kernel", s);
+        bwd_k_kernel<T, R, false><<<grid, 128, RowSmem<R>::bytes, s>>>(sl, d.n, d.b, d.t, Mq, Mk, Vt, E, Rs, Q, K, dMk, nullptr, dV);
+        prof_end(s);
+    }
     *launches += 2;
     PSK_TRY(cudaGetLastError());
     const size_t smem = (size_t)(2 * H64 * (R + 1) + 64 * 65 + 2 * 64 * (R + 1)) * sizeof(float);
     PSK_TRY(allow_smem(sketch_bwd_kernel<T, R>, smem));
     prof_begin("sketch_bwd_kernel", s);
-    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dQ);
+    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dXq, dQ);
     prof_end(s);
     prof_begin("sketch_bwd_kernel", s);
-    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dK);
+    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dXk, dK);
     prof_end(s);
     *launches += 2;
     return cudaGetLastError();

@@ -17,6 +17,7 @@ struct Dims {
     int g_heads;                      // 1 or H
     bool bf16;                        // storage type
     bool keep_states;                 // PSK_FLAG_KEEP_STATES
+    bool local;                       // PSK_FLAG_LOCAL_EXACT
     int BH() const { return B * H; }
 };
 
@@ -27,7 +28,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Scratch layout of the CUDA-core path (all fp32).
 struct CcWorkspace {
-    size_t status, Mq, Mk, Vt, Zst, E, Rst, dMq, dMk, total;
+    size_t status, Mq, Mk, Vt, Zst, E, Rst, dMq, dMk, dXq, dXk, total;
 };
 CcWorkspace cc_workspace(const Dims& d, bool backward);
 

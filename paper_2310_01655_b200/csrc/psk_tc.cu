@@ -925,7 +925,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
-    return d.bf16 && encoder() != nullptr;
+    // (exact same-block weights, Section 3.2: CUDA-core kernels only so far)
+    return d.bf16 && !d.local && encoder() != nullptr;
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
