@@ -420,7 +420,7 @@ constexpr uint32_t kZStageBytes = 16384;        // two [64 features x 128 B] box
 constexpr int kFeatBufs = kZStages;             // feature staging buffers in tensor memory, 32 columns each:
                                                 // chunk C uses buffer and stage C % 4, both freed by its MMAs
 
-template <int R>
+template <int R, bool LOCAL = false>
 struct OutSmem {
     // The prefix-state stages (first phase), the key/value tiles with the keys' split half
     // sketches (second phase) and the output staging tiles (epilogue) share one region; small
@@ -428,12 +428,16 @@ struct OutSmem {
     static constexpr uint32_t Q = 0, G = 16384;
     static constexpr uint32_t Ones = G + GImage<R>::bytes;           // 4 KB of bf16 1.0: B operand of the row sums
     static constexpr uint32_t Mq = Ones + 4096;
-    static constexpr uint32_t U = (Mq + 128 * 3 * R * 2 + 1023) / 1024 * 1024;   // split operand: 3R columns
+    // split operand: 3R columns.  (LOCAL: no split operands; the region holds the ring's last
+    // stage and then the value tile, because the query tile stays alive for the exact scores.)
+    static constexpr uint32_t kMqBytes = (LOCAL && 128 * 3 * R * 2 < 16384) ? 16384 : 128 * 3 * R * 2;
+    static constexpr uint32_t U = (Mq + kMqBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t Z = U;
     // key tile in ring stage 1, value tile in the query tile's buffer (ring stage 3), split key
     // sketches over stage 2: the stages the last chunks free first, so the first key/value tile is
     // fetched while the last chunks are still being multiplied
-    static constexpr uint32_t K = U + 16384, V = Q, Mk = U + 32768;
+    static constexpr uint32_t Z3 = LOCAL ? Mq : Q;                   // ring stage 3
+    static constexpr uint32_t K = U + 16384, V = Z3, Mk = U + 32768;
     static constexpr int kStageK = 1, kStageV = kZStages - 1;
     // last chunk that uses ring stage s (-1: none)
     __host__ __device__ static constexpr int last_chunk(int nc, int s) { return nc > s ? s + (nc - 1 - s) / kZStages * kZStages : -1; }
@@ -442,7 +446,7 @@ struct OutSmem {
     static constexpr uint32_t kMax12 = kPhase1 > kPhase2 ? kPhase1 : kPhase2;
     static constexpr uint32_t total = U + (kMax12 > kEpi ? kMax12 : kEpi);
     // stage s of the prefix-state ring; the last one is the query tile's buffer, dead after the sketch
-    __device__ static uint32_t zstage(int s) { return s < kZStages - 1 ? Z + s * kZStageBytes : Q; }
+    __device__ static uint32_t zstage(int s) { return s < kZStages - 1 ? Z + s * kZStageBytes : Z3; }
 };
 
 
@@ -450,7 +454,10 @@ struct OutSmem {
 // recomputation of the row numerators against centred prefix states; writes E = dO/d (bf16),
 // e65 = -(dO.(O - c))/d and e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32
 // accumulators rather than from the rounded O the caller holds.
-template <int R, int MODE>
+// LOCAL (Section 3.2): the same-block scores are (q_i . k_j)^2 from the raw query and key tiles
+// (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
+// they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
+template <int R, int MODE, bool LOCAL>
 __global__ void __launch_bounds__(160, (R <= 32 ? 2 : 1))
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
@@ -460,7 +467,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                   float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
                   float* __restrict__ e65, float* __restrict__ e65h, int keep_oc, int* status) {
     using F = Feat<R>;
-    using L = OutSmem<R>;
+    using L = OutSmem<R, LOCAL>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_q, bar_kv, bar_sk, bar_go, bar_mk, bar_s, bar_p, bar_pv;
@@ -529,7 +536,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 // staged" and "MMAs issued" lie the four MMA instructions and nothing else.  (The
                 // stages are refilled by the rows' side, which learns first that a buffer is free.)
                 const uint64_t zd0 = smem_desc(smem_u32(smem + L::Z), 8192, 1024, kSwz128);
-                const uint64_t zdq = smem_desc(smem_u32(smem + L::Q), 8192, 1024, kSwz128);
+                const uint64_t zdq = smem_desc(smem_u32(smem + L::Z3), 8192, 1024, kSwz128);
 #pragma unroll 1
                 for (int C = 0; C < F::NC && ok; ++C) {
                     const int s = C % kZStages;
@@ -577,11 +584,20 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 }
                 ok = ok && mbar_spin(&bar_kv, tp & 1, status, kErrTma);
                 tc_fence_after();
-                issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
-                umma_commit(&bar_sk);
-                ok = ok && mbar_spin(&bar_mk, tp & 1, status, kErrMma);
-                tc_fence_after();
-                {
+                if constexpr (LOCAL) {
+                    // scores = Q_tile K_tile^T over the head dimension
+                    constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
+                    const uint64_t qr = smem_desc(smem_u32(smem + L::Q), 0, 1024, kSwz128);
+                    const uint64_t kr = smem_desc(smem_u32(smem + L::K), 0, 1024, kSwz128);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_ss(tm + cS, desc_off(qr, k * 32), desc_off(kr, k * 32), idesc, k > 0);
+                    umma_commit(&bar_s);
+                } else {
+                    issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
+                    umma_commit(&bar_sk);
+                    ok = ok && mbar_spin(&bar_mk, tp & 1, status, kErrMma);
+                    tc_fence_after();
                     constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
 #pragma unroll
                     for (int k = 0; k < 3 * R / 16; ++k)
@@ -611,7 +627,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         tc_fence_after();
         float mq[R];
         read_half_sketch<R>(lane_tm + cSk, mq);
-        store_split_rows<R, true>(smem + L::Mq, mq, tid);
+        if constexpr (!LOCAL) store_split_rows<R, true>(smem + L::Mq, mq, tid);
         tc_fence_before();
         mbar_arrive(&bar_go);
 
@@ -667,16 +683,18 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
 #pragma unroll 1
         for (int tp = 0; tp <= tau && ok; ++tp) {
-            ok = mbar_wait(&bar_sk, (tp + 1) & 1, status, kErrMma);
-            tc_fence_after();
-            {
-                float mk[R];
-                read_half_sketch<R>(lane_tm + cSk, mk);
-                store_split_rows<R, false>(smem + L::Mk, mk, tid);
+            if constexpr (!LOCAL) {
+                ok = mbar_wait(&bar_sk, (tp + 1) & 1, status, kErrMma);
+                tc_fence_after();
+                {
+                    float mk[R];
+                    read_half_sketch<R>(lane_tm + cSk, mk);
+                    store_split_rows<R, false>(smem + L::Mk, mk, tid);
+                }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(&bar_mk);
             }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            mbar_arrive(&bar_mk);
             ok = ok && mbar_wait(&bar_s, tp & 1, status, kErrMma);
             tc_fence_after();
             // weights = squared scores (lower triangle on the diagonal tile), packed to bf16 over
@@ -697,7 +715,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 }
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
+                    float w0 = __uint_as_float(v[j]), w1 = __uint_as_float(v[j + 1]);
+                    if constexpr (LOCAL) { w0 *= w0; w1 *= w1; }          // (q . k)^2, squared once more below
                     pk[j / 2] = pack_bf16(w0 * w0, w1 * w1);
                 }
                 tmem_st16(lane_tm + cW + gq * 16, pk);
@@ -910,12 +929,20 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
     PSK_TRY((launch_states<R>(d, mK, mV, gimg, nullptr, cmean, cmean ? 1 : 0, Z, false,
                               status, s, launches)));
-    constexpr size_t smem = OutSmem<R>::total + 1024;
-    PSK_TRY(set_smem(tc_fwd_out_kernel<R, 0>, smem));
     prof_begin("tc_fwd_out_kernel", s);
-    tc_fwd_out_kernel<R, 0><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
-        mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-        denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+    if (d.local) {
+        constexpr size_t smem = OutSmem<R, true>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true>, smem)));
+        tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+    } else {
+        constexpr size_t smem = OutSmem<R, false>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false>, smem)));
+        tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+    }
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -925,8 +952,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
-    // (exact same-block weights, Section 3.2: CUDA-core kernels only so far)
-    return d.bf16 && !d.local && encoder() != nullptr;
+    // (exact same-block weights, Section 3.2: forward here, backward on the CUDA-core kernels so far)
+    return d.bf16 && !(d.local && backward) && encoder() != nullptr;
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
@@ -953,12 +980,20 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
                                   const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean,
                                   const float* denom, const bf16* dO, bf16* E, float* e65, float* e65h, int* status,
                                   cudaStream_t s, int* launches) {
-    constexpr size_t smem = OutSmem<R>::total + 1024;
-    PSK_TRY(set_smem(tc_fwd_out_kernel<R, 1>, smem));
     prof_begin("tc_bwd_recompute_kernel", s);
-    tc_fwd_out_kernel<R, 1><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
-        mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-        const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
+    if (d.local) {
+        constexpr size_t smem = OutSmem<R, true>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true>, smem)));
+        tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
+    } else {
+        constexpr size_t smem = OutSmem<R, false>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false>, smem)));
+        tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
+    }
     prof_end(s);
     ++*launches;
     return cudaGetLastError();

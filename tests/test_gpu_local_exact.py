@@ -33,16 +33,18 @@ def test_forward_and_backward_small(r, b, n, dtype):
     w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype=dtype, seed=5 * r + b)
     inp = wl.make_inputs(w, "cuda")
     args = (inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"])
-    O, den = psk.causal_attn_fwd(*args, b, flags=LOCAL)
-    dQ, dK, dV = psk.causal_attn_bwd(*args, O, den, inp["dO"], b, flags=LOCAL)
-    torch.cuda.synchronize()
-    for bi in range(w.B):
-        for hi in range(w.H):
-            (O_ref, d_ref), g = _oracle(inp, bi, hi, b, True)
-            check("O", O[bi, hi], O_ref, TOL[dtype])
-            check("denom", den[bi, hi], d_ref, TOL[dtype])
-            for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), g):
-                check(name, got[bi, hi], ref, TOL[dtype])
+    # bf16 storage: the tensor-core kernels (PATH_AUTO) and the CUDA-core kernels
+    for path in ([psk.PATH_CUDA_CORES] if dtype == "f32" else [psk.PATH_CUDA_CORES, psk.PATH_AUTO]):
+        O, den = psk.causal_attn_fwd(*args, b, path=path, flags=LOCAL)
+        dQ, dK, dV = psk.causal_attn_bwd(*args, O, den, inp["dO"], b, path=path, flags=LOCAL)
+        torch.cuda.synchronize()
+        for bi in range(w.B):
+            for hi in range(w.H):
+                (O_ref, d_ref), g = _oracle(inp, bi, hi, b, True)
+                check("O", O[bi, hi], O_ref, TOL[dtype])
+                check("denom", den[bi, hi], d_ref, TOL[dtype])
+                for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), g):
+                    check(name, got[bi, hi], ref, TOL[dtype])
 
 
 def test_single_block_is_exact_polynomial_attention():
@@ -77,10 +79,12 @@ def test_flag_changes_only_same_block_pairs():
     assert torch.equal(O3[:, :, :c], O_loc[:, :, :c]) and torch.equal(den3[:, :, :c], den[:, :, :c])
 
 
-def test_tensor_core_path_refuses_the_flag():
+def test_tensor_core_backward_refuses_the_flag():
+    # forward: tensor-core kernels; backward: CUDA-core kernels only (PATH_AUTO picks them)
     w = wl.small_workload(B=1, H=1, n=256, r=32, b=256, dtype="bf16", seed=79)
     inp = wl.make_inputs(w, "cuda")
+    args = (inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"])
+    O, den = psk.causal_attn_fwd(*args, 256, path=psk.PATH_TENSOR_CORES, flags=LOCAL)
     with pytest.raises(psk.PskError) as e:
-        psk.causal_attn_fwd(inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"], 256,
-                            path=psk.PATH_TENSOR_CORES, flags=LOCAL)
+        psk.causal_attn_bwd(*args, O, den, inp["dO"], 256, path=psk.PATH_TENSOR_CORES, flags=LOCAL)
     assert e.value.code == -2
