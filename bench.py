@@ -30,14 +30,16 @@ UNIT = "model-tokens/s"
 # flop model (GEMM flops only, per head-token); "nominal" follows the paper's statement
 # of the algorithm (r^2 features, h+1 columns, full b x b diagonal tiles)
 # ---------------------------------------------------------------------------
-def nominal_flops_per_head_token(w):
+def nominal_flops_per_head_token(w, local=False):
+    """local: exact same-block weights (Section 3.2): the b x b tiles contract over h, not r."""
     h, r, b = w.h, w.r, w.b
-    fwd = 8 * h * r + 4 * r * r * (h + 1) + 2 * b * (r + h + 1)
-    bwd = 10 * r * r * (h + 1) + 6 * b * r + 4 * b * (h + 1) + 16 * h * r
+    kd = h if local else r
+    fwd = 8 * h * r + 4 * r * r * (h + 1) + 2 * b * (kd + h + 1)
+    bwd = 10 * r * r * (h + 1) + 6 * b * kd + 4 * b * (h + 1) + 16 * h * r
     return fwd, (bwd if w.backward else 0)
 
 
-def kernel_flops_per_head_token(name, w):
+def kernel_flops_per_head_token(name, w, local=False):
     """Executed flops of one launch of a library kernel, per head-token it covers."""
     h, r, b = w.h, w.r, w.b
     k = h + 1
@@ -62,6 +64,9 @@ def kernel_flops_per_head_token(name, w):
     sk = 2 * h * 2 * r                  # one half-sketch GEMM
     tile_fwd = sk + 2 * 128 * 3 * r + 2 * 128 * h
     tile_bwd = sk + 2 * 128 * 3 * r + 2 * 128 * h + 2 * 128 * 64
+    if local:                           # scores over h, no sketch of the other tile; dX product 64 wide
+        tile_fwd = 2 * 128 * h + 2 * 128 * h
+        tile_bwd = 2 * 128 * h + 2 * 128 * h + 2 * 128 * 64
     table.update({
         "tc_state_kernel": sk * (1 if r <= 32 else 5) + 2 * FP * 80,
         "tc_fwd_out_kernel": sk + 2 * FK * 80 + other * tile_fwd,
@@ -131,15 +136,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_step(w, inp_host, head):
+def oracle_step(w, inp_host, head, local=False):
     """One bounded sample of the workload for the CPU oracle: forward (+ backward) of one
     (batch, head) slice at full n.  Returns seconds."""
     from oracle import polysketch as orc
     Q, K, V, dO, G1, G2 = inp_host[head]
+    diag = "exact" if local else "LR"
     t0 = time.perf_counter()
-    orc.causal_polysketch_attention_blocked(Q, K, V, G1, G2, w.b)
+    orc.causal_polysketch_attention_blocked(Q, K, V, G1, G2, w.b, diagonal=diag)
     if w.backward:
-        orc.causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, w.b)
+        orc.causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, w.b, diagonal=diag)
     return time.perf_counter() - t0
 
 
@@ -173,8 +179,8 @@ def run_reference(args, w):
     heads = list(range(max(1, min(2, args.steps + args.warmup))))
     data = host_head_inputs(w, heads)
     for i in range(args.warmup):
-        oracle_step(w, data, i % len(data))
-    times = [oracle_step(w, data, i % len(data)) for i in range(args.steps)]
+        oracle_step(w, data, i % len(data), args.local_exact)
+    times = [oracle_step(w, data, i % len(data), args.local_exact) for i in range(args.steps)]
     total = sum(times)
     value = (w.n * args.steps / total) / w.H          # head-tokens/s -> model-tokens/s
     line = {
@@ -183,6 +189,7 @@ def run_reference(args, w):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
                    "passes": "fwd+bwd" if w.backward else "fwd",
+                   "variant": "local_exact" if args.local_exact else "polysketch",
                    "step": "oracle on one (batch, head) slice at full n; value extrapolated over heads"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                          "sample": "%d steps x 1 head slice of %s at n=%d" % (args.steps, w.name, w.n)},
@@ -204,6 +211,8 @@ def main():
     ap.add_argument("--cpu-heads", type=int, default=12, help="head slices the CPU baseline leg times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--local-exact", action="store_true",
+                    help="exact polynomial weights inside each block (Section 3.2) instead of the headline variant")
     ap.add_argument("--no-keep-states", action="store_true",
                     help="let the backward rebuild the prefix states instead of reading the forward's")
     args = ap.parse_args()
@@ -233,6 +242,9 @@ def main():
     Q, K, V, dO, G1, G2 = (inp[k] for k in ("Q", "K", "V", "dO", "G1", "G2"))
     # forward and backward of one step share the workspace: the backward reads the forward's states
     flags = psk.FLAG_KEEP_STATES if (w.backward and not args.no_keep_states) else 0
+    keep = bool(flags)
+    if args.local_exact:
+        flags |= psk.FLAG_LOCAL_EXACT
     shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path, flags)
     ws_bytes = max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True) if w.backward else 0)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
@@ -356,7 +368,7 @@ def main():
     roof = None
     if top[0] is not None:
         name, (cnt, tot) = top
-        fl = kernel_flops_per_head_token(name, w)
+        fl = kernel_flops_per_head_token(name, w, args.local_exact)
         tensor = name.startswith("tc_")
         peak = pk["bf16_sustained"] if tensor else ALU_PEAK_TFLOPS
         achieved = (fl * w.head_tokens / ((tot / cnt) / 1e3) / 1e12) if fl else None
@@ -381,13 +393,13 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         heads = list(range(args.cpu_heads))
         data = host_head_inputs(w, heads)
-        secs = sum(oracle_step(w, data, i) for i in range(len(heads)))
+        secs = sum(oracle_step(w, data, i, args.local_exact) for i in range(len(heads)))
         cpu = {"value": (w.n * len(heads) / secs) / w.H, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": "%d (batch, head) slices of %s at full n=%d, %s; extrapolated linearly over heads"
                          % (len(heads), w.name, w.n, "fwd+bwd" if w.backward else "fwd"),
                "seconds": secs}
 
-    f_fwd, f_bwd = nominal_flops_per_head_token(w)
+    f_fwd, f_bwd = nominal_flops_per_head_token(w, args.local_exact)
     nominal_tflops = (f_fwd + f_bwd) * w.head_tokens * world * args.steps / (ms / 1e3) / 1e12
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -395,7 +407,8 @@ def main():
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
                    "passes": "fwd+bwd" if w.backward else "fwd", "path": args.path,
-                   "keep_states": bool(flags),
+                   "variant": "local_exact" if args.local_exact else "polysketch",
+                   "keep_states": keep,
                    "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
         "nominal_tflops": nominal_tflops,
         "frac_bf16_peak": {"burst": nominal_tflops / world / pk["bf16_burst"],

@@ -87,9 +87,9 @@ typedef struct {
  * unchanged.  The result now depends on b (more exact pairs with larger blocks; b = n is exact
  * degree-4 polynomial attention).  Set it on the forward and on the backward call alike; the
  * backward sends the same-block part of dQ, dK straight to Q and K instead of through the
- * sketch.  bf16 storage: the forward runs on the tensor-core kernels, the backward on the
- * CUDA-core kernels (PSK_PATH_AUTO selects them; PSK_PATH_TENSOR_CORES with this flag on the
- * backward call is PSK_ERR_UNSUPPORTED).  fp32 storage: CUDA-core kernels. */
+ * sketch.  Both paths serve it (bf16 storage: tensor-core kernels, scores from the raw bf16
+ * rows with fp32 accumulation; fp32 storage: CUDA-core kernels), and it combines with
+ * PSK_FLAG_KEEP_STATES. */
 typedef enum { PSK_FLAG_KEEP_STATES = 1, PSK_FLAG_LOCAL_EXACT = 2 } psk_flags;
 
 /* Library version (major*100 + minor). */

@@ -952,8 +952,7 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
-    // (exact same-block weights, Section 3.2: forward here, backward on the CUDA-core kernels so far)
-    return d.bf16 && !(d.local && backward) && encoder() != nullptr;
+    return d.bf16 && encoder() != nullptr;
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {

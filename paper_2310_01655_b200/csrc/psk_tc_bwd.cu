@@ -124,7 +124,12 @@ __device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint32_t own, uint
     }
 }
 
-template <int R, bool QSIDE>
+// LOCAL (Section 3.2): same-block pairs carry the exact weights x_ij^4, x_ij = q_i . k_j.  The
+// tile scores are then X_own X_other^T over the head dimension (raw bf16 rows: exact products),
+// dL/dx_ij = 4 x_ij^3 dW_ij replaces ds_ij, and it multiplies the other side's raw rows straight
+// into a dX accumulator that the sketch's backward (phase D) adds to: no half sketch of the other
+// tile, no split operands, no dM from the tiles.
+template <int R, bool QSIDE, bool LOCAL>
 __global__ void __launch_bounds__(128, (R <= 32 ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
@@ -211,6 +216,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     constexpr bool kTsA = (R <= 32);
     constexpr uint32_t cYA = cdM + 32;
     constexpr int kNdM = kTsA ? R : 64;                   // columns the dM GEMM writes
+    // LOCAL: the tiles' dX accumulator (64 columns).  Query side, r <= 32: the unused dV columns.
+    // Otherwise the dM columns -- on the key side with r <= 32 that includes the Y operand's,
+    // which phase C then reads from shared memory instead.
+    constexpr bool kTsC = kTsA && !(LOCAL && !QSIDE);
+    constexpr uint32_t cXl = (kTsA && QSIDE) ? cdV : cdM;
     uint32_t mma_uses = 0;
     bool ok = true;
 
@@ -419,7 +429,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     }
 
     // ---- phase C: same block, other-side tiles, 64 other rows at a time ----
-    store_hilo_tiles<R>(smem + L::Mown, m, tid);
+    if constexpr (!LOCAL) store_hilo_tiles<R>(smem + L::Mown, m, tid);
     const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
     bool dm_started = false;
     uint32_t oth_uses = 0;
@@ -444,17 +454,19 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             }
         }
         ok = mbar_wait(&bar_xoth, oth_uses & 1, status, kErrTma);
-        if (tid == 0) {
+        if constexpr (!LOCAL) {
+            if (tid == 0) {
+                tc_fence_after();
+                issue_sketch<R>(tm + cSk, smem + L::Xoth, smem + L::G);
+                umma_commit(&bar_mma);
+            }
+            ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
             tc_fence_after();
-            issue_sketch<R>(tm + cSk, smem + L::Xoth, smem + L::G);
-            umma_commit(&bar_mma);
         }
-        ok = ok && mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
         ok = ok && mbar_wait(&bar_yoth, oth_uses & 1, status, kErrTma);
         ++oth_uses;
-        {
+        if constexpr (!LOCAL) {
             float mo[R];
             read_half_sketch<R>(lane_tm + cSk, mo);
             store_hilo_tiles<R>(smem + L::Moth, mo, tid);
@@ -470,16 +482,24 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 // The X tile has been consumed, and every thread is past its wait for it (a
                 // barrier must not complete twice before its slowest waiter has looked): next
                 // tile's rows.
-                if (hh == 0 && tp + 1 < tp_end) {
+                // (LOCAL: the raw rows are operands of this tile's GEMMs to its end; see below)
+                if (!LOCAL && hh == 0 && tp + 1 < tp_end) {
                     mbar_expect_tx(&bar_xoth, 16384);
                     tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
                 }
-                issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
+                if constexpr (LOCAL) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)       // x = own rows . other rows, over the head dimension
+                        umma_ss(tm + cS, desc_off(smem_desc(smem_u32(smem + L::Xown), 0, 1024, kSwz128), k * 32),
+                                desc_off(smem_desc(smem_u32(smem + L::Xoth) + hh * 8192, 0, 1024, kSwz128), k * 32), idesc, k > 0);
+                } else {
+                    issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
+                }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {         // dW without its 65th-column term
                     const uint64_t yod = desc_off(smem_desc(smem_u32(smem + L::Yoth) + hh * 8192, 0, 1024, kSwz128), k * 32);
-                    if constexpr (kTsA) umma_ts(tm + cDW, tm + cYA + k * 8, yod, idesc, k > 0);
+                    if constexpr (kTsC) umma_ts(tm + cDW, tm + cYA + k * 8, yod, idesc, k > 0);
                     else umma_ss(tm + cDW, desc_off(smem_desc(smem_u32(smem + L::Yown), 0, 1024, kSwz128), k * 32), yod, idesc, k > 0);
                 }
                 umma_commit(&bar_mma);
@@ -510,8 +530,14 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                             inv = o.x; yinv = o.y;
                         }
                         const float dw = fmaf(__uint_as_float(wv[j]), inv, yinv);
-                        sv[j] = __float_as_uint((s + s) * dw);
-                        wv[j] = __float_as_uint(s * (s * inv));     // weight / d_i: the value side sees g_i / d_i
+                        if constexpr (LOCAL) {
+                            const float s2 = s * s;                     // s is x_ij here
+                            sv[j] = __float_as_uint(4.f * s * s2 * dw);
+                            wv[j] = __float_as_uint(s2 * (s2 * inv));
+                        } else {
+                            sv[j] = __float_as_uint((s + s) * dw);
+                            wv[j] = __float_as_uint(s * (s * inv));     // weight / d_i: the value side sees g_i / d_i
+                        }
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -530,11 +556,19 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 tc_fence_after();
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
                 constexpr uint32_t idesc_dm = idesc_bf16(128, kNdM, false, true);
+                if constexpr (LOCAL) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)           // dM_own += dS x M_other (its hi columns)
-                    umma_ts(tm + cdM, tm + cS + k * 8,
-                            desc_off(smem_desc(smem_u32(smem + L::Moth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc_dm,
-                            (dm_started || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < 4; ++k)       // dX_own += dx x X_other
+                        umma_ts(tm + cXl, tm + cS + k * 8,
+                                desc_off(smem_desc(smem_u32(smem + L::Xoth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
+                                (dm_started || k > 0) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)       // dM_own += dS x M_other (its hi columns)
+                        umma_ts(tm + cdM, tm + cS + k * 8,
+                                desc_off(smem_desc(smem_u32(smem + L::Moth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc_dm,
+                                (dm_started || k > 0) ? 1u : 0u);
+                }
                 if constexpr (!QSIDE) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)       // dV += W x E_other
@@ -553,6 +587,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         if (tid == 0 && tp + 1 < tp_end) {        // every MMA that read the Y tile has completed
             mbar_expect_tx(&bar_yoth, 16384);
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0 + 128, hi, bi, &bar_yoth);
+            if constexpr (LOCAL) {                // ... and the X tile
+                mbar_expect_tx(&bar_xoth, 16384);
+                tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
+            }
         }
     }
 
@@ -560,13 +598,18 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     if (ok) {
         const float rs = rsqrtf((float)R);
         // dM total = state part (registers) + tile part (tensor memory), scaled by 1/sqrt(R)
+        if constexpr (LOCAL) {
 #pragma unroll
-        for (int c0 = 0; c0 < R; c0 += 16) {
-            uint32_t v[16];
-            tmem_ld16(lane_tm + cdM + c0, v);
-            tmem_ld_wait();
+            for (int c = 0; c < R; ++c) dm[c] *= rs;
+        } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + __uint_as_float(v[j])) * rs;
+            for (int c0 = 0; c0 < R; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(lane_tm + cdM + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + __uint_as_float(v[j])) * rs;
+            }
         }
         tc_fence_before();
         __syncthreads();
@@ -580,7 +623,12 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         tc_fence_after();
     }
     if (ok) {
-        // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cdM)
+        // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cdM).
+        // LOCAL: the dM columns may hold the tiles' dX accumulator, so U goes over the sketch
+        // columns this thread has just read (dM*A2 from column 0, dM*A1 from column R), and the
+        // GEMM adds to that accumulator.
+        constexpr uint32_t cU1 = LOCAL ? cSk : cdM, cU2 = LOCAL ? cSk + R : cdM + R / 2;
+        constexpr uint32_t cDX = LOCAL ? cXl : cS;
 #pragma unroll
         for (int c0 = 0; c0 < R; c0 += 16) {
             uint32_t a1[16], a2[16], u1[8], u2[8];
@@ -594,8 +642,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 u2[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a1[2 * j]),
                                   dm[c0 + 2 * j + 1] * __uint_as_float(a1[2 * j + 1]));
             }
-            tmem_st8(lane_tm + cdM + c0 / 2, u1);
-            tmem_st8(lane_tm + cdM + R / 2 + c0 / 2, u2);
+            tmem_st8(lane_tm + cU1 + c0 / 2, u1);
+            tmem_st8(lane_tm + cU2 + c0 / 2, u2);
         }
         tmem_st_wait();
         tc_fence_before();
@@ -605,8 +653,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
 #pragma unroll
             for (int k = 0; k < 2 * R / 16; ++k)    // contraction over the 2R sketch columns
-                umma_ts(tm + cS, tm + cdM + k * 8, desc_off(smem_desc(smem_u32(smem + L::G), 0, 1024, kSwz128), k * 2048), idesc,
-                        k > 0);
+                umma_ts(tm + cDX, tm + (k < R / 16 ? cU1 + k * 8 : cU2 + (k - R / 16) * 8),
+                        desc_off(smem_desc(smem_u32(smem + L::G), 0, 1024, kSwz128), k * 2048), idesc, (LOCAL || k > 0) ? 1u : 0u);
             umma_commit(&bar_mma);
         }
         ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
@@ -620,7 +668,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
             uint32_t v[32];
-            tmem_ld32(lane_tm + cS + c0, v);
+            tmem_ld32(lane_tm + (LOCAL ? cXl : cS) + c0, v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; j += 8)
@@ -700,24 +748,28 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
     }
     constexpr size_t smem = BwdSmem<R>::total + 1024;
-    PSK_TRY(set_smem(tc_bwd_rows_kernel<R, true>, smem));
-    PSK_TRY(set_smem(tc_bwd_rows_kernel<R, false>, smem));
     const dim3 grid(d.b / 128, d.t, d.BH());
-    // query side first: it needs only the prefix states, and the row scalars just written are
-    // still in L2; the suffix states (5 GB through L2) come after it
-    prof_begin("tc_bwd_q_kernel", s);
-    tc_bwd_rows_kernel<R, true><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n, d.b, d.t,
-                                                        e65, e65h, denom, status);
-    prof_end(s);
-    ++*launches;
-    PSK_TRY(cudaGetLastError());
-    PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
-    prof_begin("tc_bwd_k_kernel", s);
-    tc_bwd_rows_kernel<R, false><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n, d.b, d.t,
-                                                         e65, e65h, denom, status);
-    prof_end(s);
-    ++*launches;
-    return cudaGetLastError();
+    auto rows = [&](auto local_c) -> cudaError_t {
+        constexpr bool LOCAL = decltype(local_c)::value;
+        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, true, LOCAL>, smem)));
+        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, false, LOCAL>, smem)));
+        // query side first: it needs only the prefix states, and the row scalars just written are
+        // still in L2; the suffix states (5 GB through L2) come after it
+        prof_begin("tc_bwd_q_kernel", s);
+        tc_bwd_rows_kernel<R, true, LOCAL><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
+                                                                   d.b, d.t, e65, e65h, denom, status);
+        prof_end(s);
+        ++*launches;
+        PSK_TRY(cudaGetLastError());
+        PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
+        prof_begin("tc_bwd_k_kernel", s);
+        tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
+                                                                    d.b, d.t, e65, e65h, denom, status);
+        prof_end(s);
+        ++*launches;
+        return cudaGetLastError();
+    };
+    return d.local ? rows(std::true_type{}) : rows(std::false_type{});
 }
 
 }  // namespace

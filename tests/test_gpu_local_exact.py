@@ -79,12 +79,45 @@ def test_flag_changes_only_same_block_pairs():
     assert torch.equal(O3[:, :, :c], O_loc[:, :, :c]) and torch.equal(den3[:, :, :c], den[:, :, :c])
 
 
-def test_tensor_core_backward_refuses_the_flag():
-    # forward: tensor-core kernels; backward: CUDA-core kernels only (PATH_AUTO picks them)
-    w = wl.small_workload(B=1, H=1, n=256, r=32, b=256, dtype="bf16", seed=79)
+@pytest.mark.parametrize("r,b,n,corr", [(32, 256, 1024, False), (16, 128, 512, True), (64, 512, 1024, True),
+                                        (32, 256, 256, True), (32, 512, 2048, False)])
+def test_tensor_core_backward_reading_the_forwards_states(r, b, n, corr):
+    # both flags: forward and backward share one workspace on the tensor-core path
+    w = wl.small_workload(B=1, H=2, n=n, r=r, b=b, dtype="bf16", seed=91 + r, correlated=corr)
     inp = wl.make_inputs(w, "cuda")
     args = (inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"])
-    O, den = psk.causal_attn_fwd(*args, 256, path=psk.PATH_TENSOR_CORES, flags=LOCAL)
-    with pytest.raises(psk.PskError) as e:
-        psk.causal_attn_bwd(*args, O, den, inp["dO"], 256, path=psk.PATH_TENSOR_CORES, flags=LOCAL)
-    assert e.value.code == -2
+    flags = psk.FLAG_KEEP_STATES | LOCAL
+    shp = psk.binding.make_shape(inp["Q"], inp["G1"], r, b, path=psk.PATH_TENSOR_CORES, flags=flags)
+    ws = torch.empty(psk.workspace_bytes(shp, True), dtype=torch.uint8, device="cuda")
+    O, den = psk.causal_attn_fwd(*args, b, path=psk.PATH_TENSOR_CORES, workspace=ws, flags=flags)
+    dQ, dK, dV = psk.causal_attn_bwd(*args, O, den, inp["dO"], b, path=psk.PATH_TENSOR_CORES, workspace=ws, flags=flags)
+    assert psk.check(ws) == 0
+    for hi in range(w.H):
+        (O_ref, d_ref), g = _oracle(inp, 0, hi, b, True)
+        check("O", O[0, hi], O_ref, TOL["bf16"])
+        check("denom", den[0, hi], d_ref, TOL["bf16"])
+        for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), g):
+            check(name, got[0, hi], ref, TOL["bf16"])
+
+
+def test_full_size_configuration_2():
+    """PSK_FLAG_LOCAL_EXACT at configuration 2's full size, as `bench.py --local-exact` runs it:
+    sampled (batch, head) slices against the block-form oracle, finiteness of the full tensors."""
+    w = wl.WORKLOADS["c2"]
+    inp = wl.make_inputs(w, "cuda")
+    Q, K, V, G1, G2 = (inp[k] for k in ("Q", "K", "V", "G1", "G2"))
+    flags = psk.FLAG_KEEP_STATES | LOCAL
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, flags=flags)
+    ws = torch.empty(psk.workspace_bytes(shp, True), dtype=torch.uint8, device="cuda")
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, workspace=ws, flags=flags)
+    grads = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, inp["dO"], w.b, workspace=ws, flags=flags)
+    assert psk.check(ws) == 0
+    for t in (O, den) + tuple(grads):
+        assert torch.isfinite(t).all()
+    assert (den >= 1).all()
+    for bi, hi in ((0, 0), (w.B - 1, w.H - 1)):
+        (O_ref, d_ref), g = _oracle(inp, bi, hi, w.b, True)
+        check("O[%d,%d]" % (bi, hi), O[bi, hi], O_ref, TOL["bf16"])
+        check("denom[%d,%d]" % (bi, hi), den[bi, hi], d_ref, TOL["bf16"])
+        for nm, got, ref in zip(("dQ", "dK", "dV"), grads, g):
+            check("%s[%d,%d]" % (nm, bi, hi), got[bi, hi], ref, TOL["bf16"])
