@@ -824,10 +824,13 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     if (warp == 4) tmem_dealloc(tm, 256);
 }
 
-// Column means of V per head: cmean[bh][c] = (1/n) sum_i V[bh][i][c].  The kernels work with
-// v - cmean (and add cmean back times the row's weight sum): an exact identity that keeps the
-// bf16 states free of the common component of the values, which otherwise cancels only after
-// rounding in the backward.  One CTA per head, fixed summation order.
+// Centre of the values of a head: cmean[bh][c] = mean of V[bh][i][c] over at most 1024 rows i
+// spread evenly over the sequence (all rows when n <= 1024).  The kernels work with v - cmean
+// (and add cmean back times the row's weight sum): an exact identity for ANY constant, which keeps
+// the bf16 states free of the common component of the values -- that component otherwise cancels
+// only after rounding in the backward.  An estimate of the mean serves that purpose as well as
+// the mean itself and costs 128 KB of reads per head instead of the whole tensor.  One CTA per
+// head, fixed summation order.
 __global__ void __launch_bounds__(1024)
 tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh, int64_t sn,
                 float* __restrict__ cmean) {
@@ -837,7 +840,9 @@ tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh
     float s[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) s[j] = 0.f;
-    for (int i = rg; i < n; i += 128) {
+    const int stride = n > 1024 ? n / 1024 : 1, count = n > 1024 ? 1024 : n;
+    for (int q = rg; q < count; q += 128) {
+        const int i = q * stride;
         const uint4 v = *reinterpret_cast<const uint4*>(base + (int64_t)i * sn);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -852,7 +857,7 @@ tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh
     if (tid < 64) {
         float acc = 0.f;
         for (int r = 0; r < 128; ++r) acc += part[r][tid];
-        cmean[(size_t)bh * 64 + tid] = acc / (float)n;
+        cmean[(size_t)bh * 64 + tid] = acc / (float)count;
     }
 }
 
