@@ -87,7 +87,9 @@ namespace {
 // block boundary it is rounded to bf16 and written out, then the block's own contribution is
 // accumulated on top -- the per-block states H_l and the scan over them are fused away.
 //   X: tensor that is sketched (K for the forward state, Q for the backward's reverse state)
-//   Y: [V] or [E(:, :64)];  y65: last column (nullptr = all ones)
+//   Y: [V] or [dO];  y65: last column (nullptr = all ones);  fscale: per-token d_i, the
+//   features of token i are divided by it (nullptr = not) -- phi(q_i)^T [dO_i | y65_i] / d_i is the
+//   suffix state's phi(q_i)^T E_i without E ever being formed
 // grid (BH).  Warp roles:
 //   NWG generator warpgroups  thread = token: read the half sketches, write their feature tiles
 //                             (dealt round-robin) as MN-major A operands into shared memory;
@@ -118,8 +120,8 @@ template <int R, int T0, int TN, int NWG>
 __global__ void __launch_bounds__(128 * (NWG + 1) + 64)
 tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
                 const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
-                const float* __restrict__ y65, const float* __restrict__ cmean, int center_mode, int reverse,
-                bf16* __restrict__ S, int* status) {
+                const float* __restrict__ y65, const float* __restrict__ fscale, const float* __restrict__ cmean,
+                int center_mode, int reverse, bf16* __restrict__ S, int* status) {
     using F = Feat<R>;
     using L = StateSmem<R, NWG>;
     extern __shared__ uint8_t smem_raw[];
@@ -333,6 +335,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
         bool ok = true;
         // last-column entry of this thread's token, requested one token tile ahead of its use
         float y_next = (y65 != nullptr && wg == 0) ? y65[(size_t)bh * n + tile_of(0) * 128 + wt] : 0.f;
+        float d_next = fscale != nullptr ? fscale[(size_t)bh * n + tile_of(0) * 128 + wt] : 1.f;
         for (int j = 0; j < NJ && ok; ++j) {
             ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
             tc_fence_after();
@@ -340,7 +343,10 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
             CircGen<R> gen;
             {
                 float m[R];
-                read_half_sketch<R>(lane_tm, m);
+                // features m_a m_b / d: both factors carry 1 / sqrt(d) (d requested a token tile ago)
+                const float sc = rsqrtf(d_next);
+                if (fscale != nullptr && j + 1 < NJ) d_next = fscale[(size_t)bh * n + tile_of(j + 1) * 128 + wt];
+                read_half_sketch<R>(lane_tm, m, sc);
                 if constexpr (F::kCirc) gen.init(m); else pack_half_sketch<R>(m, pm);
             }
             tc_fence_before();
@@ -451,9 +457,9 @@ struct OutSmem {
 
 
 // MODE 0: forward (writes O, denom, optionally O - c in fp32).  MODE 1: the backward's
-// recomputation of the row numerators against centred prefix states; writes E = dO/d (bf16),
-// e65 = -(dO.(O - c))/d and e65h = e65 - E.c (fp32), with O - c = (N' - c)/d taken from the fp32
-// accumulators rather than from the rounded O the caller holds.
+// recomputation of the row numerators against centred prefix states; writes y65 = -(dO.(O - c))
+// and e65h = -(dO.O)/d (fp32), with O - c = (N' - c)/d taken from the fp32 accumulators rather
+// than from the rounded O the caller holds.
 // LOCAL (Section 3.2): the same-block scores are (q_i . k_j)^2 from the raw query and key tiles
 // (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
 // they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
@@ -464,8 +470,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                   const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapOc,
                   const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                   const float* __restrict__ cmean, int64_t sb, int64_t sh, int64_t sn,
-                  float* __restrict__ denom, const bf16* __restrict__ dO, bf16* __restrict__ E,
-                  float* __restrict__ e65, float* __restrict__ e65h, int keep_oc, int* status) {
+                  float* __restrict__ denom, const bf16* __restrict__ dO,
+                  float* __restrict__ y65, float* __restrict__ e65h, int keep_oc, int* status) {
     using F = Feat<R>;
     using L = OutSmem<R, LOCAL>;
     extern __shared__ uint8_t smem_raw[];
@@ -801,7 +807,6 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             for (int c = 0; c < 64; c += 8) {
                 const uint4 gv = *reinterpret_cast<const uint4*>(gp + c);
                 const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-                uint32_t ew[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
@@ -810,13 +815,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     dot = fmaf(g1, acc[c + 2 * j + 1] - (rowsum + 1.f) * c1, dot);
                     ec = fmaf(g0 * inv, c0, ec);
                     ec = fmaf(g1 * inv, c1, ec);
-                    ew[j] = pack_bf16(g0 * inv, g1 * inv);
                 }
-                *reinterpret_cast<uint4*>(E + row * 64 + c) = make_uint4(ew[0], ew[1], ew[2], ew[3]);
             }
-            const float e = -dot * inv * inv;
-            e65[row] = e;
-            e65h[row] = e - ec;
+            const float y = -dot * inv;               // -(dO . (O - c))
+            y65[row] = y;
+            e65h[row] = y * inv - ec;
         }
     }
     tc_fence_before();
@@ -881,13 +884,13 @@ tc_gimage_kernel(const bf16* __restrict__ G1, const bf16* __restrict__ G2, int r
 // Prefix (or suffix) states of every head.  X is sketched, Y is the right-hand side.
 template <int R, int T0, int TN, int NWG>
 cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                               const float* y65, const float* cmean, int center_mode, bool reverse,
+                               const float* y65, const float* fscale, const float* cmean, int center_mode, bool reverse,
                                bf16* S, int* status, cudaStream_t s, int* launches) {
     constexpr size_t smem = StateSmem<R, NWG>::total + 1024;
     PSK_TRY(set_smem(tc_state_kernel<R, T0, TN, NWG>, smem));
     prof_begin("tc_state_kernel", s);
     tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 64, smem, s>>>(
-        mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, y65, cmean, center_mode, reverse ? 1 : 0, S, status);
+        mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, y65, fscale, cmean, center_mode, reverse ? 1 : 0, S, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -895,10 +898,10 @@ cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUten
 
 template <int R>
 cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                          const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
-                          cudaStream_t s, int* launches) {
+                          const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
+                          int* status, cudaStream_t s, int* launches) {
 #define PSK_SG(T0, TN, NWG) \
-    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, gimg, y65, cmean, center_mode, reverse, S, status, s, launches)))
+    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, reverse, S, status, s, launches)))
     if constexpr (R == 16) {
         PSK_SG(0, 2, 2);
     } else if constexpr (R == 32) {
@@ -932,7 +935,7 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (cmean != nullptr) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
-    PSK_TRY((launch_states<R>(d, mK, mV, gimg, nullptr, cmean, cmean ? 1 : 0, Z, false,
+    PSK_TRY((launch_states<R>(d, mK, mV, gimg, nullptr, nullptr, cmean, cmean ? 1 : 0, Z, false,
                               status, s, launches)));
     prof_begin("tc_fwd_out_kernel", s);
     if (d.local) {
@@ -940,13 +943,13 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true>, smem)));
         tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false>, smem)));
         tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            denom, nullptr, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
     }
     prof_end(s);
     ++*launches;
@@ -982,7 +985,7 @@ cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V, c
 template <int R>
 static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
                                   const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean,
-                                  const float* denom, const bf16* dO, bf16* E, float* e65, float* e65h, int* status,
+                                  const float* denom, const bf16* dO, float* y65, float* e65h, int* status,
                                   cudaStream_t s, int* launches) {
     prof_begin("tc_bwd_recompute_kernel", s);
     if (d.local) {
@@ -990,13 +993,13 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true>, smem)));
         tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
+            const_cast<float*>(denom), dO, y65, e65h, 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false>, smem)));
         tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            const_cast<float*>(denom), dO, E, e65, e65h, 0, status);
+            const_cast<float*>(denom), dO, y65, e65h, 0, status);
     }
     prof_end(s);
     ++*launches;
@@ -1005,11 +1008,11 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
 
 cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
                          const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
-                         const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches) {
+                         const bf16* dO, float* y65, float* e65h, int* status, cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
-        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
-        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, E, e65, e65h, status, s, launches);
+        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
+        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
+        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
     }
     return cudaErrorInvalidValue;
 }
@@ -1031,12 +1034,12 @@ cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s,
 }
 
 cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                      const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
-                          cudaStream_t s, int* launches) {
+                      const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
+                      int* status, cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return launch_states<16>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
-        case 32: return launch_states<32>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
-        case 64: return launch_states<64>(d, mX, mY, gimg, y65, cmean, center_mode, S, reverse, status, s, launches);
+        case 16: return launch_states<16>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
+        case 32: return launch_states<32>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
+        case 64: return launch_states<64>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
     }
     return cudaErrorInvalidValue;
 }

@@ -20,11 +20,13 @@ using namespace tc;
 namespace {
 
 // With kept states the forward left Oc = O - c (fp32).  Eight lanes x 8 columns per row (four
-// rows per warp):  E = dO / d (bf16, for the suffix states),  e65 = -(dO . Oc) / d,  e65h = e65 - E . c
+// rows per warp):  y65 = -(dO . Oc)  (the last entry of E_i times d_i, paired with centred states),
+// e65h = (y65 - dO . c) / d = -(dO . O) / d.  The rows E_i[:h] = dO_i / d_i themselves are never
+// formed: the suffix-state kernel reads dO and scales the query features by 1 / d_i instead.
 __global__ void __launch_bounds__(256)
 tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom, const float* __restrict__ cmean,
                    const float* __restrict__ Oc, int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn,
-                   bf16* __restrict__ E, float* __restrict__ e65, float* __restrict__ e65h) {
+                   float* __restrict__ y65, float* __restrict__ e65h) {
     const int row = blockIdx.x * 32 + threadIdx.x / 8, ch = threadIdx.x % 8;
     if (row >= total_rows) return;                 // total_rows is a multiple of 128: whole warps leave together
     const int bh = row / n, i = row % n;
@@ -37,7 +39,6 @@ tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom,
     const float inv = 1.f / denom[row];
     const float* c = cmean + (size_t)bh * 64 + 8 * ch;
     float dot = 0.f, ec = 0.f;
-    uint32_t ew[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
@@ -45,18 +46,15 @@ tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom,
         dot = fmaf(g1, ov[2 * j + 1], dot);
         ec = fmaf(g0 * inv, c[2 * j], ec);
         ec = fmaf(g1 * inv, c[2 * j + 1], ec);
-        ew[j] = pack_bf16(g0 * inv, g1 * inv);
     }
 #pragma unroll
     for (int s = 4; s > 0; s >>= 1) {
         dot += __shfl_xor_sync(0xffffffffu, dot, s);
         ec += __shfl_xor_sync(0xffffffffu, ec, s);
     }
-    *reinterpret_cast<uint4*>(E + (size_t)row * 64 + 8 * ch) = make_uint4(ew[0], ew[1], ew[2], ew[3]);
     if (ch == 0) {
-        const float e = -dot * inv;
-        e65[row] = e;
-        e65h[row] = e - ec;
+        y65[row] = -dot;
+        e65h[row] = -dot * inv - ec;
     }
 }
 
@@ -136,7 +134,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    const __grid_constant__ CUtensorMap mapS, const __grid_constant__ CUtensorMap mapDX,
                    const __grid_constant__ CUtensorMap mapDV, const uint8_t* __restrict__ gimg,
                    int g_heads, int H, int n, int b, int t,
-                   const float* __restrict__ e65, const float* __restrict__ e65h, const float* __restrict__ denom,
+                   const float* __restrict__ y65g, const float* __restrict__ e65h, const float* __restrict__ denom,
                    int* status) {
     using F = Feat<R>;
     using L = BwdSmem<R>;
@@ -189,7 +187,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     // (The three row scalars come from HBM.  They are requested here and first used after the half
     // sketch has been read, a few thousand cycles later: the arithmetic on them stays below.)
     const float d_raw = QSIDE ? denom[(size_t)bh * n + row0 + tid] : 1.f;
-    const float e65_raw = QSIDE ? e65[(size_t)bh * n + row0 + tid] : 1.f;
+    const float y65_raw = QSIDE ? y65g[(size_t)bh * n + row0 + tid] : 1.f;
     const float e65h_raw = QSIDE ? e65h[(size_t)bh * n + row0 + tid] : 1.f;
     // key side: the scalars of the first query tile it will meet (thread = that tile's row tid)
     float od_raw = 1.f, oe_raw = 0.f;
@@ -240,7 +238,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
     const float d_own = d_raw, inv_own = 1.f / d_own;
-    const float y65 = QSIDE ? e65_raw * d_own : 1.f, y65h = QSIDE ? e65h_raw * d_own : 1.f;
+    const float y65 = y65_raw, y65h = QSIDE ? e65h_raw * d_own : 1.f;
     // the 65th column of the A operand [Y_own | y65]: first read by phase B's MMAs, after the barrier below
     *reinterpret_cast<uint4*>(smem + L::ExtA + (tid / 8) * 128 + (tid % 8) * 16) = make_uint4(pack_bf16(y65, 0.f), 0, 0, 0);
     fence_proxy_async_smem();
@@ -716,16 +714,14 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     int* status = reinterpret_cast<int*>(ws + w.status);
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
     bf16* Rs = reinterpret_cast<bf16*>(ws + w.Rst);
-    bf16* E = reinterpret_cast<bf16*>(ws + w.E);
-    float* e65 = reinterpret_cast<float*>(ws + w.e65);
+    float* y65 = reinterpret_cast<float*>(ws + w.y65);
     float* cmean = reinterpret_cast<float*>(ws + w.vmean);
     float* e65h = reinterpret_cast<float*>(ws + w.e65h);
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
-    CUtensorMap mQ, mK, mV, mE, mG, mZ, mR, mdQ, mdK, mdV;
+    CUtensorMap mQ, mK, mV, mG, mZ, mR, mdQ, mdK, mdV;
     const int64_t nblk = (int64_t)d.BH() * d.t;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
-        !tc_map_rows(&mE, E, d.B, d.H, d.n, (int64_t)d.H * d.n * 64, (int64_t)d.n * 64, 64) ||
         !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk) ||
         !tc_map_rows(&mdQ, dQ, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mdK, dK, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
@@ -733,19 +729,19 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         return cudaErrorInvalidValue;
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
-    // prefix states of centred values; forward rows again in fp32 -> E, e65, e65h; suffix states
-    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, cmean, 1, Z, false, status, s, launches));
+    // prefix states of centred values; forward rows again in fp32 -> y65, e65h; suffix states
+    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, nullptr, cmean, 1, Z, false, status, s, launches));
     if (d.keep_states) {
         const int rows = d.BH() * d.n;
         prof_begin("tc_bwd_prep_kernel", s);
         tc_bwd_prep_kernel<<<(rows + 31) / 32, 256, 0, s>>>((const bf16*)dO, denom, cmean,
                                                            reinterpret_cast<const float*>(ws + w.Oc), d.H, d.n, rows, d.sb,
-                                                           d.sh, d.sn, E, e65, e65h);
+                                                           d.sh, d.sn, y65, e65h);
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
     } else {
-        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, E, e65, e65h, status, s, launches));
+        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, y65, e65h, status, s, launches));
     }
     constexpr size_t smem = BwdSmem<R>::total + 1024;
     const dim3 grid(d.b / 128, d.t, d.BH());
@@ -757,14 +753,15 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // still in L2; the suffix states (5 GB through L2) come after it
         prof_begin("tc_bwd_q_kernel", s);
         tc_bwd_rows_kernel<R, true, LOCAL><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
-                                                                   d.b, d.t, e65, e65h, denom, status);
+                                                                   d.b, d.t, y65, e65h, denom, status);
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
-        PSK_TRY(tc_states(d, mQ, mE, gimg, e65, cmean, 2, Rs, true, status, s, launches));
+        // suffix states: phi(q_i) / d_i against [dO_i | y65_i]
+        PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
         tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
-                                                                    d.b, d.t, e65, e65h, denom, status);
+                                                                    d.b, d.t, y65, e65h, denom, status);
         prof_end(s);
         ++*launches;
         return cudaGetLastError();

@@ -19,12 +19,12 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
 // center_mode 0: states as they are; 1: values centred by the per-head vector cmean
 // (columns < 64 become H[:, c] - cmean[c] H[:, 64]); 2: last column becomes H[:, 64] - H[:, :64] cmean.
 cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                      const float* y65, const float* cmean, int center_mode, bf16* S, bool reverse, int* status,
-                      cudaStream_t s, int* launches);
-// the backward's recomputation of the forward rows: writes E, e65, e65h (see tc_fwd_out_kernel)
+                      const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
+                      int* status, cudaStream_t s, int* launches);
+// the backward's recomputation of the forward rows: writes y65, e65h (see tc_fwd_out_kernel)
 cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
                          const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
-                         const bf16* dO, bf16* E, float* e65, float* e65h, int* status, cudaStream_t s, int* launches);
+                         const bf16* dO, float* y65, float* e65h, int* status, cudaStream_t s, int* launches);
 // gimg[g] = [G1 | G2]^T of sketch-matrix set g as the shared-memory image of the sketch GEMM's B operand
 // (2r rows x 128 B, K-major, 128-byte swizzle): the kernels fetch it with one bulk copy
 cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gimg, cudaStream_t s, int* launches);
@@ -32,7 +32,7 @@ cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gi
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
 
 // Scratch layout of the tensor-core path.
-struct TcWorkspace { size_t status, vmean, gimg, Z, Rst, E, e65, e65h, Oc, total; };
+struct TcWorkspace { size_t status, vmean, gimg, Z, Rst, y65, e65h, Oc, total; };
 
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
@@ -46,8 +46,7 @@ inline TcWorkspace tc_ws(const Dims& d, bool backward) {
     w.Z = off; off += align_up(st);
     if (backward) {
         w.Rst = off; off += align_up(st);
-        w.E = off; off += align_up(rows * 64 * sizeof(bf16));
-        w.e65 = off; off += align_up(rows * sizeof(float));
+        w.y65 = off; off += align_up(rows * sizeof(float));
         w.e65h = off; off += align_up(rows * sizeof(float));
         if (d.keep_states) { w.Oc = off; off += align_up(rows * 64 * sizeof(float)); }   // forward's O - c, fp32
     }
@@ -99,9 +98,10 @@ __device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX,
 }
 
 // m[c] = A1[c] A2[c] / sqrt(R) from the sketch accumulator (this thread's lane).
+// (`scale`: an extra factor on every entry, folded into the constant)
 template <int R>
-__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R]) {
-    const float rs = rsqrtf((float)R);
+__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R], float scale = 1.f) {
+    const float rs = rsqrtf((float)R) * scale;
 #pragma unroll
     for (int c0 = 0; c0 < R; c0 += 16) {
         uint32_t a1[16], a2[16];
