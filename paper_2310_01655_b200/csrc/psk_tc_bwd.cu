@@ -436,6 +436,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll 1
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
+        // LOCAL: the other side's raw tiles alternate between two buffers (the second one is the
+        // unused split-operand tile), so the next tile's rows can be requested a tile ahead
+        const uint32_t xo = (LOCAL && ((tp - tp_begin) & 1)) ? L::Moth : L::Xoth;
+        const uint32_t xo_next = (LOCAL && !((tp - tp_begin) & 1)) ? L::Moth : L::Xoth;
         // (this tile's rows were requested ahead: by the prologue, by phase B's last chunks, or
         // by the previous tile as soon as its own copies had been consumed)
         // Every thread is past its wait for the previous tile's last MMAs before the next commit
@@ -480,17 +484,17 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 // The X tile has been consumed, and every thread is past its wait for it (a
                 // barrier must not complete twice before its slowest waiter has looked): next
                 // tile's rows.
-                // (LOCAL: the raw rows are operands of this tile's GEMMs to its end; see below)
-                if (!LOCAL && hh == 0 && tp + 1 < tp_end) {
+                // (LOCAL: the raw rows stay operands to the tile's end; the next ones go to the other buffer)
+                if (hh == 0 && tp + 1 < tp_end) {
                     mbar_expect_tx(&bar_xoth, 16384);
-                    tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
+                    tma_load_4d(smem + xo_next, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
                 }
                 constexpr uint32_t idesc = idesc_bf16(128, 64, false, false);
                 if constexpr (LOCAL) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)       // x = own rows . other rows, over the head dimension
                         umma_ss(tm + cS, desc_off(smem_desc(smem_u32(smem + L::Xown), 0, 1024, kSwz128), k * 32),
-                                desc_off(smem_desc(smem_u32(smem + L::Xoth) + hh * 8192, 0, 1024, kSwz128), k * 32), idesc, k > 0);
+                                desc_off(smem_desc(smem_u32(smem + xo) + hh * 8192, 0, 1024, kSwz128), k * 32), idesc, k > 0);
                 } else {
                     issue_scores<R>(tm + cS, smem_u32(smem + L::Mown), smem_u32(smem + L::Moth) + hh * 8192);
                 }
@@ -558,7 +562,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
                     for (int k = 0; k < 4; ++k)       // dX_own += dx x X_other
                         umma_ts(tm + cXl, tm + cS + k * 8,
-                                desc_off(smem_desc(smem_u32(smem + L::Xoth) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
+                                desc_off(smem_desc(smem_u32(smem + xo) + hh * 8192, 0, 1024, kSwz128), k * 2048), idesc,
                                 (dm_started || k > 0) ? 1u : 0u);
                 } else {
 #pragma unroll
@@ -585,10 +589,6 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         if (tid == 0 && tp + 1 < tp_end) {        // every MMA that read the Y tile has completed
             mbar_expect_tx(&bar_yoth, 16384);
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow0 + 128, hi, bi, &bar_yoth);
-            if constexpr (LOCAL) {                // ... and the X tile
-                mbar_expect_tx(&bar_xoth, 16384);
-                tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow0 + 128, hi, bi, &bar_xoth);
-            }
         }
     }
 
