@@ -374,14 +374,15 @@ def main():
         achieved = (fl * w.head_tokens / ((tot / cnt) / 1e3) / 1e12) if fl else None
         # DRAM bytes per launch: ncu capture on the profiling-sized slice, scaled by head-tokens
         traffic = None
-        tpath = os.path.join(ROOT, "profiles", "dram_traffic_c2s.json")
+        tname = "dram_traffic_c2s_local_exact.json" if args.local_exact else "dram_traffic_c2s.json"
+        tpath = os.path.join(ROOT, "profiles", tname)
         if os.path.exists(tpath) and w.r == 32 and w.b == 256:
             per = json.load(open(tpath))["kernels"].get(name)
             if per:
                 traffic = per["dram_bytes_per_head_token"] * w.head_tokens
         roof = {"kernel": name, "bound": "tensor" if tensor else "alu", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "traffic_source": "profiles/dram_traffic_c2s.json (ncu on the c2s slice, scaled by head-tokens)" if traffic else None,
+                "traffic_source": ("profiles/%s (ncu on the c2s slice, scaled by head-tokens)" % tname) if traffic else None,
                 "flops_per_launch": fl * w.head_tokens if fl else None,
                 "peak_source": (pk["source"] + " (sustained bf16)") if tensor else "derived: 148 SM x 128 FMA x 1.965 GHz",
                 "launches": cnt, "avg_ms": tot / cnt, "share_of_kernel_time": tot / total_kernel_ms}
