@@ -774,24 +774,25 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 *reinterpret_cast<uint4*>(smem + L::So + swz128_offset(tid, c)) = v;
             }
             if (keep_oc) {
-                // kept for the backward: O - c in fp32.  (The rounded O cannot supply it: where the
-                // values share a common component, or one key dominates a row, |O - c| and
-                // |v - O| are far below |O|.)
+                // kept for the backward: O - c, rounded to bf16 AFTER the subtraction.  (The rounded
+                // O cannot supply it: where the values share a common component |O - c| is far
+                // below |O|, and bf16(O) - c would carry O's rounding error, not (O - c)'s.)
 #pragma unroll
-                for (int c = 0; c < 16; ++c)
-                    *reinterpret_cast<float4*>(smem + L::Soc + (c / 8) * 16384 + swz128_offset(tid, c % 8)) =
-                        make_float4(acc[4 * c] * inv - cm[4 * c], acc[4 * c + 1] * inv - cm[4 * c + 1],
-                                    acc[4 * c + 2] * inv - cm[4 * c + 2], acc[4 * c + 3] * inv - cm[4 * c + 3]);
+                for (int c = 0; c < 8; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16(acc[8 * c] * inv - cm[8 * c], acc[8 * c + 1] * inv - cm[8 * c + 1]);
+                    v.y = pack_bf16(acc[8 * c + 2] * inv - cm[8 * c + 2], acc[8 * c + 3] * inv - cm[8 * c + 3]);
+                    v.z = pack_bf16(acc[8 * c + 4] * inv - cm[8 * c + 4], acc[8 * c + 5] * inv - cm[8 * c + 5]);
+                    v.w = pack_bf16(acc[8 * c + 6] * inv - cm[8 * c + 6], acc[8 * c + 7] * inv - cm[8 * c + 7]);
+                    *reinterpret_cast<uint4*>(smem + L::Soc + swz128_offset(tid, c)) = v;
+                }
             }
             if (denom != nullptr && ok) denom[(size_t)bh * n + row0 + tid] = d;
             fence_proxy_async_smem();
             consumer_barrier();
             if (tid == 0 && ok) {
                 tma_store_4d(&mapO, smem + L::So, 0, row0, hi, bi);
-                if (keep_oc) {
-                    tma_store_2d(&mapOc, smem + L::Soc, 0, bh * n + row0);
-                    tma_store_2d(&mapOc, smem + L::Soc + 16384, 32, bh * n + row0);
-                }
+                if (keep_oc) tma_store_4d(&mapOc, smem + L::Soc, 0, bh * n + row0, 0, 0);
                 bulk_commit();
                 bulk_wait_read();
             }
@@ -919,14 +920,15 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     const TcWorkspace w = tc_ws<R>(d, d.keep_states);
     int* status = reinterpret_cast<int*>(ws + w.status);
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
-    float* Oc = d.keep_states ? reinterpret_cast<float*>(ws + w.Oc) : nullptr;
+    bf16* Oc = d.keep_states ? reinterpret_cast<bf16*>(ws + w.Oc) : nullptr;
     CUtensorMap mQ, mK, mV, mZ, mO, mOc;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t) ||
         !tc_map_rows(&mO, O, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
     if (Oc != nullptr) {
-        if (!tc_map_f32rows(&mOc, Oc, (int64_t)d.BH() * d.n)) return cudaErrorInvalidValue;
+        const int64_t rows = (int64_t)d.BH() * d.n;      // one [rows, 64] bf16 array
+        if (!tc_map_rows(&mOc, Oc, 1, 1, (int)rows, rows * 64, rows * 64, 64)) return cudaErrorInvalidValue;
     } else {
         mOc = mO;       // never used
     }

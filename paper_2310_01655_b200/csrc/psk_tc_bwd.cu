@@ -19,43 +19,57 @@ using namespace tc;
 
 namespace {
 
-// With kept states the forward left Oc = O - c (fp32).  Eight lanes x 8 columns per row (four
+// With kept states the forward left Oc = O - c (bf16).  Eight lanes x 8 columns per row (four
 // rows per warp):  y65 = -(dO . Oc)  (the last entry of E_i times d_i, paired with centred states),
 // e65h = (y65 - dO . c) / d = -(dO . O) / d.  The rows E_i[:h] = dO_i / d_i themselves are never
 // formed: the suffix-state kernel reads dO and scales the query features by 1 / d_i instead.
 __global__ void __launch_bounds__(256)
 tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom, const float* __restrict__ cmean,
-                   const float* __restrict__ Oc, int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn,
+                   const bf16* __restrict__ Oc, int H, int n, int total_rows, int64_t sb, int64_t sh, int64_t sn,
                    float* __restrict__ y65, float* __restrict__ e65h) {
-    const int row = blockIdx.x * 32 + threadIdx.x / 8, ch = threadIdx.x % 8;
-    if (row >= total_rows) return;                 // total_rows is a multiple of 128: whole warps leave together
-    const int bh = row / n, i = row % n;
-    const int64_t base = (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn + 8 * ch;
-    const uint4 gv = *reinterpret_cast<const uint4*>(dO + base);
-    const float4 o0 = *reinterpret_cast<const float4*>(Oc + (size_t)row * 64 + 8 * ch);
-    const float4 o1 = *reinterpret_cast<const float4*>(Oc + (size_t)row * 64 + 8 * ch + 4);
-    const float ov[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
-    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-    const float inv = 1.f / denom[row];
-    const float* c = cmean + (size_t)bh * 64 + 8 * ch;
-    float dot = 0.f, ec = 0.f;
+    // 128 rows per CTA, four per thread group: all eight 16-byte loads of a thread are in flight
+    // before the first is used.  (n and total_rows are multiples of 128: one head per CTA.)
+    const int ch = threadIdx.x % 8;
+    const int row_base = blockIdx.x * 128 + threadIdx.x / 8;
+    const int bh = row_base / n;
+    const int64_t head = (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + 8 * ch;
+    uint4 gv[4], oc[4];
+    float dn[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
-        dot = fmaf(g0, ov[2 * j], dot);
-        dot = fmaf(g1, ov[2 * j + 1], dot);
-        ec = fmaf(g0 * inv, c[2 * j], ec);
-        ec = fmaf(g1 * inv, c[2 * j + 1], ec);
+    for (int it = 0; it < 4; ++it) {
+        const int row = row_base + it * 32;
+        gv[it] = *reinterpret_cast<const uint4*>(dO + head + (int64_t)(row % n) * sn);
+        oc[it] = *reinterpret_cast<const uint4*>(Oc + (size_t)row * 64 + 8 * ch);
+        dn[it] = denom[row];
     }
+    const float4 c0 = *reinterpret_cast<const float4*>(cmean + (size_t)bh * 64 + 8 * ch);
+    const float4 c1 = *reinterpret_cast<const float4*>(cmean + (size_t)bh * 64 + 8 * ch + 4);
+    const float c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-    for (int s = 4; s > 0; s >>= 1) {
-        dot += __shfl_xor_sync(0xffffffffu, dot, s);
-        ec += __shfl_xor_sync(0xffffffffu, ec, s);
+    for (int it = 0; it < 4; ++it) {
+        const uint32_t gw[4] = {gv[it].x, gv[it].y, gv[it].z, gv[it].w};
+        const uint32_t ow[4] = {oc[it].x, oc[it].y, oc[it].z, oc[it].w};
+        float dot = 0.f, gc = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
+            dot = fmaf(g0, __uint_as_float(ow[j] << 16), dot);
+            dot = fmaf(g1, __uint_as_float(ow[j] & 0xFFFF0000u), dot);
+            gc = fmaf(g0, c[2 * j], gc);
+            gc = fmaf(g1, c[2 * j + 1], gc);
+        }
+#pragma unroll
+        for (int s = 4; s > 0; s >>= 1) {
+            dot += __shfl_xor_sync(0xffffffffu, dot, s);
+            gc += __shfl_xor_sync(0xffffffffu, gc, s);
+        }
+        if (ch == 0) {
+            const int row = row_base + it * 32;
+            y65[row] = -dot;
+            e65h[row] = -(dot + gc) / dn[it];          // -(dO . (O - c) + dO . c) / d
+        }
     }
-    if (ch == 0) {
-        y65[row] = -dot;
-        e65h[row] = -dot * inv - ec;
-    }
+    (void)total_rows;
 }
 
 constexpr int kStages = 4;
@@ -734,8 +748,8 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (d.keep_states) {
         const int rows = d.BH() * d.n;
         prof_begin("tc_bwd_prep_kernel", s);
-        tc_bwd_prep_kernel<<<(rows + 31) / 32, 256, 0, s>>>((const bf16*)dO, denom, cmean,
-                                                           reinterpret_cast<const float*>(ws + w.Oc), d.H, d.n, rows, d.sb,
+        tc_bwd_prep_kernel<<<rows / 128, 256, 0, s>>>((const bf16*)dO, denom, cmean,
+                                                           reinterpret_cast<const bf16*>(ws + w.Oc), d.H, d.n, rows, d.sb,
                                                            d.sh, d.sn, y65, e65h);
         prof_end(s);
         ++*launches;

@@ -48,7 +48,7 @@ inline TcWorkspace tc_ws(const Dims& d, bool backward) {
         w.Rst = off; off += align_up(st);
         w.y65 = off; off += align_up(rows * sizeof(float));
         w.e65h = off; off += align_up(rows * sizeof(float));
-        if (d.keep_states) { w.Oc = off; off += align_up(rows * 64 * sizeof(float)); }   // forward's O - c, fp32
+        if (d.keep_states) { w.Oc = off; off += align_up(rows * 64 * sizeof(bf16)); }   // forward's O - c
     }
     w.total = off;
     return w;
