@@ -100,10 +100,12 @@ def test_tensor_core_backward_reading_the_forwards_states(r, b, n, corr):
             check(name, got[0, hi], ref, TOL["bf16"])
 
 
-def test_full_size_configuration_2():
-    """PSK_FLAG_LOCAL_EXACT at configuration 2's full size, as `bench.py --local-exact` runs it:
-    sampled (batch, head) slices against the block-form oracle, finiteness of the full tensors."""
-    w = wl.WORKLOADS["c2"]
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_full_size_configuration(name):
+    """PSK_FLAG_LOCAL_EXACT at a benchmark configuration's full size, as `bench.py --local-exact`
+    runs it: sampled (batch, head) slices against the block-form oracle, finiteness of the full
+    tensors."""
+    w = wl.WORKLOADS[name]
     inp = wl.make_inputs(w, "cuda")
     Q, K, V, G1, G2 = (inp[k] for k in ("Q", "K", "V", "G1", "G2"))
     flags = psk.FLAG_KEEP_STATES | LOCAL

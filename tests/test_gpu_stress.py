@@ -53,3 +53,32 @@ def test_recomputing_backward_agrees_with_kept_states():
     for name, a, c in zip(("dQ", "dK", "dV"), g_plain, g_kept):
         rel = (a.double() - c.double()).norm() / c.double().norm()
         assert rel <= 1e-2, (name, float(rel))
+
+
+def _time_step(B, n, reps=3):
+    w = wl.small_workload(B=B, H=6, n=n, r=32, b=256, dtype="bf16", seed=17)
+    inp = wl.make_inputs(w, "cuda", with_dO=True)
+    Q, K, V, G1, G2, dO = (inp[k] for k in ("Q", "K", "V", "G1", "G2", "dO"))
+    flags = psk.FLAG_KEEP_STATES
+    shp = psk.binding.make_shape(Q, G1, 32, 256, flags=flags)
+    ws = torch.empty(psk.workspace_bytes(shp, True), dtype=torch.uint8, device="cuda")
+    best = float("inf")
+    for _ in range(reps + 1):                      # first repetition: warm-up
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, 256, workspace=ws, flags=flags)
+        psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, 256, workspace=ws, flags=flags)
+        e1.record()
+        torch.cuda.synchronize()
+        if _ > 0:
+            best = min(best, e0.elapsed_time(e1))
+    assert psk.check(ws) == 0
+    return best
+
+
+def test_time_is_linear_in_the_context_length():
+    """Section 3.1: the cost is linear in n at a fixed block size (exact attention would be
+    quadratic): four times the context at the same batch and heads costs about four times as much."""
+    t_1 = _time_step(B=25, n=16384)                # 150 heads: every SM has work in every kernel
+    t_4 = _time_step(B=25, n=65536)
+    assert 3.2 <= t_4 / t_1 <= 4.8, (t_1, t_4)
