@@ -25,7 +25,8 @@ causality, block-size invariance, lt-multiply against a dense triangle, central
 finite differences for every gradient, dV against the explicit weight matrix;
 for the local-exact variant (Section 3.2): one block = exact polynomial
 attention, exact features = no dependence on the block size, looped definition,
-block algorithm against the masked definition, finite differences.
+block algorithm against the masked definition, finite differences; for
+degree 2 (no sketch): looped (q.k)^2 attention, finite differences.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -340,6 +341,42 @@ def causal_polysketch_attention_backward_blocked(Q, K, V, G1, G2, dO, b, diagona
         dVt[rows] += PhiK[rows] @ R
         R = R + PhiQ[rows].T @ E[rows]
     return (_sketch_backward(Q, G1, G2, dMq) + dQl, _sketch_backward(K, G1, G2, dMk) + dKl, dVt[:, :h])
+
+
+# ---------------------------------------------------------------------------
+# Degree p = 2: Algorithm 1 with p/2 = 1 has no sketch at all (PolySketchWithNegativity(A, r, 1)
+# is A), so phi'(A) = A^{(x)2} with h^2 entries and the attention is exact degree-2 polynomial
+# attention (Section 2.1 with p = 2).
+# ---------------------------------------------------------------------------
+def causal_degree2_attention_blocked(Q, K, V, b):
+    """Section 3.1's block algorithm on phi'(A) = A^{(x)2} (Algorithm 1, p = 2), diagonal
+    blocks through (Q_l K_l^T)^2.  Returns (O, d)."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, h = V.shape
+    C = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+
+    def diag_block(l):
+        return lt((Q[l * b:(l + 1) * b] @ K[l * b:(l + 1) * b].T) ** 2)
+
+    N = lt_multiply_blocked(self_tensor(Q), self_tensor(K), C, b, diag_block)
+    d = 1.0 + N[:, h]
+    return N[:, :h] / d[:, None], d
+
+
+def causal_degree2_attention_backward(Q, K, V, dO):
+    """Gradients (dQ, dK, dV) of sum(dO * O) for the weights (q_i . k_j)^2, j <= i, through the
+    quadratic definition: ds = 2 s dW reaches Q and K directly (there is no sketch)."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, h = V.shape
+    s = Q @ K.T
+    W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = lt(E @ Vt.T)
+    ds = 2.0 * s * dW
+    return ds @ K, ds.T @ Q, W.T @ E[:, :h]
 
 
 # ---------------------------------------------------------------------------
