@@ -34,6 +34,10 @@
  *   - Supported: p = 4, h = 64, r in {16, 32, 64}, b a multiple of 128, n a multiple
  *     of b (Section 3.1 assumes b = n / t).  Anything else: PSK_ERR_UNSUPPORTED or
  *     PSK_ERR_SHAPE.
+ *   - Also p = 2 (Algorithm 1 with p/2 = 1): no sketch, m(x) = x, phi'(x) = x (x) x with
+ *     h^2 entries, i.e. exact degree-2 polynomial attention with weights (q_i . k_j)^2.
+ *     Set r = h; G1 and G2 are not read and may be null.  Served by the CUDA-core
+ *     kernels for either storage type (PSK_PATH_TENSOR_CORES: PSK_ERR_UNSUPPORTED).
  */
 #ifndef PSK_H_
 #define PSK_H_
@@ -48,7 +52,7 @@ extern "C" {
 typedef enum {
     PSK_OK = 0,
     PSK_ERR_INVALID_ARG = -1,   /* null pointer, bad enum value                      */
-    PSK_ERR_UNSUPPORTED = -2,   /* p != 4, h != 64, r not in {16,32,64}, bad path    */
+    PSK_ERR_UNSUPPORTED = -2,   /* p not 4 (or 2 with r = h), h != 64, r not in {16,32,64}, bad path */
     PSK_ERR_SHAPE = -3,         /* n % b != 0, b % 128 != 0, non-positive extents    */
     PSK_ERR_ALIGN = -4,         /* pointer or stride not 16-byte aligned             */
     PSK_ERR_WORKSPACE = -5,     /* workspace missing, misaligned or too small        */

@@ -88,6 +88,14 @@ def _ptr(t):
     return c_void_p(t.data_ptr()) if t is not None else c_void_p(0)
 
 
+def _contig(t):
+    return t.contiguous() if t is not None else None
+
+
+def _sketch_r(G1, x):
+    return G1.shape[-1] if G1 is not None else x.shape[-1]      # p = 2: the half sketch is the row, r = h
+
+
 def _stream():
     return c_void_p(torch.cuda.current_stream().cuda_stream)
 
@@ -100,7 +108,7 @@ def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, pa
     if x.dtype not in _DTYPES:
         raise ValueError("unsupported storage dtype %s" % x.dtype)
     B, H, n, h = x.shape
-    g_heads = G1.shape[0] if G1.dim() == 3 else 1
+    g_heads = G1.shape[0] if (G1 is not None and G1.dim() == 3) else 1
     return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path, flags)
 
 
@@ -132,12 +140,13 @@ def _empty_like(x):
 def sketch(X, G1, G2, r=None, b=128, want_phi=False, path=PATH_AUTO):
     """psk_sketch: returns (M [B,H,n,r] fp32, Phi [B,H,n,r*r] fp32 or None)."""
     _require_cuda(X, G1, G2)
-    r = G1.shape[-1] if r is None else r
-    shp = make_shape(X, G1, r, b, path=path)
+    p = 4 if G1 is not None else 2             # no sketch matrices: degree 2, M = X
+    r = (G1.shape[-1] if G1 is not None else X.shape[-1]) if r is None else r
+    shp = make_shape(X, G1, r, b, p, path=path)
     B, H, n, _ = X.shape
     M = torch.empty((B, H, n, r), dtype=torch.float32, device=X.device)
     Phi = torch.empty((B, H, n, r * r), dtype=torch.float32, device=X.device) if want_phi else None
-    st = lib().psk_sketch(byref(shp), _ptr(X), _ptr(G1.contiguous()), _ptr(G2.contiguous()), _ptr(M), _ptr(Phi),
+    st = lib().psk_sketch(byref(shp), _ptr(X), _ptr(_contig(G1)), _ptr(_contig(G2)), _ptr(M), _ptr(Phi),
                           _stream())
     if st != 0:
         raise PskError(st, "psk_sketch")
@@ -148,7 +157,7 @@ def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out
     """psk_causal_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, G1, G2)
     _same_layout(Q, K, V, out)
-    shp = make_shape(Q, G1, G1.shape[-1], b, p, path, flags)
+    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags)
     O = _empty_like(Q) if out is None else out
     B, H, n, _ = Q.shape
     if denom is None:
@@ -188,7 +197,7 @@ def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, works
     """psk_causal_attn_bwd: returns (dQ, dK, dV)."""
     _require_cuda(Q, K, V, G1, G2, O, denom, dO)
     _same_layout(Q, K, V, O, dO)
-    shp = make_shape(Q, G1, G1.shape[-1], b, p, path, flags)
+    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags)
     dQ, dK, dV = out if out is not None else (_empty_like(Q), _empty_like(Q), _empty_like(Q))
     _same_layout(Q, dQ, dK, dV)
     ws, nbytes = _workspace(shp, True, workspace)

@@ -40,8 +40,9 @@ int make_dims(const psk_shape* sh, Dims* d) {
     if (sh->path < PSK_PATH_AUTO || sh->path > PSK_PATH_TENSOR_CORES) return PSK_ERR_INVALID_ARG;
     if (sh->flags & ~(int32_t)(PSK_FLAG_KEEP_STATES | PSK_FLAG_LOCAL_EXACT)) return PSK_ERR_INVALID_ARG;
     if (sh->B <= 0 || sh->H <= 0 || sh->n <= 0 || sh->b <= 0) return PSK_ERR_SHAPE;
-    if (sh->p != 4 || sh->h != 64) return PSK_ERR_UNSUPPORTED;
+    if ((sh->p != 4 && sh->p != 2) || sh->h != 64) return PSK_ERR_UNSUPPORTED;
     if (sh->r != 16 && sh->r != 32 && sh->r != 64) return PSK_ERR_UNSUPPORTED;
+    if (sh->p == 2 && sh->r != sh->h) return PSK_ERR_UNSUPPORTED;      // p = 2: M = X, so r is h
     if (sh->b % 128 != 0 || sh->n % sh->b != 0) return PSK_ERR_SHAPE;
     if (sh->g_heads != 1 && sh->g_heads != sh->H) return PSK_ERR_SHAPE;
     if (sh->stride_n < sh->h || sh->stride_h <= 0 || sh->stride_b <= 0) return PSK_ERR_SHAPE;
@@ -55,7 +56,9 @@ int make_dims(const psk_shape* sh, Dims* d) {
     d->g_heads = sh->g_heads;
     d->bf16 = sh->dtype == PSK_BF16;
     d->keep_states = (sh->flags & PSK_FLAG_KEEP_STATES) != 0;
-    d->local = (sh->flags & PSK_FLAG_LOCAL_EXACT) != 0;
+    d->p = sh->p;
+    // p = 2 has no sketch error: the exact same-block weights are what it computes anyway
+    d->local = (sh->flags & PSK_FLAG_LOCAL_EXACT) != 0 && sh->p == 4;
     return PSK_OK;
 }
 
@@ -76,7 +79,7 @@ const char* psk_status_string(int status) {
     switch (status) {
         case PSK_OK: return "ok";
         case PSK_ERR_INVALID_ARG: return "invalid argument (null pointer or bad enum)";
-        case PSK_ERR_UNSUPPORTED: return "unsupported configuration (need p=4, h=64, r in {16,32,64})";
+        case PSK_ERR_UNSUPPORTED: return "unsupported configuration (need p=4 or p=2 with r=h, h=64, r in {16,32,64})";
         case PSK_ERR_SHAPE: return "bad shape (need b % 128 == 0, n % b == 0, positive extents)";
         case PSK_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
         case PSK_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
@@ -99,7 +102,7 @@ int psk_sketch(const psk_shape* shape, const void* X, const void* G1, const void
     Dims d;
     const int st = make_dims(shape, &d);
     if (st != PSK_OK) return st;
-    if (!X || !G1 || !G2 || !M_out) return PSK_ERR_INVALID_ARG;
+    if (!X || !M_out || (d.p != 2 && (!G1 || !G2))) return PSK_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(G1) || !aligned16(G2) || !aligned16(M_out) || !aligned16(Phi_out))
         return PSK_ERR_ALIGN;
     int launches = 0;
@@ -114,7 +117,7 @@ int psk_causal_attn_fwd(const psk_shape* shape, const void* Q, const void* K, co
     Dims d;
     const int st = make_dims(shape, &d);
     if (st != PSK_OK) return st;
-    if (!Q || !K || !V || !G1 || !G2 || !O) return PSK_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !O || (d.p != 2 && (!G1 || !G2))) return PSK_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(G1) || !aligned16(G2) ||
         !aligned16(O) || !aligned16(denom))
         return PSK_ERR_ALIGN;
@@ -140,7 +143,8 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
     Dims d;
     const int st = make_dims(shape, &d);
     if (st != PSK_OK) return st;
-    if (!Q || !K || !V || !G1 || !G2 || !O || !denom || !dO || !dQ || !dK || !dV) return PSK_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !O || !denom || !dO || !dQ || !dK || !dV || (d.p != 2 && (!G1 || !G2)))
+        return PSK_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(G1) || !aligned16(G2) ||
         !aligned16(O) || !aligned16(denom) || !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) ||
         !aligned16(dV))

@@ -92,6 +92,45 @@ sketch_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const
 }
 
 // ---------------------------------------------------------------------------
+// Degree p = 2 (Algorithm 1 with p/2 = 1): the "half sketch" is the row itself, M = X, and
+// phi'(x) = x (x) x has h^2 entries: exact degree-2 polynomial attention, no Gaussians.
+// Forward copy M = X (optionally Phi = X (x) X); backward dX = dM (+ add).  One warp per row.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+identity_sketch_kernel(Slice sl, int n, int total_rows, const T* __restrict__ X, float* __restrict__ M,
+                       float* __restrict__ Phi) {
+    const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (row >= total_rows) return;
+    const int64_t base = sl.row(row / n, row % n);
+    const float x0 = ldf(X + base + lane), x1 = ldf(X + base + lane + 32);
+    M[(size_t)row * 64 + lane] = x0;
+    M[(size_t)row * 64 + lane + 32] = x1;
+    if (Phi != nullptr) {
+        for (int a = 0; a < 64; ++a) {
+            const float xa = __shfl_sync(0xffffffffu, a < 32 ? x0 : x1, a % 32);
+            Phi[((size_t)row * 64 + a) * 64 + lane] = xa * x0;
+            Phi[((size_t)row * 64 + a) * 64 + lane + 32] = xa * x1;
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+identity_sketch_bwd_kernel(Slice sl, int n, int total_rows, const float* __restrict__ dM,
+                           const float* __restrict__ add, T* __restrict__ dX) {
+    const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (row >= total_rows) return;
+    const int64_t base = sl.row(row / n, row % n);
+#pragma unroll
+    for (int c = lane; c < 64; c += 32) {
+        float v = dM[(size_t)row * 64 + c];
+        if (add != nullptr) v += add[(size_t)row * 64 + c];
+        stf(dX + base + c, v);
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Row preparation: mode 0 writes V~ = [V | 1]; mode 1 writes E = [dO/d | -(dO.O)/d]
 // One warp per row.
 // ---------------------------------------------------------------------------
@@ -570,6 +609,14 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
 template <typename T, int R>
 cudaError_t launch_sketch(const Dims& d, const T* X, const T* G1, const T* G2, float* M, float* Phi,
                           cudaStream_t s, int* launches) {
+    if (d.p == 2) {           // M = X (R = 64 = h)
+        const int rows = d.BH() * d.n;
+        prof_begin("identity_sketch_kernel", s);
+        identity_sketch_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(Slice{d.H, d.sb, d.sh, d.sn}, d.n, rows, X, M, Phi);
+        prof_end(s);
+        ++*launches;
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)(2 * H64 * R + 64 * 65 + 64 * (R + 1)) * sizeof(float);
     PSK_TRY(allow_smem(sketch_kernel<T, R>, smem));
     Slice sl{d.H, d.sb, d.sh, d.sn};
@@ -674,6 +721,16 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     }
     *launches += 2;
     PSK_TRY(cudaGetLastError());
+    if (d.p == 2) {           // dX = dM (+ the same-block part that bypassed it)
+        prof_begin("identity_sketch_bwd_kernel", s);
+        identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMq, dXq, dQ);
+        prof_end(s);
+        prof_begin("identity_sketch_bwd_kernel", s);
+        identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMk, dXk, dK);
+        prof_end(s);
+        *launches += 2;
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)(2 * H64 * (R + 1) + 64 * 65 + 2 * 64 * (R + 1)) * sizeof(float);
     PSK_TRY(allow_smem(sketch_bwd_kernel<T, R>, smem));
     prof_begin("sketch_bwd_kernel", s);

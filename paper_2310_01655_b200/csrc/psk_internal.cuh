@@ -13,6 +13,7 @@ namespace psk {
 // Validated problem description handed to the launchers.
 struct Dims {
     int B, H, n, h, r, b, t;          // t = n / b blocks per head (Section 3.1)
+    int p;                            // degree: 4, or 2 (no sketch: the half sketch is the row itself, r = h)
     int64_t sb, sh, sn;               // element strides of the [B,H,n,h] tensors
     int g_heads;                      // 1 or H
     bool bf16;                        // storage type

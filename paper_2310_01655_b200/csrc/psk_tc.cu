@@ -962,7 +962,7 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
-    return d.bf16 && encoder() != nullptr;
+    return d.bf16 && d.p == 4 && encoder() != nullptr;      // (p = 2: CUDA-core kernels)
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
