@@ -66,17 +66,6 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// [rows, 64] fp32, contiguous; box = 128 rows x 32 columns (128 B), 128-byte swizzle.
-bool tc_map_f32rows(CUtensorMap* m, const void* base, int64_t rows) {
-    EncodeFn enc = encoder();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {64, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {256};
-    cuuint32_t box[2] = {32, 128}, es[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, es,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 namespace {
 
@@ -447,8 +436,8 @@ struct OutSmem {
     static constexpr int kStageK = 1, kStageV = kZStages - 1;
     // last chunk that uses ring stage s (-1: none)
     __host__ __device__ static constexpr int last_chunk(int nc, int s) { return nc > s ? s + (nc - 1 - s) / kZStages * kZStages : -1; }
-    static constexpr uint32_t So = U, Soc = U + 16384;               // O tile (bf16), two fp32 half tiles
-    static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2, kEpi = 49152;
+    static constexpr uint32_t So = U, Soc = U + 16384;               // O tile, O - c tile (bf16 each)
+    static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2, kEpi = 32768;
     static constexpr uint32_t kMax12 = kPhase1 > kPhase2 ? kPhase1 : kPhase2;
     static constexpr uint32_t total = U + (kMax12 > kEpi ? kMax12 : kEpi);
     // stage s of the prefix-state ring; the last one is the query tile's buffer, dead after the sketch

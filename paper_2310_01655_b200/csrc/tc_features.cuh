@@ -147,12 +147,10 @@ struct CircGen {
 template <int R>
 struct CircUntensor {
     float mr[R], dr[R];
-    int steps;
 
     __device__ __forceinline__ void init(const float (&m)[R]) {
 #pragma unroll
         for (int a = 0; a < R; ++a) { mr[a] = m[a]; dr[a] = 0.f; }
-        steps = 0;
     }
     // xe / xo: gradients of the features of shifts 2j / 2j+1 (fp32 bit patterns, a = 0 .. r-1)
     __device__ __forceinline__ void even(const uint32_t* xe, const float (&m)[R], float (&dm)[R]) {
