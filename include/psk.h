@@ -157,6 +157,20 @@ size_t psk_static_scratch_bytes(void);
 int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void* K, const void* V,
                                const void* G1, const void* G2, void* O, float* denom, void* stream);
 
+/* Block lower-triangular multiplication for arbitrary feature matrices (Section 3.1):
+ *   Out = lt(A B^T) C,   A, B: [batch, n, m],  C, Out: [batch, n, k],  all fp32, contiguous, DEVICE,
+ * computed as  H_l = B_l^T C_l,  Z_l = sum_{j<l} H_j,  rows of block l = lt(A_l B_l^T) C_l + A_l Z_l
+ * over blocks of b rows: O(n b (m + k) + n m k) instead of O(n^2 (m + k)).  The attention
+ * calls above are this algorithm with A = phi'(Q), B = phi'(K), C = [V | 1] and the features
+ * generated on the fly; this call takes any feature matrices (the paper uses it for other
+ * feature maps too).  CUDA-core kernels, fp32 arithmetic.  Needs b % 32 == 0, n % b == 0,
+ * 1 <= k <= 128 (else PSK_ERR_SHAPE); `workspace` (DEVICE) of at least
+ * psk_lt_multiply_workspace_bytes() bytes (0 for a bad shape) holds the t = n / b states
+ * of every batch entry.  Enqueues on `stream` and returns. */
+size_t psk_lt_multiply_workspace_bytes(int batch, int n, int m, int k, int b);
+int psk_lt_multiply(int batch, int n, int m, int k, int b, const float* A, const float* B, const float* C,
+                    float* Out, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, then reports PSK_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` abandoned a bounded wait, PSK_ERR_CUDA if the stream is in error,
  * else PSK_OK.  Never traps. */

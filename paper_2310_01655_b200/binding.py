@@ -63,6 +63,10 @@ def lib():
     L.psk_check.restype = c_int
     L.psk_check.argtypes = [c_void_p, c_void_p]
     L.psk_last_launch_count.restype = c_int
+    L.psk_lt_multiply_workspace_bytes.restype = c_size_t
+    L.psk_lt_multiply_workspace_bytes.argtypes = [c_int] * 5
+    L.psk_lt_multiply.restype = c_int
+    L.psk_lt_multiply.argtypes = [c_int] * 5 + [c_void_p] * 5 + [c_size_t, c_void_p]
     L.psk_profile_enable.restype = c_int
     L.psk_profile_enable.argtypes = [c_int]
     L.psk_profile_count.restype = c_int
@@ -248,3 +252,24 @@ def feature_table(r: int):
     if n < 0:
         raise PskError(n, "psk_feature_table")
     return a[:n].copy(), b[:n].copy(), w[:n].copy()
+
+
+def lt_multiply(A, B, C, b, workspace=None):
+    """psk_lt_multiply: lt(A B^T) C for fp32 CUDA tensors A, B [batch, n, m] and C [batch, n, k]."""
+    _require_cuda(A, B, C)
+    for t in (A, B, C):
+        if t.dtype != torch.float32 or t.dim() != 3 or not t.is_contiguous():
+            raise ValueError("lt_multiply expects contiguous fp32 [batch, n, *] tensors")
+    batch, n, m = A.shape
+    k = C.shape[2]
+    if B.shape != A.shape or C.shape[:2] != A.shape[:2]:
+        raise ValueError("lt_multiply: A, B [batch, n, m] and C [batch, n, k] must agree")
+    need = int(lib().psk_lt_multiply_workspace_bytes(batch, n, m, k, b))
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=A.device)
+    out = torch.empty_like(C)
+    st = lib().psk_lt_multiply(batch, n, m, k, b, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _ptr(workspace),
+                               workspace.numel() if workspace is not None else 0, _stream())
+    if st != 0:
+        raise PskError(st, "psk_lt_multiply")
+    return out
