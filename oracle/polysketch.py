@@ -26,7 +26,9 @@ finite differences for every gradient, dV against the explicit weight matrix;
 for the local-exact variant (Section 3.2): one block = exact polynomial
 attention, exact features = no dependence on the block size, looped definition,
 block algorithm against the masked definition, finite differences; for
-degree 2 (no sketch): looped (q.k)^2 attention, finite differences.
+degree 2 (no sketch): looped (q.k)^2 attention, finite differences; for degree 8:
+the recursion written out, Monte-Carlo mean (q.k)^4 of the half sketch, exact
+features, block algorithm against the definition, finite differences.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -377,6 +379,73 @@ def causal_degree2_attention_backward(Q, K, V, dO):
     dW = lt(E @ Vt.T)
     ds = 2.0 * s * dW
     return ds @ K, ds.T @ Q, W.T @ E[:, :h]
+
+
+# ---------------------------------------------------------------------------
+# Degree p = 8: one more level of Algorithm 1's recursion.  PolySketchWithNegativity(A, r, 4)
+# combines two independent degree-2 sketches M1, M2 of A through two r x r Gaussians,
+#   M = sqrt(1/r) [(M1 Gc1) * (M2 Gc2)],   M1 = sqrt(1/r) [(A Ga1) * (A Ga2)],  M2 likewise with Gb,
+# and phi'(A) = M^{(x)2}: <phi'(q), phi'(k)> = (M_q . M_k)^2 approximates (q . k)^8.
+# Everything after the half sketch M is the p = 4 algorithm unchanged.
+# ---------------------------------------------------------------------------
+def half_sketch_degree4(X, gaussians):
+    """PolySketchWithNegativity(X, r, 4) with gaussians = [Ga1, Ga2, Gb1, Gb2, Gc1, Gc2]."""
+    M, rest = polysketch_with_negativity(X, list(gaussians), 4)
+    assert len(rest) == 0
+    return M
+
+
+def causal_attention_blocked_from_half_sketches(Mq, Mk, V, b):
+    """Section 3.1 on phi' = M^{(x)2} for given half sketches (diagonal blocks through (L R^T)^2)."""
+    Mq, Mk, V = _f64(Mq), _f64(Mk), _f64(V)
+    n, h = V.shape
+    C = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+
+    def diag_block(l):
+        return lt((Mq[l * b:(l + 1) * b] @ Mk[l * b:(l + 1) * b].T) ** 2)
+
+    N = lt_multiply_blocked(self_tensor(Mq), self_tensor(Mk), C, b, diag_block)
+    d = 1.0 + N[:, h]
+    return N[:, :h] / d[:, None], d
+
+
+def causal_polysketch8_attention(Q, K, V, gaussians):
+    """Section 3 with phi' = PolySketchNonNegative(., r, 8): the n x n definition.  Returns (O, d)."""
+    s = half_sketch_degree4(Q, gaussians) @ half_sketch_degree4(K, gaussians).T
+    W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
+def _sketch_degree4_backward(X, gaussians, dM):
+    """Chain rule through M = sqrt(1/r) [(M1 Gc1) * (M2 Gc2)] and the two degree-2 sketches."""
+    X = _f64(X)
+    Ga1, Ga2, Gb1, Gb2, Gc1, Gc2 = (_f64(g) for g in gaussians)
+    r = Gc1.shape[1]
+    rs = 1.0 / np.sqrt(r)
+    M1 = rs * (X @ Ga1) * (X @ Ga2)
+    M2 = rs * (X @ Gb1) * (X @ Gb2)
+    C1, C2 = M1 @ Gc1, M2 @ Gc2
+    dM1 = (rs * dM * C2) @ Gc1.T
+    dM2 = (rs * dM * C1) @ Gc2.T
+    return _sketch_backward(X, Ga1, Ga2, dM1) + _sketch_backward(X, Gb1, Gb2, dM2)
+
+
+def causal_polysketch8_attention_backward(Q, K, V, gaussians, dO):
+    """Gradients (dQ, dK, dV) of sum(dO * O) for degree 8, through the quadratic definition."""
+    V = _f64(V)
+    n, h = V.shape
+    Mq, Mk = half_sketch_degree4(Q, gaussians), half_sketch_degree4(K, gaussians)
+    s = Mq @ Mk.T
+    W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = lt(E @ Vt.T)
+    ds = 2.0 * s * dW
+    return (_sketch_degree4_backward(Q, gaussians, ds @ Mk), _sketch_degree4_backward(K, gaussians, ds.T @ Mq),
+            W.T @ E[:, :h])
 
 
 # ---------------------------------------------------------------------------
