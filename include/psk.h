@@ -38,6 +38,12 @@
  *     h^2 entries, i.e. exact degree-2 polynomial attention with weights (q_i . k_j)^2.
  *     Set r = h; G1 and G2 are not read and may be null.  Served by the CUDA-core
  *     kernels for either storage type (PSK_PATH_TENSOR_CORES: PSK_ERR_UNSUPPORTED).
+ *   - Also p = 8 (one more level of Algorithm 1's recursion): two independent degree-2
+ *     sketches M1 = sqrt(1/r)[(x Ga1)*(x Ga2)], M2 = sqrt(1/r)[(x Gb1)*(x Gb2)] combined as
+ *     m(x) = sqrt(1/r)[(M1 Gc1)*(M2 Gc2)] with Gc1, Gc2 of r x r; phi'(x) = m (x) m as for p = 4,
+ *     so the weights approximate (q_i . k_j)^8.  G1 then holds [Ga1; Gb1; Gc1] and G2 holds
+ *     [Ga2; Gb2; Gc2], each [g_heads, 2h + r, r] contiguous.  CUDA-core kernels only; not
+ *     with PSK_FLAG_LOCAL_EXACT (PSK_ERR_UNSUPPORTED).
  */
 #ifndef PSK_H_
 #define PSK_H_
@@ -52,7 +58,7 @@ extern "C" {
 typedef enum {
     PSK_OK = 0,
     PSK_ERR_INVALID_ARG = -1,   /* null pointer, bad enum value                      */
-    PSK_ERR_UNSUPPORTED = -2,   /* p not 4 (or 2 with r = h), h != 64, r not in {16,32,64}, bad path */
+    PSK_ERR_UNSUPPORTED = -2,   /* p not 4, 8 (or 2 with r = h), h != 64, r not in {16,32,64}, bad path */
     PSK_ERR_SHAPE = -3,         /* n % b != 0, b % 128 != 0, non-positive extents    */
     PSK_ERR_ALIGN = -4,         /* pointer or stride not 16-byte aligned             */
     PSK_ERR_WORKSPACE = -5,     /* workspace missing, misaligned or too small        */

@@ -40,7 +40,9 @@ int make_dims(const psk_shape* sh, Dims* d) {
     if (sh->path < PSK_PATH_AUTO || sh->path > PSK_PATH_TENSOR_CORES) return PSK_ERR_INVALID_ARG;
     if (sh->flags & ~(int32_t)(PSK_FLAG_KEEP_STATES | PSK_FLAG_LOCAL_EXACT)) return PSK_ERR_INVALID_ARG;
     if (sh->B <= 0 || sh->H <= 0 || sh->n <= 0 || sh->b <= 0) return PSK_ERR_SHAPE;
-    if ((sh->p != 4 && sh->p != 2) || sh->h != 64) return PSK_ERR_UNSUPPORTED;
+    if ((sh->p != 4 && sh->p != 2 && sh->p != 8) || sh->h != 64) return PSK_ERR_UNSUPPORTED;
+    // exact same-block weights are built for degree 4 (and are what degree 2 computes anyway)
+    if (sh->p == 8 && (sh->flags & PSK_FLAG_LOCAL_EXACT)) return PSK_ERR_UNSUPPORTED;
     if (sh->r != 16 && sh->r != 32 && sh->r != 64) return PSK_ERR_UNSUPPORTED;
     if (sh->p == 2 && sh->r != sh->h) return PSK_ERR_UNSUPPORTED;      // p = 2: M = X, so r is h
     if (sh->b % 128 != 0 || sh->n % sh->b != 0) return PSK_ERR_SHAPE;
@@ -79,7 +81,7 @@ const char* psk_status_string(int status) {
     switch (status) {
         case PSK_OK: return "ok";
         case PSK_ERR_INVALID_ARG: return "invalid argument (null pointer or bad enum)";
-        case PSK_ERR_UNSUPPORTED: return "unsupported configuration (need p=4 or p=2 with r=h, h=64, r in {16,32,64})";
+        case PSK_ERR_UNSUPPORTED: return "unsupported configuration (need p=4, p=8 or p=2 with r=h; h=64; r in {16,32,64})";
         case PSK_ERR_SHAPE: return "bad shape (need b % 128 == 0, n % b == 0, positive extents)";
         case PSK_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
         case PSK_ERR_WORKSPACE: return "workspace missing, misaligned or too small";

@@ -131,6 +131,152 @@ identity_sketch_bwd_kernel(Slice sl, int n, int total_rows, const float* __restr
 }
 
 // ---------------------------------------------------------------------------
+// Degree p = 8: one more level of Algorithm 1's recursion.  Two independent degree-2 sketches
+//   M1 = (X Ga1)*(X Ga2)/sqrt(r),  M2 = (X Gb1)*(X Gb2)/sqrt(r)
+// are combined through r x r Gaussians,  M = (M1 Gc1)*(M2 Gc2)/sqrt(r); phi' = M (x) M as before.
+// G1 holds [Ga1; Gb1; Gc1] and G2 holds [Ga2; Gb2; Gc2], each (2h + r) x r row-major per head.
+// 32 rows per CTA; the Gaussians are read from global memory (they stay in cache).
+// ---------------------------------------------------------------------------
+template <int R> struct Sk8 {
+    static constexpr int kRows = 32, kLd = R + 1;
+    static constexpr int kGRows = 2 * H64 + R;             // rows of one packed Gaussian set
+    static constexpr int X = 0;                            // [32][65]
+    static constexpr int A1 = X + kRows * 65, A2 = A1 + kRows * kLd, B1 = A2 + kRows * kLd, B2 = B1 + kRows * kLd;
+    static constexpr int M1 = B2 + kRows * kLd, M2 = M1 + kRows * kLd, C1 = M2 + kRows * kLd, C2 = C1 + kRows * kLd;
+    static constexpr int total = C2 + kRows * kLd;
+    static constexpr size_t bytes = (size_t)total * sizeof(float);
+};
+
+// shared by the forward and the backward: X tile -> A1, A2, B1, B2, M1, M2, C1 = M1 Gc1, C2 = M2 Gc2
+template <typename T, int R>
+__device__ __forceinline__ void sketch8_forward_tile(float* smem, Slice sl, const T* __restrict__ X,
+                                                     const T* __restrict__ g1, const T* __restrict__ g2,
+                                                     int bh, int i0, int tid) {
+    using L = Sk8<R>;
+    for (int e = tid; e < L::kRows * H64; e += 256) {
+        const int rr = e / H64, c = e % H64;
+        smem[L::X + rr * 65 + c] = ldf(X + sl.row(bh, i0 + rr) + c);
+    }
+    __syncthreads();
+    const float rs = rsqrtf((float)R);
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, c = e % R;
+        float a1 = 0.f, a2 = 0.f, b1 = 0.f, b2 = 0.f;
+        for (int t = 0; t < H64; ++t) {
+            const float x = smem[L::X + rr * 65 + t];
+            a1 = fmaf(x, ldf(g1 + t * R + c), a1);
+            a2 = fmaf(x, ldf(g2 + t * R + c), a2);
+            b1 = fmaf(x, ldf(g1 + (H64 + t) * R + c), b1);
+            b2 = fmaf(x, ldf(g2 + (H64 + t) * R + c), b2);
+        }
+        const int o = rr * L::kLd + c;
+        smem[L::A1 + o] = a1; smem[L::A2 + o] = a2; smem[L::B1 + o] = b1; smem[L::B2 + o] = b2;
+        smem[L::M1 + o] = a1 * a2 * rs;
+        smem[L::M2 + o] = b1 * b2 * rs;
+    }
+    __syncthreads();
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, c = e % R;
+        float c1 = 0.f, c2 = 0.f;
+        for (int k = 0; k < R; ++k) {
+            c1 = fmaf(smem[L::M1 + rr * L::kLd + k], ldf(g1 + (2 * H64 + k) * R + c), c1);
+            c2 = fmaf(smem[L::M2 + rr * L::kLd + k], ldf(g2 + (2 * H64 + k) * R + c), c2);
+        }
+        smem[L::C1 + rr * L::kLd + c] = c1;
+        smem[L::C2 + rr * L::kLd + c] = c2;
+    }
+    __syncthreads();
+}
+
+template <typename T, int R>
+__global__ void __launch_bounds__(256)
+sketch8_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const T* __restrict__ G2,
+               int g_heads, int n, float* __restrict__ M_out, float* __restrict__ Phi_out) {
+    extern __shared__ float smem[];
+    using L = Sk8<R>;
+    const int bh = blockIdx.y, i0 = blockIdx.x * L::kRows, tid = threadIdx.x;
+    const int g = (g_heads == 1) ? 0 : (bh % sl.H);
+    const T* g1 = G1 + (size_t)g * L::kGRows * R;
+    const T* g2 = G2 + (size_t)g * L::kGRows * R;
+    sketch8_forward_tile<T, R>(smem, sl, X, g1, g2, bh, i0, tid);
+    const float rs = rsqrtf((float)R);
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, c = e % R;
+        const float m = smem[L::C1 + rr * L::kLd + c] * smem[L::C2 + rr * L::kLd + c] * rs;
+        smem[L::M1 + rr * L::kLd + c] = m;                 // (M1 is dead: keep M for Phi)
+        M_out[((size_t)bh * n + i0 + rr) * R + c] = m;
+    }
+    if (Phi_out != nullptr) {
+        __syncthreads();
+        for (int e = tid; e < L::kRows * R * R; e += 256) {
+            const int rr = e / (R * R), f = e % (R * R);
+            Phi_out[((size_t)bh * n + i0 + rr) * R * R + f] =
+                smem[L::M1 + rr * L::kLd + f / R] * smem[L::M1 + rr * L::kLd + f % R];
+        }
+    }
+}
+
+// Chain rule through the degree-8 half sketch (forward values recomputed):
+//   dC1 = dM*C2/sqrt(r), dC2 = dM*C1/sqrt(r);  dM1 = dC1 Gc1^T, dM2 = dC2 Gc2^T;
+//   dA1 = dM1*A2/sqrt(r), dA2 = dM1*A1/sqrt(r), dB1 = dM2*B2/sqrt(r), dB2 = dM2*B1/sqrt(r);
+//   dX = dA1 Ga1^T + dA2 Ga2^T + dB1 Gb1^T + dB2 Gb2^T.
+template <typename T, int R>
+__global__ void __launch_bounds__(256)
+sketch8_bwd_kernel(Slice sl, const T* __restrict__ X, const T* __restrict__ G1, const T* __restrict__ G2,
+                   int g_heads, int n, const float* __restrict__ dM, T* __restrict__ dX) {
+    extern __shared__ float smem[];
+    using L = Sk8<R>;
+    const int bh = blockIdx.y, i0 = blockIdx.x * L::kRows, tid = threadIdx.x;
+    const int g = (g_heads == 1) ? 0 : (bh % sl.H);
+    const T* g1 = G1 + (size_t)g * L::kGRows * R;
+    const T* g2 = G2 + (size_t)g * L::kGRows * R;
+    sketch8_forward_tile<T, R>(smem, sl, X, g1, g2, bh, i0, tid);
+    const float rs = rsqrtf((float)R);
+    // dC1, dC2 over C1, C2 (each entry is read and written by one thread)
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, c = e % R, o = rr * L::kLd + c;
+        const float gm = dM[((size_t)bh * n + i0 + rr) * R + c] * rs;
+        const float c1 = smem[L::C1 + o], c2 = smem[L::C2 + o];
+        smem[L::C1 + o] = gm * c2;
+        smem[L::C2 + o] = gm * c1;
+    }
+    __syncthreads();
+    // dM1, dM2 over M1, M2 (M1, M2 themselves are no longer needed)
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, k = e % R;
+        float d1 = 0.f, d2 = 0.f;
+        for (int c = 0; c < R; ++c) {
+            d1 = fmaf(smem[L::C1 + rr * L::kLd + c], ldf(g1 + (2 * H64 + k) * R + c), d1);
+            d2 = fmaf(smem[L::C2 + rr * L::kLd + c], ldf(g2 + (2 * H64 + k) * R + c), d2);
+        }
+        smem[L::M1 + rr * L::kLd + k] = d1;
+        smem[L::M2 + rr * L::kLd + k] = d2;
+    }
+    __syncthreads();
+    // dA1, dA2, dB1, dB2 over A1, A2, B1, B2
+    for (int e = tid; e < L::kRows * R; e += 256) {
+        const int rr = e / R, c = e % R, o = rr * L::kLd + c;
+        const float d1 = smem[L::M1 + o] * rs, d2 = smem[L::M2 + o] * rs;
+        const float a1 = smem[L::A1 + o], a2 = smem[L::A2 + o], b1 = smem[L::B1 + o], b2 = smem[L::B2 + o];
+        smem[L::A1 + o] = d1 * a2; smem[L::A2 + o] = d1 * a1;
+        smem[L::B1 + o] = d2 * b2; smem[L::B2 + o] = d2 * b1;
+    }
+    __syncthreads();
+    for (int e = tid; e < L::kRows * H64; e += 256) {
+        const int rr = e / H64, t = e % H64;
+        float dx = 0.f;
+        for (int c = 0; c < R; ++c) {
+            const int o = rr * L::kLd + c;
+            dx = fmaf(smem[L::A1 + o], ldf(g1 + t * R + c), dx);
+            dx = fmaf(smem[L::A2 + o], ldf(g2 + t * R + c), dx);
+            dx = fmaf(smem[L::B1 + o], ldf(g1 + (H64 + t) * R + c), dx);
+            dx = fmaf(smem[L::B2 + o], ldf(g2 + (H64 + t) * R + c), dx);
+        }
+        stf(dX + sl.row(bh, i0 + rr) + t, dx);
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Row preparation: mode 0 writes V~ = [V | 1]; mode 1 writes E = [dO/d | -(dO.O)/d]
 // One warp per row.
 // ---------------------------------------------------------------------------
@@ -617,6 +763,15 @@ cudaError_t launch_sketch(const Dims& d, const T* X, const T* G1, const T* G2, f
         ++*launches;
         return cudaGetLastError();
     }
+    if (d.p == 8) {           // one more recursion level: packed Gaussians [Ga; Gb; Gc]
+        PSK_TRY((allow_smem(sketch8_kernel<T, R>, Sk8<R>::bytes)));
+        prof_begin("sketch8_kernel", s);
+        sketch8_kernel<T, R><<<dim3(d.n / Sk8<R>::kRows, d.BH()), 256, Sk8<R>::bytes, s>>>(
+            Slice{d.H, d.sb, d.sh, d.sn}, X, G1, G2, d.g_heads, d.n, M, Phi);
+        prof_end(s);
+        ++*launches;
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)(2 * H64 * R + 64 * 65 + 64 * (R + 1)) * sizeof(float);
     PSK_TRY(allow_smem(sketch_kernel<T, R>, smem));
     Slice sl{d.H, d.sb, d.sh, d.sn};
@@ -727,6 +882,18 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
         prof_end(s);
         prof_begin("identity_sketch_bwd_kernel", s);
         identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMk, dXk, dK);
+        prof_end(s);
+        *launches += 2;
+        return cudaGetLastError();
+    }
+    if (d.p == 8) {
+        PSK_TRY((allow_smem(sketch8_bwd_kernel<T, R>, Sk8<R>::bytes)));
+        const dim3 grid8(d.n / Sk8<R>::kRows, d.BH());
+        prof_begin("sketch8_bwd_kernel", s);
+        sketch8_bwd_kernel<T, R><<<grid8, 256, Sk8<R>::bytes, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dQ);
+        prof_end(s);
+        prof_begin("sketch8_bwd_kernel", s);
+        sketch8_bwd_kernel<T, R><<<grid8, 256, Sk8<R>::bytes, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dK);
         prof_end(s);
         *launches += 2;
         return cudaGetLastError();

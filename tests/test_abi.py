@@ -58,7 +58,7 @@ def test_workspace_size_formula(L):
 
 
 @pytest.mark.parametrize("field,value,code", [
-    ("p", 2, -2), ("p", 8, -2), ("h", 128, -2), ("r", 48, -2),
+    ("p", 2, -2), ("p", 6, -2), ("p", 16, -2), ("h", 128, -2), ("r", 48, -2),      # (p = 2 needs r = h)
     ("b", 100, -3), ("n", 500, -3), ("B", 0, -3), ("g_heads", 3, -3),
     ("dtype", 7, -1), ("path", 9, -1), ("flags", 6, -1), ("stride_n", 66, -4),
 ])
