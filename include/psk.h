@@ -177,6 +177,20 @@ size_t psk_lt_multiply_workspace_bytes(int batch, int n, int m, int k, int b);
 int psk_lt_multiply(int batch, int n, int m, int k, int b, const float* A, const float* B, const float* C,
                     float* Out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Recurrent form: one new token per (batch, head) per call (inference at O(r^2 h) per token,
+ * whatever the context length).  With the running state S (r^2 x 65 per head, fp32)
+ *   S <- S + phi'(k_t) [v_t | 1]^T,   N = phi'(q_t)^T S,   d = 1 + N[64],   o_t = N[:64] / d,
+ * which is row t of psk_causal_attn_fwd (without PSK_FLAG_LOCAL_EXACT) when the calls are made
+ * for t = 0, 1, ... on a state that started as zeros.  q, k, v, o: [B, H, h] contiguous DEVICE
+ * arrays of the shape's dtype; G1, G2 as for the other calls; `state`: DEVICE array of
+ * psk_decode_state_bytes(shape) bytes, [B*H][r*r][65] fp32, rows in the Kronecker order
+ * a*r + b, owned and zero-initialised by the caller, updated in place; `denom` ([B, H] fp32,
+ * DEVICE) may be null.  Of the shape only B, H, h, r, p (= 4), dtype, g_heads are read;
+ * flags must be 0.  CUDA-core kernel; one pass over the state per call. */
+size_t psk_decode_state_bytes(const psk_shape* shape);
+int psk_decode_step(const psk_shape* shape, const void* q, const void* k, const void* v, const void* G1,
+                    const void* G2, float* state, void* o, float* denom, void* stream);
+
 /* Synchronises `stream`, then reports PSK_ERR_TIMEOUT if a kernel of the last call that
  * used `workspace` abandoned a bounded wait, PSK_ERR_CUDA if the stream is in error,
  * else PSK_OK.  Never traps. */

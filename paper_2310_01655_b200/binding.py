@@ -67,6 +67,10 @@ def lib():
     L.psk_lt_multiply_workspace_bytes.argtypes = [c_int] * 5
     L.psk_lt_multiply.restype = c_int
     L.psk_lt_multiply.argtypes = [c_int] * 5 + [c_void_p] * 5 + [c_size_t, c_void_p]
+    L.psk_decode_state_bytes.restype = c_size_t
+    L.psk_decode_state_bytes.argtypes = [POINTER(Shape)]
+    L.psk_decode_step.restype = c_int
+    L.psk_decode_step.argtypes = [POINTER(Shape)] + [c_void_p] * 9
     L.psk_profile_enable.restype = c_int
     L.psk_profile_enable.argtypes = [c_int]
     L.psk_profile_count.restype = c_int
@@ -273,3 +277,28 @@ def lt_multiply(A, B, C, b, workspace=None):
     if st != 0:
         raise PskError(st, "psk_lt_multiply")
     return out
+
+
+def decode_state(B, H, r, device="cuda"):
+    """Zero state for decode_step: [B, H, r*r, 65] fp32."""
+    return torch.zeros((B, H, r * r, 65), dtype=torch.float32, device=device)
+
+
+def decode_step(q, k, v, G1, G2, state):
+    """psk_decode_step: q, k, v [B, H, h]; updates `state` in place; returns (o [B, H, h], denom [B, H])."""
+    _require_cuda(q, k, v, G1, G2, state)
+    B, H, h = q.shape
+    r = G1.shape[-1]
+    g_heads = G1.shape[0] if G1.dim() == 3 else 1
+    if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and state.is_contiguous()):
+        raise ValueError("decode_step expects contiguous tensors")
+    shp = Shape(B, H, 1, h, r, 4, 128, _DTYPES[q.dtype], H * h, h, h, g_heads, PATH_AUTO, 0)
+    if state.numel() * 4 != int(lib().psk_decode_state_bytes(byref(shp))):
+        raise ValueError("decode_step: state must be [B, H, r*r, 65] fp32")
+    o = torch.empty_like(q)
+    den = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    st = lib().psk_decode_step(byref(shp), _ptr(q), _ptr(k), _ptr(v), _ptr(_contig(G1)), _ptr(_contig(G2)),
+                               _ptr(state), _ptr(o), _ptr(den), _stream())
+    if st != 0:
+        raise PskError(st, "psk_decode_step")
+    return o, den
