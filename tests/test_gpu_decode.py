@@ -54,14 +54,17 @@ def test_bad_arguments_and_step_time():
     for _ in range(3):
         psk.decode_step(q, k, v, inp["G1"], inp["G2"], state)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    # device time of the kernel itself (events the library records around its launch): a Python
+    # caller cannot issue steps as fast as they run
+    psk.profile_enable(True)
     for _ in range(20):
         psk.decode_step(q, k, v, inp["G1"], inp["G2"], state)
-    e1.record()
     torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / 20
+    recs = [ms for name, ms in psk.profile_records() if name == "decode_step_kernel"]
+    psk.profile_enable(False)
+    assert len(recs) == 20
+    us = 1e3 * sorted(recs)[len(recs) // 2]
     moved = 2 * state.numel() * 4                     # the state is read and written once
     print("decode step: %.1f us for 384 heads, %.0f GB/s of state traffic" % (us, moved / us / 1e3))
     assert torch.isfinite(state).all()
-    assert moved / (us * 1e-6) > 1.0e12               # streams the state at more than 1 TB/s
+    assert moved / (us * 1e-6) > 2.0e12               # streams the state at more than 2 TB/s
