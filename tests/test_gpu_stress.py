@@ -14,12 +14,13 @@ from paper_2310_01655_b200 import inputs as wl
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("local", [False, True])
 @pytest.mark.parametrize("r,b,n", [(32, 256, 16384), (16, 128, 4096), (64, 512, 8192)])
-def test_repeated_calls_agree_bitwise(r, b, n):
+def test_repeated_calls_agree_bitwise(r, b, n, local):
     w = wl.small_workload(B=2, H=6, n=n, r=r, b=b, dtype="bf16", seed=700 + r)
     inp = wl.make_inputs(w, "cuda", with_dO=True)
     Q, K, V, G1, G2, dO = (inp[k] for k in ("Q", "K", "V", "G1", "G2", "dO"))
-    flags = psk.FLAG_KEEP_STATES
+    flags = psk.FLAG_KEEP_STATES | (psk.FLAG_LOCAL_EXACT if local else 0)
     shp = psk.binding.make_shape(Q, G1, r, b, flags=flags)
     ws = torch.zeros(psk.workspace_bytes(shp, True), dtype=torch.uint8, device="cuda")
     first = None
