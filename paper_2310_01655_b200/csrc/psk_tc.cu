@@ -425,7 +425,7 @@ struct OutSmem {
     static constexpr uint32_t Mq = Ones + 4096;
     // split operand: 3R columns.  (LOCAL: no split operands; the region holds the ring's last
     // stage and then the value tile, because the query tile stays alive for the exact scores.)
-    static constexpr uint32_t kMqBytes = (LOCAL && 128 * 3 * R * 2 < 16384) ? 16384 : 128 * 3 * R * 2;
+    static constexpr uint32_t kMqBytes = LOCAL ? 16384 : 128 * 3 * R * 2;
     static constexpr uint32_t U = (Mq + kMqBytes + 1023) / 1024 * 1024;
     static constexpr uint32_t Z = U;
     // key tile in ring stage 1, value tile in the query tile's buffer (ring stage 3), split key
@@ -437,7 +437,7 @@ struct OutSmem {
     // last chunk that uses ring stage s (-1: none)
     __host__ __device__ static constexpr int last_chunk(int nc, int s) { return nc > s ? s + (nc - 1 - s) / kZStages * kZStages : -1; }
     static constexpr uint32_t So = U, Soc = U + 16384;               // O tile, O - c tile (bf16 each)
-    static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + 128 * 3 * R * 2, kEpi = 32768;
+    static constexpr uint32_t kPhase1 = (kZStages - 1) * kZStageBytes, kPhase2 = 32768 + (LOCAL ? 0 : 128 * 3 * R * 2), kEpi = 32768;
     static constexpr uint32_t kMax12 = kPhase1 > kPhase2 ? kPhase1 : kPhase2;
     static constexpr uint32_t total = U + (kMax12 > kEpi ? kMax12 : kEpi);
     // stage s of the prefix-state ring; the last one is the query tile's buffer, dead after the sketch
@@ -453,7 +453,7 @@ struct OutSmem {
 // (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
 // they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
 template <int R, int MODE, bool LOCAL>
-__global__ void __launch_bounds__(160, (R <= 32 ? 2 : 1))
+__global__ void __launch_bounds__(160, ((R <= 32 || LOCAL) ? 2 : 1))
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
                   const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapOc,
