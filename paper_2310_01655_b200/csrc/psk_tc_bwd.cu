@@ -72,10 +72,9 @@ tc_bwd_prep_kernel(const bf16* __restrict__ dO, const float* __restrict__ denom,
     (void)total_rows;
 }
 
-constexpr int kStages = 4;
 constexpr uint32_t kBoxBytes = 16384;      // two [64 features x 128 B] boxes: state columns 0..63, 64..79
 
-template <int R>
+template <int R, bool LOCAL = false, bool QSIDE = false>
 struct BwdSmem {
     // every tile: 128 rows x 128 B, 128-byte swizzle
     static constexpr uint32_t kM = HiLoTiles<R>::N * 16384;      // [hi | lo] half-sketch operand
@@ -84,20 +83,26 @@ struct BwdSmem {
     static constexpr uint32_t ExtA = G + GImage<R>::bytes;       // [128 x 16] un-swizzled
     static constexpr uint32_t Eoth = ExtA + 4096;        // 128 x (1/d, e65h) of the other side's rows
     static constexpr uint32_t U = Eoth + 1024;
-    static constexpr uint32_t Box = U;                   // phase B: kStages state boxes
+    static constexpr uint32_t Box = U;                   // phase B: kSt state boxes
     static constexpr int NC = Feat<R>::NC;
+    // stages of the state-chunk ring: four; three on the query side for r = 64 with exact
+    // same-block weights, which then fits two CTAs per SM (no split-operand tiles in that variant;
+    // the key side, at 255 registers and 225 KB of code, ran slower as two CTAs and keeps four)
+    static constexpr int kSt = (R > 32 && LOCAL && QSIDE) ? 3 : 4;
     // Phase C tiles.  r <= 32 (two CTAs per SM): they reuse the boxes' memory, each tile in the
     // stage that the last chunks free first, so the first other-side tile is fetched while the
-    // last chunks are still being processed.  r = 64 (one CTA per SM): memory of their own.
-    static constexpr bool kAlias = (R <= 32);
-    static constexpr int sX = NC >= 4 ? (NC - 4) % 4 : 3, sY = NC >= 4 ? (NC - 3) % 4 : 0;
-    static constexpr int sMo = NC >= 4 ? (NC - 2) % 4 : 1, sMn = NC >= 4 ? (NC - 1) % 4 : 2;
-    static constexpr uint32_t C0 = U + kStages * kBoxBytes;
+    // last chunks are still being processed.  r = 64 (one CTA per SM): memory of their own,
+    // except with exact same-block weights, where X, Y and the second X buffer are all there is.
+    static constexpr bool kAlias = (R <= 32) || LOCAL;
+    static constexpr int sX = NC >= kSt ? (NC - kSt) % kSt : 3, sY = NC >= kSt ? (NC - kSt + 1) % kSt : 0;
+    static constexpr int sMo = NC >= kSt ? (NC - kSt + 2) % kSt : 1, sMn = NC >= kSt ? (NC - 1) % kSt : 2;
+    static constexpr uint32_t C0 = U + kSt * kBoxBytes;
     static constexpr uint32_t Xoth = kAlias ? U + sX * kBoxBytes : C0;
     static constexpr uint32_t Yoth = kAlias ? U + sY * kBoxBytes : C0 + 16384;
     static constexpr uint32_t Moth = kAlias ? U + sMo * kBoxBytes : C0 + 32768;
     static constexpr uint32_t Mown = kAlias ? U + sMn * kBoxBytes : C0 + 32768 + kM;
-    static_assert(!kAlias || kM == kBoxBytes, "aliased layout: one tile per stage");
+    static_assert(!kAlias || LOCAL || kM == kBoxBytes, "aliased layout: one tile per stage");
+    static_assert(kSt == 4 || NC >= kSt, "three stages: only with many chunks");
     static constexpr uint32_t total = kAlias ? C0 : C0 + 32768 + 2 * kM;
     // output staging (epilogue): dX, dV tiles
     static constexpr uint32_t Sx = U, Sv = U + 16384;
@@ -142,7 +147,7 @@ __device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint32_t own, uint
 // into a dX accumulator that the sketch's backward (phase D) adds to: no half sketch of the other
 // tile, no split operands, no dM from the tiles.
 template <int R, bool QSIDE, bool LOCAL>
-__global__ void __launch_bounds__(128, (R <= 32 ? 2 : 1))
+__global__ void __launch_bounds__(128, ((R <= 32 || (LOCAL && QSIDE)) ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
                    const __grid_constant__ CUtensorMap mapS, const __grid_constant__ CUtensorMap mapDX,
@@ -151,10 +156,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    const float* __restrict__ y65g, const float* __restrict__ e65h, const float* __restrict__ denom,
                    int* status) {
     using F = Feat<R>;
-    using L = BwdSmem<R>;
+    using L = BwdSmem<R, LOCAL, QSIDE>;
+    constexpr int kStages = L::kSt;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_own, bar_xoth, bar_yoth, bar_mma, bar_phi[2], bar_box[kStages];
+    __shared__ uint64_t bar_own, bar_xoth, bar_yoth, bar_mma, bar_phi[2], bar_box[4];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
@@ -314,11 +320,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             } else if (L::kAlias) {
                 // the last chunks free the stages that the first other-side tile goes into
                 const int orow_first = l * b + (QSIDE ? 0 : tau) * 128;
-                if (F::NC >= kStages && C == F::NC - 4) {
+                if (F::NC >= kStages && C == F::NC - kStages) {
                     mbar_expect_tx(&bar_xoth, 16384);
                     tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow_first, hi, bi, &bar_xoth);
                 }
-                if (C == (F::NC >= kStages ? F::NC - 3 : 0)) {
+                if (C == (F::NC >= kStages ? F::NC - kStages + 1 : 0)) {
                     mbar_expect_tx(&bar_yoth, 16384);
                     tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow_first, hi, bi, &bar_yoth);
                 }
@@ -757,12 +763,12 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     } else {
         PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, y65, e65h, status, s, launches));
     }
-    constexpr size_t smem = BwdSmem<R>::total + 1024;
     const dim3 grid(d.b / 128, d.t, d.BH());
     auto rows = [&](auto local_c) -> cudaError_t {
         constexpr bool LOCAL = decltype(local_c)::value;
+        constexpr size_t smem = BwdSmem<R, LOCAL, true>::total + 1024, smem_k = BwdSmem<R, LOCAL, false>::total + 1024;
         PSK_TRY((set_smem(tc_bwd_rows_kernel<R, true, LOCAL>, smem)));
-        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, false, LOCAL>, smem)));
+        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, false, LOCAL>, smem_k)));
         // query side first: it needs only the prefix states, and the row scalars just written are
         // still in L2; the suffix states (5 GB through L2) come after it
         prof_begin("tc_bwd_q_kernel", s);
@@ -774,7 +780,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // suffix states: phi(q_i) / d_i against [dO_i | y65_i]
         PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
-        tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
+        tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
                                                                     d.b, d.t, y65, e65h, denom, status);
         prof_end(s);
         ++*launches;
