@@ -80,6 +80,10 @@ typedef struct {
     int32_t g_heads;            /* 1 or H */
     int32_t path;               /* psk_path */
     int32_t flags;              /* bit set of psk_flags, 0 for none */
+    int32_t seq_segments;       /* tensor-core path: runs of blocks a head's sequence is cut into for the
+                                   prefix scan over block states (Section 3.1 notes that the prefix sums
+                                   can be computed in parallel); 0 = the library chooses (1 unless there
+                                   are too few heads to fill the GPU); must divide n / b */
 } psk_shape;
 
 /* PSK_FLAG_KEEP_STATES (tensor-core path; ignored by the CUDA-core path): set on BOTH the
@@ -195,6 +199,20 @@ int psk_decode_step(const psk_shape* shape, const void* q, const void* k, const 
  * used `workspace` abandoned a bounded wait, PSK_ERR_CUDA if the stream is in error,
  * else PSK_OK.  Never traps. */
 int psk_check(const void* workspace, void* stream);
+
+/* Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait inside the
+ * tensor-core kernels (on a TMA load, an MMA, another warp) is bounded by wall time: a wait that
+ * is not satisfied within about one second records a code in the workspace's status word and
+ * returns, after which the rest of that thread block runs through without waiting again, so a lost
+ * signal costs about a second and can never hang the GPU.  This call exercises exactly that path:
+ * it enqueues one small kernel whose 128 threads wait, through the same code with the limit
+ * `limit_ns` (1 .. 100 000 000), on a barrier that nobody completes.  Afterwards
+ * psk_check(workspace, stream) returns PSK_ERR_TIMEOUT, and four uint64 values at byte offset 64
+ * of the workspace (DEVICE) report: nanoseconds the first wait took, nanoseconds a second wait on
+ * the same barrier took (it must return at once), and the number of threads whose first / second
+ * wait reported failure (128 each).  The next regular call on the workspace clears the status
+ * word.  `workspace`: DEVICE, at least 256 bytes, 256-byte aligned. */
+int psk_selftest_wait_timeout(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* stream);
 
 /* Number of kernel launches the last forward / backward call on this thread enqueued
  * (for launch accounting in benchmarks). */

@@ -25,14 +25,15 @@ class Shape(Structure):
     _fields_ = [("B", c_int32), ("H", c_int32), ("n", c_int32), ("h", c_int32), ("r", c_int32),
                 ("p", c_int32), ("b", c_int32), ("dtype", c_int32),
                 ("stride_b", c_int64), ("stride_h", c_int64), ("stride_n", c_int64),
-                ("g_heads", c_int32), ("path", c_int32), ("flags", c_int32)]
+                ("g_heads", c_int32), ("path", c_int32), ("flags", c_int32), ("seq_segments", c_int32)]
 
 
 _lib = None
 
 
 def library_path() -> str:
-    return os.path.join(_PKG, "libpsk.so")
+    """libpsk.so beside this file, or the library the environment variable PSK_LIBRARY names."""
+    return os.environ.get("PSK_LIBRARY") or os.path.join(_PKG, "libpsk.so")
 
 
 def lib():
@@ -62,6 +63,8 @@ def lib():
     L.psk_causal_attn_fwd_static.argtypes = [P] + [c_void_p] * 8
     L.psk_check.restype = c_int
     L.psk_check.argtypes = [c_void_p, c_void_p]
+    L.psk_selftest_wait_timeout.restype = c_int
+    L.psk_selftest_wait_timeout.argtypes = [c_void_p, c_size_t, ctypes.c_uint64, c_void_p]
     L.psk_last_launch_count.restype = c_int
     L.psk_lt_multiply_workspace_bytes.restype = c_size_t
     L.psk_lt_multiply_workspace_bytes.argtypes = [c_int] * 5
@@ -109,7 +112,7 @@ def _stream():
 
 
 def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, path: int = PATH_AUTO,
-               flags: int = 0) -> Shape:
+               flags: int = 0, seq_segments: int = 0) -> Shape:
     """Shape descriptor for a [B,H,n,h] tensor `x` (its strides are used for all eight tensors)."""
     if x.dim() != 4 or x.stride(3) != 1:
         raise ValueError("expected a [B,H,n,h] tensor with a contiguous last dimension")
@@ -117,7 +120,8 @@ def make_shape(x: torch.Tensor, G1: torch.Tensor, r: int, b: int, p: int = 4, pa
         raise ValueError("unsupported storage dtype %s" % x.dtype)
     B, H, n, h = x.shape
     g_heads = G1.shape[0] if (G1 is not None and G1.dim() == 3) else 1
-    return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path, flags)
+    return Shape(B, H, n, h, r, p, b, _DTYPES[x.dtype], x.stride(0), x.stride(1), x.stride(2), g_heads, path, flags,
+                 seq_segments)
 
 
 def workspace_bytes(shape: Shape, for_backward: bool) -> int:
@@ -161,11 +165,12 @@ def sketch(X, G1, G2, r=None, b=128, want_phi=False, path=PATH_AUTO):
     return M, Phi
 
 
-def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out=None, denom=None, flags=0):
+def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out=None, denom=None, flags=0,
+                    seq_segments=0):
     """psk_causal_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, G1, G2)
     _same_layout(Q, K, V, out)
-    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags)
+    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags, seq_segments)
     O = _empty_like(Q) if out is None else out
     B, H, n, _ = Q.shape
     if denom is None:
@@ -201,11 +206,12 @@ def causal_attn_fwd_static(Q, K, V, G1, G2, b, p=4, out=None, denom=None):
     return O, denom
 
 
-def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, workspace=None, out=None, flags=0):
+def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, workspace=None, out=None, flags=0,
+                    seq_segments=0):
     """psk_causal_attn_bwd: returns (dQ, dK, dV)."""
     _require_cuda(Q, K, V, G1, G2, O, denom, dO)
     _same_layout(Q, K, V, O, dO)
-    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags)
+    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags, seq_segments)
     dQ, dK, dV = out if out is not None else (_empty_like(Q), _empty_like(Q), _empty_like(Q))
     _same_layout(Q, dQ, dK, dV)
     ws, nbytes = _workspace(shp, True, workspace)
@@ -220,6 +226,18 @@ def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, works
 def check(workspace) -> int:
     """psk_check: synchronises the current stream and returns the device-side status."""
     return int(lib().psk_check(_ptr(workspace), _stream()))
+
+
+def selftest_wait_timeout(workspace, limit_ns: int):
+    """psk_selftest_wait_timeout: makes a bounded device-side wait run out (nothing hangs or traps).
+    Returns (ns of the first wait, ns of the second wait, threads failed first, threads failed second)
+    after synchronising; psk_check(workspace) then reports the timeout."""
+    st = lib().psk_selftest_wait_timeout(_ptr(workspace), workspace.numel(), int(limit_ns), _stream())
+    if st != 0:
+        raise PskError(st, "psk_selftest_wait_timeout")
+    torch.cuda.current_stream().synchronize()
+    rep = workspace[64:96].view(torch.int64).cpu().tolist()
+    return tuple(int(x) for x in rep)
 
 
 def last_launch_count() -> int:
@@ -292,7 +310,7 @@ def decode_step(q, k, v, G1, G2, state):
     g_heads = G1.shape[0] if G1.dim() == 3 else 1
     if not (q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and state.is_contiguous()):
         raise ValueError("decode_step expects contiguous tensors")
-    shp = Shape(B, H, 1, h, r, 4, 128, _DTYPES[q.dtype], H * h, h, h, g_heads, PATH_AUTO, 0)
+    shp = Shape(B, H, 1, h, r, 4, 128, _DTYPES[q.dtype], H * h, h, h, g_heads, PATH_AUTO, 0, 0)
     if state.numel() * 4 != int(lib().psk_decode_state_bytes(byref(shp))):
         raise ValueError("decode_step: state must be [B, H, r*r, 65] fp32")
     o = torch.empty_like(q)

@@ -61,6 +61,10 @@ int make_dims(const psk_shape* sh, Dims* d) {
     d->p = sh->p;
     // p = 2 has no sketch error: the exact same-block weights are what it computes anyway
     d->local = (sh->flags & PSK_FLAG_LOCAL_EXACT) != 0 && sh->p == 4;
+    d->noncausal = false;
+    if (sh->seq_segments < 0) return PSK_ERR_INVALID_ARG;
+    if (sh->seq_segments > 1 && d->t % sh->seq_segments != 0) return PSK_ERR_SHAPE;
+    d->seq_segments = sh->seq_segments;
     return PSK_OK;
 }
 

@@ -19,6 +19,8 @@ struct Dims {
     bool bf16;                        // storage type
     bool keep_states;                 // PSK_FLAG_KEEP_STATES
     bool local;                       // PSK_FLAG_LOCAL_EXACT
+    bool noncausal;                   // PSK_FLAG_NONCAUSAL: no lt(), one global state per head
+    int seq_segments;                 // runs a head's sequence is cut into for the state scan; 0 = library's choice
     int BH() const { return B * H; }
 };
 

@@ -70,338 +70,6 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk) {
 namespace {
 
 // ---------------------------------------------------------------------------
-// Prefix states of one head, sequentially along the sequence (Section 3.1, Z_l = sum_{j<l} H_j):
-//   S[l] = sum over blocks before l (after l when `reverse`) of phi(X_blk)^T [Y_blk | y65]
-// for feature tiles [T0, T0+TN).  The running sum never leaves tensor memory (fp32); at every
-// block boundary it is rounded to bf16 and written out, then the block's own contribution is
-// accumulated on top -- the per-block states H_l and the scan over them are fused away.
-//   X: tensor that is sketched (K for the forward state, Q for the backward's reverse state)
-//   Y: [V] or [dO];  y65: last column (nullptr = all ones);  fscale: per-token d_i, the
-//   features of token i are divided by it (nullptr = not) -- phi(q_i)^T [dO_i | y65_i] / d_i is the
-//   suffix state's phi(q_i)^T E_i without E ever being formed
-// grid (BH).  Warp roles:
-//   NWG generator warpgroups  thread = token: read the half sketches, write their feature tiles
-//                             (dealt round-robin) as MN-major A operands into shared memory;
-//   1 store warpgroup         thread = feature row: at block boundaries reads the accumulators,
-//                             centres, rounds and stores them;
-//   1 feeder warp             one thread issues every TMA load, sketch GEMM and state GEMM.
-// Stored layout S[blk][FP][80]: one row per feature, 64 state columns, the last column, zeros.
-// ---------------------------------------------------------------------------
-template <int R, int NWG>
-struct StateSmem {
-    static constexpr uint32_t X = 0;                     // 2 x 16 KB: rows to sketch
-    static constexpr uint32_t Y = 32768;                 // 2 x (16 KB values + 16 KB last-column chunk)
-    static constexpr uint32_t kYSlot = 32768;
-    static constexpr uint32_t G = Y + 2 * kYSlot;
-    static constexpr uint32_t A0 = G + (2 * R * 128 < 1024 ? 1024 : 2 * R * 128);
-    static constexpr uint32_t St = A0 + NWG * 32768;     // one state tile on its way out: 128 rows x 160 B
-    static constexpr bool kStaged = St + 128 * 160 + 2048 <= 232448;     // where it fits (r <= 32)
-    static constexpr uint32_t total = St + (kStaged ? 128 * 160 : 0);
-};
-
-__device__ __forceinline__ void wg_barrier(int wg) {
-    asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
-}
-
-constexpr int kErrState = 3;
-
-template <int R, int T0, int TN, int NWG>
-__global__ void __launch_bounds__(128 * (NWG + 1) + 64)
-tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
-                const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
-                const float* __restrict__ y65, const float* __restrict__ fscale, const float* __restrict__ cmean,
-                int center_mode, int reverse, bf16* __restrict__ S, int* status) {
-    using F = Feat<R>;
-    using L = StateSmem<R, NWG>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = align1024(smem_raw);
-    __shared__ uint64_t bar_fullx[2], bar_fully[2], bar_yfree[2], bar_ext[2], bar_sk, bar_mread, bar_drain[2];
-    __shared__ uint64_t bar_aready[NWG], bar_afree[NWG], bar_accfull[TN], bar_accread[TN];
-    __shared__ uint32_t tmem_slot;
-    __shared__ __align__(16) float cm[64];
-    const int tid = threadIdx.x, wg = tid / 128, wt = tid % 128, warp = tid / 32;
-    const int bh = blockIdx.x;
-    const int hi = bh % H, bi = bh / H;
-    const int g = g_heads == 1 ? 0 : hi;
-    const int tpb = b / 128, NJ = n / 128;               // token tiles per block / per head
-    constexpr int kThreads = 128 * (NWG + 1) + 64;
-
-    if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&bar_fullx[i], 1); mbar_init(&bar_fully[i], 1); mbar_init(&bar_yfree[i], 1);
-            mbar_init(&bar_ext[i], 1);
-        }
-        mbar_init(&bar_sk, 1); mbar_init(&bar_mread, NWG); mbar_init(&bar_drain[0], 1); mbar_init(&bar_drain[1], 1);
-        for (int i = 0; i < NWG; ++i) { mbar_init(&bar_aready[i], 1); mbar_init(&bar_afree[i], 1); }
-        for (int i = 0; i < TN; ++i) { mbar_init(&bar_accread[i], 4); mbar_init(&bar_accfull[i], 1); }
-        mbar_fence_init();
-        tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapY);
-    }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
-    if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
-    // last-column chunks of both slots: zero, and column 0 = 1 when the last column is all ones
-    for (int e = tid; e < 2 * 1024; e += kThreads) {
-        const int s = e / 1024, i = e % 1024;
-        reinterpret_cast<uint4*>(smem + L::Y + s * L::kYSlot + 16384)[i] = make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
-    if (y65 == nullptr && tid < 128) {
-        *reinterpret_cast<bf16*>(smem + L::Y + 16384 + swz128_offset(tid, 0)) = __float2bfloat16_rn(1.f);
-        *reinterpret_cast<bf16*>(smem + L::Y + L::kYSlot + 16384 + swz128_offset(tid, 0)) = __float2bfloat16_rn(1.f);
-    }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tm = tmem_slot;
-    constexpr uint32_t kAcc = 2 * R;                      // accumulators start after the sketch columns
-    auto tile_of = [&](int j) { return reverse ? (NJ - 1 - j) : j; };
-
-    if (wg == NWG + 1) {
-        // =============================== feeders ===============================
-        // Two issuing threads in two warps.  The first loads the tiles and issues the sketch
-        // GEMMs, the second issues the state GEMMs: between two of its MMAs lies as little as
-        // possible (each satisfied wait, commit or TMA issue costs a single thread about a
-        // hundred cycles, during which the tensor pipe would idle).
-        if (tid == 128 * (NWG + 1)) {
-            bool ok = true;
-            auto load_x = [&](int j) {
-                // the first tile's barrier also covers the sketch matrices' image
-                mbar_expect_tx(&bar_fullx[j & 1], 16384 + (j == 0 ? GImage<R>::bytes : 0u));
-                if (j == 0) bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_fullx[0]);
-                tma_load_4d(smem + L::X + (j & 1) * 16384, &mapX, 0, tile_of(j) * 128, hi, bi, &bar_fullx[j & 1]);
-            };
-            auto load_y = [&](int j) {
-                mbar_expect_tx(&bar_fully[j & 1], 16384);
-                tma_load_4d(smem + L::Y + (j & 1) * L::kYSlot, &mapY, 0, tile_of(j) * 128, hi, bi, &bar_fully[j & 1]);
-            };
-            load_x(0);
-            if (NJ > 1) load_x(1);
-            load_y(0);
-            ok = mbar_wait(&bar_fullx[0], 0, status, kErrTma);
-            tc_fence_after();
-            issue_sketch<R>(tm, smem + L::X, smem + L::G);
-            umma_commit(&bar_sk);
-            for (int j = 0; j + 1 < NJ && ok; ++j) {
-                // sketch of the next token tile, as soon as this tile's half sketches are read out
-                ok = mbar_wait(&bar_mread, j & 1, status, kErrState);
-                ok = ok && mbar_wait(&bar_fullx[(j + 1) & 1], ((j + 1) >> 1) & 1, status, kErrTma);
-                tc_fence_after();
-                issue_sketch<R>(tm, smem + L::X + ((j + 1) & 1) * 16384, smem + L::G);
-                umma_commit(&bar_sk);
-                if (j + 2 < NJ) load_x(j + 2);            // its slot: sketch j has completed (it was read)
-                // values of the next token tile: their slot held tile j-1
-                if (j >= 1) ok = ok && mbar_wait(&bar_yfree[(j + 1) & 1], ((j - 1) >> 1) & 1, status, kErrState);
-                load_y(j + 1);
-            }
-            // drain: every sketch GEMM has completed before tensor memory is released.  (A barrier
-            // of its own: completing bar_sk once more, right behind the last sketch, could flip it
-            // twice before a generator thread has looked.)
-            umma_commit(&bar_drain[0]);
-            mbar_wait(&bar_drain[0], 0, status, kErrMma);
-        } else if (tid == 128 * (NWG + 1) + 32) {
-            constexpr uint32_t idesc_state = idesc_bf16(128, 80, true, true);
-            bool ok = true;
-            uint32_t a_cnt[NWG];
-#pragma unroll
-            for (int i = 0; i < NWG; ++i) a_cnt[i] = 0;
-            uint64_t ad[NWG];
-#pragma unroll
-            for (int i = 0; i < NWG; ++i) ad[i] = smem_desc(smem_u32(smem + L::A0 + i * 32768), 16384, 1024, kSwz128);
-            const uint64_t yd0 = smem_desc(smem_u32(smem + L::Y), 16384, 1024, kSwz128);
-            for (int j = 0; j < NJ && ok; ++j) {
-                ok = mbar_spin(&bar_fully[j & 1], (j >> 1) & 1, status, kErrTma);
-                if (y65 != nullptr) ok = ok && mbar_spin(&bar_ext[j & 1], (j >> 1) & 1, status, kErrState);
-                const bool boundary = (j % tpb == 0) && j > 0;
-                const uint64_t yd = desc_off(yd0, (j & 1) * L::kYSlot);
-                const uint32_t acc0 = j > 0 ? 1u : 0u;
-                static_for<0, TN>([&](auto ic) {
-                    constexpr int I = decltype(ic)::value;
-                    constexpr int w = I % NWG;
-                    // the store warpgroup has taken this accumulator's values for the boundary
-                    if (boundary) ok = ok && mbar_spin(&bar_accread[I], ((j / tpb) - 1) & 1, status, kErrState);
-                    ok = ok && mbar_spin(&bar_aready[w], a_cnt[w] & 1, status, kErrState);
-                    ++a_cnt[w];
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        umma_ss(tm + kAcc + 80 * I, desc_off(ad[w], k * 2048), desc_off(yd, k * 2048), idesc_state, k > 0 ? 1u : acc0);
-                    umma_commit(&bar_afree[w]);
-                    // last token tile of a block: this accumulator is complete, and the store
-                    // warpgroup may take it while the remaining tiles are still being issued
-                    if ((j + 1) % tpb == 0) umma_commit(&bar_accfull[I]);
-                });
-                umma_commit(&bar_yfree[j & 1]);
-            }
-            // drain: every state GEMM has completed before tensor memory is released
-            umma_commit(&bar_drain[1]);
-            mbar_wait(&bar_drain[1], 0, status, kErrMma);
-        }
-    } else if (wg == NWG) {
-        // ============================ store warpgroup ============================
-        // Tiles leave through shared memory: a warp's 32 rows of 160 B are one contiguous 5 KB
-        // piece of the state array, which the warp writes out in ten 512-byte rows of lanes.
-        // (Rows stored by their threads directly would be 10 scattered 16-byte stores each: the L1
-        // data path, which the MMA operands and the generators' tiles also go through, is this
-        // kernel's busiest unit.)
-        const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
-        uint8_t* stage = smem + L::St;
-        bool ok = true;
-        for (int p = 0; p < t && ok; ++p) {
-            const int l = reverse ? (t - 1 - p) : p;
-            static_for<0, TN>([&](auto ic) {
-                constexpr int I = decltype(ic)::value;
-                if (p > 0) {
-                    ok = ok && mbar_wait(&bar_accfull[I], (p - 1) & 1, status, kErrMma);
-                    tc_fence_after();
-                }
-                // centred values, in fp32, without touching the operands (the mode only selects
-                // coefficients):  mode 1: sum phi (y - c)^T = H[:, :64] - H[:, 64] c^T
-                //                 mode 2: last column H[:, 64] - H[:, :64] c
-                float last = 0.f, corr = 0.f;
-                if (p > 0) {
-                    uint32_t v[16];
-                    tmem_ld16(lane_tm + kAcc + 80 * I + 64, v);
-                    tmem_ld_wait();
-                    last = __uint_as_float(v[0]);
-                }
-                const float k1 = center_mode == 1 ? -last : 0.f, k2 = center_mode == 2 ? 1.f : 0.f;
-                // the row's pair weight (tc_features.cuh) goes into the stored state; 0 on padding rows
-                const float wgt = F::weight((T0 + I) * 128 + wt);
-                // this thread's feature row: 80 bf16 = ten 16-byte pieces of the staging tile
-                if constexpr (L::kStaged) __syncwarp();       // the previous tile has been read back
-                uint4* const grow = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + wt) * 80);
-                uint4* dst = L::kStaged ? reinterpret_cast<uint4*>(stage + wt * 160) : grow;
-#pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 16) {
-                    uint32_t v[16];
-                    if (p > 0) {
-                        tmem_ld16(lane_tm + kAcc + 80 * I + c0, v);
-                        tmem_ld_wait();
-                        if (c0 == 48) {          // last read of this accumulator: hand it back
-                            tc_fence_before();
-                            if (wt % 32 == 0) mbar_arrive(&bar_accread[I]);
-                        }
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) v[q] = 0u;
-                    }
-                    uint32_t pk[8];
-                    float cv[16];
-#pragma unroll
-                    for (int q = 0; q < 16; q += 4) {
-                        const float4 c4 = *reinterpret_cast<const float4*>(&cm[c0 + q]);
-                        cv[q] = c4.x; cv[q + 1] = c4.y; cv[q + 2] = c4.z; cv[q + 3] = c4.w;
-                    }
-#pragma unroll
-                    for (int q = 0; q < 16; q += 2) {
-                        const float x0 = fmaf(k1, cv[q], __uint_as_float(v[q]));
-                        const float x1 = fmaf(k1, cv[q + 1], __uint_as_float(v[q + 1]));
-                        corr = fmaf(k2 * cv[q], x0, corr);
-                        corr = fmaf(k2 * cv[q + 1], x1, corr);
-                        pk[q / 2] = pack_bf16(x0 * wgt, x1 * wgt);
-                    }
-                    dst[c0 / 8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    dst[c0 / 8 + 1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                }
-                dst[8] = make_uint4(pack_bf16((last - corr) * wgt, 0.f), 0, 0, 0);
-                dst[9] = make_uint4(0, 0, 0, 0);
-                if constexpr (L::kStaged) {
-                    __syncwarp();
-                    const int w32 = wt & ~31, lane = wt & 31;
-                    const uint4* src = reinterpret_cast<const uint4*>(stage + w32 * 160);
-                    uint4* out = reinterpret_cast<uint4*>(S + (((size_t)bh * t + l) * F::FP + (size_t)(T0 + I) * 128 + w32) * 80);
-#pragma unroll
-                    for (int i = 0; i < 10; ++i) out[i * 32 + lane] = src[i * 32 + lane];
-                }
-            });
-        }
-    } else {
-        // ============================= generators =============================
-        const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
-        uint8_t* sA = smem + L::A0 + wg * 32768;
-        uint32_t a_uses = 0;                              // times this warpgroup's buffer has been filled
-        bool ok = true;
-        // last-column entry of this thread's token, requested one token tile ahead of its use
-        float y_next = (y65 != nullptr && wg == 0) ? y65[(size_t)bh * n + tile_of(0) * 128 + wt] : 0.f;
-        float d_next = fscale != nullptr ? fscale[(size_t)bh * n + tile_of(0) * 128 + wt] : 1.f;
-        for (int j = 0; j < NJ && ok; ++j) {
-            ok = mbar_wait(&bar_sk, j & 1, status, kErrMma);
-            tc_fence_after();
-            PackedM<R> pm;
-            CircGen<R> gen;
-            {
-                float m[R];
-                // features m_a m_b / d: both factors carry 1 / sqrt(d) (d requested a token tile ago)
-                const float sc = rsqrtf(d_next);
-                if (fscale != nullptr && j + 1 < NJ) d_next = fscale[(size_t)bh * n + tile_of(j + 1) * 128 + wt];
-                read_half_sketch<R>(lane_tm, m, sc);
-                if constexpr (F::kCirc) gen.init(m); else pack_half_sketch<R>(m, pm);
-            }
-            tc_fence_before();
-            wg_barrier(wg);
-            if (wt == 0) mbar_arrive(&bar_mread);
-            if (y65 != nullptr && wg == 0) {
-                // last-column chunk of this token tile; its slot is free once tile j-2's MMAs are done
-                if (j >= 2) ok = ok && mbar_wait(&bar_yfree[j & 1], ((j >> 1) - 1) & 1, status, kErrState);
-                const float y = y_next;
-                if (j + 1 < NJ) y_next = y65[(size_t)bh * n + tile_of(j + 1) * 128 + wt];
-                *reinterpret_cast<bf16*>(smem + L::Y + (j & 1) * L::kYSlot + 16384 + swz128_offset(wt, 0)) =
-                    __float2bfloat16_rn(y);
-                fence_proxy_async_smem();
-                wg_barrier(0);
-                if (wt == 0) mbar_arrive(&bar_ext[j & 1]);
-            }
-            if constexpr (F::kCirc) {
-                // this warpgroup's tiles wg, wg + NWG, ...: the same loop body on a rotated copy of m
-                static_assert(T0 == 0, "circulant order: one launch covers every tile");
-                constexpr int kTileSteps = 128 / (2 * R);
-                for (int i = 0; i < wg; ++i) gen.template skip<kTileSteps>();
-#pragma unroll 1
-                for (int I = wg; I < TN && ok; I += NWG) {
-                    if (a_uses > 0) ok = ok && mbar_wait(&bar_afree[wg], (a_uses - 1) & 1, status, kErrMma);
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t pk[32];
-                        gen.chunk(pk);
-#pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            *reinterpret_cast<uint4*>(sA + half * 16384 + swz128_offset(wt, c)) =
-                                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                    }
-                    fence_proxy_async_smem();
-                    wg_barrier(wg);
-                    if (wt == 0) mbar_arrive(&bar_aready[wg]);
-                    ++a_uses;
-                    gen.template skip<(NWG - 1) * kTileSteps>();
-                }
-            } else {
-                static_for<0, TN>([&](auto ic) {
-                    constexpr int I = decltype(ic)::value;
-                    if (I % NWG == wg) {
-                        if (a_uses > 0) ok = ok && mbar_wait(&bar_afree[wg], (a_uses - 1) & 1, status, kErrMma);
-                        static_for<0, 16>([&](auto cc) {
-                            constexpr int C = decltype(cc)::value;
-                            uint32_t pk[4];
-                            gen_features<R, (T0 + I) * 128 + C * 8, 4>(pm, pk);
-                            *reinterpret_cast<uint4*>(sA + (C / 8) * 16384 + swz128_offset(wt, C % 8)) =
-                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        });
-                        fence_proxy_async_smem();
-                        wg_barrier(wg);
-                        if (wt == 0) mbar_arrive(&bar_aready[wg]);
-                        ++a_uses;
-                    }
-                });
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 512);
-}
-
-// ---------------------------------------------------------------------------
 // Forward output rows (Section 3.1): for a 128-row tile of block l,
 //   N = phi_w(Q) Z_l  (tensor memory A operand x TMA-fed Z chunks, N = 80: column 64 = normaliser)
 //     + sum over key tiles of the same block  lt((M_q M_k^T)^2) [V | 1]
@@ -480,6 +148,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         mbar_init(&bar_mk, 128); mbar_init(&bar_p, 128); mbar_init(&bar_go, 128);
         for (int s = 0; s < kZStages; ++s) mbar_init(&bar_z[s], 1);
         for (int s = 0; s < kFeatBufs; ++s) { mbar_init(&bar_feat[s], 128); mbar_init(&bar_a[s], 1); }
+        cta_giveup_init();
         mbar_fence_init();
         tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV); tma_prefetch_desc(&mapZ);
         mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
@@ -871,38 +540,6 @@ tc_gimage_kernel(const bf16* __restrict__ G1, const bf16* __restrict__ G2, int r
 // host launchers
 // ---------------------------------------------------------------------------
 
-// Prefix (or suffix) states of every head.  X is sketched, Y is the right-hand side.
-template <int R, int T0, int TN, int NWG>
-cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                               const float* y65, const float* fscale, const float* cmean, int center_mode, bool reverse,
-                               bf16* S, int* status, cudaStream_t s, int* launches) {
-    constexpr size_t smem = StateSmem<R, NWG>::total + 1024;
-    PSK_TRY(set_smem(tc_state_kernel<R, T0, TN, NWG>, smem));
-    prof_begin("tc_state_kernel", s);
-    tc_state_kernel<R, T0, TN, NWG><<<d.BH(), 128 * (NWG + 1) + 64, smem, s>>>(
-        mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, y65, fscale, cmean, center_mode, reverse ? 1 : 0, S, status);
-    prof_end(s);
-    ++*launches;
-    return cudaGetLastError();
-}
-
-template <int R>
-cudaError_t launch_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                          const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
-                          int* status, cudaStream_t s, int* launches) {
-#define PSK_SG(T0, TN, NWG) \
-    PSK_TRY((launch_state_group<R, T0, TN, NWG>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, reverse, S, status, s, launches)))
-    if constexpr (R == 16) {
-        PSK_SG(0, 2, 2);
-    } else if constexpr (R == 32) {
-        PSK_SG(0, 5, 3);
-    } else {
-        PSK_SG(0, 4, 3); PSK_SG(4, 4, 3); PSK_SG(8, 3, 3); PSK_SG(11, 3, 3); PSK_SG(14, 3, 3);
-    }
-#undef PSK_SG
-    return cudaSuccess;
-}
-
 template <int R>
 cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
                      void* O, float* denom, char* ws, cudaStream_t s, int* launches) {
@@ -926,8 +563,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (cmean != nullptr) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
-    PSK_TRY((launch_states<R>(d, mK, mV, gimg, nullptr, nullptr, cmean, cmean ? 1 : 0, Z, false,
-                              status, s, launches)));
+    PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, nullptr, cmean, cmean ? 1 : 0, Z, false,
+                      reinterpret_cast<float*>(ws + w.tot), status, s, launches));
     prof_begin("tc_fwd_out_kernel", s);
     if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
@@ -1022,17 +659,6 @@ cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s,
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
-}
-
-cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
-                      const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
-                      int* status, cudaStream_t s, int* launches) {
-    switch (d.r) {
-        case 16: return launch_states<16>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
-        case 32: return launch_states<32>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
-        case 64: return launch_states<64>(d, mX, mY, gimg, y65, fscale, cmean, center_mode, S, reverse, status, s, launches);
-    }
-    return cudaErrorInvalidValue;
 }
 
 }  // namespace psk

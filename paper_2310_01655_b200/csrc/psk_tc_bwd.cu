@@ -174,6 +174,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         mbar_init(&bar_own, 1); mbar_init(&bar_xoth, 1); mbar_init(&bar_yoth, 1); mbar_init(&bar_mma, 1);
         mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
         for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
+        cta_giveup_init();
         mbar_fence_init();
         tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
         tma_prefetch_desc(&mapYoth); tma_prefetch_desc(&mapS);
@@ -737,6 +738,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     float* y65 = reinterpret_cast<float*>(ws + w.y65);
     float* cmean = reinterpret_cast<float*>(ws + w.vmean);
     float* e65h = reinterpret_cast<float*>(ws + w.e65h);
+    float* tot = reinterpret_cast<float*>(ws + w.tot);
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     CUtensorMap mQ, mK, mV, mG, mZ, mR, mdQ, mdK, mdV;
     const int64_t nblk = (int64_t)d.BH() * d.t;
@@ -750,7 +752,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
     // prefix states of centred values; forward rows again in fp32 -> y65, e65h; suffix states
-    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, nullptr, cmean, 1, Z, false, status, s, launches));
+    if (!d.keep_states) PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, nullptr, cmean, 1, Z, false, tot, status, s, launches));
     if (d.keep_states) {
         const int rows = d.BH() * d.n;
         prof_begin("tc_bwd_prep_kernel", s);
@@ -778,7 +780,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         ++*launches;
         PSK_TRY(cudaGetLastError());
         // suffix states: phi(q_i) / d_i against [dO_i | y65_i]
-        PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, status, s, launches));
+        PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, tot, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
         tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
                                                                     d.b, d.t, y65, e65h, denom, status);

@@ -18,9 +18,14 @@ bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
 // per-block states of every head + prefix (reverse = false) or suffix (reverse = true) scan
 // center_mode 0: states as they are; 1: values centred by the per-head vector cmean
 // (columns < 64 become H[:, c] - cmean[c] H[:, 64]); 2: last column becomes H[:, 64] - H[:, :64] cmean.
+// `tot`: scratch of tc_state_total_bytes(d) bytes for the segment totals (may be null when that is 0).
+// Non-causal (d.noncausal): one state per head, the sum over the whole sequence, stored as block 0.
 cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& mY, const uint8_t* gimg,
                       const float* y65, const float* fscale, const float* cmean, int center_mode, bf16* S, bool reverse,
-                      int* status, cudaStream_t s, int* launches);
+                      float* tot, int* status, cudaStream_t s, int* launches);
+// runs a head's blocks are cut into by the state kernel (1 = one CTA group walks the whole head)
+int tc_state_segments(const Dims& d);
+size_t tc_state_total_bytes(const Dims& d);
 // the backward's recomputation of the forward rows: writes y65, e65h (see tc_fwd_out_kernel)
 cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
                          const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
@@ -32,17 +37,18 @@ cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gi
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
 
 // Scratch layout of the tensor-core path.
-struct TcWorkspace { size_t status, vmean, gimg, Z, Rst, y65, e65h, Oc, total; };
+struct TcWorkspace { size_t status, vmean, gimg, tot, Z, Rst, y65, e65h, Oc, total; };
 
 template <int R>
 inline TcWorkspace tc_ws(const Dims& d, bool backward) {
     TcWorkspace w{};
-    const size_t st = (size_t)d.BH() * d.t * tc::Feat<R>::FP * 80 * sizeof(bf16);
+    const size_t st = (size_t)d.BH() * (d.noncausal ? 1 : d.t) * tc::Feat<R>::FP * 80 * sizeof(bf16);
     const size_t rows = (size_t)d.BH() * d.n;
     size_t off = 0;
     w.status = off; off += kStatusBytes;
     w.vmean = off; off += align_up((size_t)d.BH() * 64 * sizeof(float));
     w.gimg = off; off += align_up((size_t)d.g_heads * 2 * R * 128);
+    w.tot = off; off += align_up(tc_state_total_bytes(d));
     w.Z = off; off += align_up(st);
     if (backward) {
         w.Rst = off; off += align_up(st);

@@ -47,9 +47,27 @@ __device__ __forceinline__ bool mbar_try_wait_addr(uint32_t bar_addr, uint32_t p
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return mbar_try_wait_addr(smem_u32(bar), parity);
 }
-// Bounded wait: gives up after kSpinLimit polls, records `code` in *status (global) and
-// returns false; the caller then leaves its loop, so a lost signal cannot hang the GPU.
-constexpr uint32_t kSpinLimit = 1u << 20;
+// Bounded waits.  A wait that is not satisfied at once goes to an out-of-line loop that gives up
+// when kWaitLimitNs of wall time (%globaltimer) have passed.  The loser records `code` in *status
+// (global), raises the CTA's give-up flag (shared memory) and returns false.  From then on every
+// wait of that CTA that is not satisfied at once returns false without waiting, so the CTA runs
+// through the rest of its work at full speed: the first lost signal costs one limit, nothing after
+// it costs anything.  Kernels therefore never have to leave a loop early because a wait failed --
+// which matters wherever a loop contains a barrier that counts its participants.
+// Every kernel that waits calls cta_giveup_init() from one thread before its first block-wide
+// barrier, and may read cta_gave_up() after its last one to skip its global stores.
+constexpr uint64_t kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ volatile int* cta_giveup_flag() {
+    __shared__ int flag;
+    return &flag;
+}
+__device__ __forceinline__ void cta_giveup_init() { *cta_giveup_flag() = 0; }
+__device__ __forceinline__ bool cta_gave_up() { return *cta_giveup_flag() != 0; }
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -61,39 +79,67 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// The bounded spin is one out-of-line copy: waits are everywhere in straight-line kernel code, and
-// instruction fetch is what those kernels run out of first.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, int* status, int code) {
-#pragma unroll 1
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait_addr(bar_addr, parity)) return true;
-    }
+__device__ __forceinline__ bool wait_failed(int* status, int code) {
+    *cta_giveup_flag() = 1;
     if (status != nullptr) atomicCAS(status, 0, code);
     return false;
+}
+// The bounded loop is one out-of-line copy: waits are everywhere in straight-line kernel code, and
+// instruction fetch is what those kernels run out of first.  Nothing precedes the first poll
+// (nearly every wait ends inside it, and whatever came before it would delay the waiter's
+// wake-up); the flag is read after a poll that came back without the barrier, the clock every
+// 1024 such polls.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, int* status, int code,
+                                                   uint64_t limit_ns) {
+    uint64_t t0 = 0;
+#pragma unroll 1
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 1024; ++i) {
+            if (mbar_try_wait_addr(bar_addr, parity)) return true;
+            if (cta_gave_up()) return false;
+        }
+        const uint64_t now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > limit_ns) break;
+    }
+    return wait_failed(status, code);
 }
 // Bounded wait by polling only (no suspension): for a lone issuing thread, whose wake-up latency
 // is on the critical path of everything it feeds and whose polling costs no one else issue slots.
-static __device__ __noinline__ bool mbar_spin_slow(uint32_t bar_addr, uint32_t parity, int* status, int code) {
+// Flag every 64 polls, clock every 4096.
+static __device__ __noinline__ bool mbar_spin_slow(uint32_t bar_addr, uint32_t parity, int* status, int code,
+                                                   uint64_t limit_ns) {
+    uint64_t t0 = 0;
 #pragma unroll 1
-    for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.b32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
-        if (ok) return true;
+    for (;;) {
+#pragma unroll 1
+        for (int g = 0; g < 64; ++g) {
+#pragma unroll 1
+            for (int i = 0; i < 64; ++i) {
+                uint32_t ok;
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\t"
+                    "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                    "selp.b32 %0, 1, 0, p;\n\t}"
+                    : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
+                if (ok) return true;
+            }
+            if (cta_gave_up()) return false;
+        }
+        const uint64_t now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > limit_ns) break;
     }
-    if (status != nullptr) atomicCAS(status, 0, code);
-    return false;
+    return wait_failed(status, code);
 }
 __device__ __forceinline__ bool mbar_spin(uint64_t* bar, uint32_t parity, int* status, int code) {
     if (mbar_test(bar, parity)) return true;
-    return mbar_spin_slow(smem_u32(bar), parity, status, code);
+    return mbar_spin_slow(smem_u32(bar), parity, status, code, kWaitLimitNs);
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code) {
     if (mbar_test(bar, parity)) return true;       // already complete: no suspension round trip
-    return mbar_wait_slow(smem_u32(bar), parity, status, code);
+    return mbar_wait_slow(smem_u32(bar), parity, status, code, kWaitLimitNs);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {

@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(L):
 
 
 def good():
-    return Shape(1, 2, 512, 64, 32, 4, 256, 1, 2 * 512 * 64, 512 * 64, 64, 2, 0, 0)
+    return Shape(1, 2, 512, 64, 32, 4, 256, 1, 2 * 512 * 64, 512 * 64, 64, 2, 0, 0, 0)
 
 
 def test_status_strings(L):
