@@ -29,7 +29,10 @@ block algorithm against the masked definition, finite differences; for
 degree 2 (no sketch): looped (q.k)^2 attention, finite differences; for degree 8:
 the recursion written out, Monte-Carlo mean (q.k)^4 of the half sketch, exact
 features, block algorithm against the definition, finite differences.
-No function here is "parity unpinned".
+the non-causal form of Section 3: looped (q.k)^4 attention over all keys, invariance
+under a joint permutation of keys and values, last row of the causal form, linear-time
+evaluation against the definition, finite differences.
+Every function in this file has at least one such pin.
 """
 from __future__ import annotations
 
@@ -446,6 +449,80 @@ def causal_polysketch8_attention_backward(Q, K, V, gaussians, dO):
     ds = 2.0 * s * dW
     return (_sketch_degree4_backward(Q, gaussians, ds @ Mk), _sketch_degree4_backward(K, gaussians, ds.T @ Mq),
             W.T @ E[:, :h])
+
+
+# ---------------------------------------------------------------------------
+# Section 3, first formula: Polysketch attention WITHOUT the causal mask,
+#   D~^{-1} phi'(Q) phi'(K)^T V,   D~ = diag(1 + phi'(Q) phi'(K)^T 1),
+# which the paper evaluates in time linear in n by forming phi'(K)^T V first.
+# ---------------------------------------------------------------------------
+def attention_from_features(PhiQ, PhiK, V):
+    """The definition: all n x n weights <phi'(q_i), phi'(k_j)>, no mask.  Returns (O, d)."""
+    W = _f64(PhiQ) @ _f64(PhiK).T
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
+def polysketch_attention(Q, K, V, G1, G2):
+    """Non-causal Polysketch attention from the definition (features materialised)."""
+    return attention_from_features(polysketch_non_negative(Q, G1, G2), polysketch_non_negative(K, G1, G2), V)
+
+
+def polysketch_attention_linear(Q, K, V, G1, G2):
+    """The same in time linear in n (Section 3): one state S = phi'(K)^T [V | 1] per head, then
+    every row is phi'(q_i)^T S; its last entry is the normaliser's sum."""
+    V = _f64(V)
+    n, h = V.shape
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    S = polysketch_non_negative(K, G1, G2).T @ Vt
+    N = polysketch_non_negative(Q, G1, G2) @ S
+    d = 1.0 + N[:, h]
+    return N[:, :h] / d[:, None], d
+
+
+def polysketch_attention_backward(Q, K, V, G1, G2, dO):
+    """Gradients (dQ, dK, dV) of sum(dO * O) for the non-causal form, through the n x n
+    definition: W_ij = s_ij^2 for every pair, dL/dW_ij = E_i . V~_j (derivation above)."""
+    V = _f64(V)
+    n, h = V.shape
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    s = Mq @ Mk.T
+    W = s * s
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = E @ Vt.T
+    dV = W.T @ E[:, :h]
+    ds = 2.0 * s * dW
+    return (_sketch_backward(Q, G1, G2, ds @ Mk), _sketch_backward(K, G1, G2, ds.T @ Mq), dV)
+
+
+def polysketch_attention_backward_linear(Q, K, V, G1, G2, dO):
+    """The same gradients in time linear in n: with S = phi'(K)^T V~ and R = phi'(Q)^T E,
+    d phi'(q_i) = S E_i,  d phi'(k_j) = R V~_j,  dV~_j = R^T phi'(k_j), and
+    dm = (mat(d phi') + mat(d phi')^T) m  because phi'(m)[a*r+b] = m_a m_b."""
+    V = _f64(V)
+    n, h = V.shape
+    r = _f64(G1).shape[1]
+    Mq, Mk = half_sketch(Q, G1, G2), half_sketch(K, G1, G2)
+    Pq, Pk = self_tensor(Mq), self_tensor(Mk)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    S = Pk.T @ Vt
+    N = Pq @ S
+    d = 1.0 + N[:, h]
+    O = N[:, :h] / d[:, None]
+    E = _backward_rows(O, d, dO)
+    R = Pq.T @ E
+    dPq = E @ S.T
+    dPk = Vt @ R.T
+    dV = (Pk @ R)[:, :h]
+
+    def untensor(dP, M):
+        D = dP.reshape(n, r, r)
+        return np.einsum("nab,nb->na", D + D.transpose(0, 2, 1), M)
+
+    return (_sketch_backward(Q, G1, G2, untensor(dPq, Mq)), _sketch_backward(K, G1, G2, untensor(dPk, Mk)), dV)
 
 
 # ---------------------------------------------------------------------------
