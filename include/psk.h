@@ -103,8 +103,17 @@ typedef struct {
  * backward sends the same-block part of dQ, dK straight to Q and K instead of through the
  * sketch.  Both paths serve it (bf16 storage: tensor-core kernels, scores from the raw bf16
  * rows with fp32 accumulation; fp32 storage: CUDA-core kernels), and it combines with
- * PSK_FLAG_KEEP_STATES. */
-typedef enum { PSK_FLAG_KEEP_STATES = 1, PSK_FLAG_LOCAL_EXACT = 2 } psk_flags;
+ * PSK_FLAG_KEEP_STATES.
+ *
+ * PSK_FLAG_NONCAUSAL: Polysketch attention without the causal mask (Section 3, first formula):
+ *   O = D~^{-1} phi'(Q) phi'(K)^T V,   D~ = diag(1 + phi'(Q) phi'(K)^T 1),
+ * evaluated in time linear in n through ONE state phi'(K)^T [V | 1] per head (the sum over the whole
+ * sequence) instead of per-block prefix sums; the backward uses that state and the single state
+ * phi'(Q)^T E.  b still sets the launch granularity (a multiple of 128 dividing n) but no longer
+ * changes the result.  Set it on the forward and on the backward call alike.  Tensor-core path only
+ * (bf16 storage, p = 4), not with PSK_FLAG_LOCAL_EXACT: otherwise PSK_ERR_UNSUPPORTED.  Combines
+ * with PSK_FLAG_KEEP_STATES. */
+typedef enum { PSK_FLAG_KEEP_STATES = 1, PSK_FLAG_LOCAL_EXACT = 2, PSK_FLAG_NONCAUSAL = 4 } psk_flags;
 
 /* Library version (major*100 + minor). */
 int psk_version(void);

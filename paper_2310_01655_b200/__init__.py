@@ -11,11 +11,11 @@ from .binding import (PskError, Shape, lib, library_path, sketch, lt_multiply, d
                       workspace_bytes, check, last_launch_count, status_string,
                       profile_enable, profile_records,
                       PATH_AUTO, PATH_CUDA_CORES, PATH_TENSOR_CORES, FLAG_KEEP_STATES,
-                      FLAG_LOCAL_EXACT)
+                      FLAG_LOCAL_EXACT, FLAG_NONCAUSAL)
 
 __all__ = ["PskError", "Shape", "lib", "library_path", "sketch", "lt_multiply", "decode_state", "decode_step", "causal_attn_fwd", "causal_attn_bwd", "causal_attn_fwd_static",
            "static_scratch_bytes",
            "workspace_bytes", "check", "last_launch_count", "status_string",
            "profile_enable", "profile_records",
            "PATH_AUTO", "PATH_CUDA_CORES", "PATH_TENSOR_CORES", "FLAG_KEEP_STATES",
-           "FLAG_LOCAL_EXACT"]
+           "FLAG_LOCAL_EXACT", "FLAG_NONCAUSAL"]

@@ -10,6 +10,7 @@ import torch
 PATH_AUTO, PATH_CUDA_CORES, PATH_TENSOR_CORES = 0, 1, 2
 FLAG_KEEP_STATES = 1
 FLAG_LOCAL_EXACT = 2
+FLAG_NONCAUSAL = 4
 _DTYPES = {torch.float32: 0, torch.bfloat16: 1}
 _PKG = os.path.dirname(os.path.abspath(__file__))
 

@@ -38,7 +38,7 @@ int make_dims(const psk_shape* sh, Dims* d) {
     if (sh == nullptr) return PSK_ERR_INVALID_ARG;
     if (sh->dtype != PSK_F32 && sh->dtype != PSK_BF16) return PSK_ERR_INVALID_ARG;
     if (sh->path < PSK_PATH_AUTO || sh->path > PSK_PATH_TENSOR_CORES) return PSK_ERR_INVALID_ARG;
-    if (sh->flags & ~(int32_t)(PSK_FLAG_KEEP_STATES | PSK_FLAG_LOCAL_EXACT)) return PSK_ERR_INVALID_ARG;
+    if (sh->flags & ~(int32_t)(PSK_FLAG_KEEP_STATES | PSK_FLAG_LOCAL_EXACT | PSK_FLAG_NONCAUSAL)) return PSK_ERR_INVALID_ARG;
     if (sh->B <= 0 || sh->H <= 0 || sh->n <= 0 || sh->b <= 0) return PSK_ERR_SHAPE;
     if ((sh->p != 4 && sh->p != 2 && sh->p != 8) || sh->h != 64) return PSK_ERR_UNSUPPORTED;
     // exact same-block weights are built for degree 4 (and are what degree 2 computes anyway)
@@ -61,9 +61,14 @@ int make_dims(const psk_shape* sh, Dims* d) {
     d->p = sh->p;
     // p = 2 has no sketch error: the exact same-block weights are what it computes anyway
     d->local = (sh->flags & PSK_FLAG_LOCAL_EXACT) != 0 && sh->p == 4;
-    d->noncausal = false;
+    d->noncausal = (sh->flags & PSK_FLAG_NONCAUSAL) != 0;
+    // without the mask there are no blocks to treat exactly, and only the degree-4 tensor-core kernels serve it
+    if (d->noncausal && ((sh->flags & PSK_FLAG_LOCAL_EXACT) || sh->p != 4 || sh->dtype != PSK_BF16 ||
+                         sh->path == PSK_PATH_CUDA_CORES))
+        return PSK_ERR_UNSUPPORTED;
     if (sh->seq_segments < 0) return PSK_ERR_INVALID_ARG;
-    if (sh->seq_segments > 1 && d->t % sh->seq_segments != 0) return PSK_ERR_SHAPE;
+    // runs start at block boundaries (at 128-row tiles when there is no mask and hence no block)
+    if (sh->seq_segments > 1 && (d->noncausal ? sh->n / 128 : d->t) % sh->seq_segments != 0) return PSK_ERR_SHAPE;
     d->seq_segments = sh->seq_segments;
     return PSK_OK;
 }

@@ -128,7 +128,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                   const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                   const float* __restrict__ cmean, int64_t sb, int64_t sh, int64_t sn,
                   float* __restrict__ denom, const bf16* __restrict__ dO,
-                  float* __restrict__ y65, float* __restrict__ e65h, int keep_oc, int* status) {
+                  float* __restrict__ y65, float* __restrict__ e65h, int keep_oc, int noncausal, int* status) {
     using F = Feat<R>;
     using L = OutSmem<R, LOCAL>;
     extern __shared__ uint8_t smem_raw[];
@@ -141,7 +141,10 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
     const int row0 = l * b + tau * 128;
-    const int blk = bh * t + l;
+    // Non-causal (Section 3, first formula): one state per head, the sum over the whole sequence,
+    // multiplies every row tile, and there are no same-block tiles.
+    const int blk = noncausal ? bh : bh * t + l;
+    const bool has_prefix = noncausal || l > 0;
 
     if (tid == 0) {
         mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_sk, 1); mbar_init(&bar_s, 1); mbar_init(&bar_pv, 1);
@@ -154,7 +157,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
         tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
         bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
-        if (l > 0) {
+        if (has_prefix) {
             for (int c = 0; c < kZStages - 1 && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_z[c], kZStageBytes);
                 tma_load_3d(smem + L::zstage(c), &mapZ, 0, c * 64, blk, &bar_z[c]);
@@ -184,14 +187,14 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tc_fence_after();
             issue_sketch<R>(tm + cSk, smem + L::Q, smem + L::G);
             umma_commit(&bar_sk);
-            if (l > 0 && kZStages - 1 < F::NC) {
+            if (has_prefix && kZStages - 1 < F::NC) {
                 // the query tile has been consumed: its buffer becomes the ring's last stage
                 ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);
                 mbar_expect_tx(&bar_z[kZStages - 1], kZStageBytes);
                 tma_load_3d(smem + L::zstage(kZStages - 1), &mapZ, 0, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
                 tma_load_3d(smem + L::zstage(kZStages - 1) + 8192, &mapZ, 64, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
             }
-            if (l > 0) {
+            if (has_prefix) {
                 // earlier blocks: weighted features (tensor memory) x prefix state chunks.
                 // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step,
                 // the second 64-column group (columns 64..79) 8192 B further on
@@ -216,6 +219,8 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         if (k < ksteps) umma_ts(tm + cO, at + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
                     umma_commit(&bar_a[s]);
                 }
+            }
+            if (has_prefix && !noncausal) {
                 // first key/value tile of the same block, each into its stage as soon as the last
                 // chunk that used it has been multiplied
                 constexpr int cK = L::last_chunk(F::NC, L::kStageK), cV = L::last_chunk(F::NC, L::kStageV);
@@ -238,8 +243,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             // every row has read the query sketch (the first key sketch overwrites its columns, and
             // bar_sk must not complete a second time before its slowest waiter has seen the first)
             ok = ok && mbar_spin(&bar_go, 0, status, kErrMma);
+            const int tp_last = noncausal ? -1 : tau;
 #pragma unroll 1
-            for (int tp = 0; tp <= tau && ok; ++tp) {
+            for (int tp = 0; tp <= tp_last && ok; ++tp) {
                 if (tp > 0) ok = mbar_spin(&bar_pv, (tp - 1) & 1, status, kErrMma);   // K, V, Mk, weights are free
                 if (tp > 0 || l == 0) {       // (block l > 0: the first tile was requested above)
                     mbar_expect_tx(&bar_kv, 32768);
@@ -295,7 +301,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         tc_fence_before();
         mbar_arrive(&bar_go);
 
-        if (l > 0) {
+        if (has_prefix) {
             if constexpr (F::kCirc) {
                 CircGen<R> gen;
                 gen.init(mq);
@@ -345,8 +351,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
         }
 
+        const int tp_last = noncausal ? -1 : tau;
 #pragma unroll 1
-        for (int tp = 0; tp <= tau && ok; ++tp) {
+        for (int tp = 0; tp <= tp_last && ok; ++tp) {
             if constexpr (!LOCAL) {
                 ok = mbar_wait(&bar_sk, (tp + 1) & 1, status, kErrMma);
                 tc_fence_after();
@@ -389,7 +396,10 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tc_fence_before();
             mbar_arrive(&bar_p);
         }
-        ok = ok && mbar_wait(&bar_pv, tau & 1, status, kErrMma);
+        if (noncausal)      // the last chunk's MMAs (no same-block tiles follow them)
+            ok = ok && mbar_wait(&bar_a[(F::NC - 1) % kFeatBufs], ((F::NC - 1) / kFeatBufs) & 1, status, kErrMma);
+        else
+            ok = ok && mbar_wait(&bar_pv, tau & 1, status, kErrMma);
         tc_fence_after();
 
         // ---- epilogue ----
@@ -402,17 +412,19 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 32; ++j) acc[c0 + j] = __uint_as_float(v[j]);
         }
-        float noff = 0.f, rowsum;             // normaliser parts: earlier blocks, same block
+        float noff = 0.f, rowsum = 0.f;       // normaliser parts: earlier blocks, same block
         {
             uint32_t v[16];
-            if (l > 0) {
+            if (has_prefix) {
                 tmem_ld16(lane_tm + cO + 64, v);
                 tmem_ld_wait();
                 noff = __uint_as_float(v[0]);
             }
-            tmem_ld16(lane_tm + cN, v);
-            tmem_ld_wait();
-            rowsum = __uint_as_float(v[0]);
+            if (!noncausal) {
+                tmem_ld16(lane_tm + cN, v);
+                tmem_ld_wait();
+                rowsum = __uint_as_float(v[0]);
+            }
         }
         if constexpr (MODE == 0) {
             const float d = 1.f + rowsum + noff;
@@ -549,7 +561,8 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     bf16* Oc = d.keep_states ? reinterpret_cast<bf16*>(ws + w.Oc) : nullptr;
     CUtensorMap mQ, mK, mV, mZ, mO, mOc;
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
-        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * d.t) ||
+        !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * (d.noncausal ? 1 : d.t)) ||
         !tc_map_rows(&mO, O, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
     if (Oc != nullptr) {
@@ -571,13 +584,13 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true>, smem)));
         tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false>, smem)));
         tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, status);
+            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     }
     prof_end(s);
     ++*launches;
@@ -621,13 +634,13 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true>, smem)));
         tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            const_cast<float*>(denom), dO, y65, e65h, 0, status);
+            const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false>, smem)));
         tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
-            const_cast<float*>(denom), dO, y65, e65h, 0, status);
+            const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     }
     prof_end(s);
     ++*launches;

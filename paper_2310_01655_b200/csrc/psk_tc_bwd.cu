@@ -154,7 +154,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    const __grid_constant__ CUtensorMap mapDV, const uint8_t* __restrict__ gimg,
                    int g_heads, int H, int n, int b, int t,
                    const float* __restrict__ y65g, const float* __restrict__ e65h, const float* __restrict__ denom,
-                   int* status) {
+                   int noncausal, int* status) {
     using F = Feat<R>;
     using L = BwdSmem<R, LOCAL, QSIDE>;
     constexpr int kStages = L::kSt;
@@ -166,9 +166,10 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
     const int row0 = l * b + tau * 128;
-    const int blk = bh * t + l;
+    // Non-causal: every row tile meets the head's single global state and no same-block tiles.
+    const int blk = noncausal ? bh : bh * t + l;
     const int ntiles = b / 128;
-    const bool has_state = QSIDE ? (l > 0) : (l < t - 1);
+    const bool has_state = noncausal || (QSIDE ? (l > 0) : (l < t - 1));
 
     if (tid == 0) {
         mbar_init(&bar_own, 1); mbar_init(&bar_xoth, 1); mbar_init(&bar_yoth, 1); mbar_init(&bar_mma, 1);
@@ -191,11 +192,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         }
         // first other-side tile: at once where its memory is free from the start
         const int orow_first = l * b + (QSIDE ? 0 : tau) * 128;
-        if (!has_state || !L::kAlias || F::NC < kStages) {
+        if (!noncausal && (!has_state || !L::kAlias || F::NC < kStages)) {
             mbar_expect_tx(&bar_xoth, 16384);
             tma_load_4d(smem + L::Xoth, &mapXoth, 0, orow_first, hi, bi, &bar_xoth);
         }
-        if (!has_state || !L::kAlias) {
+        if (!noncausal && (!has_state || !L::kAlias)) {
             mbar_expect_tx(&bar_yoth, 16384);
             tma_load_4d(smem + L::Yoth, &mapYoth, 0, orow_first, hi, bi, &bar_yoth);
         }
@@ -318,7 +319,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 mbar_expect_tx(&bar_box[stage], kBoxBytes);
                 tma_load_3d(smem + L::Box + stage * kBoxStride, &mapS, 0, (C + kStages) * 64, blk, &bar_box[stage]);
                 tma_load_3d(smem + L::Box + stage * kBoxStride + 8192, &mapS, 64, (C + kStages) * 64, blk, &bar_box[stage]);
-            } else if (L::kAlias) {
+            } else if (L::kAlias && !noncausal) {
                 // the last chunks free the stages that the first other-side tile goes into
                 const int orow_first = l * b + (QSIDE ? 0 : tau) * 128;
                 if (F::NC >= kStages && C == F::NC - kStages) {
@@ -449,7 +450,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     // ---- phase C: same block, other-side tiles, 64 other rows at a time ----
     if constexpr (!LOCAL) store_hilo_tiles<R>(smem + L::Mown, m, tid);
-    const int tp_begin = QSIDE ? 0 : tau, tp_end = QSIDE ? tau + 1 : ntiles;
+    const int tp_begin = QSIDE ? 0 : tau, tp_end = noncausal ? tp_begin : (QSIDE ? tau + 1 : ntiles);
     bool dm_started = false;
     uint32_t oth_uses = 0;
     float2* oth_col = reinterpret_cast<float2*>(smem + L::Eoth);   // other rows: (1/d, -(g . O)/d)
@@ -626,8 +627,9 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 uint32_t v[16];
                 tmem_ld16(lane_tm + cdM + c0, v);
                 tmem_ld_wait();
+                // (no same-block tiles ran: nothing was accumulated there)
 #pragma unroll
-                for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + __uint_as_float(v[j])) * rs;
+                for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + (dm_started ? __uint_as_float(v[j]) : 0.f)) * rs;
             }
         }
         tc_fence_before();
@@ -741,7 +743,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     float* tot = reinterpret_cast<float*>(ws + w.tot);
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     CUtensorMap mQ, mK, mV, mG, mZ, mR, mdQ, mdK, mdV;
-    const int64_t nblk = (int64_t)d.BH() * d.t;
+    const int64_t nblk = (int64_t)d.BH() * (d.noncausal ? 1 : d.t);
     if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
@@ -775,7 +777,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // still in L2; the suffix states (5 GB through L2) come after it
         prof_begin("tc_bwd_q_kernel", s);
         tc_bwd_rows_kernel<R, true, LOCAL><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
-                                                                   d.b, d.t, y65, e65h, denom, status);
+                                                                   d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
@@ -783,7 +785,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, tot, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
         tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
-                                                                    d.b, d.t, y65, e65h, denom, status);
+                                                                    d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
         return cudaGetLastError();
