@@ -68,7 +68,9 @@ def kernel_flops_per_head_token(name, w, local=False):
         tile_fwd = 2 * 128 * h + 2 * 128 * h
         tile_bwd = 2 * 128 * h + 2 * 128 * h + 2 * 128 * 64
     table.update({
-        "tc_state_kernel": sk * (1 if r <= 32 else 5) + 2 * FP * 80,
+        # (r = 64: a state set is built by five launches that split the feature tiles between them and
+        # each redo the half sketch; the figure is the average launch)
+        "tc_state_kernel": sk + 2 * FP * 80 / (1 if r <= 32 else 5),
         "tc_fwd_out_kernel": sk + 2 * FK * 80 + other * tile_fwd,
         "tc_bwd_recompute_kernel": sk + 2 * FK * 80 + other * tile_fwd,
         "tc_bwd_q_kernel": 2 * sk + 2 * FK * 80 + other * tile_bwd + 2 * 2 * r * 64,
@@ -199,6 +201,71 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def executed_flops_per_step(w, kernels, local):
+    """Sum over the library's kernels of the MMA flops they issued in one step (None-flop kernels are
+    memory-bound helpers and add nothing)."""
+    total = 0.0
+    for name, (cnt, _ms, steps) in kernels.items():
+        key = {"tc_state_total_kernel": "tc_state_kernel"}.get(name, name)
+        fl = kernel_flops_per_head_token(key, w, local)
+        if fl:
+            total += fl * w.head_tokens * cnt / steps
+    return total
+
+
+def time_other_config(psk, wl, name, steps, warmup, local, pk, device_index):
+    """A short timed run of another benchmark configuration (same step definition as the headline):
+    ms per step, nominal and executed TFLOP/s with their fractions of the measured peaks, clocks."""
+    import torch
+    w = wl.WORKLOADS[name]
+    inp = wl.make_inputs(w, "cuda", with_dO=True)
+    Q, K, V, dO, G1, G2 = (inp[k] for k in ("Q", "K", "V", "dO", "G1", "G2"))
+    flags = (psk.FLAG_KEEP_STATES if w.backward else 0) | (psk.FLAG_LOCAL_EXACT if local else 0)
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, psk.PATH_AUTO, flags)
+    ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True) if w.backward else 0),
+                     dtype=torch.uint8, device="cuda")
+    O = torch.empty_like(Q)
+    den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
+    grads = tuple(torch.empty_like(Q) for _ in range(3)) if w.backward else None
+
+    def step():
+        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, psk.PATH_AUTO, ws, O, den, flags)
+        if w.backward:
+            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, psk.PATH_AUTO, ws, grads, flags)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    psk.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.stop()
+    agg = {}
+    for kname, t in psk.profile_records():
+        a = agg.setdefault(kname, [0, 0.0, steps])
+        a[0] += 1; a[1] += t
+    psk.profile_enable(False)
+    if psk.check(ws) != 0:
+        raise RuntimeError("device-side error while timing %s" % name)
+    f_fwd, f_bwd = nominal_flops_per_head_token(w, local)
+    nominal = (f_fwd + f_bwd) * w.head_tokens / (ms / 1e3) / 1e12
+    executed = executed_flops_per_step(w, agg, local) / (ms / 1e3) / 1e12
+    return {"B": w.B, "H": w.H, "n": w.n, "r": w.r, "b": w.b, "passes": "fwd+bwd" if w.backward else "fwd",
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "model_tokens_per_s": w.model_tokens / (ms / 1e3),
+            "nominal_tflops": nominal, "executed_tflops": executed,
+            "frac_nominal": {"burst": nominal / pk["bf16_burst"], "sustained": nominal / pk["bf16_sustained"]},
+            "frac_executed": {"burst": executed / pk["bf16_burst"], "sustained": executed / pk["bf16_sustained"]},
+            "kernels_ms_per_launch": {k: round(v[1] / v[0], 3) for k, v in sorted(agg.items(), key=lambda kv: -kv[1][1])},
+            "clocks": clocks}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -213,6 +280,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--local-exact", action="store_true",
                     help="exact polynomial weights inside each block (Section 3.2) instead of the headline variant")
+    ap.add_argument("--others", default="c1,c3,c4",
+                    help="other configurations timed briefly after the headline one (N = 1 only); '' for none")
+    ap.add_argument("--other-steps", type=int, default=5)
     ap.add_argument("--no-keep-states", action="store_true",
                     help="let the backward rebuild the prefix states instead of reading the forward's")
     args = ap.parse_args()
@@ -381,7 +451,9 @@ def main():
             if per:
                 traffic = per["dram_bytes_per_head_token"] * w.head_tokens
         roof = {"kernel": name, "bound": "tensor" if tensor else "alu", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                "unit": "TFLOP/s", "frac": (achieved / peak) if achieved else None,
+                "frac_sustained": (achieved / pk["bf16_sustained"]) if (achieved and tensor) else None,
+                "frac_burst": (achieved / pk["bf16_burst"]) if (achieved and tensor) else None, "traffic": traffic,
                 "traffic_source": ("profiles/%s (ncu on the c2s slice, scaled by head-tokens)" % tname) if traffic else None,
                 "flops_per_launch": fl * w.head_tokens if fl else None,
                 "peak_source": (pk["source"] + " (sustained bf16)") if tensor else "derived: 148 SM x 128 FMA x 1.965 GHz",
@@ -402,6 +474,19 @@ def main():
 
     f_fwd, f_bwd = nominal_flops_per_head_token(w, args.local_exact)
     nominal_tflops = (f_fwd + f_bwd) * w.head_tokens * world * args.steps / (ms / 1e3) / 1e12
+    # flops the kernels actually issued (symmetric features, masked tiles skipped): the figure the
+    # fraction of peak is claimed on; the nominal one counts the paper's statement of the algorithm
+    executed_tflops = executed_flops_per_step(w, {k: (v[0], v[1], args.steps) for k, v in agg.items()},
+                                              args.local_exact) * world / (ms / args.steps / 1e3) / 1e12
+    # the headline tensors go before the other configurations are built
+    others = None
+    if world == 1 and args.others:
+        del Q, K, V, dO, O, den, grads, ws, inp
+        torch.cuda.empty_cache()
+        others = {}
+        for name in [x for x in args.others.split(",") if x and x != w.name]:
+            others[name] = time_other_config(psk, wl, name, args.other_steps, args.warmup, args.local_exact, pk, local)
+            torch.cuda.empty_cache()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -411,10 +496,17 @@ def main():
                    "variant": "local_exact" if args.local_exact else "polysketch",
                    "keep_states": keep,
                    "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
-        "nominal_tflops": nominal_tflops,
+        "nominal_tflops": nominal_tflops, "executed_tflops": executed_tflops,
         "frac_bf16_peak": {"burst": nominal_tflops / world / pk["bf16_burst"],
                            "sustained": nominal_tflops / world / pk["bf16_sustained"],
-                           "nominal_2250": nominal_tflops / world / 2250.0, "source": pk["source"]},
+                           "nominal_2250": nominal_tflops / world / 2250.0, "source": pk["source"],
+                           "flops": "nominal (paper's statement: r^2 features, full b x b tiles)"},
+        "frac_bf16_peak_executed": {"burst": executed_tflops / world / pk["bf16_burst"],
+                                    "sustained": executed_tflops / world / pk["bf16_sustained"],
+                                    "nominal_2250": executed_tflops / world / 2250.0, "source": pk["source"],
+                                    "flops": "executed MMA flops (symmetric features, masked tiles skipped)"},
+        "ms_x_sm_mhz": (ms / args.steps) * clocks["sm_mhz"] if (clocks and clocks.get("sm_mhz")) else None,
+        "other_configs": others,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0], "roofline": roof, "kernels": kernels,
         "cpu_baseline": cpu,
     }
