@@ -166,7 +166,8 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
  *   - Shapes whose forward scratch (psk_workspace_bytes with path = PSK_PATH_CUDA_CORES)
  *     exceeds the array are refused with PSK_ERR_WORKSPACE before any launch.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call outside any stream capture.
+ *     current); make that first call outside any stream capture.  The address is kept for the life
+ *     of the process: do not call cudaDeviceReset on a device between calls.
  *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - All calls on a device share the one array and it keeps the previous call's bytes;
  *     the call zeroes the part that must start at zero.  Two calls that overlap on the

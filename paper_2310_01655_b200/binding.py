@@ -139,6 +139,17 @@ def _workspace(shape, for_backward, workspace):
     return workspace, workspace.numel()
 
 
+def _check_sketch_matrices(*gs):
+    for g in gs:
+        if g is not None and not g.is_contiguous():
+            raise ValueError("G1 and G2 must be contiguous [g_heads, h, r] tensors")
+
+
+def _check_keep_states(flags, workspace):
+    if (flags & FLAG_KEEP_STATES) and workspace is None:
+        raise ValueError("FLAG_KEEP_STATES needs a caller-owned workspace shared by the forward and the backward call")
+
+
 def _same_layout(ref, *ts):
     for t in ts:
         if t is not None and (t.shape != ref.shape or t.stride() != ref.stride() or t.dtype != ref.dtype):
@@ -170,6 +181,8 @@ def causal_attn_fwd(Q, K, V, G1, G2, b, p=4, path=PATH_AUTO, workspace=None, out
                     seq_segments=0):
     """psk_causal_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, G1, G2)
+    _check_sketch_matrices(G1, G2)
+    _check_keep_states(flags, workspace)
     _same_layout(Q, K, V, out)
     shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags, seq_segments)
     O = _empty_like(Q) if out is None else out
@@ -194,8 +207,9 @@ def causal_attn_fwd_static(Q, K, V, G1, G2, b, p=4, out=None, denom=None):
     and nothing is allocated by the call itself; `out` and `denom` must be supplied by such
     a caller (they are created here only as a convenience when omitted)."""
     _require_cuda(Q, K, V, G1, G2)
+    _check_sketch_matrices(G1, G2)
     _same_layout(Q, K, V, out)
-    shp = make_shape(Q, G1, G1.shape[-1], b, p, PATH_CUDA_CORES)
+    shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, PATH_CUDA_CORES)
     O = _empty_like(Q) if out is None else out
     B, H, n, _ = Q.shape
     if denom is None:
@@ -211,6 +225,8 @@ def causal_attn_bwd(Q, K, V, G1, G2, O, denom, dO, b, p=4, path=PATH_AUTO, works
                     seq_segments=0):
     """psk_causal_attn_bwd: returns (dQ, dK, dV)."""
     _require_cuda(Q, K, V, G1, G2, O, denom, dO)
+    _check_sketch_matrices(G1, G2)
+    _check_keep_states(flags, workspace)
     _same_layout(Q, K, V, O, dO)
     shp = make_shape(Q, G1, _sketch_r(G1, Q), b, p, path, flags, seq_segments)
     dQ, dK, dV = out if out is not None else (_empty_like(Q), _empty_like(Q), _empty_like(Q))

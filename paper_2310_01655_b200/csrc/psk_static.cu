@@ -21,7 +21,8 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 char* g_scratch_ptr[kMaxDevices] = {nullptr};
 
-// Device address of the scratch array on the current device, resolved once per device.
+// Device address of the scratch array on the current device, resolved once per device and kept for
+// the life of the process (it does not survive a cudaDeviceReset of that device).
 int scratch_for_current_device(char** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PSK_ERR_CUDA;
@@ -55,7 +56,7 @@ int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void
         // Invalid shape: let the regular entry point name the reason (it fails before any launch).
         return psk_causal_attn_fwd(&sh, Q, K, V, G1, G2, O, denom, nullptr, 0, stream);
     }
-    if (!Q || !K || !V || !G1 || !G2 || !O) return PSK_ERR_INVALID_ARG;
+    if (!Q || !K || !V || !O || (sh.p != 2 && (!G1 || !G2))) return PSK_ERR_INVALID_ARG;   // p = 2 reads no G
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(G1) || !aligned16(G2) ||
         !aligned16(O) || !aligned16(denom))
         return PSK_ERR_ALIGN;

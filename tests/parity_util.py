@@ -43,3 +43,26 @@ def check(name, got, ref, tol):
     err = orc.rel_l2(got.detach().cpu().to(torch.float64).numpy(), ref)
     assert np.isfinite(err) and err <= tol, "%s: rel L2 %.3e > %.1e" % (name, err, tol)
     return err
+
+
+def tile_errors(got, ref, rows=128):
+    """Relative L2 of every tile of `rows` consecutive rows of a [n, ...] tensor: the slice-level norm
+    is dominated by late rows (large normalisers), so the worst tile is reported beside it."""
+    g = got.detach().cpu().to(torch.float64).numpy()
+    g = g.reshape(g.shape[0], -1)
+    r = np.asarray(ref, dtype=np.float64).reshape(g.shape[0], -1)
+    n = g.shape[0] // rows * rows
+    num = np.linalg.norm((g[:n] - r[:n]).reshape(n // rows, -1), axis=1)
+    den = np.linalg.norm(r[:n].reshape(n // rows, -1), axis=1)
+    return num / np.maximum(den, 1e-300)
+
+
+def check_tiles(name, got, ref, tol, first_block_rows, rows=128):
+    """Per-tile bound for tiles beyond the first block (every row there has at least a block of keys
+    behind it); the first block's worst tile is returned for the record, not asserted: a row with one
+    or two keys has a single cancelling score and is outside what a tensor-level tolerance covers."""
+    e = tile_errors(got, ref, rows)
+    k = first_block_rows // rows
+    later = float(e[k:].max()) if len(e) > k else 0.0
+    assert np.isfinite(e).all() and later <= tol, "%s: worst 128-row tile beyond the first block %.3e > %.1e" % (name, later, tol)
+    return float(e[:k].max()) if k else 0.0, later

@@ -7,7 +7,7 @@ import torch
 
 import paper_2310_01655_b200 as psk
 from paper_2310_01655_b200 import inputs as wl
-from parity_util import TOL, check, oracle_backward, oracle_forward, oracle_rows
+from parity_util import TOL, check, check_tiles, oracle_backward, oracle_forward, oracle_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +47,10 @@ def test_full_size_configuration(name):
         O_ref, d_ref = oracle_forward(inp, bi, hi, w.b)
         check("%s O[%d,%d]" % (name, bi, hi), O[bi, hi], O_ref, tol)
         check("%s denom[%d,%d]" % (name, bi, hi), den[bi, hi], d_ref, tol)
+        # the slice norm cannot see a bad tile among thousands: every 128-row tile beyond the first
+        # block holds the same tolerance on its own; the first block's figure is printed (run with -s)
+        first, later = check_tiles("%s O[%d,%d]" % (name, bi, hi), O[bi, hi], O_ref, tol, w.b)
+        print("%s O[%d,%d]: worst 128-row tile, first block %.2e, later blocks %.2e" % (name, bi, hi, first, later))
         if idx == 0:
             # single rows straight from the definition (quadratic form, no blocks)
             rows = [0, 1, w.b - 1, w.b, w.n // 2 + 3, w.n - 1]
@@ -66,3 +70,5 @@ def test_full_size_configuration(name):
         if w.backward and idx < 2:
             for nm, got, ref in zip(("dQ", "dK", "dV"), grads, oracle_backward(inp, bi, hi, w.b)):
                 check("%s %s[%d,%d]" % (name, nm, bi, hi), got[bi, hi], ref, tol)
+                first, later = check_tiles("%s %s[%d,%d]" % (name, nm, bi, hi), got[bi, hi], ref, 2 * tol, w.b)
+                print("%s %s[%d,%d]: worst 128-row tile, first block %.2e, later blocks %.2e" % (name, nm, bi, hi, first, later))

@@ -141,3 +141,59 @@ def test_device_status_word_is_clean():
     psk.causal_attn_fwd(inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"], 128, workspace=ws)
     assert psk.check(ws) == 0
     assert psk.last_launch_count() > 0
+
+
+@pytest.mark.parametrize("r,b,n", [(32, 1024, 2048), (16, 384, 768), (64, 1024, 1024), (32, 640, 1280)])
+@pytest.mark.parametrize("flags", [0, psk.FLAG_KEEP_STATES, psk.FLAG_LOCAL_EXACT | psk.FLAG_KEEP_STATES])
+def test_many_tiles_per_block_on_the_tensor_cores(r, b, n, flags):
+    # blocks of 3, 5 and 8 row tiles (the paper's own b = 1024 among them): the rings of state chunks,
+    # the aliased tile buffers and the "last chunk" bookkeeping all depend on the tile count
+    w = wl.small_workload(B=1, H=2, n=n, r=r, b=b, dtype="bf16", seed=7 * r + b)
+    inp = wl.make_inputs(w, "cuda")
+    Q, K, V, G1, G2, dO = (inp[k] for k in ("Q", "K", "V", "G1", "G2", "dO"))
+    shp = psk.binding.make_shape(Q, G1, r, b, flags=flags)
+    ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True)), dtype=torch.uint8, device="cuda")
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b, workspace=ws, flags=flags)
+    grads = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, workspace=ws, flags=flags)
+    assert psk.check(ws) == 0
+    diag = "exact" if flags & psk.FLAG_LOCAL_EXACT else "LR"
+    for hi in range(w.H):
+        f = lambda k: wl.head_slice_f64(inp[k], 0, hi)
+        g1, g2 = g_slice(G1, hi), g_slice(G2, hi)
+        O_ref, d_ref = orc.causal_polysketch_attention_blocked(f("Q"), f("K"), f("V"), g1, g2, b, diagonal=diag)
+        refs = (O_ref, d_ref) + tuple(orc.causal_polysketch_attention_backward_blocked(
+            f("Q"), f("K"), f("V"), g1, g2, f("dO"), b, diagonal=diag))
+        for nm, got, ref in zip(("O", "denom", "dQ", "dK", "dV"), (O, den) + tuple(grads), refs):
+            check("%s[%d]" % (nm, hi), got[0, hi], ref, TOL["bf16"])
+
+
+def test_strided_views_and_one_shared_sketch_on_the_tensor_cores():
+    # [B, n, H, h] storage viewed as [B, H, n, h] (TMA maps with non-dense strides), one G pair for all heads
+    B, H, n, r, b = 2, 3, 512, 32, 256
+    w = wl.small_workload(B=B, H=H, n=n, r=r, b=b, dtype="bf16", seed=91)
+    inp = wl.make_inputs(w, "cuda")
+    view = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)      # same values, strides of [B, n, H, h]
+    Q, K, V, dO = (view(inp[k]) for k in ("Q", "K", "V", "dO"))
+    assert not Q.is_contiguous()
+    G1, G2 = inp["G1"][:1].contiguous(), inp["G2"][:1].contiguous()
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b)
+    dQ, dK, dV = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b)
+    assert O.stride() == Q.stride() and dQ.stride() == Q.stride()
+    one = dict(inp, G1=G1, G2=G2)
+    for bi, hi in ((0, 0), (1, 2)):
+        O_ref, d_ref = oracle_forward(one, bi, hi, b)
+        check("O", O[bi, hi], O_ref, TOL["bf16"])
+        check("denom", den[bi, hi], d_ref, TOL["bf16"])
+        for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), oracle_backward(one, bi, hi, b)):
+            check(nm, got[bi, hi], ref, TOL["bf16"])
+
+
+def test_binding_refuses_kept_states_without_a_workspace_and_strided_sketch_matrices():
+    w = wl.small_workload(B=1, H=2, n=256, r=32, b=128, dtype="bf16", seed=92)
+    inp = wl.make_inputs(w, "cuda")
+    args = (inp["Q"], inp["K"], inp["V"], inp["G1"], inp["G2"], 128)
+    with pytest.raises(ValueError):
+        psk.causal_attn_fwd(*args, flags=psk.FLAG_KEEP_STATES)
+    Gs = torch.empty((2, 64, 64), dtype=torch.bfloat16, device="cuda")[:, :, :32]
+    with pytest.raises(ValueError):
+        psk.causal_attn_fwd(inp["Q"], inp["K"], inp["V"], Gs, Gs, 128)

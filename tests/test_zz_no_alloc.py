@@ -9,6 +9,8 @@ import torch
 
 import paper_2310_01655_b200 as psk
 from paper_2310_01655_b200 import inputs as wl
+from oracle import polysketch as orc
+from parity_util import check, oracle_forward
 
 pytestmark = pytest.mark.gpu
 
@@ -43,6 +45,25 @@ def test_static_scratch_forward_matches_regular_forward_twice(dtype, tol):
         torch.cuda.synchronize()
         assert torch.isfinite(O.float()).all() and torch.isfinite(den).all()
         assert _rel(O, O_ref) <= tol and _rel(den, den_ref) <= tol
+        # and against the oracle itself, not only against the library's other entry point
+        for hi in range(w.H):
+            O_orc, d_orc = oracle_forward(inp, 0, hi, b)
+            check("static O[%d]" % hi, O[0, hi], O_orc, tol)
+            check("static denom[%d]" % hi, den[0, hi], d_orc, tol)
+
+
+def test_static_scratch_degree_two_takes_no_sketch_matrices():
+    # p = 2 reads no G1, G2: null pointers are valid here as they are for the regular forward
+    w = wl.small_workload(B=1, H=2, n=256, r=64, b=128, dtype="f32", seed=54)
+    inp = wl.make_inputs(w, "cuda")
+    Q, K, V = 0.5 * inp["Q"], 0.5 * inp["K"], inp["V"]
+    O, den = psk.causal_attn_fwd_static(Q, K, V, None, None, 128, p=2)
+    torch.cuda.synchronize()
+    for hi in range(w.H):
+        f = lambda t: t[0, hi].double().cpu().numpy()
+        O_ref, d_ref = orc.causal_degree2_attention_blocked(f(Q), f(K), f(V), 128)
+        check("static p=2 O[%d]" % hi, O[0, hi], O_ref, 1e-4)
+        check("static p=2 denom[%d]" % hi, den[0, hi], d_ref, 1e-4)
 
 
 def test_static_scratch_refuses_oversized_problems():
