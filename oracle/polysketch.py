@@ -32,6 +32,9 @@ features, block algorithm against the definition, finite differences.
 the non-causal form of Section 3: looped (q.k)^4 attention over all keys, invariance
 under a joint permutation of keys and values, last row of the causal form, linear-time
 evaluation against the definition, finite differences.
+for the learnable sketch (Algorithm 2): one row evaluated entry by entry, the bound |M| <= sqrt(r),
+weights under which each network reduces to x -> LN(x) G so that the result approaches the random
+sketch's, finite differences for inputs and every parameter group.
 Every function in this file has at least one such pin.
 """
 from __future__ import annotations
@@ -523,6 +526,165 @@ def polysketch_attention_backward_linear(Q, K, V, G1, G2, dO):
         return np.einsum("nab,nb->na", D + D.transpose(0, 2, 1), M)
 
     return (_sketch_backward(Q, G1, G2, untensor(dPq, Mq)), _sketch_backward(K, G1, G2, untensor(dPk, Mk)), dV)
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 2 (appendix "Replacing Random Projections with Learnable Transformations"):
+# the products M_1 G_1 and M_2 G_2 of Algorithm 1 become f_1(M_1), f_2(M_2) for two dense networks
+# of equal structure and separate parameters, and the result goes through
+# sqrt(r) tanh(sqrt(1/r) [f_1 * f_2]).  Each network: output dimension r, three hidden layers of
+# sizes [8r, r, 8r], gelu after the first and the third hidden layer, layer normalisation before the
+# input and before the second hidden layer.
+# Readings where the appendix is silent: dense layers carry biases; each layer normalisation has a
+# learnable gain and bias and eps = 1e-6 inside the square root; gelu is x Phi(x) (the erf form);
+# one pair of networks serves every head.  For p = 4 the recursion bottoms out at M_1 = M_2 = A.
+# A network's parameters are a dict with keys
+#   g0, c0 (h)  W1 (h x 8r), b1 (8r)  g1, c1 (8r)  W2 (8r x r), b2 (r)  W3 (r x 8r), b3 (8r)  W4 (8r x r), b4 (r).
+# ---------------------------------------------------------------------------
+LN_EPS = 1e-6
+NET_KEYS = ("g0", "c0", "W1", "b1", "g1", "c1", "W2", "b2", "W3", "b3", "W4", "b4")
+
+
+def _erf(x):
+    import math
+    return np.vectorize(math.erf, otypes=[F64])(x)
+
+
+def gelu(x):
+    x = _f64(x)
+    return 0.5 * x * (1.0 + _erf(x / np.sqrt(2.0)))
+
+
+def _gelu_grad(x):
+    x = _f64(x)
+    return 0.5 * (1.0 + _erf(x / np.sqrt(2.0))) + x * np.exp(-0.5 * x * x) / np.sqrt(2.0 * np.pi)
+
+
+def layer_norm(x, gain, bias):
+    x = _f64(x)
+    mu = x.mean(axis=1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=1, keepdims=True)
+    return (x - mu) / np.sqrt(var + LN_EPS) * _f64(gain) + _f64(bias)
+
+
+def learned_net(X, P):
+    """One network f of Algorithm 2 applied to the rows of X."""
+    z0 = layer_norm(X, P["g0"], P["c0"])
+    a1 = gelu(z0 @ _f64(P["W1"]) + _f64(P["b1"]))
+    z1 = layer_norm(a1, P["g1"], P["c1"])
+    a2 = z1 @ _f64(P["W2"]) + _f64(P["b2"])
+    a3 = gelu(a2 @ _f64(P["W3"]) + _f64(P["b3"]))
+    return a3 @ _f64(P["W4"]) + _f64(P["b4"])
+
+
+def learned_half_sketch(X, P1, P2):
+    """LearnablePolysketchWithNegativity(X, r, 2): sqrt(r) tanh(sqrt(1/r) [f_1(X) * f_2(X)])."""
+    f1, f2 = learned_net(X, P1), learned_net(X, P2)
+    r = f1.shape[1]
+    return np.sqrt(r) * np.tanh(f1 * f2 / np.sqrt(r))
+
+
+def causal_learned_polysketch_attention(Q, K, V, P1, P2):
+    """Section 3 with phi' = LearnablePolysketchNonNegative(., r, 4) = M^{(x)2}: the n x n definition."""
+    s = learned_half_sketch(Q, P1, P2) @ learned_half_sketch(K, P1, P2).T
+    W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    return (W @ _f64(V)) / d[:, None], d
+
+
+def causal_learned_polysketch_attention_blocked(Q, K, V, P1, P2, b, diagonal="LR"):
+    """The same by Section 3.1's block algorithm; diagonal="exact" gives the same-block pairs the
+    weights (q_i . k_j)^4 of Section 3.2 (the paper's "learned + local" variant)."""
+    Mq, Mk = learned_half_sketch(Q, P1, P2), learned_half_sketch(K, P1, P2)
+    if diagonal == "LR":
+        return causal_attention_blocked_from_half_sketches(Mq, Mk, V, b)
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, h = V.shape
+    C = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+
+    def diag_block(l):
+        return lt((Q[l * b:(l + 1) * b] @ K[l * b:(l + 1) * b].T) ** 4)
+
+    N = lt_multiply_blocked(self_tensor(Mq), self_tensor(Mk), C, b, diag_block)
+    d = 1.0 + N[:, h]
+    return N[:, :h] / d[:, None], d
+
+
+def _layer_norm_backward(x, gain, dz):
+    """z = n * gain + bias with n = (x - mean) / sqrt(var + eps): returns (dx, dgain, dbias)."""
+    x, dz = _f64(x), _f64(dz)
+    mu = x.mean(axis=1, keepdims=True)
+    sig = np.sqrt(((x - mu) ** 2).mean(axis=1, keepdims=True) + LN_EPS)
+    nrm = (x - mu) / sig
+    dn = dz * _f64(gain)
+    dx = (dn - dn.mean(axis=1, keepdims=True) - nrm * (dn * nrm).mean(axis=1, keepdims=True)) / sig
+    return dx, (dz * nrm).sum(axis=0), dz.sum(axis=0)
+
+
+def learned_net_backward(X, P, df):
+    """Gradients of sum(df * f(X)): (dX, dict of parameter gradients)."""
+    X = _f64(X)
+    W1, W2, W3, W4 = (_f64(P[k]) for k in ("W1", "W2", "W3", "W4"))
+    z0 = layer_norm(X, P["g0"], P["c0"])
+    p1 = z0 @ W1 + _f64(P["b1"])
+    a1 = gelu(p1)
+    z1 = layer_norm(a1, P["g1"], P["c1"])
+    a2 = z1 @ W2 + _f64(P["b2"])
+    p3 = a2 @ W3 + _f64(P["b3"])
+    a3 = gelu(p3)
+    df = _f64(df)
+    g = {"W4": a3.T @ df, "b4": df.sum(axis=0)}
+    dp3 = (df @ W4.T) * _gelu_grad(p3)
+    g["W3"], g["b3"] = a2.T @ dp3, dp3.sum(axis=0)
+    da2 = dp3 @ W3.T
+    g["W2"], g["b2"] = z1.T @ da2, da2.sum(axis=0)
+    da1, g["g1"], g["c1"] = _layer_norm_backward(a1, P["g1"], da2 @ W2.T)
+    dp1 = da1 * _gelu_grad(p1)
+    g["W1"], g["b1"] = z0.T @ dp1, dp1.sum(axis=0)
+    dX, g["g0"], g["c0"] = _layer_norm_backward(X, P["g0"], dp1 @ W1.T)
+    return dX, g
+
+
+def learned_half_sketch_backward(X, P1, P2, dM):
+    """Gradients of sum(dM * M) for M = learned_half_sketch(X, P1, P2): (dX, grads of P1, grads of P2)."""
+    f1, f2 = learned_net(X, P1), learned_net(X, P2)
+    r = f1.shape[1]
+    t = np.tanh(f1 * f2 / np.sqrt(r))
+    du = _f64(dM) * (1.0 - t * t)                 # d/du of sqrt(r) tanh(u / sqrt(r)) at u = f1 * f2
+    dX1, g1 = learned_net_backward(X, P1, du * f2)
+    dX2, g2 = learned_net_backward(X, P2, du * f1)
+    return dX1 + dX2, g1, g2
+
+
+def causal_learned_polysketch_attention_backward(Q, K, V, P1, P2, dO, b=None, diagonal="LR"):
+    """Gradients (dQ, dK, dV, grads of P1, grads of P2) of sum(dO * O), through the n x n definition.
+    The networks see the queries and the keys, so their gradients are the sum of both uses.
+    diagonal="exact" (with the block size b): same-block pairs carry (q_i . k_j)^4, whose gradient
+    reaches Q and K directly."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, h = V.shape
+    Mq, Mk = learned_half_sketch(Q, P1, P2), learned_half_sketch(K, P1, P2)
+    s = Mq @ Mk.T
+    if diagonal == "exact":
+        same = same_block(n, b)
+        x = Q @ K.T
+        W = lt(np.where(same, x ** 4, s * s))
+    else:
+        same = np.zeros((n, n), dtype=bool)
+        x = np.zeros((n, n))
+        W = lt(s * s)
+    d = 1.0 + W.sum(axis=1)
+    O = (W @ V) / d[:, None]
+    E = _backward_rows(O, d, dO)
+    Vt = np.concatenate([V, np.ones((n, 1), dtype=F64)], axis=1)
+    dW = lt(E @ Vt.T)
+    ds = np.where(same, 0.0, 2.0 * s * dW)
+    dx = np.where(same, 4.0 * x ** 3 * dW, 0.0)
+    dQ, gq1, gq2 = learned_half_sketch_backward(Q, P1, P2, ds @ Mk)
+    dK, gk1, gk2 = learned_half_sketch_backward(K, P1, P2, ds.T @ Mq)
+    g1 = {k: gq1[k] + gk1[k] for k in NET_KEYS}
+    g2 = {k: gq2[k] + gk2[k] for k in NET_KEYS}
+    return dQ + dx @ K, dK + dx.T @ Q, W.T @ E[:, :h], g1, g2
 
 
 # ---------------------------------------------------------------------------
