@@ -177,6 +177,38 @@ size_t psk_static_scratch_bytes(void);
 int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void* K, const void* V,
                                const void* G1, const void* G2, void* O, float* denom, void* stream);
 
+/* Learnable sketches (Algorithm 2 in the appendix, "Replacing Random Projections with Learnable
+ * Transformations"; Section 3's paragraph on learnable sketches).  The products x G1 and x G2 of
+ * the degree-2 level become f1(x) and f2(x) for two dense networks of equal structure and separate
+ * parameters, and the half sketch is
+ *     m(x) = sqrt(r) tanh( sqrt(1/r) [ f1(x) * f2(x) ] ),          |m| <= sqrt(r);
+ * features m (x) m, the block algorithm and everything else are as for the random sketch.
+ * Each network: layer normalisation of the input, dense h -> 8r, gelu, layer normalisation, dense
+ * 8r -> r, dense r -> 8r, gelu, dense 8r -> r (output dimension r, hidden layers [8r, r, 8r], gelu after
+ * the first and the third, normalisation before the input and before the second hidden layer).
+ * Where the paper is silent this library takes: dense layers with biases, normalisations with a
+ * learnable gain and bias and eps = 1e-6, gelu(x) = x Phi(x), one pair of networks for all heads.
+ *   params   DEVICE fp32 [2][psk_learned_param_count(h, r)]: network 1 then network 2, each packed as
+ *            g0[h] c0[h] | W1[h][8r] b1[8r] | g1[8r] c1[8r] | W2[8r][r] b2[r] | W3[r][8r] b3[8r] | W4[8r][r] b4[r]
+ *            (gain, bias of a normalisation; row-major weight [in][out], bias of a dense layer)
+ *   dparams  DEVICE fp32, same layout: dL/dparams, overwritten by psk_learned_attn_bwd (summed over
+ *            the batch, the heads and both uses of the networks, on Q and on K; accumulated with
+ *            floating-point atomics, so its last bits are not reproducible from run to run)
+ * The other arguments, the workspace rules and the error codes are those of psk_sketch,
+ * psk_causal_attn_fwd and psk_causal_attn_bwd; `shape` needs p = 4, g_heads and path are ignored,
+ * PSK_FLAG_LOCAL_EXACT is honoured (the paper's "learned + local" variant), PSK_FLAG_NONCAUSAL is
+ * not supported here.  CUDA-core kernels (fp32 arithmetic) for either storage type; workspace size from
+ * psk_learned_workspace_bytes. */
+size_t psk_learned_param_count(int h, int r);
+size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward);
+int psk_learned_sketch(const psk_shape* shape, const void* X, const float* params, float* M_out, float* Phi_out,
+                       void* stream);
+int psk_learned_attn_fwd(const psk_shape* shape, const void* Q, const void* K, const void* V, const float* params,
+                         void* O, float* denom, void* workspace, size_t workspace_bytes, void* stream);
+int psk_learned_attn_bwd(const psk_shape* shape, const void* Q, const void* K, const void* V, const float* params,
+                         const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV,
+                         float* dparams, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Block lower-triangular multiplication for arbitrary feature matrices (Section 3.1):
  *   Out = lt(A B^T) C,   A, B: [batch, n, m],  C, Out: [batch, n, k],  all fp32, contiguous, DEVICE,
  * computed as  H_l = B_l^T C_l,  Z_l = sum_{j<l} H_j,  rows of block l = lt(A_l B_l^T) C_l + A_l Z_l

@@ -75,6 +75,16 @@ def lib():
     L.psk_decode_state_bytes.argtypes = [POINTER(Shape)]
     L.psk_decode_step.restype = c_int
     L.psk_decode_step.argtypes = [POINTER(Shape)] + [c_void_p] * 9
+    L.psk_learned_param_count.restype = c_size_t
+    L.psk_learned_param_count.argtypes = [c_int, c_int]
+    L.psk_learned_workspace_bytes.restype = c_size_t
+    L.psk_learned_workspace_bytes.argtypes = [P, c_int]
+    L.psk_learned_sketch.restype = c_int
+    L.psk_learned_sketch.argtypes = [P] + [c_void_p] * 5
+    L.psk_learned_attn_fwd.restype = c_int
+    L.psk_learned_attn_fwd.argtypes = [P] + [c_void_p] * 7 + [c_size_t, c_void_p]
+    L.psk_learned_attn_bwd.restype = c_int
+    L.psk_learned_attn_bwd.argtypes = [P] + [c_void_p] * 12 + [c_size_t, c_void_p]
     L.psk_profile_enable.restype = c_int
     L.psk_profile_enable.argtypes = [c_int]
     L.psk_profile_count.restype = c_int
@@ -312,6 +322,95 @@ def lt_multiply(A, B, C, b, workspace=None):
     if st != 0:
         raise PskError(st, "psk_lt_multiply")
     return out
+
+
+# ---- learnable sketch (Algorithm 2): parameter packing and the three calls ----
+LEARNED_KEYS = ("g0", "c0", "W1", "b1", "g1", "c1", "W2", "b2", "W3", "b3", "W4", "b4")
+
+
+def learned_param_count(h: int, r: int) -> int:
+    """Floats in one network's packed parameter vector (0 for unsupported h, r)."""
+    return int(lib().psk_learned_param_count(int(h), int(r)))
+
+
+def learned_shapes(h: int, r: int):
+    m = 8 * r
+    return {"g0": (h,), "c0": (h,), "W1": (h, m), "b1": (m,), "g1": (m,), "c1": (m,), "W2": (m, r), "b2": (r,),
+            "W3": (r, m), "b3": (m,), "W4": (m, r), "b4": (r,)}
+
+
+def pack_learned_params(P1, P2, device="cuda"):
+    """Two dicts of arrays (keys LEARNED_KEYS) -> the fp32 [2, count] tensor the library reads."""
+    rows = []
+    for P in (P1, P2):
+        rows.append(torch.cat([torch.as_tensor(P[k], dtype=torch.float32).reshape(-1) for k in LEARNED_KEYS]))
+    return torch.stack(rows).to(device).contiguous()
+
+
+def unpack_learned_params(flat, h: int, r: int):
+    """The inverse of pack_learned_params (for gradients): a pair of dicts of tensors."""
+    out = []
+    for row in flat:
+        o, P = 0, {}
+        for k, shp in learned_shapes(h, r).items():
+            cnt = 1
+            for x in shp:
+                cnt *= x
+            P[k] = row[o:o + cnt].reshape(shp)
+            o += cnt
+        out.append(P)
+    return out[0], out[1]
+
+
+def _learned_shape(x, r, b, flags):
+    return make_shape(x, None, r, b, 4, PATH_CUDA_CORES, flags)
+
+
+def learned_sketch(X, params, r, want_phi=False):
+    """psk_learned_sketch: (M [B,H,n,r] fp32, Phi [B,H,n,r*r] fp32 or None)."""
+    _require_cuda(X, params)
+    B, H, n, _ = X.shape
+    shp = _learned_shape(X, r, 128, 0)
+    M = torch.empty((B, H, n, r), dtype=torch.float32, device=X.device)
+    Phi = torch.empty((B, H, n, r * r), dtype=torch.float32, device=X.device) if want_phi else None
+    st = lib().psk_learned_sketch(byref(shp), _ptr(X), _ptr(params), _ptr(M), _ptr(Phi), _stream())
+    if st != 0:
+        raise PskError(st, "psk_learned_sketch")
+    return M, Phi
+
+
+def learned_attn_fwd(Q, K, V, params, r, b, flags=0, workspace=None):
+    """psk_learned_attn_fwd: returns (O, denom)."""
+    _require_cuda(Q, K, V, params)
+    _same_layout(Q, K, V)
+    shp = _learned_shape(Q, r, b, flags)
+    need = int(lib().psk_learned_workspace_bytes(byref(shp), 0))
+    ws = workspace if workspace is not None else torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
+    B, H, n, _ = Q.shape
+    O = _empty_like(Q)
+    den = torch.empty((B, H, n), dtype=torch.float32, device=Q.device)
+    st = lib().psk_learned_attn_fwd(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(params), _ptr(O), _ptr(den), _ptr(ws),
+                                    ws.numel() if need else 0, _stream())
+    if st != 0:
+        raise PskError(st, "psk_learned_attn_fwd")
+    return O, den
+
+
+def learned_attn_bwd(Q, K, V, params, O, denom, dO, r, b, flags=0, workspace=None):
+    """psk_learned_attn_bwd: returns (dQ, dK, dV, dparams [2, count] fp32)."""
+    _require_cuda(Q, K, V, params, O, denom, dO)
+    _same_layout(Q, K, V, O, dO)
+    shp = _learned_shape(Q, r, b, flags)
+    need = int(lib().psk_learned_workspace_bytes(byref(shp), 1))
+    ws = workspace if workspace is not None else torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
+    dQ, dK, dV = _empty_like(Q), _empty_like(Q), _empty_like(Q)
+    dparams = torch.empty_like(params)
+    st = lib().psk_learned_attn_bwd(byref(shp), _ptr(Q), _ptr(K), _ptr(V), _ptr(params), _ptr(O), _ptr(denom), _ptr(dO),
+                                    _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dparams), _ptr(ws), ws.numel() if need else 0,
+                                    _stream())
+    if st != 0:
+        raise PskError(st, "psk_learned_attn_bwd")
+    return dQ, dK, dV, dparams
 
 
 def decode_state(B, H, r, device="cuda"):

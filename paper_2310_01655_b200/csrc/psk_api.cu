@@ -175,6 +175,87 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
     return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
 }
 
+// ---- learnable sketch (Algorithm 2): the same calls with network parameters in place of G1, G2 ----
+static int learned_dims(const psk_shape* shape, psk_shape* sh, Dims* d) {
+    if (shape == nullptr) return PSK_ERR_INVALID_ARG;
+    *sh = *shape;
+    sh->path = PSK_PATH_CUDA_CORES;
+    sh->g_heads = 1;
+    if (sh->p != 4) return PSK_ERR_UNSUPPORTED;
+    const int st = make_dims(sh, d);
+    if (st != PSK_OK) return st;
+    d->learned = true;
+    return PSK_OK;
+}
+
+size_t psk_learned_param_count(int h, int r) {
+    if (h != 64 || (r != 16 && r != 32 && r != 64)) return 0;
+    return learned_param_count(h, r);
+}
+
+size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward) {
+    psk_shape sh; Dims d;
+    if (learned_dims(shape, &sh, &d) != PSK_OK) return 0;
+    return cc_workspace(d, for_backward != 0).total;
+}
+
+int psk_learned_sketch(const psk_shape* shape, const void* X, const float* params, float* M_out, float* Phi_out,
+                       void* stream) {
+    psk_shape sh; Dims d;
+    const int st = learned_dims(shape, &sh, &d);
+    if (st != PSK_OK) return st;
+    if (!X || !params || !M_out) return PSK_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(params) || !aligned16(M_out) || !aligned16(Phi_out)) return PSK_ERR_ALIGN;
+    d.lparams = params;
+    int launches = 0;
+    const cudaError_t e = cc_sketch(d, X, nullptr, nullptr, M_out, Phi_out, (cudaStream_t)stream, &launches);
+    g_last_launches = launches;
+    return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
+}
+
+int psk_learned_attn_fwd(const psk_shape* shape, const void* Q, const void* K, const void* V, const float* params,
+                         void* O, float* denom, void* workspace, size_t workspace_bytes, void* stream) {
+    psk_shape sh; Dims d;
+    const int st = learned_dims(shape, &sh, &d);
+    if (st != PSK_OK) return st;
+    if (!Q || !K || !V || !O || !params) return PSK_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(params) || !aligned16(O) || !aligned16(denom))
+        return PSK_ERR_ALIGN;
+    const size_t need = cc_workspace(d, false).total;
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign)) return PSK_ERR_WORKSPACE;
+    d.lparams = params;
+    cudaStream_t s = (cudaStream_t)stream;
+    int launches = 0;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
+    if (e == cudaSuccess) e = cc_fwd(d, Q, K, V, nullptr, nullptr, O, denom, (char*)workspace, s, &launches);
+    g_last_launches = launches;
+    return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
+}
+
+int psk_learned_attn_bwd(const psk_shape* shape, const void* Q, const void* K, const void* V, const float* params,
+                         const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV,
+                         float* dparams, void* workspace, size_t workspace_bytes, void* stream) {
+    psk_shape sh; Dims d;
+    const int st = learned_dims(shape, &sh, &d);
+    if (st != PSK_OK) return st;
+    if (!Q || !K || !V || !O || !denom || !dO || !dQ || !dK || !dV || !params || !dparams) return PSK_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(params) || !aligned16(O) || !aligned16(denom) ||
+        !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(dparams))
+        return PSK_ERR_ALIGN;
+    const size_t need = cc_workspace(d, true).total;
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign)) return PSK_ERR_WORKSPACE;
+    d.lparams = params;
+    d.dlparams = dparams;
+    cudaStream_t s = (cudaStream_t)stream;
+    int launches = 0;
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
+    // the kernels add into the gradient array: it starts at zero
+    if (e == cudaSuccess) e = cudaMemsetAsync(dparams, 0, 2 * learned_param_count(d.h, d.r) * sizeof(float), s);
+    if (e == cudaSuccess) e = cc_bwd(d, Q, K, V, nullptr, nullptr, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches);
+    g_last_launches = launches;
+    return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
+}
+
 int psk_check(const void* workspace, void* stream) {
     if (!workspace) return PSK_ERR_INVALID_ARG;
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PSK_ERR_CUDA;

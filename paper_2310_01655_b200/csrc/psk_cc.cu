@@ -755,6 +755,7 @@ cudaError_t allow_smem(K kernel, size_t bytes) {
 template <typename T, int R>
 cudaError_t launch_sketch(const Dims& d, const T* X, const T* G1, const T* G2, float* M, float* Phi,
                           cudaStream_t s, int* launches) {
+    if (d.learned) return learned_sketch(d, X, M, Phi, s, launches);      // Algorithm 2: two dense networks
     if (d.p == 2) {           // M = X (R = 64 = h)
         const int rows = d.BH() * d.n;
         prof_begin("identity_sketch_kernel", s);
@@ -876,6 +877,10 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     }
     *launches += 2;
     PSK_TRY(cudaGetLastError());
+    if (d.learned) {          // back through the two networks; their gradients collect both uses
+        PSK_TRY(learned_sketch_bwd(d, Q, dMq, dXq, dQ, s, launches));
+        return learned_sketch_bwd(d, K, dMk, dXk, dK, s, launches);
+    }
     if (d.p == 2) {           // dX = dM (+ the same-block part that bypassed it)
         prof_begin("identity_sketch_bwd_kernel", s);
         identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMq, dXq, dQ);

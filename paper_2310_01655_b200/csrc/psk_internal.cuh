@@ -21,6 +21,10 @@ struct Dims {
     bool local;                       // PSK_FLAG_LOCAL_EXACT
     bool noncausal;                   // PSK_FLAG_NONCAUSAL: no lt(), one global state per head
     int seq_segments;                 // runs a head's sequence is cut into for the state scan; 0 = library's choice
+    // learnable sketch (Algorithm 2): the half sketch comes from two dense networks instead of G1, G2
+    bool learned = false;
+    const float* lparams = nullptr;   // packed parameters of both networks (psk_learned.cu)
+    float* dlparams = nullptr;        // their gradients (backward only)
     int BH() const { return B * H; }
 };
 
@@ -46,6 +50,13 @@ cudaError_t cc_bwd(const Dims& d, const void* Q, const void* K, const void* V,
                    const void* G1, const void* G2, const void* O, const float* denom,
                    const void* dO, void* dQ, void* dK, void* dV,
                    char* ws, cudaStream_t s, int* launches);
+
+// Learnable sketch (CUDA cores): M = sqrt(r) tanh(f1(x) * f2(x) / sqrt(r)) and its backward
+// (dX = chain rule + `add`; parameter gradients are added to d.dlparams).
+size_t learned_param_count(int h, int r);
+cudaError_t learned_sketch(const Dims& d, const void* X, float* M, float* Phi, cudaStream_t s, int* launches);
+cudaError_t learned_sketch_bwd(const Dims& d, const void* X, const float* dM, const float* add, void* dX,
+                               cudaStream_t s, int* launches);
 
 // Tensor-core (bf16 operands, fp32 accumulation) launchers.
 size_t tc_workspace_bytes(const Dims& d, bool backward);

@@ -1,0 +1,98 @@
+"""Learnable sketch (Algorithm 2 of the appendix) on the GPU against the oracle: the half sketch, causal
+attention on it forward and backward, with the gradients of every parameter group, also with exact
+same-block weights (the paper's "learned + local" variant)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_01655_b200 as psk
+from paper_2310_01655_b200 import binding, inputs as wl
+from oracle import polysketch as orc
+from parity_util import TOL, check
+from paper_2310_01655_b200.inputs import head_slice_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def make_net(g, h, r):
+    m = 8 * r
+    return {"g0": 1.0 + 0.1 * g.standard_normal(h), "c0": 0.1 * g.standard_normal(h),
+            "W1": g.standard_normal((h, m)) / np.sqrt(h), "b1": 0.1 * g.standard_normal(m),
+            "g1": 1.0 + 0.1 * g.standard_normal(m), "c1": 0.1 * g.standard_normal(m),
+            "W2": g.standard_normal((m, r)) / np.sqrt(m), "b2": 0.1 * g.standard_normal(r),
+            "W3": g.standard_normal((r, m)) / np.sqrt(r), "b3": 0.1 * g.standard_normal(m),
+            "W4": 1.5 * g.standard_normal((m, r)) / np.sqrt(m), "b4": 0.1 * g.standard_normal(r)}
+
+
+def nets(r, seed):
+    g = np.random.default_rng(seed)
+    P1, P2 = make_net(g, 64, r), make_net(g, 64, r)
+    # the library reads fp32 parameters: the oracle gets exactly those values
+    flat = binding.pack_learned_params(P1, P2)
+    Q1, Q2 = binding.unpack_learned_params(flat.double().cpu(), 64, r)
+    return flat, {k: v.numpy() for k, v in Q1.items()}, {k: v.numpy() for k, v in Q2.items()}
+
+
+@pytest.mark.parametrize("r", [16, 32, 64])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_half_sketch(r, dtype):
+    assert binding.learned_param_count(64, r) == 2 * 64 + 8 * 64 * r + 24 * r * r + 34 * r
+    w = wl.small_workload(B=1, H=2, n=128, r=r, dtype=dtype, seed=60 + r)
+    inp = wl.make_inputs(w, "cuda")
+    flat, P1, P2 = nets(r, 1)
+    M, Phi = binding.learned_sketch(inp["Q"], flat, r, want_phi=True)
+    assert float(M.abs().max()) <= np.sqrt(r) * (1 + 1e-6)
+    for hi in range(w.H):
+        Mref = orc.learned_half_sketch(head_slice_f64(inp["Q"], 0, hi), P1, P2)
+        check("M", M[0, hi], Mref, 2e-5)
+        check("Phi", Phi[0, hi], orc.self_tensor(Mref), 4e-5)
+
+
+@pytest.mark.parametrize("r,b,n", [(16, 128, 256), (32, 128, 384), (64, 256, 256)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("local", [False, True])
+def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype, local):
+    w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype=dtype, seed=70 + r)
+    inp = wl.make_inputs(w, "cuda")
+    if local:
+        # (q . k)^4 next to weights bounded by r^2: keep the exact pairs on the same scale
+        inp["Q"], inp["K"] = (0.35 * inp["Q"].float()).to(inp["Q"].dtype), (0.35 * inp["K"].float()).to(inp["K"].dtype)
+    flat, P1, P2 = nets(r, 2)
+    flags = psk.FLAG_LOCAL_EXACT if local else 0
+    Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
+    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags)
+    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags)
+    torch.cuda.synchronize()
+    tol = TOL[dtype]
+    diag = "exact" if local else "LR"
+    g1_sum = {k: 0.0 for k in orc.NET_KEYS}
+    g2_sum = {k: 0.0 for k in orc.NET_KEYS}
+    for bi in range(w.B):
+        for hi in range(w.H):
+            f = lambda k: head_slice_f64(inp[k], bi, hi)
+            O_ref, d_ref = orc.causal_learned_polysketch_attention_blocked(f("Q"), f("K"), f("V"), P1, P2, b, diagonal=diag)
+            check("O", O[bi, hi], O_ref, tol)
+            check("denom", den[bi, hi], d_ref, tol)
+            gq, gk, gv, g1, g2 = orc.causal_learned_polysketch_attention_backward(f("Q"), f("K"), f("V"), P1, P2, f("dO"), b, diag)
+            # the oracle's backward starts from its own fp64 forward, as the other parity tests do
+            for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), (gq, gk, gv)):
+                check(nm, got[bi, hi], ref, tol)
+            for k in orc.NET_KEYS:
+                g1_sum[k] = g1_sum[k] + g1[k]
+                g2_sum[k] = g2_sum[k] + g2[k]
+    # parameter gradients are sums over the batch, the heads and both uses of the networks
+    d1, d2 = binding.unpack_learned_params(dflat, 64, r)
+    for which, (got, ref) in enumerate(((d1, g1_sum), (d2, g2_sum))):
+        for k in orc.NET_KEYS:
+            check("net %d %s" % (which + 1, k), got[k], ref[k], 5 * tol if dtype == "bf16" else 2e-3)
+
+
+def test_refusals():
+    w = wl.small_workload(B=1, H=1, n=256, r=32, b=128, dtype="f32", seed=5)
+    inp = wl.make_inputs(w, "cuda")
+    flat, _, _ = nets(32, 3)
+    with pytest.raises(psk.PskError):
+        binding.learned_attn_fwd(inp["Q"], inp["K"], inp["V"], flat, 32, 128, psk.FLAG_NONCAUSAL)
+    with pytest.raises(psk.PskError):
+        binding.learned_attn_fwd(inp["Q"], inp["K"], inp["V"], flat, 32, 100)
+    assert binding.learned_param_count(48, 32) == 0
