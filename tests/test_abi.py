@@ -60,7 +60,9 @@ def test_workspace_size_formula(L):
 @pytest.mark.parametrize("field,value,code", [
     ("p", 2, -2), ("p", 6, -2), ("p", 16, -2), ("h", 128, -2), ("r", 48, -2),      # (p = 2 needs r = h)
     ("b", 100, -3), ("n", 500, -3), ("B", 0, -3), ("g_heads", 3, -3),
-    ("dtype", 7, -1), ("path", 9, -1), ("flags", 6, -1), ("stride_n", 66, -4),
+    ("dtype", 7, -1), ("path", 9, -1), ("flags", 8, -1), ("stride_n", 66, -4),
+    ("flags", 6, -2),                                   # no mask together with exact same-block weights
+    ("seq_segments", -1, -1), ("seq_segments", 3, -3),   # runs must divide the n / b = 2 blocks
 ])
 def test_bad_shapes_are_rejected_before_any_launch(L, field, value, code):
     s = good()
