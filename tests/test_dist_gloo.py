@@ -33,6 +33,39 @@ WORKER = textwrap.dedent("""
 """) % ROOT
 
 
+SEQ_WORKER = textwrap.dedent("""
+    # A sequence cut over the ranks: every rank holds n / world consecutive rows of one head.  Its
+    # rows' outputs are the causal result inside the shard plus phi'(Q_shard) times the sum of the
+    # earlier shards' end states -- which is what exclusive_prefix_over_ranks delivers.
+    import os, sys
+    sys.path.insert(0, %r)
+    import numpy as np, torch
+    from paper_2310_01655_b200 import dist_util as du
+    from oracle import polysketch as orc
+    rank, world, local = du.env_rank()
+    assert du.init("gloo")
+    g = np.random.default_rng(7)                      # the same full problem on every rank
+    n, h, r = 48, 6, 4
+    Q, K, V = (g.standard_normal((n, h)) for _ in range(3))
+    G1, G2 = g.standard_normal((h, r)), g.standard_normal((h, r))
+    O_full, d_full = orc.causal_polysketch_attention(Q, K, V, G1, G2)
+    lo, hi = rank * n // world, (rank + 1) * n // world
+    Qs, Ks, Vs = Q[lo:hi], K[lo:hi], V[lo:hi]
+    Vt = np.concatenate([Vs, np.ones((hi - lo, 1))], axis=1)
+    total = orc.polysketch_non_negative(Ks, G1, G2).T @ Vt          # this shard's end state
+    start = du.exclusive_prefix_over_ranks(torch.from_numpy(total)).numpy()
+    if rank == 0:
+        assert np.all(start == 0)
+    W = orc.causal_weights(Qs, Ks, G1, G2)                           # pairs inside the shard
+    N = W @ Vt + orc.polysketch_non_negative(Qs, G1, G2) @ start     # + everything before the shard
+    d = 1.0 + N[:, h]
+    np.testing.assert_allclose(d, d_full[lo:hi], rtol=1e-11)
+    np.testing.assert_allclose(N[:, :h] / d[:, None], O_full[lo:hi], rtol=1e-10, atol=1e-12)
+    du.shutdown()
+    print("rank", rank, "ok")
+""") % ROOT
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
@@ -42,12 +75,21 @@ def _free_port():
 
 
 def test_two_gloo_ranks(tmp_path):
+    _run_ranks(tmp_path, WORKER, 2)
+
+
+def test_sequence_shards_exchange_their_end_states(tmp_path):
+    _run_ranks(tmp_path, SEQ_WORKER, 2)
+    _run_ranks(tmp_path, SEQ_WORKER, 3)
+
+
+def _run_ranks(tmp_path, source, world):
     script = tmp_path / "worker.py"
-    script.write_text(WORKER)
+    script.write_text(source)
     port = _free_port()
     procs = []
-    for rank in range(2):
-        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", LOCAL_RANK=str(rank),
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
                    MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
         procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
                                       stderr=subprocess.STDOUT, text=True))
