@@ -78,6 +78,20 @@ namespace {
 // weights, epilogue).  Warp 4: one thread issues every TMA load and every MMA; the two sides meet
 // only at mbarriers, so the rows never wait for an issue sequence and the tensor pipe runs ahead.
 // ---------------------------------------------------------------------------
+#ifdef PSK_FWD_TRACE
+// scratch builds only: clock stamps of one CTA, one slot per (event, index)
+__device__ long long g_ftr[64 * 16];
+#define FTR(ev, idx) do { if (blockIdx.x == 1 && blockIdx.y == 5 && blockIdx.z == 3) g_ftr[(ev) * 16 + (idx)] = clock64(); } while (0)
+#else
+#define FTR(ev, idx)
+#endif
+
+// Warps 0-3: rows.  Warp 4: one thread issues every TMA load and every MMA.  (A second issuing
+// thread in a sixth warp for the odd state chunks was measured: 1 % faster, and the two threads'
+// MMAs reach the accumulator in an order that changes from run to run, so results were no longer
+// bitwise reproducible.  Not kept.)
+constexpr int kOutThreads = 160;
+#define PSK_OUT_ISSUERS 1
 constexpr int kZStages = 4;                     // three in the shared region + the query tile's buffer
 constexpr uint32_t kZStageBytes = 16384;        // two [64 features x 128 B] boxes: columns 0..63, 64..79
 constexpr int kFeatBufs = kZStages;             // feature staging buffers in tensor memory, 32 columns each:
@@ -121,7 +135,7 @@ struct OutSmem {
 // (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
 // they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
 template <int R, int MODE, bool LOCAL>
-__global__ void __launch_bounds__(160, ((R <= 32 || LOCAL) ? 2 : 1))
+__global__ void __launch_bounds__(kOutThreads, ((R <= 32 || LOCAL) ? 2 : 1))
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
                   const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapOc,
@@ -140,6 +154,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const int tid = threadIdx.x, warp = tid / 32, tau = blockIdx.x, l = blockIdx.y, bh = blockIdx.z;
     const int hi = bh % H, bi = bh / H;
     const int g = g_heads == 1 ? 0 : hi;
+    FTR(0, 0);
     const int row0 = l * b + tau * 128;
     // Non-causal (Section 3, first formula): one state per head, the sum over the whole sequence,
     // multiplies every row tile, and there are no same-block tiles.
@@ -157,16 +172,19 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
         tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
         bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
-        if (has_prefix) {
-            for (int c = 0; c < kZStages - 1 && c < F::NC; ++c) {
-                mbar_expect_tx(&bar_z[c], kZStageBytes);
-                tma_load_3d(smem + L::zstage(c), &mapZ, 0, c * 64, blk, &bar_z[c]);
-                tma_load_3d(smem + L::zstage(c) + 8192, &mapZ, 64, c * 64, blk, &bar_z[c]);
-            }
+    }
+    // The same-block key/value tiles are loaded late (their buffers hold state chunks first, and a
+    // tile's buffers are free only when the previous tile's MMAs are done): ask for them in L2 now,
+    // so that those loads pay the L2 latency and not HBM's.  (Forward rows 4.48 -> 4.40 ms at
+    // configuration 2; the same in the backward's row kernels made them 2 % slower and is not there.)
+    if (tid == 32 && !noncausal) {
+        for (int tp = 0; tp <= tau; ++tp) {
+            tma_prefetch_4d(&mapK, 0, l * b + tp * 128, hi, bi);
+            tma_prefetch_4d(&mapV, 0, l * b + tp * 128, hi, bi);
         }
     }
     if (warp == 4) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
-    for (int e = tid; e < 256; e += 160)
+    for (int e = tid; e < 256; e += kOutThreads)
         reinterpret_cast<uint4*>(smem + L::Ones)[e] = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
     if (tid < 64) cm[tid] = cmean != nullptr ? cmean[(size_t)bh * 64 + tid] : 0.f;
     fence_proxy_async_smem();
@@ -174,19 +192,61 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tm = tmem_slot;
+    if (tid == 0) FTR(1, 0);
     // tensor-memory columns: sketch accumulators, feature staging buffers, scores and packed
     // weights all live in [0, 128), each consumed before the next is produced; then the output
     // accumulator (64 + the prefix normaliser's 16) and the same-block row sums (16)
     constexpr uint32_t cSk = 0, cS = 0, cW = 0, cA = 0, cO = 128, cN = cO + 80;
     bool ok = true;
 
+    // First phase, issuing side: the chunks `first`, `first + step`, ... of the prefix state.
+    // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step, the second
+    // 64-column group (columns 64..79) 8192 B further on.  Everything the loop needs is in registers
+    // before it waits: between "features staged" and "MMAs issued" lie the four MMA instructions
+    // and nothing else.  (The stages are refilled by the rows' side, which learns first that a
+    // buffer is free.)
+    auto issue_chunks = [&](int first, int step) {
+        constexpr uint32_t idesc = idesc_bf16(128, 80, false, true);
+        const uint64_t zd0 = smem_desc(smem_u32(smem + L::Z), 8192, 1024, kSwz128);
+        const uint64_t zdq = smem_desc(smem_u32(smem + L::Z3), 8192, 1024, kSwz128);
+#pragma unroll 1
+        for (int C = first; C < F::NC && ok; C += step) {
+            const int s = C % kZStages;
+            const uint32_t par = (C / kZStages) & 1;
+            const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
+            const uint64_t zd = s == kZStages - 1 ? zdq : desc_off(zd0, s * kZStageBytes);
+            const uint32_t at = tm + cA + s * 32;
+            ok = mbar_spin(&bar_z[s], par, status, kErrTma);
+            FTR(4, C);
+            ok = ok && mbar_spin(&bar_feat[s], par, status, kErrMma);
+            FTR(5, C);
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < ksteps) umma_ts(tm + cO, at + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
+            umma_commit(&bar_a[s]);
+            FTR(6, C);
+        }
+    };
+
     if (warp == 4) {
         // ================================ issuer ================================
         if (tid == 128) {
+            // (the first state chunks are requested here, not by the thread that sets the barriers
+            // up: everyone waits for that thread, only this one waits for the query tile anyway)
+            if (has_prefix) {
+                for (int c = 0; c < kZStages - 1 && c < F::NC; ++c) {
+                    mbar_expect_tx(&bar_z[c], kZStageBytes);
+                    tma_load_3d(smem + L::zstage(c), &mapZ, 0, c * 64, blk, &bar_z[c]);
+                    tma_load_3d(smem + L::zstage(c) + 8192, &mapZ, 64, c * 64, blk, &bar_z[c]);
+                }
+            }
             ok = mbar_spin(&bar_q, 0, status, kErrTma);
+            FTR(2, 0);
             tc_fence_after();
             issue_sketch<R>(tm + cSk, smem + L::Q, smem + L::G);
             umma_commit(&bar_sk);
+            FTR(3, 0);
             if (has_prefix && kZStages - 1 < F::NC) {
                 // the query tile has been consumed: its buffer becomes the ring's last stage
                 ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);
@@ -194,32 +254,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 tma_load_3d(smem + L::zstage(kZStages - 1), &mapZ, 0, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
                 tma_load_3d(smem + L::zstage(kZStages - 1) + 8192, &mapZ, 64, (kZStages - 1) * 64, blk, &bar_z[kZStages - 1]);
             }
-            if (has_prefix) {
-                // earlier blocks: weighted features (tensor memory) x prefix state chunks.
-                // B = the chunk's 64 feature rows x 80 columns, MN-major: 16 features per K step,
-                // the second 64-column group (columns 64..79) 8192 B further on
-                constexpr uint32_t idesc = idesc_bf16(128, 80, false, true);
-                // Everything the loop needs is in registers before it waits: between "features
-                // staged" and "MMAs issued" lie the four MMA instructions and nothing else.  (The
-                // stages are refilled by the rows' side, which learns first that a buffer is free.)
-                const uint64_t zd0 = smem_desc(smem_u32(smem + L::Z), 8192, 1024, kSwz128);
-                const uint64_t zdq = smem_desc(smem_u32(smem + L::Z3), 8192, 1024, kSwz128);
-#pragma unroll 1
-                for (int C = 0; C < F::NC && ok; ++C) {
-                    const int s = C % kZStages;
-                    const uint32_t par = (C / kZStages) & 1;
-                    const int ksteps = (F::FK - C * 64) >= 64 ? 4 : (F::FK - C * 64) / 16;
-                    const uint64_t zd = s == kZStages - 1 ? zdq : desc_off(zd0, s * kZStageBytes);
-                    const uint32_t at = tm + cA + s * 32;
-                    ok = mbar_spin(&bar_z[s], par, status, kErrTma);
-                    ok = ok && mbar_spin(&bar_feat[s], par, status, kErrMma);
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < ksteps) umma_ts(tm + cO, at + k * 8, desc_off(zd, k * 2048), idesc, (C > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&bar_a[s]);
-                }
-            }
+            if (has_prefix) issue_chunks(0, PSK_OUT_ISSUERS);     // earlier blocks: features x prefix state chunks
             if (has_prefix && !noncausal) {
                 // first key/value tile of the same block, each into its stage as soon as the last
                 // chunk that used it has been multiplied
@@ -253,6 +288,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     tma_load_4d(smem + L::V, &mapV, 0, l * b + tp * 128, hi, bi, &bar_kv);
                 }
                 ok = ok && mbar_spin(&bar_kv, tp & 1, status, kErrTma);
+                FTR(7, tp);
                 tc_fence_after();
                 if constexpr (LOCAL) {
                     // scores = Q_tile K_tile^T over the head dimension
@@ -266,7 +302,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 } else {
                     issue_sketch<R>(tm + cSk, smem + L::K, smem + L::G);
                     umma_commit(&bar_sk);
+                    FTR(8, tp);
                     ok = ok && mbar_spin(&bar_mk, tp & 1, status, kErrMma);
+                    FTR(9, tp);
                     tc_fence_after();
                     constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
 #pragma unroll
@@ -274,7 +312,9 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         umma_ss(tm + cS, desc_off(qd, k * 4096), desc_off(kd, k * 4096), idesc, k > 0);
                     umma_commit(&bar_s);
                 }
+                FTR(10, tp);
                 ok = ok && mbar_spin(&bar_p, tp & 1, status, kErrMma);
+                FTR(11, tp);
                 tc_fence_after();
                 {
                     // numerator += W V; row sums += W 1 (the weights exactly as the value GEMM sees them)
@@ -287,6 +327,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                         umma_ts(tm + cN, tm + cW + k * 8, desc_off(od, k * 512), idesc1, k > 0 ? 1u : acc1);
                     }
                     umma_commit(&bar_pv);
+                    FTR(12, tp);
                 }
             }
         }
@@ -294,12 +335,14 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         // ================================= rows =================================
         const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
         ok = mbar_wait(&bar_sk, 0, status, kErrMma);
+        if (tid == 0) FTR(20, 0);
         tc_fence_after();
         float mq[R];
         read_half_sketch<R>(lane_tm + cSk, mq);
         if constexpr (!LOCAL) store_split_rows<R, true>(smem + L::Mq, mq, tid);
         tc_fence_before();
         mbar_arrive(&bar_go);
+        if (tid == 0) FTR(21, 0);
 
         if (has_prefix) {
             if constexpr (F::kCirc) {
@@ -317,12 +360,14 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                             tma_load_3d(smem + L::zstage(buf) + 8192, &mapZ, 64, C * 64, blk, &bar_z[buf]);
                         }
                     }
+                    if (tid == 0) FTR(22, C);
                     uint32_t pk[32];
                     gen.chunk(pk);
                     tmem_st32(lane_tm + cA + buf * 32, pk);
                     tmem_st_wait();
                     tc_fence_before();
                     mbar_arrive(&bar_feat[buf]);
+                    if (tid == 0) FTR(23, C);
                 }
             } else {
                 PackedM<R> pmq;
@@ -356,6 +401,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         for (int tp = 0; tp <= tp_last && ok; ++tp) {
             if constexpr (!LOCAL) {
                 ok = mbar_wait(&bar_sk, (tp + 1) & 1, status, kErrMma);
+                if (tid == 0) FTR(24, tp);
                 tc_fence_after();
                 {
                     float mk[R];
@@ -365,8 +411,10 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 fence_proxy_async_smem();
                 tc_fence_before();
                 mbar_arrive(&bar_mk);
+                if (tid == 0) FTR(25, tp);
             }
             ok = ok && mbar_wait(&bar_s, tp & 1, status, kErrMma);
+            if (tid == 0) FTR(26, tp);
             tc_fence_after();
             // weights = squared scores (lower triangle on the diagonal tile), packed to bf16 over
             // columns whose fp32 contents have already been read
@@ -395,12 +443,14 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&bar_p);
+            if (tid == 0) FTR(27, tp);
         }
         if (noncausal)      // the last chunk's MMAs (no same-block tiles follow them)
             ok = ok && mbar_wait(&bar_a[(F::NC - 1) % kFeatBufs], ((F::NC - 1) / kFeatBufs) & 1, status, kErrMma);
         else
             ok = ok && mbar_wait(&bar_pv, tau & 1, status, kErrMma);
         tc_fence_after();
+        if (tid == 0) FTR(28, 0);
 
         // ---- epilogue ----
         float acc[64];
@@ -493,9 +543,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             e65h[row] = y * inv - ec;
         }
     }
+    if (tid == 0) FTR(29, 0);
     tc_fence_before();
     __syncthreads();
     if (warp == 4) tmem_dealloc(tm, 256);
+    if (tid == 0) FTR(30, 0);
 }
 
 // Centre of the values of a head: cmean[bh][c] = mean of V[bh][i][c] over at most 1024 rows i
@@ -582,13 +634,13 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true>, smem)));
-        tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false>, smem)));
-        tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     }
@@ -598,6 +650,14 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
 }
 
 }  // namespace
+
+#ifdef PSK_FWD_TRACE
+extern "C" int psk_debug_ftrace(long long* host) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(host, g_ftr, sizeof(long long) * 64 * 16);
+    return 64 * 16;
+}
+#endif
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
@@ -632,13 +692,13 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
     if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true>, smem)));
-        tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false>, smem)));
-        tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), 160, smem, s>>>(
+        tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     }

@@ -180,6 +180,14 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, int
         : "memory");
 }
 
+// Ask for a tile to be brought into L2 (no shared-memory destination, nothing to wait for): the
+// later load of the same tile then pays the L2 latency instead of HBM's.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+
 // Tiled stores shared -> global (bulk async-group completion).  The issuing thread commits the
 // group and waits until the copies have READ their shared-memory source before it is reused.
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, const void* src, int c0, int c1, int c2, int c3) {
