@@ -283,6 +283,8 @@ def main():
     ap.add_argument("--others", default="c1,c3,c4",
                     help="other configurations timed briefly after the headline one (N = 1 only); '' for none")
     ap.add_argument("--other-steps", type=int, default=5)
+    ap.add_argument("--seq-segments", type=int, default=0,
+                    help="runs a head's blocks are cut into for the state scan (0: the library chooses)")
     ap.add_argument("--no-keep-states", action="store_true",
                     help="let the backward rebuild the prefix states instead of reading the forward's")
     args = ap.parse_args()
@@ -315,7 +317,8 @@ def main():
     keep = bool(flags)
     if args.local_exact:
         flags |= psk.FLAG_LOCAL_EXACT
-    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path, flags)
+    segs = args.seq_segments
+    shp = psk.binding.make_shape(Q, G1, w.r, w.b, w.p, path, flags, segs)
     ws_bytes = max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True) if w.backward else 0)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     O = torch.empty_like(Q)
@@ -324,10 +327,10 @@ def main():
     launches = [0]
 
     def step():
-        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den, flags)
+        psk.causal_attn_fwd(Q, K, V, G1, G2, w.b, w.p, path, ws, O, den, flags, segs)
         n = psk.last_launch_count()
         if w.backward:
-            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, path, ws, grads, flags)
+            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, w.b, w.p, path, ws, grads, flags, segs)
             n += psk.last_launch_count()
         launches[0] += n
 
@@ -396,10 +399,10 @@ def main():
                 if ev_out[k] is not None:
                     s_comp.wait_event(ev_out[k])             # step i-2's results have left this output set
                 d = dev_in[k]
-                psk.causal_attn_fwd(d["Q"], d["K"], d["V"], G1, G2, w.b, w.p, path, ws, dev_out[k][0], dev_den[k], flags)
+                psk.causal_attn_fwd(d["Q"], d["K"], d["V"], G1, G2, w.b, w.p, path, ws, dev_out[k][0], dev_den[k], flags, segs)
                 if w.backward:
                     psk.causal_attn_bwd(d["Q"], d["K"], d["V"], G1, G2, dev_out[k][0], dev_den[k], d["dO"], w.b, w.p,
-                                        path, ws, tuple(dev_out[k][1:]), flags)
+                                        path, ws, tuple(dev_out[k][1:]), flags, segs)
                 ev_comp[k] = torch.cuda.Event(); ev_comp[k].record(s_comp)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(ev_comp[k])
@@ -494,7 +497,7 @@ def main():
         "config": {"workload": w.name, "B": w.B, "H": w.H, "n": w.n, "h": w.h, "r": w.r, "p": w.p, "b": w.b,
                    "passes": "fwd+bwd" if w.backward else "fwd", "path": args.path,
                    "variant": "local_exact" if args.local_exact else "polysketch",
-                   "keep_states": keep,
+                   "keep_states": keep, "seq_segments": segs,
                    "l2": "inputs larger than L2 (no flush)", "per_gpu_batch": w.B},
         "nominal_tflops": nominal_tflops, "executed_tflops": executed_tflops,
         "frac_bf16_peak": {"burst": nominal_tflops / world / pk["bf16_burst"],
