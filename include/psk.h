@@ -36,8 +36,9 @@
  *     PSK_ERR_SHAPE.
  *   - Also p = 2 (Algorithm 1 with p/2 = 1): no sketch, m(x) = x, phi'(x) = x (x) x with
  *     h^2 entries, i.e. exact degree-2 polynomial attention with weights (q_i . k_j)^2.
- *     Set r = h; G1 and G2 are not read and may be null.  Served by the CUDA-core
- *     kernels for either storage type (PSK_PATH_TENSOR_CORES: PSK_ERR_UNSUPPORTED).
+ *     Set r = h; G1 and G2 are not read and may be null.  bf16 storage runs on the tensor
+ *     cores (the same kernels, with the rows taken as their own half sketch), fp32 storage on
+ *     the CUDA cores.
  *   - Also p = 8 (one more level of Algorithm 1's recursion): two independent degree-2
  *     sketches M1 = sqrt(1/r)[(x Ga1)*(x Ga2)], M2 = sqrt(1/r)[(x Gb1)*(x Gb2)] combined as
  *     m(x) = sqrt(1/r)[(M1 Gc1)*(M2 Gc2)] with Gc1, Gc2 of r x r; phi'(x) = m (x) m as for p = 4,

@@ -55,6 +55,8 @@ int make_dims(const psk_shape* sh, Dims* d) {
     d->B = sh->B; d->H = sh->H; d->n = sh->n; d->h = sh->h; d->r = sh->r; d->b = sh->b;
     d->t = sh->n / sh->b;
     d->sb = sh->stride_b; d->sh = sh->stride_h; d->sn = sh->stride_n;
+    d->xsb = d->sb; d->xsh = d->sh; d->xsn = d->sn;
+    d->sketch_linear = sh->p == 2;          // degree 2: the rows are their own half sketch
     d->g_heads = sh->g_heads;
     d->bf16 = sh->dtype == PSK_BF16;
     d->keep_states = (sh->flags & PSK_FLAG_KEEP_STATES) != 0;

@@ -21,6 +21,10 @@ struct Dims {
     bool local;                       // PSK_FLAG_LOCAL_EXACT
     bool noncausal;                   // PSK_FLAG_NONCAUSAL: no lt(), one global state per head
     int seq_segments;                 // runs a head's sequence is cut into for the state scan; 0 = library's choice
+    // tensor-core kernels: the tensors they "sketch" already hold the half sketch (tc_common.cuh,
+    // read_half_sketch); `xsb, xsh, xsn` are the strides of those tensors and of their gradients
+    bool sketch_linear = false;
+    int64_t xsb = 0, xsh = 0, xsn = 0;
     // learnable sketch (Algorithm 2): the half sketch comes from two dense networks instead of G1, G2
     bool learned = false;
     const float* lparams = nullptr;   // packed parameters of both networks (psk_learned.cu)

@@ -134,7 +134,8 @@ struct OutSmem {
 // LOCAL (Section 3.2): the same-block scores are (q_i . k_j)^2 from the raw query and key tiles
 // (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
 // they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
-template <int R, int MODE, bool LOCAL>
+// LIN: the rows hold a given half sketch (tc_common.cuh, read_half_sketch).
+template <int R, int MODE, bool LOCAL, bool LIN>
 __global__ void __launch_bounds__(kOutThreads, ((R <= 32 || LOCAL) ? 2 : 1))
 tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
@@ -143,6 +144,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                   const float* __restrict__ cmean, int64_t sb, int64_t sh, int64_t sn,
                   float* __restrict__ denom, const bf16* __restrict__ dO,
                   float* __restrict__ y65, float* __restrict__ e65h, int keep_oc, int noncausal, int* status) {
+    constexpr bool lin = LIN;
     using F = Feat<R>;
     using L = OutSmem<R, LOCAL>;
     extern __shared__ uint8_t smem_raw[];
@@ -338,7 +340,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         if (tid == 0) FTR(20, 0);
         tc_fence_after();
         float mq[R];
-        read_half_sketch<R>(lane_tm + cSk, mq);
+        read_half_sketch<R>(lane_tm + cSk, mq, 1.f, lin != 0);
         if constexpr (!LOCAL) store_split_rows<R, true>(smem + L::Mq, mq, tid);
         tc_fence_before();
         mbar_arrive(&bar_go);
@@ -405,7 +407,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 tc_fence_after();
                 {
                     float mk[R];
-                    read_half_sketch<R>(lane_tm + cSk, mk);
+                    read_half_sketch<R>(lane_tm + cSk, mk, 1.f, lin != 0);
                     store_split_rows<R, false>(smem + L::Mk, mk, tid);
                 }
                 fence_proxy_async_smem();
@@ -589,13 +591,16 @@ tc_vmean_kernel(const bf16* __restrict__ V, int H, int n, int64_t sb, int64_t sh
 
 // Image of [G1 | G2]^T (set g of the sketch matrices, each [64 x r] row-major) in the layout the
 // sketch GEMM reads from shared memory: row nn < 2r = sketch column, 64 head dimensions, swizzled.
+// (lin: "G1" = I for r = 64, [I; I] padded with zero rows for r <= 32, "G2" = 0: the sketch GEMM then
+// returns the row itself, or the sum of its [hi | lo] halves, see read_half_sketch)
 __global__ void __launch_bounds__(128)
-tc_gimage_kernel(const bf16* __restrict__ G1, const bf16* __restrict__ G2, int r, uint8_t* __restrict__ gimg) {
+tc_gimage_kernel(const bf16* __restrict__ G1, const bf16* __restrict__ G2, int r, int lin, uint8_t* __restrict__ gimg) {
     const int g = blockIdx.x;
     uint8_t* img = gimg + (size_t)g * 2 * r * 128;
     for (int e = threadIdx.x; e < 2 * r * 64; e += 128) {
         const int nn = e / 64, k = e % 64;
-        const bf16 v = (nn < r ? G1 : G2)[(size_t)g * 64 * r + k * r + (nn % r)];
+        const bf16 v = lin ? __float2bfloat16_rn((nn < r && (k == nn || (r <= 32 && k == r + nn))) ? 1.f : 0.f)
+                           : (nn < r ? G1 : G2)[(size_t)g * 64 * r + k * r + (nn % r)];
         *reinterpret_cast<bf16*>(img + swz128_offset(nn, k / 8) + (k % 8) * 2) = v;
     }
 }
@@ -612,7 +617,7 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     bf16* Z = reinterpret_cast<bf16*>(ws + w.Z);
     bf16* Oc = d.keep_states ? reinterpret_cast<bf16*>(ws + w.Oc) : nullptr;
     CUtensorMap mQ, mK, mV, mZ, mO, mOc;
-    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_states(&mZ, Z, Feat<R>::FP, (int64_t)d.BH() * (d.noncausal ? 1 : d.t)) ||
         !tc_map_rows(&mO, O, d.B, d.H, d.n, d.sb, d.sh, d.sn))
@@ -633,14 +638,20 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     prof_begin("tc_fwd_out_kernel", s);
     if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
-        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true>, smem)));
-        tc_fwd_out_kernel<R, 0, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true, false>, smem)));
+        tc_fwd_out_kernel<R, 0, true, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
+    } else if (d.sketch_linear) {
+        constexpr size_t smem = OutSmem<R, false>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false, true>, smem)));
+        tc_fwd_out_kernel<R, 0, false, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
-        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false>, smem)));
-        tc_fwd_out_kernel<R, 0, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false, false>, smem)));
+        tc_fwd_out_kernel<R, 0, false, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     }
@@ -661,7 +672,9 @@ extern "C" int psk_debug_ftrace(long long* host) {
 
 bool tc_supported(const Dims& d, bool backward) {
     (void)backward;
-    return d.bf16 && d.p == 4 && encoder() != nullptr;      // (p = 2: CUDA-core kernels)
+    // p = 2 (the rows are their own half sketch, r = h) runs the same kernels in "linear" mode;
+    // p = 8: CUDA-core kernels (or the tensor cores through the given-half-sketch route of psk_api.cu)
+    return d.bf16 && (d.p == 4 || d.p == 2 || d.sketch_linear) && encoder() != nullptr;
 }
 
 size_t tc_workspace_bytes(const Dims& d, bool backward) {
@@ -691,14 +704,20 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
     prof_begin("tc_bwd_recompute_kernel", s);
     if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
-        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true>, smem)));
-        tc_fwd_out_kernel<R, 1, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true, false>, smem)));
+        tc_fwd_out_kernel<R, 1, true, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
+    } else if (d.sketch_linear) {
+        constexpr size_t smem = OutSmem<R, false>::total + 1024;
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false, true>, smem)));
+        tc_fwd_out_kernel<R, 1, false, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
-        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false>, smem)));
-        tc_fwd_out_kernel<R, 1, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+        PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false, false>, smem)));
+        tc_fwd_out_kernel<R, 1, false, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
             mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     }
@@ -720,7 +739,7 @@ cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap
 
 cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gimg, cudaStream_t s, int* launches) {
     prof_begin("tc_gimage_kernel", s);
-    tc_gimage_kernel<<<d.g_heads, 128, 0, s>>>((const bf16*)G1, (const bf16*)G2, d.r, gimg);
+    tc_gimage_kernel<<<d.g_heads, 128, 0, s>>>((const bf16*)G1, (const bf16*)G2, d.r, d.sketch_linear ? 1 : 0, gimg);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();

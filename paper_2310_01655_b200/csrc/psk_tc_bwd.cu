@@ -146,7 +146,9 @@ __device__ __forceinline__ void issue_scores(uint32_t d_tmem, uint32_t own, uint
 // dL/dx_ij = 4 x_ij^3 dW_ij replaces ds_ij, and it multiplies the other side's raw rows straight
 // into a dX accumulator that the sketch's backward (phase D) adds to: no half sketch of the other
 // tile, no split operands, no dM from the tiles.
-template <int R, bool QSIDE, bool LOCAL>
+// LIN: the rows hold a given half sketch (tc_common.cuh, read_half_sketch); a template parameter, not
+// an argument: the key side sits at the register limit, and the flag as an argument cost it 4 %.
+template <int R, bool QSIDE, bool LOCAL, bool LIN>
 __global__ void __launch_bounds__(128, ((R <= 32 || (LOCAL && QSIDE)) ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
@@ -155,6 +157,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                    int g_heads, int H, int n, int b, int t,
                    const float* __restrict__ y65g, const float* __restrict__ e65h, const float* __restrict__ denom,
                    int noncausal, int* status) {
+    constexpr bool lin = LIN;
     using F = Feat<R>;
     using L = BwdSmem<R, LOCAL, QSIDE>;
     constexpr int kStages = L::kSt;
@@ -255,7 +258,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     ++mma_uses;
     tc_fence_after();
     float m[R], dm[R];
-    read_half_sketch<R>(lane_tm + cSk, m);
+    read_half_sketch<R>(lane_tm + cSk, m, 1.f, lin != 0);
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
@@ -492,7 +495,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         ++oth_uses;
         if constexpr (!LOCAL) {
             float mo[R];
-            read_half_sketch<R>(lane_tm + cSk, mo);
+            read_half_sketch<R>(lane_tm + cSk, mo, 1.f, lin != 0);
             store_hilo_tiles<R>(smem + L::Moth, mo, tid);
         }
         const bool diag = (tp == tau);
@@ -616,7 +619,8 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 
     // ---- phase D: through the sketch, dX = ((dM*A2) G1^T + (dM*A1) G2^T) / sqrt(R) ----
     if (ok) {
-        const float rs = rsqrtf((float)R);
+        // (a given half sketch has no 1/sqrt(R) of its own)
+        const float rs = lin ? 1.f : rsqrtf((float)R);
         // dM total = state part (registers) + tile part (tensor memory), scaled by 1/sqrt(R)
         if constexpr (LOCAL) {
 #pragma unroll
@@ -658,10 +662,11 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                u1[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a2[2 * j]),
-                                  dm[c0 + 2 * j + 1] * __uint_as_float(a2[2 * j + 1]));
-                u2[j] = pack_bf16(dm[c0 + 2 * j] * __uint_as_float(a1[2 * j]),
-                                  dm[c0 + 2 * j + 1] * __uint_as_float(a1[2 * j + 1]));
+                // given half sketch: dX = dM "G1"^T with that identity-like matrix, and nothing through "G2"
+                u1[j] = pack_bf16(dm[c0 + 2 * j] * (lin ? 1.f : __uint_as_float(a2[2 * j])),
+                                  dm[c0 + 2 * j + 1] * (lin ? 1.f : __uint_as_float(a2[2 * j + 1])));
+                u2[j] = pack_bf16(lin ? 0.f : dm[c0 + 2 * j] * __uint_as_float(a1[2 * j]),
+                                  lin ? 0.f : dm[c0 + 2 * j + 1] * __uint_as_float(a1[2 * j + 1]));
             }
             tmem_st8(lane_tm + cU1 + c0 / 2, u1);
             tmem_st8(lane_tm + cU2 + c0 / 2, u2);
@@ -744,11 +749,11 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     if (!d.keep_states) PSK_TRY(tc_vmean(d, V, cmean, s, launches));
     CUtensorMap mQ, mK, mV, mG, mZ, mR, mdQ, mdK, mdV;
     const int64_t nblk = (int64_t)d.BH() * (d.noncausal ? 1 : d.t);
-    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+    if (!tc_map_rows(&mQ, Q, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) || !tc_map_rows(&mK, K, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) ||
         !tc_map_rows(&mV, V, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_rows(&mG, dO, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
         !tc_map_states(&mZ, Z, Feat<R>::FP, nblk) || !tc_map_states(&mR, Rs, Feat<R>::FP, nblk) ||
-        !tc_map_rows(&mdQ, dQ, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mdK, dK, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+        !tc_map_rows(&mdQ, dQ, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) || !tc_map_rows(&mdK, dK, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) ||
         !tc_map_rows(&mdV, dV, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
@@ -768,15 +773,16 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, y65, e65h, status, s, launches));
     }
     const dim3 grid(d.b / 128, d.t, d.BH());
-    auto rows = [&](auto local_c) -> cudaError_t {
+    auto rows = [&](auto local_c, auto lin_c) -> cudaError_t {
         constexpr bool LOCAL = decltype(local_c)::value;
+        constexpr bool LIN = decltype(lin_c)::value;
         constexpr size_t smem = BwdSmem<R, LOCAL, true>::total + 1024, smem_k = BwdSmem<R, LOCAL, false>::total + 1024;
-        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, true, LOCAL>, smem)));
-        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, false, LOCAL>, smem_k)));
+        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, true, LOCAL, LIN>, smem)));
+        PSK_TRY((set_smem(tc_bwd_rows_kernel<R, false, LOCAL, LIN>, smem_k)));
         // query side first: it needs only the prefix states, and the row scalars just written are
         // still in L2; the suffix states (5 GB through L2) come after it
         prof_begin("tc_bwd_q_kernel", s);
-        tc_bwd_rows_kernel<R, true, LOCAL><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
+        tc_bwd_rows_kernel<R, true, LOCAL, LIN><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
                                                                    d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
@@ -784,13 +790,14 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // suffix states: phi(q_i) / d_i against [dO_i | y65_i]
         PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, tot, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
-        tc_bwd_rows_kernel<R, false, LOCAL><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
+        tc_bwd_rows_kernel<R, false, LOCAL, LIN><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
                                                                     d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
         return cudaGetLastError();
     };
-    return d.local ? rows(std::true_type{}) : rows(std::false_type{});
+    if (d.sketch_linear) return rows(std::false_type{}, std::true_type{});      // (never with exact same-block weights)
+    return d.local ? rows(std::true_type{}, std::false_type{}) : rows(std::false_type{}, std::false_type{});
 }
 
 }  // namespace

@@ -93,7 +93,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
                 const float* __restrict__ y65, const float* __restrict__ fscale, const float* __restrict__ cmean,
                 int center_mode, int reverse, int nseg_arg, int mode_arg, int use_init, float* __restrict__ tot,
-                bf16* __restrict__ S, int* status) {
+                bf16* __restrict__ S, int lin, int* status) {
     using F = Feat<R>;
     using L = StateSmem<R, NWG>;
     extern __shared__ uint8_t smem_raw[];
@@ -359,7 +359,7 @@ tc_state_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant_
                 // features m_a m_b / d: both factors carry 1 / sqrt(d) (d requested a token tile ago)
                 const float sc = rsqrtf(d_next);
                 if (fscale != nullptr && j + 1 < NJs) d_next = fscale[(size_t)bh * n + tile_of(j + 1) * 128 + wt];
-                read_half_sketch<R>(lane_tm, m, sc);
+                read_half_sketch<R>(lane_tm, m, sc, lin != 0);
                 if constexpr (F::kCirc) gen.init(m); else pack_half_sketch<R>(m, pm);
             }
             tc_fence_before();
@@ -489,12 +489,12 @@ cudaError_t launch_state_group(const Dims& d, const CUtensorMap& mX, const CUten
         PSK_TRY((set_smem(tc_state_kernel<R, T0, TN, NWG, false>, smem)));
         tc_state_kernel<R, T0, TN, NWG, false><<<dim3(d.BH(), 1), 128 * (NWG + 1) + 64, smem, s>>>(
             mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, a.y65, a.fscale, a.cmean, a.center_mode, a.reverse ? 1 : 0, 1,
-            kModePrefix, 0, a.tot, a.S, status);
+            kModePrefix, 0, a.tot, a.S, d.sketch_linear ? 1 : 0, status);
     } else {
         PSK_TRY((set_smem(tc_state_kernel<R, T0, TN, NWG, true>, smem)));
         tc_state_kernel<R, T0, TN, NWG, true><<<dim3(d.BH(), a.segs_launched), 128 * (NWG + 1) + 64, smem, s>>>(
             mX, mY, gimg, d.g_heads, d.H, d.n, d.b, d.t, a.y65, a.fscale, a.cmean, a.center_mode, a.reverse ? 1 : 0, a.nseg,
-            a.mode, a.use_init ? 1 : 0, a.tot, a.S, status);
+            a.mode, a.use_init ? 1 : 0, a.tot, a.S, d.sketch_linear ? 1 : 0, status);
     }
     prof_end(s);
     ++*launches;

@@ -32,6 +32,7 @@ cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap
                          const bf16* dO, float* y65, float* e65h, int* status, cudaStream_t s, int* launches);
 // gimg[g] = [G1 | G2]^T of sketch-matrix set g as the shared-memory image of the sketch GEMM's B operand
 // (2r rows x 128 B, K-major, 128-byte swizzle): the kernels fetch it with one bulk copy
+// (d.sketch_linear: the image of [I | 0] or [I; I | 0] instead, G1 and G2 are not read)
 cudaError_t tc_gimage(const Dims& d, const void* G1, const void* G2, uint8_t* gimg, cudaStream_t s, int* launches);
 // cmean[bh][c] = mean over the n rows of V[bh][:, c]  (deterministic reduction)
 cudaError_t tc_vmean(const Dims& d, const void* V, float* cmean, cudaStream_t s, int* launches);
@@ -105,9 +106,13 @@ __device__ __forceinline__ void issue_sketch(uint32_t d_tmem, const uint8_t* sX,
 
 // m[c] = A1[c] A2[c] / sqrt(R) from the sketch accumulator (this thread's lane).
 // (`scale`: an extra factor on every entry, folded into the constant)
+// `linear`: the half sketch is given, not formed here: the "rows to sketch" are the half sketch
+// itself (degree 2: m = x), or its two bf16 terms side by side ([hi | lo]), and the first half of the
+// sketch GEMM against an identity-like matrix ([I], [I; I]) just carries it into tensor memory in
+// fp32: m[c] = A1[c].
 template <int R>
-__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R], float scale = 1.f) {
-    const float rs = rsqrtf((float)R) * scale;
+__device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[R], float scale = 1.f, bool linear = false) {
+    const float rs = linear ? scale : rsqrtf((float)R) * scale;
 #pragma unroll
     for (int c0 = 0; c0 < R; c0 += 16) {
         uint32_t a1[16], a2[16];
@@ -115,7 +120,7 @@ __device__ __forceinline__ void read_half_sketch(uint32_t lane_tmem, float (&m)[
         tmem_ld16(lane_tmem + R + c0, a2);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) m[c0 + j] = __uint_as_float(a1[j]) * __uint_as_float(a2[j]) * rs;
+        for (int j = 0; j < 16; ++j) m[c0 + j] = __uint_as_float(a1[j]) * (linear ? 1.f : __uint_as_float(a2[j])) * rs;
     }
 }
 
