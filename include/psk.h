@@ -43,8 +43,10 @@
  *     sketches M1 = sqrt(1/r)[(x Ga1)*(x Ga2)], M2 = sqrt(1/r)[(x Gb1)*(x Gb2)] combined as
  *     m(x) = sqrt(1/r)[(M1 Gc1)*(M2 Gc2)] with Gc1, Gc2 of r x r; phi'(x) = m (x) m as for p = 4,
  *     so the weights approximate (q_i . k_j)^8.  G1 then holds [Ga1; Gb1; Gc1] and G2 holds
- *     [Ga2; Gb2; Gc2], each [g_heads, 2h + r, r] contiguous.  CUDA-core kernels only; not
- *     with PSK_FLAG_LOCAL_EXACT (PSK_ERR_UNSUPPORTED).
+ *     [Ga2; Gb2; Gc2], each [g_heads, 2h + r, r] contiguous.  Not with PSK_FLAG_LOCAL_EXACT
+ *     (PSK_ERR_UNSUPPORTED).  fp32 storage and r = 64: CUDA-core kernels.  bf16 storage with
+ *     r <= 32: the half sketches are formed by the CUDA-core sketch kernels and the attention on
+ *     them runs on the tensor cores (PSK_PATH_CUDA_CORES forces the CUDA-core kernels throughout).
  */
 #ifndef PSK_H_
 #define PSK_H_
@@ -196,9 +198,12 @@ int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void
  *            the batch, the heads and both uses of the networks, on Q and on K; accumulated with
  *            floating-point atomics, so its last bits are not reproducible from run to run)
  * The other arguments, the workspace rules and the error codes are those of psk_sketch,
- * psk_causal_attn_fwd and psk_causal_attn_bwd; `shape` needs p = 4, g_heads and path are ignored,
+ * psk_causal_attn_fwd and psk_causal_attn_bwd; `shape` needs p = 4, g_heads is ignored,
  * PSK_FLAG_LOCAL_EXACT is honoured (the paper's "learned + local" variant), PSK_FLAG_NONCAUSAL is
- * not supported here.  CUDA-core kernels (fp32 arithmetic) for either storage type; workspace size from
+ * not supported here.  The networks always run on the CUDA cores in fp32; the attention on their half
+ * sketches runs on the tensor cores for bf16 storage with r <= 32 and sketched same-block weights
+ * (`path` = PSK_PATH_CUDA_CORES forces the CUDA-core kernels, PSK_PATH_TENSOR_CORES refuses what the
+ * tensor-core route does not serve), else on the CUDA cores.  Workspace size from
  * psk_learned_workspace_bytes. */
 size_t psk_learned_param_count(int h, int r);
 size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward);

@@ -362,8 +362,8 @@ def unpack_learned_params(flat, h: int, r: int):
     return out[0], out[1]
 
 
-def _learned_shape(x, r, b, flags):
-    return make_shape(x, None, r, b, 4, PATH_CUDA_CORES, flags)
+def _learned_shape(x, r, b, flags, path=PATH_AUTO):
+    return make_shape(x, None, r, b, 4, path, flags)
 
 
 def learned_sketch(X, params, r, want_phi=False):
@@ -379,11 +379,11 @@ def learned_sketch(X, params, r, want_phi=False):
     return M, Phi
 
 
-def learned_attn_fwd(Q, K, V, params, r, b, flags=0, workspace=None):
+def learned_attn_fwd(Q, K, V, params, r, b, flags=0, workspace=None, path=PATH_AUTO):
     """psk_learned_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, params)
     _same_layout(Q, K, V)
-    shp = _learned_shape(Q, r, b, flags)
+    shp = _learned_shape(Q, r, b, flags, path)
     need = int(lib().psk_learned_workspace_bytes(byref(shp), 0))
     ws = workspace if workspace is not None else torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
     B, H, n, _ = Q.shape
@@ -396,11 +396,11 @@ def learned_attn_fwd(Q, K, V, params, r, b, flags=0, workspace=None):
     return O, den
 
 
-def learned_attn_bwd(Q, K, V, params, O, denom, dO, r, b, flags=0, workspace=None):
+def learned_attn_bwd(Q, K, V, params, O, denom, dO, r, b, flags=0, workspace=None, path=PATH_AUTO):
     """psk_learned_attn_bwd: returns (dQ, dK, dV, dparams [2, count] fp32)."""
     _require_cuda(Q, K, V, params, O, denom, dO)
     _same_layout(Q, K, V, O, dO)
-    shp = _learned_shape(Q, r, b, flags)
+    shp = _learned_shape(Q, r, b, flags, path)
     need = int(lib().psk_learned_workspace_bytes(byref(shp), 1))
     ws = workspace if workspace is not None else torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device)
     dQ, dK, dV = _empty_like(Q), _empty_like(Q), _empty_like(Q)

@@ -75,11 +75,19 @@ int make_dims(const psk_shape* sh, Dims* d) {
     return PSK_OK;
 }
 
-// 0 = CUDA cores, 1 = tensor cores, <0 = error
+// 0 = CUDA cores, 1 = tensor cores, 2 = tensor cores on half sketches formed by the CUDA-core sketch
+// kernels (degree 8, learnable sketch), <0 = error
 int pick_path(const psk_shape* sh, const Dims& d, bool backward) {
     if (sh->path == PSK_PATH_CUDA_CORES) return 0;
+    if (given_supported(d)) return 2;
+    if (d.p == 8 || d.learned) return sh->path == PSK_PATH_TENSOR_CORES ? PSK_ERR_UNSUPPORTED : 0;
     if (sh->path == PSK_PATH_TENSOR_CORES) return (d.bf16 && tc_supported(d, backward)) ? 1 : PSK_ERR_UNSUPPORTED;
     return (d.bf16 && tc_supported(d, backward)) ? 1 : 0;
+}
+
+size_t path_workspace(int path, const Dims& d, bool backward) {
+    return path == 2 ? given_workspace_bytes(d, backward)
+                     : (path == 1 ? tc_workspace_bytes(d, backward) : cc_workspace(d, backward).total);
 }
 
 }  // namespace
@@ -107,7 +115,7 @@ size_t psk_workspace_bytes(const psk_shape* shape, int for_backward) {
     if (make_dims(shape, &d) != PSK_OK) return 0;
     const int path = pick_path(shape, d, for_backward != 0);
     if (path < 0) return 0;
-    return path == 1 ? tc_workspace_bytes(d, for_backward != 0) : cc_workspace(d, for_backward != 0).total;
+    return path_workspace(path, d, for_backward != 0);
 }
 
 int psk_sketch(const psk_shape* shape, const void* X, const void* G1, const void* G2,
@@ -143,8 +151,9 @@ int psk_causal_attn_fwd(const psk_shape* shape, const void* Q, const void* K, co
     int launches = 0;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
     if (e == cudaSuccess)
-        e = path == 1 ? tc_fwd(d, Q, K, V, G1, G2, O, denom, (char*)workspace, s, &launches)
-                      : cc_fwd(d, Q, K, V, G1, G2, O, denom, (char*)workspace, s, &launches);
+        e = path == 2 ? given_fwd(d, Q, K, V, G1, G2, O, denom, (char*)workspace, s, &launches)
+            : path == 1 ? tc_fwd(d, Q, K, V, G1, G2, O, denom, (char*)workspace, s, &launches)
+                        : cc_fwd(d, Q, K, V, G1, G2, O, denom, (char*)workspace, s, &launches);
     g_last_launches = launches;
     return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
 }
@@ -171,8 +180,9 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
     int launches = 0;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
     if (e == cudaSuccess)
-        e = path == 1 ? tc_bwd(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches)
-                      : cc_bwd(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches);
+        e = path == 2 ? given_bwd(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches)
+            : path == 1 ? tc_bwd(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches)
+                        : cc_bwd(d, Q, K, V, G1, G2, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches);
     g_last_launches = launches;
     return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
 }
@@ -181,14 +191,19 @@ int psk_causal_attn_bwd(const psk_shape* shape, const void* Q, const void* K, co
 static int learned_dims(const psk_shape* shape, psk_shape* sh, Dims* d) {
     if (shape == nullptr) return PSK_ERR_INVALID_ARG;
     *sh = *shape;
-    sh->path = PSK_PATH_CUDA_CORES;
     sh->g_heads = 1;
     if (sh->p != 4) return PSK_ERR_UNSUPPORTED;
+    // (validated as a CUDA-core call; the tensor-core route below adds its own conditions)
+    const int32_t want = sh->path;
+    sh->path = PSK_PATH_CUDA_CORES;
     const int st = make_dims(sh, d);
     if (st != PSK_OK) return st;
     d->learned = true;
+    sh->path = want;
+    if (want == PSK_PATH_TENSOR_CORES && !given_supported(*d)) return PSK_ERR_UNSUPPORTED;
     return PSK_OK;
 }
+static bool learned_on_tc(const psk_shape& sh, const Dims& d) { return sh.path != PSK_PATH_CUDA_CORES && given_supported(d); }
 
 size_t psk_learned_param_count(int h, int r) {
     if (h != 64 || (r != 16 && r != 32 && r != 64)) return 0;
@@ -198,7 +213,7 @@ size_t psk_learned_param_count(int h, int r) {
 size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward) {
     psk_shape sh; Dims d;
     if (learned_dims(shape, &sh, &d) != PSK_OK) return 0;
-    return cc_workspace(d, for_backward != 0).total;
+    return learned_on_tc(sh, d) ? given_workspace_bytes(d, for_backward != 0) : cc_workspace(d, for_backward != 0).total;
 }
 
 int psk_learned_sketch(const psk_shape* shape, const void* X, const float* params, float* M_out, float* Phi_out,
@@ -223,13 +238,16 @@ int psk_learned_attn_fwd(const psk_shape* shape, const void* Q, const void* K, c
     if (!Q || !K || !V || !O || !params) return PSK_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(params) || !aligned16(O) || !aligned16(denom))
         return PSK_ERR_ALIGN;
-    const size_t need = cc_workspace(d, false).total;
+    const bool tcp = learned_on_tc(sh, d);
+    const size_t need = tcp ? given_workspace_bytes(d, false) : cc_workspace(d, false).total;
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign)) return PSK_ERR_WORKSPACE;
     d.lparams = params;
     cudaStream_t s = (cudaStream_t)stream;
     int launches = 0;
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
-    if (e == cudaSuccess) e = cc_fwd(d, Q, K, V, nullptr, nullptr, O, denom, (char*)workspace, s, &launches);
+    if (e == cudaSuccess)
+        e = tcp ? given_fwd(d, Q, K, V, nullptr, nullptr, O, denom, (char*)workspace, s, &launches)
+                : cc_fwd(d, Q, K, V, nullptr, nullptr, O, denom, (char*)workspace, s, &launches);
     g_last_launches = launches;
     return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
 }
@@ -244,7 +262,8 @@ int psk_learned_attn_bwd(const psk_shape* shape, const void* Q, const void* K, c
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(params) || !aligned16(O) || !aligned16(denom) ||
         !aligned16(dO) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(dparams))
         return PSK_ERR_ALIGN;
-    const size_t need = cc_workspace(d, true).total;
+    const bool tcp = learned_on_tc(sh, d);
+    const size_t need = tcp ? given_workspace_bytes(d, true) : cc_workspace(d, true).total;
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) % kAlign)) return PSK_ERR_WORKSPACE;
     d.lparams = params;
     d.dlparams = dparams;
@@ -253,7 +272,9 @@ int psk_learned_attn_bwd(const psk_shape* shape, const void* Q, const void* K, c
     cudaError_t e = cudaMemsetAsync(workspace, 0, kStatusBytes, s);
     // the kernels add into the gradient array: it starts at zero
     if (e == cudaSuccess) e = cudaMemsetAsync(dparams, 0, 2 * learned_param_count(d.h, d.r) * sizeof(float), s);
-    if (e == cudaSuccess) e = cc_bwd(d, Q, K, V, nullptr, nullptr, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches);
+    if (e == cudaSuccess)
+        e = tcp ? given_bwd(d, Q, K, V, nullptr, nullptr, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches)
+                : cc_bwd(d, Q, K, V, nullptr, nullptr, O, denom, dO, dQ, dK, dV, (char*)workspace, s, &launches);
     g_last_launches = launches;
     return e == cudaSuccess ? PSK_OK : PSK_ERR_CUDA;
 }

@@ -830,6 +830,38 @@ cudaError_t fwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     return cudaGetLastError();
 }
 
+// Chain rule through the half sketch of one tensor: dX from dM (+ `add`, the part of the gradient
+// that reached X directly through exact same-block weights).
+template <typename T, int R>
+cudaError_t launch_sketch_bwd(const Dims& d, const T* X, const T* G1, const T* G2, const float* dM, const float* add,
+                              T* dX, cudaStream_t s, int* launches) {
+    Slice sl{d.H, d.sb, d.sh, d.sn};
+    const int rows = d.BH() * d.n;
+    if (d.learned) return learned_sketch_bwd(d, X, dM, add, dX, s, launches);     // two networks; gradients add up
+    if (d.p == 2) {           // dX = dM (+ add)
+        prof_begin("identity_sketch_bwd_kernel", s);
+        identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dM, add, dX);
+        prof_end(s);
+        ++*launches;
+        return cudaGetLastError();
+    }
+    if (d.p == 8) {
+        PSK_TRY((allow_smem(sketch8_bwd_kernel<T, R>, Sk8<R>::bytes)));
+        prof_begin("sketch8_bwd_kernel", s);
+        sketch8_bwd_kernel<T, R><<<dim3(d.n / Sk8<R>::kRows, d.BH()), 256, Sk8<R>::bytes, s>>>(sl, X, G1, G2, d.g_heads, d.n, dM, dX);
+        prof_end(s);
+        ++*launches;
+        return cudaGetLastError();
+    }
+    const size_t smem = (size_t)(2 * H64 * (R + 1) + 64 * 65 + 2 * 64 * (R + 1)) * sizeof(float);
+    PSK_TRY(allow_smem(sketch_bwd_kernel<T, R>, smem));
+    prof_begin("sketch_bwd_kernel", s);
+    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, X, G1, G2, d.g_heads, d.n, dM, add, dX);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
 template <typename T, int R>
 cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T* G1, const T* G2,
                      const T* O, const float* denom, const T* dO, T* dQ, T* dK, T* dV,
@@ -877,42 +909,8 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
     }
     *launches += 2;
     PSK_TRY(cudaGetLastError());
-    if (d.learned) {          // back through the two networks; their gradients collect both uses
-        PSK_TRY(learned_sketch_bwd(d, Q, dMq, dXq, dQ, s, launches));
-        return learned_sketch_bwd(d, K, dMk, dXk, dK, s, launches);
-    }
-    if (d.p == 2) {           // dX = dM (+ the same-block part that bypassed it)
-        prof_begin("identity_sketch_bwd_kernel", s);
-        identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMq, dXq, dQ);
-        prof_end(s);
-        prof_begin("identity_sketch_bwd_kernel", s);
-        identity_sketch_bwd_kernel<T><<<(rows + 7) / 8, 256, 0, s>>>(sl, d.n, rows, dMk, dXk, dK);
-        prof_end(s);
-        *launches += 2;
-        return cudaGetLastError();
-    }
-    if (d.p == 8) {
-        PSK_TRY((allow_smem(sketch8_bwd_kernel<T, R>, Sk8<R>::bytes)));
-        const dim3 grid8(d.n / Sk8<R>::kRows, d.BH());
-        prof_begin("sketch8_bwd_kernel", s);
-        sketch8_bwd_kernel<T, R><<<grid8, 256, Sk8<R>::bytes, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dQ);
-        prof_end(s);
-        prof_begin("sketch8_bwd_kernel", s);
-        sketch8_bwd_kernel<T, R><<<grid8, 256, Sk8<R>::bytes, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dK);
-        prof_end(s);
-        *launches += 2;
-        return cudaGetLastError();
-    }
-    const size_t smem = (size_t)(2 * H64 * (R + 1) + 64 * 65 + 2 * 64 * (R + 1)) * sizeof(float);
-    PSK_TRY(allow_smem(sketch_bwd_kernel<T, R>, smem));
-    prof_begin("sketch_bwd_kernel", s);
-    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, Q, G1, G2, d.g_heads, d.n, dMq, dXq, dQ);
-    prof_end(s);
-    prof_begin("sketch_bwd_kernel", s);
-    sketch_bwd_kernel<T, R><<<dim3(d.n / 64, d.BH()), 256, smem, s>>>(sl, K, G1, G2, d.g_heads, d.n, dMk, dXk, dK);
-    prof_end(s);
-    *launches += 2;
-    return cudaGetLastError();
+    PSK_TRY((launch_sketch_bwd<T, R>(d, Q, G1, G2, dMq, dXq, dQ, s, launches)));
+    return launch_sketch_bwd<T, R>(d, K, G1, G2, dMk, dXk, dK, s, launches);
 }
 
 #define PSK_DISPATCH(CALL_F32, CALL_BF16)                                   \
@@ -934,6 +932,13 @@ cudaError_t bwd_impl(const Dims& d, const T* Q, const T* K, const T* V, const T*
 cudaError_t cc_sketch(const Dims& d, const void* X, const void* G1, const void* G2,
                       float* M_out, float* Phi_out, cudaStream_t s, int* launches) {
 #define C_ (launch_sketch<T, R>(d, (const T*)X, (const T*)G1, (const T*)G2, M_out, Phi_out, s, launches))
+    PSK_DISPATCH(C_, C_)
+#undef C_
+}
+
+cudaError_t cc_sketch_bwd(const Dims& d, const void* X, const void* G1, const void* G2, const float* dM,
+                          const float* add, void* dX, cudaStream_t s, int* launches) {
+#define C_ (launch_sketch_bwd<T, R>(d, (const T*)X, (const T*)G1, (const T*)G2, dM, add, (T*)dX, s, launches))
     PSK_DISPATCH(C_, C_)
 #undef C_
 }

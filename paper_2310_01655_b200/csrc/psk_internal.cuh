@@ -62,6 +62,19 @@ cudaError_t learned_sketch(const Dims& d, const void* X, float* M, float* Phi, c
 cudaError_t learned_sketch_bwd(const Dims& d, const void* X, const float* dM, const float* add, void* dX,
                                cudaStream_t s, int* launches);
 
+cudaError_t cc_sketch_bwd(const Dims& d, const void* X, const void* G1, const void* G2, const float* dM,
+                          const float* add, void* dX, cudaStream_t s, int* launches);
+
+// Degree 8 and the learnable sketch on the tensor cores: half sketches by the CUDA-core sketch
+// kernels, attention on them by the tensor-core kernels (psk_given.cu).
+bool given_supported(const Dims& d);
+size_t given_workspace_bytes(const Dims& d, bool backward);
+cudaError_t given_fwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
+                      void* O, float* denom, char* ws, cudaStream_t s, int* launches);
+cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
+                      const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV, char* ws,
+                      cudaStream_t s, int* launches);
+
 // Tensor-core (bf16 operands, fp32 accumulation) launchers.
 size_t tc_workspace_bytes(const Dims& d, bool backward);
 bool tc_supported(const Dims& d, bool backward);

@@ -24,9 +24,13 @@ def _oracle_gaussians(G1, G2, hi, h):
     return [a[:h], b[:h], a[h:2 * h], b[h:2 * h], a[2 * h:], b[2 * h:]]
 
 
-@pytest.mark.parametrize("r,b,n,dtype", [(16, 128, 384, "f32"), (32, 256, 512, "f32"), (64, 128, 256, "f32"),
-                                         (32, 128, 128, "f32"), (32, 256, 768, "bf16")])
-def test_forward_and_backward(r, b, n, dtype):
+@pytest.mark.parametrize("r,b,n,dtype,path", [
+    (16, 128, 384, "f32", psk.PATH_AUTO), (32, 256, 512, "f32", psk.PATH_AUTO), (64, 128, 256, "f32", psk.PATH_AUTO),
+    (32, 128, 128, "f32", psk.PATH_AUTO), (32, 256, 768, "bf16", psk.PATH_CUDA_CORES), (64, 256, 512, "bf16", psk.PATH_AUTO),
+    # bf16 storage, r <= 32: half sketches by the sketch kernels, attention on them by the tensor-core kernels
+    (32, 256, 768, "bf16", psk.PATH_TENSOR_CORES), (16, 128, 640, "bf16", psk.PATH_AUTO), (32, 512, 1024, "bf16", psk.PATH_AUTO),
+])
+def test_forward_and_backward(r, b, n, dtype, path):
     # rows scaled down: (q.k)^8 with |q|^2 = h would leave fp32's comfortable range
     w = wl.small_workload(B=1, H=2, n=n, r=r, b=b, dtype=dtype, seed=500 + r)
     inp = wl.make_inputs(w, "cuda")
@@ -34,9 +38,14 @@ def test_forward_and_backward(r, b, n, dtype):
     Q, K = (inp["Q"].float() * 0.25).to(tdt), (inp["K"].float() * 0.25).to(tdt)
     V, dO = inp["V"], inp["dO"]
     G1, G2 = _packed_gaussians(w.H, 64, r, 600 + r, tdt)
-    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b, p=8)
-    dQ, dK, dV = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, p=8)
+    psk.profile_enable(True)
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b, p=8, path=path)
+    dQ, dK, dV = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, p=8, path=path)
     torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    on_tc = dtype == "bf16" and r <= 32 and path != psk.PATH_CUDA_CORES
+    assert ("tc_fwd_out_kernel" in kernels) == on_tc and ("sketch8_kernel" in kernels) and (("fwd_out_kernel" in kernels) != on_tc)
     for hi in range(w.H):
         q, k, v, g = (x[0, hi].double().cpu().numpy() for x in (Q, K, V, dO))
         Gs = _oracle_gaussians(G1, G2, hi, 64)
@@ -64,3 +73,29 @@ def test_sketch_call_and_refusals():
     with pytest.raises(psk.PskError) as e:
         psk.causal_attn_fwd(X, X, inp["V"], G1, G2, 128, p=8, flags=psk.FLAG_LOCAL_EXACT)
     assert e.value.code == -2
+    with pytest.raises(psk.PskError) as e:      # fp32 storage has no tensor-core route
+        psk.causal_attn_fwd(X, X, inp["V"], G1, G2, 128, p=8, path=psk.PATH_TENSOR_CORES)
+    assert e.value.code == -2
+
+
+def test_kept_states_on_the_tensor_cores():
+    r, b, n = 32, 256, 1024
+    w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype="bf16", seed=510)
+    inp = wl.make_inputs(w, "cuda")
+    Q, K = (inp["Q"].float() * 0.25).bfloat16(), (inp["K"].float() * 0.25).bfloat16()
+    V, dO = inp["V"], inp["dO"]
+    G1, G2 = _packed_gaussians(w.H, 64, r, 611, torch.bfloat16)
+    shp = psk.binding.make_shape(Q, G1, r, b, 8, flags=psk.FLAG_KEEP_STATES)
+    ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True)), dtype=torch.uint8, device="cuda")
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b, p=8, workspace=ws, flags=psk.FLAG_KEEP_STATES)
+    dQ, dK, dV = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, p=8, workspace=ws, flags=psk.FLAG_KEEP_STATES)
+    assert psk.check(ws) == 0
+    for bi, hi in ((0, 1), (1, 0)):
+        q, k, v, g = (x[bi, hi].double().cpu().numpy() for x in (Q, K, V, dO))
+        Gs = _oracle_gaussians(G1, G2, hi, 64)
+        Mq, Mk = orc.half_sketch_degree4(q, Gs), orc.half_sketch_degree4(k, Gs)
+        O_ref, d_ref = orc.causal_attention_blocked_from_half_sketches(Mq, Mk, v, b)
+        check("O", O[bi, hi], O_ref, TOL["bf16"])
+        check("denom", den[bi, hi], d_ref, TOL["bf16"])
+        for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), orc.causal_polysketch8_attention_backward(q, k, v, Gs, g)):
+            check(name, got[bi, hi], ref, TOL["bf16"])

@@ -49,9 +49,11 @@ def test_half_sketch(r, dtype):
 
 
 @pytest.mark.parametrize("r,b,n", [(16, 128, 256), (32, 128, 384), (64, 256, 256)])
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype,path", [("f32", psk.PATH_AUTO), ("bf16", psk.PATH_CUDA_CORES), ("bf16", psk.PATH_AUTO)])
 @pytest.mark.parametrize("local", [False, True])
-def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype, local):
+def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype, path, local):
+    # (bf16 storage, r <= 32, sketched same-block weights: PATH_AUTO is the tensor-core route on half
+    # sketches formed by the networks; everything else runs on the CUDA cores)
     w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype=dtype, seed=70 + r)
     inp = wl.make_inputs(w, "cuda")
     if local:
@@ -60,9 +62,14 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
     flat, P1, P2 = nets(r, 2)
     flags = psk.FLAG_LOCAL_EXACT if local else 0
     Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
-    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags)
-    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags)
+    psk.profile_enable(True)
+    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags, path=path)
+    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags, path=path)
     torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    on_tc = dtype == "bf16" and r <= 32 and not local and path != psk.PATH_CUDA_CORES
+    assert ("tc_bwd_k_kernel" in kernels) == on_tc and "learned_sketch_bwd_kernel" in kernels
     tol = TOL[dtype]
     diag = "exact" if local else "LR"
     g1_sum = {k: 0.0 for k in orc.NET_KEYS}
@@ -95,4 +102,6 @@ def test_refusals():
         binding.learned_attn_fwd(inp["Q"], inp["K"], inp["V"], flat, 32, 128, psk.FLAG_NONCAUSAL)
     with pytest.raises(psk.PskError):
         binding.learned_attn_fwd(inp["Q"], inp["K"], inp["V"], flat, 32, 100)
+    with pytest.raises(psk.PskError):            # fp32 storage has no tensor-core route
+        binding.learned_attn_fwd(inp["Q"], inp["K"], inp["V"], flat, 32, 128, path=psk.PATH_TENSOR_CORES)
     assert binding.learned_param_count(48, 32) == 0
