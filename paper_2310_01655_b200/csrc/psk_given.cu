@@ -13,7 +13,7 @@ namespace psk {
 
 namespace {
 
-struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, total; };
+struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, ltc, total; };
 
 Dims linear_dims(const Dims& d) {
     Dims l = d;
@@ -37,6 +37,7 @@ GivenWs given_ws(const Dims& d, bool backward) {
         w.dSq = off; off += align_up(rows * 64 * sizeof(bf16));                     // gradient of the [hi | lo] columns
         w.dSk = off; off += align_up(rows * 64 * sizeof(bf16));
     }
+    if (d.learned && learned_tc_supported(d)) { w.ltc = off; off += align_up(learned_tc_workspace_bytes(d, backward)); }
     w.total = off;
     return w;
 }
@@ -77,13 +78,16 @@ unsplit_kernel(const bf16* __restrict__ dS, int r, size_t rows, float* __restric
 }
 
 cudaError_t half_sketches(const Dims& d, const void* Q, const void* K, const void* G1, const void* G2, char* ws,
-                          const GivenWs& w, cudaStream_t s, int* launches) {
+                          const GivenWs& w, bool backward, cudaStream_t s, int* launches) {
     const size_t rows = (size_t)d.BH() * d.n;
     const void* X[2] = {Q, K};
     const size_t mo[2] = {w.Mq, w.Mk}, so[2] = {w.Sq, w.Sk};
+    const bool nets_on_tc = d.learned && learned_tc_supported(d);
+    if (nets_on_tc) PSK_TRY(learned_tc_prepare(d, backward, ws + w.ltc, s, launches));
     for (int i = 0; i < 2; ++i) {
         float* M = reinterpret_cast<float*>(ws + mo[i]);
-        PSK_TRY(cc_sketch(d, X[i], G1, G2, M, nullptr, s, launches));
+        if (nets_on_tc) PSK_TRY(learned_tc_sketch(d, X[i], M, ws + w.ltc, reinterpret_cast<int*>(ws + w.tc), s, launches));
+        else PSK_TRY(cc_sketch(d, X[i], G1, G2, M, nullptr, s, launches));
         prof_begin("split_kernel", s);
         split_kernel<<<(unsigned)((rows * 8 + 255) / 256), 256, 0, s>>>(M, d.r, rows, reinterpret_cast<bf16*>(ws + so[i]));
         prof_end(s);
@@ -105,7 +109,7 @@ size_t given_workspace_bytes(const Dims& d, bool backward) { return given_ws(d, 
 cudaError_t given_fwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
                       void* O, float* denom, char* ws, cudaStream_t s, int* launches) {
     const GivenWs w = given_ws(d, d.keep_states);
-    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, s, launches));
+    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, false, s, launches));
     return tc_fwd(linear_dims(d), ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, ws + w.tc, s, launches);
 }
 
@@ -114,12 +118,13 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
                       cudaStream_t s, int* launches) {
     const GivenWs w = given_ws(d, true);
     const size_t rows = (size_t)d.BH() * d.n;
-    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, s, launches));
+    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, true, s, launches));
     PSK_TRY(tc_bwd(linear_dims(d), ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, dO, ws + w.dSq, ws + w.dSk, dV,
                    ws + w.tc, s, launches));
     const void* X[2] = {Q, K};
     void* dX[2] = {dQ, dK};
     const size_t mo[2] = {w.Mq, w.Mk}, go[2] = {w.dSq, w.dSk};
+    const bool nets_on_tc = d.learned && learned_tc_supported(d);
     for (int i = 0; i < 2; ++i) {
         float* dM = reinterpret_cast<float*>(ws + mo[i]);       // m itself is no longer needed
         prof_begin("unsplit_kernel", s);
@@ -127,8 +132,10 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
-        PSK_TRY(cc_sketch_bwd(d, X[i], G1, G2, dM, nullptr, dX[i], s, launches));
+        if (nets_on_tc) PSK_TRY(learned_tc_sketch_bwd(d, X[i], dM, nullptr, dX[i], ws + w.ltc, reinterpret_cast<int*>(ws + w.tc), s, launches));
+        else PSK_TRY(cc_sketch_bwd(d, X[i], G1, G2, dM, nullptr, dX[i], s, launches));
     }
+    if (nets_on_tc) PSK_TRY(learned_tc_finish(d, ws + w.ltc, s, launches));
     return cudaSuccess;
 }
 

@@ -1,0 +1,868 @@
+// Learnable sketch (Algorithm 2 of the paper's appendix) with its dense layers on the tensor
+// cores: bf16 operands, fp32 accumulation in tensor memory, r <= 32 (8r <= 256), h = 64.
+//
+//   f(x) = W4^T gelu(W3^T (W2^T LN1(gelu(W1^T LN0(x) + b1)) + b2) + b3) + b4      (two such networks)
+//   M    = sqrt(r) tanh(f_1(x) * f_2(x) / sqrt(r))
+//
+// Rows are processed in chunks; inside a chunk every layer is one launch of tc_dense_kernel
+// (128 rows per CTA: activations by TMA, the layer's weights as the MN-major B operand, the
+// accumulator read back by thread = row, where bias, gelu and the layer normalisations are plain
+// per-thread loops), with the activations the backward needs kept in the workspace as bf16.
+// The gains of the normalisations are folded into the following layer's weights
+// (z W = n (diag(g) W) + c W), so the normalised activations n are the GEMM operands and
+// their gradients come out of the GEMM with the gain already applied.  Weight gradients are
+// sums over ALL rows of outer products: tc_wgrad_kernel accumulates P^T S over a slab of rows in
+// tensor memory and adds the result to an fp32 accumulator once per slab; gains, biases and the
+// folded terms are taken from those accumulators and from column sums by a last small kernel.
+// Every r-wide array is padded to 64 columns and every 8r-wide one to 256 (zeros), so two GEMM
+// shapes, 64 -> 256 and 256 -> 64, serve all sixteen layer passes.
+#include "tc_common.cuh"
+
+namespace psk {
+
+namespace {
+
+using namespace tc;
+
+constexpr float kLnEps = 1e-6f;
+constexpr size_t kChunkRows = (size_t)1 << 20;        // rows per pass over the layers
+constexpr int kMat = 64 * 256;                        // elements of one operand matrix
+constexpr int kBank = 12;                             // operand matrices per network
+constexpr int kVec = 256 + 64 + 256 + 64;             // folded biases of one network: b1' | b2' | b3 | b4
+constexpr int kSums = 256 + 64 + 256 + 64;            // column sums of one network: dp1 | da2 | dp3 | df
+
+__device__ __forceinline__ float gelu_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
+__device__ __forceinline__ float gelu_grad_f(float x) {
+    return 0.5f * (1.f + erff(x * 0.70710678118654752f)) + x * __expf(-0.5f * x * x) * 0.3989422804014327f;
+}
+
+struct NetLayout {
+    int h, r, m;
+    int g0, c0, W1, b1, g1, c1, W2, b2, W3, b3, W4, b4, count;
+    __host__ __device__ NetLayout(int h_, int r_) : h(h_), r(r_), m(8 * r_) {
+        int o = 0;
+        g0 = o; o += h; c0 = o; o += h;
+        W1 = o; o += h * m; b1 = o; o += m;
+        g1 = o; o += m; c1 = o; o += m;
+        W2 = o; o += m * r; b2 = o; o += r;
+        W3 = o; o += r * m; b3 = o; o += m;
+        W4 = o; o += m * r; b4 = o; o += r;
+        count = o;
+    }
+};
+
+// ---------------------------------------------------------------------------
+// operand bank: per network eight bf16 matrices and the folded biases
+//   0: diag(g0) W1  [64][256]     4: W4^T           [64][256]
+//   1: diag(g1) W2  [256][64]     5: W3^T           [256][64]
+//   2: W3           [64][256]     6: (diag(g1) W2)^T [64][256]
+//   3: W4           [256][64]     7: (diag(g0) W1)^T [256][64]
+//   8..11: what rounding 0..3 to bf16 left over (the forward multiplies by hi + lo)
+// (rows / columns beyond r or 8r are zero)
+// ---------------------------------------------------------------------------
+__device__ float bank_entry(const NetLayout& nl, const float* P, int which, int row, int col) {
+    const int r = nl.r, m = nl.m;
+    switch (which) {
+        case 0: return col < m ? P[nl.g0 + row] * P[nl.W1 + row * m + col] : 0.f;                  // [k][j]
+        case 1: return (row < m && col < r) ? P[nl.g1 + row] * P[nl.W2 + row * r + col] : 0.f;      // [j][c]
+        case 2: return (row < r && col < m) ? P[nl.W3 + row * m + col] : 0.f;                       // [c][j]
+        case 3: return (row < m && col < r) ? P[nl.W4 + row * r + col] : 0.f;                       // [j][c]
+        case 4: return (col < m && row < r) ? P[nl.W4 + col * r + row] : 0.f;                       // [c][j]
+        case 5: return (row < m && col < r) ? P[nl.W3 + col * m + row] : 0.f;                       // [j][c]
+        case 6: return (col < m && row < r) ? P[nl.g1 + col] * P[nl.W2 + col * r + row] : 0.f;      // [c][j]
+        default: return row < m ? P[nl.g0 + col] * P[nl.W1 + col * m + row] : 0.f;                  // [j][k]
+    }
+}
+
+__global__ void __launch_bounds__(256)
+ltc_bank_kernel(int h, int r, const float* __restrict__ params, bf16* __restrict__ bank, float* __restrict__ vec) {
+    const NetLayout nl(h, r);
+    const int net = blockIdx.y;
+    const float* P = params + (size_t)net * nl.count;
+    const int e = blockIdx.x * 256 + threadIdx.x;
+    if (e < 8 * kMat) {
+        const int which = e / kMat, idx = e % kMat;
+        const int cols = (which % 2 == 0) ? 256 : 64;
+        const float v = bank_entry(nl, P, which, idx / cols, idx % cols);
+        const bf16 hi = __float2bfloat16_rn(v);
+        bank[(size_t)net * kBank * kMat + e] = hi;
+        if (which < 4) bank[(size_t)net * kBank * kMat + 8 * kMat + e] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    } else if (e < 8 * kMat + kVec) {
+        const int v = e - 8 * kMat;
+        float out = 0.f;
+        if (v < 256) {                                   // b1' = c0 W1 + b1
+            if (v < nl.m) { out = P[nl.b1 + v]; for (int k = 0; k < h; ++k) out = fmaf(P[nl.c0 + k], P[nl.W1 + k * nl.m + v], out); }
+        } else if (v < 320) {                            // b2' = c1 W2 + b2
+            const int c = v - 256;
+            if (c < r) { out = P[nl.b2 + c]; for (int j = 0; j < nl.m; ++j) out = fmaf(P[nl.c1 + j], P[nl.W2 + j * r + c], out); }
+        } else if (v < 576) {
+            if (v - 320 < nl.m) out = P[nl.b3 + v - 320];
+        } else {
+            if (v - 576 < r) out = P[nl.b4 + v - 576];
+        }
+        vec[(size_t)net * kVec + v] = out;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// dense layer: Out[128 rows x ND] = epilogue(A[128 x KD] B[KD x ND])
+// ---------------------------------------------------------------------------
+enum { EPI_LN = 0, EPI_B64 = 1, EPI_GELU = 2, EPI_F32 = 3, EPI_DGELU = 4, EPI_LNBWD = 5 };
+
+struct DenseArgs {
+    const float* bias;      // [ND] or null
+    bf16* out0;             // bf16 outputs, [rows][ND]
+    bf16* out1;
+    bf16* out2;
+    float* outf;            // EPI_F32: [rows][ncols]; EPI_LN: 1 / sigma of every row
+    const float* rs;        // EPI_LNBWD: 1 / sigma of every row
+    int ncols;              // EPI_F32: columns stored; EPI_LN, EPI_LNBWD, EPI_DGELU, EPI_GELU: live columns (8r)
+    int accumulate;         // EPI_F32: add to what is there
+};
+
+__device__ __forceinline__ void store8(bf16* dst, const float* v) {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+// v = hi + lo as two bf16 terms
+__device__ __forceinline__ void store8_split(bf16* hi, bf16* lo, const float* v) {
+    float h[8], l[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { h[i] = __bfloat162float(__float2bfloat16_rn(v[i])); l[i] = v[i] - h[i]; }
+    store8(hi, h);
+    store8(lo, l);
+}
+__device__ __forceinline__ void load8(const uint8_t* tile, int row, int col, float* v) {
+    // `tile`: [128 rows x 256 columns] bf16 as four 128-byte-swizzled [128 x 64] tiles
+    const uint4 q = *reinterpret_cast<const uint4*>(tile + (col / 64) * 16384 + swz128_offset(row, (col % 64) / 8));
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+// SPLIT (the forward's layers): activations and weights are both hi + lo pairs of bf16 arrays and
+// the product is A_hi B_hi + A_lo B_hi + A_hi B_lo.  A half sketch feeds fourth powers of
+// cancelling sums; single bf16 operands (2^-9 per entry, four layers deep) would leave percents of
+// error on the attention's output, the pairs leave 2^-17.
+template <int KD, int ND, int EPI, bool SPLIT>
+struct DenseSmem {
+    static constexpr int kA1 = 128 * KD * 2, kB1 = KD * ND * 2;
+    static constexpr int kA = kA1 * (SPLIT ? 2 : 1), kB = kB1 * (SPLIT ? 2 : 1);
+    static constexpr int kSides = EPI == EPI_DGELU ? 1 : (EPI == EPI_LNBWD ? 2 : 0);
+    static constexpr int bytes = kA + kB + kSides * 65536 + 1024;
+};
+
+template <int KD, int ND, int EPI, bool SPLIT>
+__global__ void __launch_bounds__(128)
+ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mA2,
+                 const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2,
+                 const __grid_constant__ CUtensorMap mS0, const __grid_constant__ CUtensorMap mS1, DenseArgs a,
+                 int* status) {
+    static_assert((KD == 64 && ND == 256) || (KD == 256 && ND == 64), "two GEMM shapes");
+    static_assert(!SPLIT || DenseSmem<KD, ND, EPI, SPLIT>::kSides == 0, "the forward's layers have no side tiles");
+    using L = DenseSmem<KD, ND, EPI, SPLIT>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sA = align1024(smem_raw);
+    uint8_t* sB = sA + L::kA;
+    uint8_t* sS = sB + L::kB;
+    __shared__ uint64_t bar_ld, bar_side, bar_mma;
+    __shared__ uint32_t tm_slot;
+    __shared__ float s_bias[ND];
+    const int tid = threadIdx.x, warp = tid / 32;
+    const int tile = blockIdx.x;
+    if (tid == 0) {
+        cta_giveup_init();
+        mbar_init(&bar_ld, 1); mbar_init(&bar_side, 1); mbar_init(&bar_mma, 1);
+        mbar_fence_init();
+    }
+    if (warp == 0) { tmem_alloc(&tm_slot, ND); tmem_relinquish(); }
+    for (int j = tid; j < ND; j += 128) s_bias[j] = a.bias != nullptr ? a.bias[j] : 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tm_slot;
+    if (tid == 0) {
+        mbar_expect_tx(&bar_ld, L::kA + L::kB);
+#pragma unroll
+        for (int s = 0; s < KD / 64; ++s) tma_load_2d(sA + s * 16384, &mA, s * 64, tile * 128, &bar_ld);
+#pragma unroll
+        for (int g = 0; g < ND / 64; ++g) tma_load_2d(sB + g * KD * 128, &mB, g * 64, 0, &bar_ld);
+        if constexpr (SPLIT) {
+#pragma unroll
+            for (int s = 0; s < KD / 64; ++s) tma_load_2d(sA + L::kA1 + s * 16384, &mA2, s * 64, tile * 128, &bar_ld);
+#pragma unroll
+            for (int g = 0; g < ND / 64; ++g) tma_load_2d(sB + L::kB1 + g * KD * 128, &mB2, g * 64, 0, &bar_ld);
+        }
+        if constexpr (L::kSides > 0) {
+            mbar_expect_tx(&bar_side, L::kSides * 65536);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) tma_load_2d(sS + g * 16384, &mS0, g * 64, tile * 128, &bar_side);
+            if constexpr (L::kSides > 1) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) tma_load_2d(sS + 65536 + g * 16384, &mS1, g * 64, tile * 128, &bar_side);
+            }
+        }
+        if (mbar_wait(&bar_ld, 0, status, kErrTma)) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, ND, false, true);
+#pragma unroll
+            for (int part = 0; part < (SPLIT ? 3 : 1); ++part) {
+                const uint64_t ad = smem_desc(smem_u32(sA) + (part == 1 ? L::kA1 : 0), 0, 1024, kSwz128);
+                const uint64_t bd = smem_desc(smem_u32(sB) + (part == 2 ? L::kB1 : 0), KD * 128, 1024, kSwz128);
+#pragma unroll
+                for (int k = 0; k < KD / 16; ++k)
+                    umma_ss(tm, desc_off(ad, (k / 4) * 16384 + (k % 4) * 32), desc_off(bd, k * 2048), idesc, (part > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&bar_mma);
+        }
+    }
+    bool ok = mbar_wait(&bar_mma, 0, status, kErrMma);
+    if constexpr (L::kSides > 0) ok = ok && mbar_wait(&bar_side, 0, status, kErrTma);
+    tc_fence_after();
+    const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
+    const size_t row = (size_t)tile * 128 + tid;
+    if (ok) {
+        if constexpr (EPI == EPI_B64) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    if constexpr (SPLIT) store8_split(a.out0 + row * 64 + c0 + j, a.out1 + row * 64 + c0 + j, v + j);
+                    else store8(a.out0 + row * 64 + c0 + j, v + j);
+                }
+            }
+        } else if constexpr (EPI == EPI_F32) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                if (c0 < a.ncols) {
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+                    float* dst = a.outf + row * a.ncols + c0;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        if (c0 + j < a.ncols) {
+                            float4 o = make_float4(__uint_as_float(u[j]) + s_bias[c0 + j], __uint_as_float(u[j + 1]) + s_bias[c0 + j + 1],
+                                                   __uint_as_float(u[j + 2]) + s_bias[c0 + j + 2], __uint_as_float(u[j + 3]) + s_bias[c0 + j + 3]);
+                            if (a.accumulate) {
+                                const float4 p = *reinterpret_cast<const float4*>(dst + j);
+                                o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+                            }
+                            *reinterpret_cast<float4*>(dst + j) = o;
+                        }
+                    }
+                }
+            }
+        } else if constexpr (EPI == EPI_GELU) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float p[32], g[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    p[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
+                    g[j] = (c0 + j < a.ncols) ? gelu_f(p[j]) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    store8(a.out0 + row * 256 + c0 + j, p + j);
+                    store8_split(a.out1 + row * 256 + c0 + j, a.out2 + row * 256 + c0 + j, g + j);
+                }
+            }
+        } else if constexpr (EPI == EPI_LN) {
+            // pass 1: pre-activation out, gelu back into tensor memory, sums
+            float s = 0.f, ss = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float p[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    p[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
+                    const float g = (c0 + j < a.ncols) ? gelu_f(p[j]) : 0.f;
+                    s += g; ss = fmaf(g, g, ss);
+                    u[j] = __float_as_uint(g);
+                }
+                tmem_st32(lane_tm + c0, u);
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, p + j);
+            }
+            tmem_st_wait();
+            const float inv = 1.f / (float)a.ncols;
+            const float mu = s * inv;
+            const float rs = rsqrtf(fmaxf(ss * inv - mu * mu, 0.f) + kLnEps);
+            a.outf[row] = rs;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float nrm[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) nrm[j] = (c0 + j < a.ncols) ? (__uint_as_float(u[j]) - mu) * rs : 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) store8_split(a.out1 + row * 256 + c0 + j, a.out2 + row * 256 + c0 + j, nrm + j);
+            }
+        } else if constexpr (EPI == EPI_DGELU) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float o[32];
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    float p[8];
+                    load8(sS, tid, c0 + j, p);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) o[j + q] = (c0 + j + q < a.ncols) ? __uint_as_float(u[j + q]) * gelu_grad_f(p[q]) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, o + j);
+            }
+        } else {   // EPI_LNBWD: back through n = (g - mu) / sigma and g = gelu(p)
+            float s1 = 0.f, s2 = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    float nrm[8];
+                    load8(sS, tid, c0 + j, nrm);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { const float dn = __uint_as_float(u[j + q]); s1 += dn; s2 = fmaf(dn, nrm[q], s2); }
+                }
+            }
+            const float inv = 1.f / (float)a.ncols;
+            const float m1 = s1 * inv, m2 = s2 * inv, rs = a.rs[row];
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + c0, u);
+                tmem_ld_wait();
+                float o[32];
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    float nrm[8], p[8];
+                    load8(sS, tid, c0 + j, nrm);
+                    load8(sS + 65536, tid, c0 + j, p);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        o[j + q] = (c0 + j + q < a.ncols) ? rs * (__uint_as_float(u[j + q]) - m1 - nrm[q] * m2) * gelu_grad_f(p[q]) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, o + j);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, ND);
+}
+
+// ---------------------------------------------------------------------------
+// weight gradients: Gt[256][64] += sum over a slab of rows of P[row][:]^T S[row][:]
+// (P: [rows][256] bf16, S: [rows][64] bf16; both tiles go to the tensor cores as TMA left them:
+// P^T is an MN-major A operand, S an MN-major B operand, the contraction runs over the rows)
+// ---------------------------------------------------------------------------
+constexpr int kWgStage = 65536 + 16384;
+constexpr int kWgSmem = 2 * kWgStage + 1024;
+
+__global__ void __launch_bounds__(128)
+ltc_wgrad_kernel(const __grid_constant__ CUtensorMap mP, const __grid_constant__ CUtensorMap mS, float* __restrict__ Gt,
+                 int ntiles, int tiles_per_cta, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align1024(smem_raw);
+    __shared__ uint64_t bar_full[2], bar_free[2], bar_done;
+    __shared__ uint32_t tm_slot;
+    const int tid = threadIdx.x, warp = tid / 32;
+    const int t0 = blockIdx.x * tiles_per_cta;
+    const int T = min(tiles_per_cta, ntiles - t0);
+    if (tid == 0) {
+        cta_giveup_init();
+        mbar_init(&bar_full[0], 1); mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1);
+        mbar_init(&bar_done, 1);
+        mbar_fence_init();
+    }
+    if (warp == 0) { tmem_alloc(&tm_slot, 128); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tm_slot;
+    if (tid == 0) {
+        auto load = [&](int j) {
+            const int s = j & 1;
+            uint8_t* sP = smem + s * kWgStage;
+            mbar_expect_tx(&bar_full[s], kWgStage);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) tma_load_2d(sP + g * 16384, &mP, g * 64, (t0 + j) * 128, &bar_full[s]);
+            tma_load_2d(sP + 65536, &mS, 0, (t0 + j) * 128, &bar_full[s]);
+        };
+        load(0);
+        if (T > 1) load(1);
+        constexpr uint32_t idesc = idesc_bf16(128, 64, true, true);
+        bool ok = true;
+        for (int j = 0; j < T && ok; ++j) {
+            const int s = j & 1;
+            ok = mbar_spin(&bar_full[s], (j >> 1) & 1, status, kErrTma);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t base = smem_u32(smem + s * kWgStage);
+            const uint64_t sd = smem_desc(base + 65536, 0, 1024, kSwz128);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const uint64_t pd = smem_desc(base + half * 32768, 16384, 1024, kSwz128);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_ss(tm + half * 64, desc_off(pd, k * 2048), desc_off(sd, k * 2048), idesc, (j > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&bar_free[s]);
+            if (j + 2 < T) {
+                ok = mbar_spin(&bar_free[s], (j >> 1) & 1, status, kErrMma);
+                if (ok) load(j + 2);
+            }
+        }
+        if (ok) umma_commit(&bar_done);
+    }
+    const bool ok = mbar_wait(&bar_done, 0, status, kErrMma);
+    tc_fence_after();
+    if (ok) {
+        const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld32(lane_tm + half * 64 + c0, u);
+                tmem_ld_wait();
+                float* dst = Gt + (size_t)(half * 128 + tid) * 64 + c0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) atomicAdd(dst + j, __uint_as_float(u[j]));
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 128);
+}
+
+// ---------------------------------------------------------------------------
+// CUDA-core helpers around the layers
+// ---------------------------------------------------------------------------
+struct Slice {
+    int H, n; int64_t sb, sh, sn;
+    __device__ int64_t row(size_t R) const {
+        const int bh = (int)(R / n), i = (int)(R % n);
+        return (int64_t)(bh / H) * sb + (int64_t)(bh % H) * sh + (int64_t)i * sn;
+    }
+};
+
+// n0 = (x - mean) / sigma of every row (one warp per row, two columns per lane), 1 / sigma kept
+__global__ void __launch_bounds__(256)
+ltc_ln0_kernel(Slice sl, const bf16* __restrict__ X, size_t row0, int rows, bf16* __restrict__ n0, bf16* __restrict__ n0_lo,
+               float* __restrict__ rs0) {
+    const int lane = threadIdx.x % 32;
+    const int i = blockIdx.x * 8 + threadIdx.x / 32;
+    if (i >= rows) return;
+    const __nv_bfloat162 x2 = *reinterpret_cast<const __nv_bfloat162*>(X + sl.row(row0 + i) + 2 * lane);
+    const float a = __low2float(x2), b = __high2float(x2);
+    float s = a + b;
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mu = s * (1.f / 64.f);
+    float v = (a - mu) * (a - mu) + (b - mu) * (b - mu);
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const float rs = rsqrtf(v * (1.f / 64.f) + kLnEps);
+    const float na = (a - mu) * rs, nb = (b - mu) * rs;
+    const float ha = __bfloat162float(__float2bfloat16_rn(na)), hb = __bfloat162float(__float2bfloat16_rn(nb));
+    *reinterpret_cast<uint32_t*>(n0 + (size_t)i * 64 + 2 * lane) = pack_bf16(ha, hb);
+    *reinterpret_cast<uint32_t*>(n0_lo + (size_t)i * 64 + 2 * lane) = pack_bf16(na - ha, nb - hb);
+    if (lane == 0) rs0[i] = rs;
+}
+
+// dX = back through the first normalisation of the summed gradient of n0 (+ add)
+__global__ void __launch_bounds__(256)
+ltc_ln0_bwd_kernel(Slice sl, size_t row0, int rows, const float* __restrict__ dn0, const bf16* __restrict__ n0,
+                   const float* __restrict__ rs0, const float* __restrict__ add, bf16* __restrict__ dX) {
+    const int lane = threadIdx.x % 32;
+    const int i = blockIdx.x * 8 + threadIdx.x / 32;
+    if (i >= rows) return;
+    const float2 d = *reinterpret_cast<const float2*>(dn0 + (size_t)i * 64 + 2 * lane);
+    const __nv_bfloat162 n2 = *reinterpret_cast<const __nv_bfloat162*>(n0 + (size_t)i * 64 + 2 * lane);
+    const float na = __low2float(n2), nb = __high2float(n2);
+    float s1 = d.x + d.y, s2 = d.x * na + d.y * nb;
+    for (int o = 16; o > 0; o >>= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s2 += __shfl_xor_sync(0xffffffffu, s2, o); }
+    const float m1 = s1 * (1.f / 64.f), m2 = s2 * (1.f / 64.f), rs = rs0[i];
+    float oa = rs * (d.x - m1 - na * m2), ob = rs * (d.y - m1 - nb * m2);
+    if (add != nullptr) {
+        const float2 q = *reinterpret_cast<const float2*>(add + (row0 + i) * 64 + 2 * lane);
+        oa += q.x; ob += q.y;
+    }
+    *reinterpret_cast<uint32_t*>(dX + sl.row(row0 + i) + 2 * lane) = pack_bf16(oa, ob);
+}
+
+// M = sqrt(r) tanh(f1 f2 / sqrt(r))
+__global__ void __launch_bounds__(256)
+ltc_combine_kernel(const float* __restrict__ f1, const float* __restrict__ f2, int r, size_t count, float* __restrict__ M) {
+    const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= count) return;
+    const float sr = sqrtf((float)r);
+    M[e] = sr * tanhf(f1[e] * f2[e] / sr);
+}
+
+// df1 = dM (1 - t^2) f2, df2 = dM (1 - t^2) f1 as bf16 rows of 64 columns (zero beyond r)
+__global__ void __launch_bounds__(256)
+ltc_combine_bwd_kernel(const float* __restrict__ f1, const float* __restrict__ f2, const float* __restrict__ dM, int r,
+                       size_t rows, bf16* __restrict__ df1, bf16* __restrict__ df2) {
+    const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= rows * 64) return;
+    const size_t row = e / 64;
+    const int c = (int)(e % 64);
+    float o1 = 0.f, o2 = 0.f;
+    if (c < r) {
+        const float a = f1[row * r + c], b = f2[row * r + c];
+        const float t = tanhf(a * b * rsqrtf((float)r));
+        const float du = dM[row * r + c] * (1.f - t * t);
+        o1 = du * b; o2 = du * a;
+    }
+    df1[e] = __float2bfloat16_rn(o1);
+    df2[e] = __float2bfloat16_rn(o2);
+}
+
+// out[c] += sum over rows of A[row][c]   (A: [rows][W] bf16, W = 64 or 256; 256 rows per CTA)
+__global__ void __launch_bounds__(256)
+ltc_colsum_kernel(const bf16* __restrict__ A, int W, int rows, float* __restrict__ out) {
+    const int c = threadIdx.x % W, sub = threadIdx.x / W, step = 256 / W;
+    const int r0 = blockIdx.x * 256, r1 = min(rows, r0 + 256);
+    float acc = 0.f;
+    for (int i = r0 + sub; i < r1; i += step) acc += __bfloat162float(A[(size_t)i * W + c]);
+    atomicAdd(out + c, acc);
+}
+
+// parameter gradients of one network from the four accumulators and the column sums
+//   G1t = dp1^T n0, G2 = n1^T da2, G3t = dp3^T a2, G4 = a3^T df   (each [256][64])
+__global__ void __launch_bounds__(256)
+ltc_finish_kernel(int h, int r, const float* __restrict__ params, const float* __restrict__ G, const float* __restrict__ sums,
+                  float* __restrict__ dparams) {
+    const NetLayout nl(h, r);
+    const int net = blockIdx.y, m = nl.m;
+    const float* P = params + (size_t)net * nl.count;
+    float* dP = dparams + (size_t)net * nl.count;
+    const float* G1t = G + (size_t)net * 4 * kMat;
+    const float* G2 = G1t + kMat;
+    const float* G3t = G2 + kMat;
+    const float* G4 = G3t + kMat;
+    const float* s_dp1 = sums + (size_t)net * kSums;
+    const float* s_da2 = s_dp1 + 256;
+    const float* s_dp3 = s_da2 + 64;
+    const float* s_df = s_dp3 + 256;
+    const int e = blockIdx.x * 256 + threadIdx.x;
+    if (e >= nl.count) return;
+    float g = 0.f;
+    if (e < nl.c0) {                                           // dg0[k] = sum_j W1[k][j] G1t[j][k]
+        const int k = e - nl.g0;
+        for (int j = 0; j < m; ++j) g = fmaf(P[nl.W1 + k * m + j], G1t[j * 64 + k], g);
+    } else if (e < nl.W1) {                                    // dc0[k] = sum_j W1[k][j] s_dp1[j]
+        const int k = e - nl.c0;
+        for (int j = 0; j < m; ++j) g = fmaf(P[nl.W1 + k * m + j], s_dp1[j], g);
+    } else if (e < nl.b1) {                                    // dW1[k][j] = g0[k] G1t[j][k] + c0[k] s_dp1[j]
+        const int k = (e - nl.W1) / m, j = (e - nl.W1) % m;
+        g = P[nl.g0 + k] * G1t[j * 64 + k] + P[nl.c0 + k] * s_dp1[j];
+    } else if (e < nl.g1) {
+        g = s_dp1[e - nl.b1];
+    } else if (e < nl.c1) {                                    // dg1[j] = sum_c W2[j][c] G2[j][c]
+        const int j = e - nl.g1;
+        for (int c = 0; c < r; ++c) g = fmaf(P[nl.W2 + j * r + c], G2[j * 64 + c], g);
+    } else if (e < nl.W2) {                                    // dc1[j] = sum_c W2[j][c] s_da2[c]
+        const int j = e - nl.c1;
+        for (int c = 0; c < r; ++c) g = fmaf(P[nl.W2 + j * r + c], s_da2[c], g);
+    } else if (e < nl.b2) {                                    // dW2[j][c] = g1[j] G2[j][c] + c1[j] s_da2[c]
+        const int j = (e - nl.W2) / r, c = (e - nl.W2) % r;
+        g = P[nl.g1 + j] * G2[j * 64 + c] + P[nl.c1 + j] * s_da2[c];
+    } else if (e < nl.W3) {
+        g = s_da2[e - nl.b2];
+    } else if (e < nl.b3) {                                    // dW3[c][j] = G3t[j][c]
+        const int c = (e - nl.W3) / m, j = (e - nl.W3) % m;
+        g = G3t[j * 64 + c];
+    } else if (e < nl.W4) {
+        g = s_dp3[e - nl.b3];
+    } else if (e < nl.b4) {                                    // dW4[j][c] = G4[j][c]
+        const int j = (e - nl.W4) / r, c = (e - nl.W4) % r;
+        g = G4[j * 64 + c];
+    } else {
+        g = s_df[e - nl.b4];
+    }
+    dP[e] += g;
+}
+
+// ---------------------------------------------------------------------------
+// host
+// ---------------------------------------------------------------------------
+struct NetBuf { size_t p1, n1, n1_lo, p3, a3, a3_lo, a2, a2_lo, rs1, f; };
+struct LtcWs {
+    size_t bank, vec, G, sums, n0, n0_lo, rs0, df[2], dp3, da2, dp1, dn0, total;
+    NetBuf net[2];
+    size_t C;
+};
+
+LtcWs ltc_ws(const Dims& d, bool backward) {
+    LtcWs w{};
+    const size_t rows = (size_t)d.BH() * d.n;
+    w.C = rows < kChunkRows ? rows : kChunkRows;
+    const size_t C = w.C;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes); return o; };
+    w.bank = take((size_t)2 * kBank * kMat * sizeof(bf16));
+    w.vec = take((size_t)2 * kVec * sizeof(float));
+    w.G = take((size_t)2 * 4 * kMat * sizeof(float));       // G and sums are zeroed together
+    w.sums = take((size_t)2 * kSums * sizeof(float));
+    w.n0 = take(C * 64 * sizeof(bf16));
+    w.n0_lo = take(C * 64 * sizeof(bf16));
+    w.rs0 = take(C * sizeof(float));
+    for (int t = 0; t < 2; ++t) {
+        w.net[t].p1 = take(C * 256 * sizeof(bf16));
+        w.net[t].n1 = take(C * 256 * sizeof(bf16));
+        w.net[t].n1_lo = take(C * 256 * sizeof(bf16));
+        w.net[t].p3 = take(C * 256 * sizeof(bf16));
+        w.net[t].a3 = take(C * 256 * sizeof(bf16));
+        w.net[t].a3_lo = take(C * 256 * sizeof(bf16));
+        w.net[t].a2 = take(C * 64 * sizeof(bf16));
+        w.net[t].a2_lo = take(C * 64 * sizeof(bf16));
+        w.net[t].rs1 = take(C * sizeof(float));
+        w.net[t].f = take(C * d.r * sizeof(float));
+    }
+    if (backward) {
+        w.df[0] = take(C * 64 * sizeof(bf16));
+        w.df[1] = take(C * 64 * sizeof(bf16));
+        w.dp3 = take(C * 256 * sizeof(bf16));
+        w.da2 = take(C * 64 * sizeof(bf16));
+        w.dp1 = take(C * 256 * sizeof(bf16));
+        w.dn0 = take(C * 64 * sizeof(float));
+    }
+    w.total = off;
+    return w;
+}
+
+struct Maps {                       // tensor maps over the chunk buffers (built once per call)
+    CUtensorMap bank[2][kBank];
+    CUtensorMap n0, n0_lo, df[2], dp3, da2, dp1;
+    CUtensorMap p1[2], n1[2], n1_lo[2], p3[2], a3[2], a3_lo[2], a2[2], a2_lo[2];
+};
+
+bool build_maps(const LtcWs& w, char* ws, bool backward, Maps* M) {
+    const int64_t C = (int64_t)w.C;
+    bool ok = true;
+    for (int t = 0; t < 2; ++t) {
+        for (int i = 0; i < kBank; ++i) {
+            const bf16* base = reinterpret_cast<const bf16*>(ws + w.bank) + ((size_t)t * kBank + i) * kMat;
+            ok = ok && ((i % 2 == 0) ? tc_map_2d(&M->bank[t][i], base, 256, 64, 64) : tc_map_2d(&M->bank[t][i], base, 64, 256, 256));
+        }
+        ok = ok && tc_map_2d(&M->p1[t], ws + w.net[t].p1, 256, C, 128) && tc_map_2d(&M->n1[t], ws + w.net[t].n1, 256, C, 128) &&
+             tc_map_2d(&M->p3[t], ws + w.net[t].p3, 256, C, 128) && tc_map_2d(&M->a3[t], ws + w.net[t].a3, 256, C, 128) &&
+             tc_map_2d(&M->a2[t], ws + w.net[t].a2, 64, C, 128) && tc_map_2d(&M->n1_lo[t], ws + w.net[t].n1_lo, 256, C, 128) &&
+             tc_map_2d(&M->a3_lo[t], ws + w.net[t].a3_lo, 256, C, 128) && tc_map_2d(&M->a2_lo[t], ws + w.net[t].a2_lo, 64, C, 128);
+    }
+    ok = ok && tc_map_2d(&M->n0, ws + w.n0, 64, C, 128) && tc_map_2d(&M->n0_lo, ws + w.n0_lo, 64, C, 128);
+    if (backward)
+        ok = ok && tc_map_2d(&M->df[0], ws + w.df[0], 64, C, 128) && tc_map_2d(&M->df[1], ws + w.df[1], 64, C, 128) &&
+             tc_map_2d(&M->dp3, ws + w.dp3, 256, C, 128) && tc_map_2d(&M->da2, ws + w.da2, 64, C, 128) &&
+             tc_map_2d(&M->dp1, ws + w.dp1, 256, C, 128);
+    return ok;
+}
+
+// backward's layers: single bf16 operands, side tiles S0, S1 where the epilogue needs them
+template <int KD, int ND, int EPI>
+cudaError_t dense(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mS0, const CUtensorMap& mS1,
+                  const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
+    auto kern = ltc_dense_kernel<KD, ND, EPI, false>;
+    constexpr int smem = DenseSmem<KD, ND, EPI, false>::bytes;
+    PSK_TRY(set_smem(kern, smem));
+    prof_begin("ltc_dense_kernel", s);
+    kern<<<tiles, 128, smem, s>>>(mA, mA, mB, mB, mS0, mS1, a, status);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+// forward's layers: hi + lo operand pairs
+template <int KD, int ND, int EPI>
+cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
+                        const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
+    auto kern = ltc_dense_kernel<KD, ND, EPI, true>;
+    constexpr int smem = DenseSmem<KD, ND, EPI, true>::bytes;
+    PSK_TRY(set_smem(kern, smem));
+    prof_begin("ltc_dense_kernel", s);
+    kern<<<tiles, 128, smem, s>>>(mA, mA2, mB, mB2, mA, mA, a, status);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t wgrad(const CUtensorMap& mP, const CUtensorMap& mS, float* Gt, int tiles, int* status, cudaStream_t s,
+                  int* launches) {
+    PSK_TRY(set_smem(ltc_wgrad_kernel, kWgSmem));
+    int per = (tiles + 295) / 296;            // about two CTAs per SM, but at least four tiles per result added
+    if (per < 4) per = tiles < 4 ? tiles : 4;
+    const int grid = (tiles + per - 1) / per;
+    prof_begin("ltc_wgrad_kernel", s);
+    ltc_wgrad_kernel<<<grid, 128, kWgSmem, s>>>(mP, mS, Gt, tiles, per, status);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t colsum(const bf16* A, int W, int rows, float* out, cudaStream_t s, int* launches) {
+    prof_begin("ltc_colsum_kernel", s);
+    ltc_colsum_kernel<<<(rows + 255) / 256, 256, 0, s>>>(A, W, rows, out);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+// forward of both networks on `c` rows starting at row0: activations and f into the chunk buffers
+cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const void* X, size_t row0, int c, char* ws,
+                          int* status, cudaStream_t s, int* launches) {
+    const Slice sl{d.H, d.n, d.sb, d.sh, d.sn};
+    const int tiles = c / 128, m = 8 * d.r;
+    prof_begin("ltc_ln0_kernel", s);
+    ltc_ln0_kernel<<<(c + 7) / 8, 256, 0, s>>>(sl, (const bf16*)X, row0, c, (bf16*)(ws + w.n0), (bf16*)(ws + w.n0_lo), (float*)(ws + w.rs0));
+    prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    for (int t = 0; t < 2; ++t) {
+        const NetBuf& nb = w.net[t];
+        const float* vec = (const float*)(ws + w.vec) + (size_t)t * kVec;
+        DenseArgs a{};
+        a = DenseArgs{vec, (bf16*)(ws + nb.p1), (bf16*)(ws + nb.n1), (bf16*)(ws + nb.n1_lo), (float*)(ws + nb.rs1), nullptr, m, 0};
+        PSK_TRY((dense_split<64, 256, EPI_LN>(M.n0, M.n0_lo, M.bank[t][0], M.bank[t][8], a, tiles, status, s, launches)));
+        a = DenseArgs{vec + 256, (bf16*)(ws + nb.a2), (bf16*)(ws + nb.a2_lo), nullptr, nullptr, nullptr, 0, 0};
+        PSK_TRY((dense_split<256, 64, EPI_B64>(M.n1[t], M.n1_lo[t], M.bank[t][1], M.bank[t][9], a, tiles, status, s, launches)));
+        a = DenseArgs{vec + 320, (bf16*)(ws + nb.p3), (bf16*)(ws + nb.a3), (bf16*)(ws + nb.a3_lo), nullptr, nullptr, m, 0};
+        PSK_TRY((dense_split<64, 256, EPI_GELU>(M.a2[t], M.a2_lo[t], M.bank[t][2], M.bank[t][10], a, tiles, status, s, launches)));
+        a = DenseArgs{vec + 576, nullptr, nullptr, nullptr, (float*)(ws + nb.f), nullptr, d.r, 0};
+        PSK_TRY((dense_split<256, 64, EPI_F32>(M.a3[t], M.a3_lo[t], M.bank[t][3], M.bank[t][11], a, tiles, status, s, launches)));
+    }
+    return cudaSuccess;
+}
+
+}  // namespace
+
+bool learned_tc_supported(const Dims& d) { return d.bf16 && d.learned && d.h == 64 && d.r <= 32 && d.r % 4 == 0; }
+
+size_t learned_tc_workspace_bytes(const Dims& d, bool backward) { return ltc_ws(d, backward).total; }
+
+// operand bank of both networks; backward: also clears the gradient accumulators
+cudaError_t learned_tc_prepare(const Dims& d, bool backward, char* ws, cudaStream_t s, int* launches) {
+    const LtcWs w = ltc_ws(d, backward);
+    prof_begin("ltc_bank_kernel", s);
+    ltc_bank_kernel<<<dim3((8 * kMat + kVec + 255) / 256, 2), 256, 0, s>>>(d.h, d.r, d.lparams, (bf16*)(ws + w.bank), (float*)(ws + w.vec));
+    prof_end(s);
+    ++*launches;
+    PSK_TRY(cudaGetLastError());
+    if (backward) PSK_TRY(cudaMemsetAsync(ws + w.G, 0, (w.sums - w.G) + (size_t)2 * kSums * sizeof(float), s));
+    return cudaSuccess;
+}
+
+cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* Mout, char* ws, int* status, cudaStream_t s, int* launches) {
+    const LtcWs w = ltc_ws(d, false);            // the forward's buffers come first in either layout
+    Maps M;
+    if (!build_maps(w, ws, false, &M)) return cudaErrorInvalidValue;
+    const size_t rows = (size_t)d.BH() * d.n;
+    for (size_t row0 = 0; row0 < rows; row0 += w.C) {
+        const int c = (int)(rows - row0 < w.C ? rows - row0 : w.C);
+        PSK_TRY(forward_chunk(d, w, M, X, row0, c, ws, status, s, launches));
+        const size_t cnt = (size_t)c * d.r;
+        prof_begin("ltc_combine_kernel", s);
+        ltc_combine_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, s>>>((const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f),
+                                                                         d.r, cnt, Mout + row0 * d.r);
+        prof_end(s);
+        ++*launches;
+        PSK_TRY(cudaGetLastError());
+    }
+    return cudaSuccess;
+}
+
+// dX = chain rule of sum(dM * M) through both networks (+ add); the weight-gradient
+// accumulators in the workspace grow by this tensor's share (learned_tc_finish turns them into
+// parameter gradients)
+cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const float* add, void* dX, char* ws,
+                                  int* status, cudaStream_t s, int* launches) {
+    const LtcWs w = ltc_ws(d, true);
+    Maps M;
+    if (!build_maps(w, ws, true, &M)) return cudaErrorInvalidValue;
+    const Slice sl{d.H, d.n, d.sb, d.sh, d.sn};
+    const size_t rows = (size_t)d.BH() * d.n;
+    const int m = 8 * d.r;
+    for (size_t row0 = 0; row0 < rows; row0 += w.C) {
+        const int c = (int)(rows - row0 < w.C ? rows - row0 : w.C);
+        const int tiles = c / 128;
+        PSK_TRY(forward_chunk(d, w, M, X, row0, c, ws, status, s, launches));
+        prof_begin("ltc_combine_bwd_kernel", s);
+        ltc_combine_bwd_kernel<<<(unsigned)(((size_t)c * 64 + 255) / 256), 256, 0, s>>>(
+            (const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f), dM + row0 * d.r, d.r, (size_t)c,
+            (bf16*)(ws + w.df[0]), (bf16*)(ws + w.df[1]));
+        prof_end(s);
+        ++*launches;
+        PSK_TRY(cudaGetLastError());
+        for (int t = 0; t < 2; ++t) {
+            const NetBuf& nb = w.net[t];
+            float* G = (float*)(ws + w.G) + (size_t)t * 4 * kMat;
+            float* sums = (float*)(ws + w.sums) + (size_t)t * kSums;
+            DenseArgs a{};
+            // dp3 = (df W4^T) * gelu'(p3);  dW4 ~ a3^T df
+            a = DenseArgs{nullptr, (bf16*)(ws + w.dp3), nullptr, nullptr, nullptr, nullptr, m, 0};
+            PSK_TRY((dense<64, 256, EPI_DGELU>(M.df[t], M.bank[t][4], M.p3[t], M.p3[t], a, tiles, status, s, launches)));
+            PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, tiles, status, s, launches));
+            PSK_TRY(colsum((const bf16*)(ws + w.df[t]), 64, c, sums + 576, s, launches));
+            // da2 = dp3 W3^T;  dW3 ~ dp3^T a2
+            PSK_TRY(wgrad(M.dp3, M.a2[t], G + 2 * kMat, tiles, status, s, launches));
+            PSK_TRY(colsum((const bf16*)(ws + w.dp3), 256, c, sums + 320, s, launches));
+            a = DenseArgs{nullptr, (bf16*)(ws + w.da2), nullptr, nullptr, nullptr, nullptr, 0, 0};
+            PSK_TRY((dense<256, 64, EPI_B64>(M.dp3, M.bank[t][5], M.n0, M.n0, a, tiles, status, s, launches)));
+            // dp1 = LN1 backward(da2 (g1 W2)^T) * gelu'(p1);  dW2 ~ n1^T da2
+            PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, tiles, status, s, launches));
+            PSK_TRY(colsum((const bf16*)(ws + w.da2), 64, c, sums + 256, s, launches));
+            a = DenseArgs{nullptr, (bf16*)(ws + w.dp1), nullptr, nullptr, nullptr, (const float*)(ws + nb.rs1), m, 0};
+            PSK_TRY((dense<64, 256, EPI_LNBWD>(M.da2, M.bank[t][6], M.n1[t], M.p1[t], a, tiles, status, s, launches)));
+            // dn0 (+)= dp1 (g0 W1)^T;  dW1 ~ dp1^T n0
+            PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, tiles, status, s, launches));
+            PSK_TRY(colsum((const bf16*)(ws + w.dp1), 256, c, sums + 0, s, launches));
+            a = DenseArgs{nullptr, nullptr, nullptr, nullptr, (float*)(ws + w.dn0), nullptr, 64, t};
+            PSK_TRY((dense<256, 64, EPI_F32>(M.dp1, M.bank[t][7], M.n0, M.n0, a, tiles, status, s, launches)));
+        }
+        prof_begin("ltc_ln0_bwd_kernel", s);
+        ltc_ln0_bwd_kernel<<<(c + 7) / 8, 256, 0, s>>>(sl, row0, c, (const float*)(ws + w.dn0), (const bf16*)(ws + w.n0),
+                                                      (const float*)(ws + w.rs0), add, (bf16*)dX);
+        prof_end(s);
+        ++*launches;
+        PSK_TRY(cudaGetLastError());
+    }
+    return cudaSuccess;
+}
+
+// parameter gradients (added to d.dlparams) from everything learned_tc_sketch_bwd accumulated
+cudaError_t learned_tc_finish(const Dims& d, char* ws, cudaStream_t s, int* launches) {
+    const LtcWs w = ltc_ws(d, true);
+    const int count = NetLayout(d.h, d.r).count;
+    prof_begin("ltc_finish_kernel", s);
+    ltc_finish_kernel<<<dim3((count + 255) / 256, 2), 256, 0, s>>>(d.h, d.r, d.lparams, (const float*)(ws + w.G),
+                                                                   (const float*)(ws + w.sums), d.dlparams);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace psk

@@ -52,6 +52,18 @@ bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t 
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// Row-major [rows][cols] bf16 matrix (cols a multiple of 64); box = box_rows rows x 64 columns,
+// 128-byte swizzle.
+bool tc_map_2d(CUtensorMap* m, const void* base, int cols, int64_t rows, int box_rows) {
+    EncodeFn enc = encoder();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows}, es[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 // States S[nblk][FP][80] bf16 (feature-major rows: 64 state columns, the last column, 15 zeros).
 // Box = 64 features x 64 columns; a second box at column 64 brings the last column (columns
 // beyond 80 lie outside the tensor and arrive as zeros).

@@ -69,7 +69,10 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
     kernels = {name for name, _ in psk.profile_records()}
     psk.profile_enable(False)
     on_tc = dtype == "bf16" and r <= 32 and not local and path != psk.PATH_CUDA_CORES
-    assert ("tc_bwd_k_kernel" in kernels) == on_tc and "learned_sketch_bwd_kernel" in kernels
+    assert ("tc_bwd_k_kernel" in kernels) == on_tc
+    # on that route the networks run on the tensor cores too (dense layers and weight gradients)
+    assert ("ltc_dense_kernel" in kernels and "ltc_wgrad_kernel" in kernels) == on_tc
+    assert ("learned_sketch_bwd_kernel" in kernels) == (not on_tc)
     tol = TOL[dtype]
     diag = "exact" if local else "LR"
     g1_sum = {k: 0.0 for k in orc.NET_KEYS}
