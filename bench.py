@@ -266,6 +266,69 @@ def time_other_config(psk, wl, name, steps, warmup, local, pk, device_index):
             "clocks": clocks}
 
 
+def time_variant(psk, wl, name, base, steps, warmup, device_index):
+    """A short timed run of another member of the family at the headline configuration's B, H, n
+    (forward + backward, bf16): "learned" = the learnable sketch of the appendix (r = 32, b = 256, parameter
+    gradients included), "p2" = exact degree-2 attention (r = h = 64, b = 512), "p8" = degree 8 (r = 32)."""
+    import torch
+    binding = psk.binding
+    r, b, p = {"learned": (32, 256, 4), "p2": (64, 512, 2), "p8": (32, 256, 8)}[name]
+    w = wl.Workload(name, base.B, base.H, base.n, base.h, r, 4, b, "bf16", True, base.data_seed, base.g_seed)
+    inp = wl.make_inputs(w, "cuda", with_dO=True)
+    Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
+    flags = psk.FLAG_KEEP_STATES
+    O = torch.empty_like(Q)
+    den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
+    grads = tuple(torch.empty_like(Q) for _ in range(3))
+    if name == "learned":
+        flat = binding.pack_learned_params(*wl.learned_network_params(w.h, r, base.g_seed))
+        ws = torch.empty(binding.learned_workspace_bytes(Q, r, b), dtype=torch.uint8, device="cuda")
+
+        def step():
+            o, d = binding.learned_attn_fwd(Q, K, V, flat, r, b, 0, ws)
+            binding.learned_attn_bwd(Q, K, V, flat, o, d, dO, r, b, 0, ws)
+    else:
+        if p == 2:
+            Q.mul_(0.5); K.mul_(0.5)        # (q.k)^2 with |q|^2 = 64: keep the weights on the headline's scale
+            G1 = G2 = None
+        else:
+            Q.mul_(0.5); K.mul_(0.5)
+            gen = torch.Generator(device="cpu").manual_seed(base.g_seed)
+            G1 = torch.randn(w.H, 2 * w.h + r, r, generator=gen).to(Q.dtype).cuda()
+            G2 = torch.randn(w.H, 2 * w.h + r, r, generator=gen).to(Q.dtype).cuda()
+        shp = binding.make_shape(Q, G1, r, b, p, psk.PATH_AUTO, flags)
+        ws = torch.empty(max(psk.workspace_bytes(shp, False), psk.workspace_bytes(shp, True)), dtype=torch.uint8, device="cuda")
+
+        def step():
+            psk.causal_attn_fwd(Q, K, V, G1, G2, b, p, psk.PATH_AUTO, ws, O, den, flags)
+            psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, p, psk.PATH_AUTO, ws, grads, flags)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    psk.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.stop()
+    agg = {}
+    for kname, t in psk.profile_records():
+        agg[kname] = agg.get(kname, 0.0) + t
+    psk.profile_enable(False)
+    if psk.check(ws) != 0:
+        raise RuntimeError("device-side error while timing %s" % name)
+    return {"B": w.B, "H": w.H, "n": w.n, "r": r, "b": b, "p": p, "passes": "fwd+bwd", "steps": steps, "warmup": warmup,
+            "ms_per_step": ms, "model_tokens_per_s": w.model_tokens / (ms / 1e3),
+            "kernels_ms_per_step": {k: round(v / steps, 3) for k, v in sorted(agg.items(), key=lambda kv: -kv[1])},
+            "clocks": clocks}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -283,6 +346,9 @@ def main():
     ap.add_argument("--others", default="c1,c3,c4",
                     help="other configurations timed briefly after the headline one (N = 1 only); '' for none")
     ap.add_argument("--other-steps", type=int, default=5)
+    ap.add_argument("--variants", default="learned,p2,p8",
+                    help="other members of the family timed briefly at the headline's B, H, n (N=1 only; '' = none)")
+    ap.add_argument("--variant-steps", type=int, default=2)
     ap.add_argument("--seq-segments", type=int, default=0,
                     help="runs a head's blocks are cut into for the state scan (0: the library chooses)")
     ap.add_argument("--no-keep-states", action="store_true",
@@ -490,6 +556,12 @@ def main():
         for name in [x for x in args.others.split(",") if x and x != w.name]:
             others[name] = time_other_config(psk, wl, name, args.other_steps, args.warmup, args.local_exact, pk, local)
             torch.cuda.empty_cache()
+    variants = None
+    if world == 1 and args.variants:
+        variants = {}
+        for name in [x for x in args.variants.split(",") if x]:
+            variants[name] = time_variant(psk, wl, name, w, args.variant_steps, 1, local)
+            torch.cuda.empty_cache()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -509,7 +581,7 @@ def main():
                                     "nominal_2250": executed_tflops / world / 2250.0, "source": pk["source"],
                                     "flops": "executed MMA flops (symmetric features, masked tiles skipped)"},
         "ms_x_sm_mhz": (ms / args.steps) * clocks["sm_mhz"] if (clocks and clocks.get("sm_mhz")) else None,
-        "other_configs": others,
+        "other_configs": others, "variants": variants,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0], "roofline": roof, "kernels": kernels,
         "cpu_baseline": cpu,
     }

@@ -379,6 +379,12 @@ def learned_sketch(X, params, r, want_phi=False):
     return M, Phi
 
 
+def learned_workspace_bytes(Q, r, b, flags=0, for_backward=True, path=PATH_AUTO):
+    """psk_learned_workspace_bytes for tensors laid out like Q (the backward's covers the forward's)."""
+    shp = _learned_shape(Q, r, b, flags, path)
+    return int(lib().psk_learned_workspace_bytes(byref(shp), 1 if for_backward else 0))
+
+
 def learned_attn_fwd(Q, K, V, params, r, b, flags=0, workspace=None, path=PATH_AUTO):
     """psk_learned_attn_fwd: returns (O, denom)."""
     _require_cuda(Q, K, V, params)

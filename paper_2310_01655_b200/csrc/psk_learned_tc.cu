@@ -31,10 +31,23 @@ constexpr int kBank = 12;                             // operand matrices per ne
 constexpr int kVec = 256 + 64 + 256 + 64;             // folded biases of one network: b1' | b2' | b3 | b4
 constexpr int kSums = 256 + 64 + 256 + 64;            // column sums of one network: dp1 | da2 | dp3 | df
 
-__device__ __forceinline__ float gelu_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
-__device__ __forceinline__ float gelu_grad_f(float x) {
-    return 0.5f * (1.f + erff(x * 0.70710678118654752f)) + x * __expf(-0.5f * x * x) * 0.3989422804014327f;
+// Phi(x) and the normal density at x.  erf by a five-term rational approximation in
+// t = 1 / (1 + 0.3275911 z), z = |x| / sqrt(2) (absolute error 1.5e-7), whose exponential
+// exp(-z^2) = exp(-x^2 / 2) is the density's too.
+__device__ __forceinline__ void normal_parts(float x, float& cdf, float& pdf) {
+    const float z = fabsf(x) * 0.70710678118654752f;
+    const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
+    const float e = __expf(-z * z);
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float q = 0.5f * poly * t * e;                 // 1 - Phi(|x|)
+    cdf = x >= 0.f ? 1.f - q : q;
+    pdf = 0.3989422804014327f * e;
 }
+__device__ __forceinline__ float gelu_f(float x) { float c, d; normal_parts(x, c, d); return x * c; }
+__device__ __forceinline__ float gelu_grad_f(float x) { float c, d; normal_parts(x, c, d); return fmaf(x, d, c); }
 
 struct NetLayout {
     int h, r, m;
@@ -114,9 +127,9 @@ struct DenseArgs {
     bf16* out0;             // bf16 outputs, [rows][ND]
     bf16* out1;
     bf16* out2;
-    float* outf;            // EPI_F32: [rows][ncols]; EPI_LN: 1 / sigma of every row
-    const float* rs;        // EPI_LNBWD: 1 / sigma of every row
-    int ncols;              // EPI_F32: columns stored; EPI_LN, EPI_LNBWD, EPI_DGELU, EPI_GELU: live columns (8r)
+    float* outf;            // EPI_F32: [rows][ncols]
+    const float* rs;        // (unused by the narrow layers)
+    int ncols;              // EPI_F32: columns stored
     int accumulate;         // EPI_F32: add to what is there
 };
 
@@ -131,17 +144,6 @@ __device__ __forceinline__ void store8_split(bf16* hi, bf16* lo, const float* v)
     store8(hi, h);
     store8(lo, l);
 }
-__device__ __forceinline__ void load8(const uint8_t* tile, int row, int col, float* v) {
-    // `tile`: [128 rows x 256 columns] bf16 as four 128-byte-swizzled [128 x 64] tiles
-    const uint4 q = *reinterpret_cast<const uint4*>(tile + (col / 64) * 16384 + swz128_offset(row, (col % 64) / 8));
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        v[2 * i] = __uint_as_float(w[i] << 16);
-        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-}
-
 // SPLIT (the forward's layers): activations and weights are both hi + lo pairs of bf16 arrays and
 // the product is A_hi B_hi + A_lo B_hi + A_hi B_lo.  A half sketch feeds fourth powers of
 // cancelling sums; single bf16 operands (2^-9 per entry, four layers deep) would leave percents of
@@ -150,8 +152,8 @@ template <int KD, int ND, int EPI, bool SPLIT>
 struct DenseSmem {
     static constexpr int kA1 = 128 * KD * 2, kB1 = KD * ND * 2;
     static constexpr int kA = kA1 * (SPLIT ? 2 : 1), kB = kB1 * (SPLIT ? 2 : 1);
-    static constexpr int kSides = EPI == EPI_DGELU ? 1 : (EPI == EPI_LNBWD ? 2 : 0);
-    static constexpr int bytes = kA + kB + kSides * 65536 + 1024;
+    static constexpr int kSides = 0;
+    static constexpr int bytes = kA + kB + 1024;
 };
 
 template <int KD, int ND, int EPI, bool SPLIT>
@@ -160,8 +162,7 @@ ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
                  const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2,
                  const __grid_constant__ CUtensorMap mS0, const __grid_constant__ CUtensorMap mS1, DenseArgs a,
                  int* status) {
-    static_assert((KD == 64 && ND == 256) || (KD == 256 && ND == 64), "two GEMM shapes");
-    static_assert(!SPLIT || DenseSmem<KD, ND, EPI, SPLIT>::kSides == 0, "the forward's layers have no side tiles");
+    static_assert(KD == 256 && ND == 64 && (EPI == EPI_B64 || EPI == EPI_F32), "the 256 -> 64 layers");
     using L = DenseSmem<KD, ND, EPI, SPLIT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sA = align1024(smem_raw);
@@ -261,117 +262,323 @@ ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
                     }
                 }
             }
-        } else if constexpr (EPI == EPI_GELU) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-                float p[32], g[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    p[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
-                    g[j] = (c0 + j < a.ncols) ? gelu_f(p[j]) : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    store8(a.out0 + row * 256 + c0 + j, p + j);
-                    store8_split(a.out1 + row * 256 + c0 + j, a.out2 + row * 256 + c0 + j, g + j);
-                }
-            }
-        } else if constexpr (EPI == EPI_LN) {
-            // pass 1: pre-activation out, gelu back into tensor memory, sums
-            float s = 0.f, ss = 0.f;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-                float p[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    p[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
-                    const float g = (c0 + j < a.ncols) ? gelu_f(p[j]) : 0.f;
-                    s += g; ss = fmaf(g, g, ss);
-                    u[j] = __float_as_uint(g);
-                }
-                tmem_st32(lane_tm + c0, u);
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, p + j);
-            }
-            tmem_st_wait();
-            const float inv = 1.f / (float)a.ncols;
-            const float mu = s * inv;
-            const float rs = rsqrtf(fmaxf(ss * inv - mu * mu, 0.f) + kLnEps);
-            a.outf[row] = rs;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-                float nrm[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) nrm[j] = (c0 + j < a.ncols) ? (__uint_as_float(u[j]) - mu) * rs : 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) store8_split(a.out1 + row * 256 + c0 + j, a.out2 + row * 256 + c0 + j, nrm + j);
-            }
-        } else if constexpr (EPI == EPI_DGELU) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-                float o[32];
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    float p[8];
-                    load8(sS, tid, c0 + j, p);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) o[j + q] = (c0 + j + q < a.ncols) ? __uint_as_float(u[j + q]) * gelu_grad_f(p[q]) : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, o + j);
-            }
-        } else {   // EPI_LNBWD: back through n = (g - mu) / sigma and g = gelu(p)
-            float s1 = 0.f, s2 = 0.f;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    float nrm[8];
-                    load8(sS, tid, c0 + j, nrm);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) { const float dn = __uint_as_float(u[j + q]); s1 += dn; s2 = fmaf(dn, nrm[q], s2); }
-                }
-            }
-            const float inv = 1.f / (float)a.ncols;
-            const float m1 = s1 * inv, m2 = s2 * inv, rs = a.rs[row];
-#pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t u[32];
-                tmem_ld32(lane_tm + c0, u);
-                tmem_ld_wait();
-                float o[32];
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    float nrm[8], p[8];
-                    load8(sS, tid, c0 + j, nrm);
-                    load8(sS + 65536, tid, c0 + j, p);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        o[j + q] = (c0 + j + q < a.ncols) ? rs * (__uint_as_float(u[j + q]) - m1 - nrm[q] * m2) * gelu_grad_f(p[q]) : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 256 + c0 + j, o + j);
-            }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tm, ND);
+}
+
+// ---------------------------------------------------------------------------
+// wide layer: Out[128 rows x 256] = epilogue(A[128 x 64] B[64 x 256]).  256 threads: the two
+// warpgroups share the rows (thread = row) and take two 64-column groups each; every output
+// leaves as TMA stores of [128 x 64] tiles staged in shared memory.  SPLIT (forward): hi + lo
+// operand pairs, the staging tiles lie over the operands (dead once the MMAs have completed).
+// Backward: single operands, side tiles (the forward's activations) by TMA, the output written
+// in place over the side tile it consumed.
+// ---------------------------------------------------------------------------
+struct WideArgs {
+    const float* bias;      // [256] or null
+    float* rs_out;          // EPI_LN: 1 / sigma of every row
+    const float* rs_in;     // EPI_LNBWD
+    int ncols;              // live columns (8r)
+};
+
+template <int EPI, bool SPLIT>
+struct WideSmem {
+    static constexpr int kA1 = 16384, kB1 = 32768;
+    static constexpr int kA = kA1 * (SPLIT ? 2 : 1), kB = kB1 * (SPLIT ? 2 : 1);
+    static constexpr int kSides = EPI == EPI_DGELU ? 1 : (EPI == EPI_LNBWD ? 2 : 0);
+    static constexpr int bytes = kA + kB + kSides * 65536 + 1024;
+    static_assert(!SPLIT || kA + kB == 2 * 3 * 16384, "three staging tiles per warpgroup over the operands");
+    static_assert(SPLIT == (kSides == 0), "forward: pairs and no side tiles; backward: the reverse");
+};
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+// 8 consecutive columns of a row of a 128-byte-swizzled [128 x 64] bf16 tile
+__device__ __forceinline__ void tile_put8(uint8_t* tile, int row, int chunk, const float* v) {
+    *reinterpret_cast<uint4*>(tile + swz128_offset(row, chunk)) =
+        make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+__device__ __forceinline__ void tile_put8_split(uint8_t* hi_tile, uint8_t* lo_tile, int row, int chunk, const float* v) {
+    float h[8], l[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { h[i] = __bfloat162float(__float2bfloat16_rn(v[i])); l[i] = v[i] - h[i]; }
+    tile_put8(hi_tile, row, chunk, h);
+    tile_put8(lo_tile, row, chunk, l);
+}
+__device__ __forceinline__ void tile_get8(const uint8_t* tile, int row, int chunk, float* v) {
+    const uint4 q = *reinterpret_cast<const uint4*>(tile + swz128_offset(row, chunk));
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+template <int EPI, bool SPLIT>
+__global__ void __launch_bounds__(256)
+ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mA2,
+                const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2,
+                const __grid_constant__ CUtensorMap mS0, const __grid_constant__ CUtensorMap mS1,
+                const __grid_constant__ CUtensorMap mO0, const __grid_constant__ CUtensorMap mO1,
+                const __grid_constant__ CUtensorMap mO2, WideArgs a, int* status) {
+    using L = WideSmem<EPI, SPLIT>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sA = align1024(smem_raw);
+    uint8_t* sB = sA + L::kA;
+    uint8_t* sS = sB + L::kB;
+    __shared__ uint64_t bar_ld, bar_side, bar_mma;
+    __shared__ uint32_t tm_slot;
+    __shared__ float s_bias[256];
+    __shared__ float2 s_part[2][128];
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int wg = warp / 4, rowt = (warp % 4) * 32 + lane;
+    const int tile = blockIdx.x;
+    if (tid == 0) {
+        cta_giveup_init();
+        mbar_init(&bar_ld, 1); mbar_init(&bar_side, 1); mbar_init(&bar_mma, 1);
+        mbar_fence_init();
+    }
+    if (warp == 0) { tmem_alloc(&tm_slot, 256); tmem_relinquish(); }
+    s_bias[tid] = a.bias != nullptr ? a.bias[tid] : 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tm_slot;
+    if (tid == 0) {
+        mbar_expect_tx(&bar_ld, L::kA + L::kB);
+        tma_load_2d(sA, &mA, 0, tile * 128, &bar_ld);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tma_load_2d(sB + g * 8192, &mB, g * 64, 0, &bar_ld);
+        if constexpr (SPLIT) {
+            tma_load_2d(sA + L::kA1, &mA2, 0, tile * 128, &bar_ld);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) tma_load_2d(sB + L::kB1 + g * 8192, &mB2, g * 64, 0, &bar_ld);
+        }
+        if constexpr (L::kSides > 0) {
+            mbar_expect_tx(&bar_side, L::kSides * 65536);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) tma_load_2d(sS + g * 16384, &mS0, g * 64, tile * 128, &bar_side);
+            if constexpr (L::kSides > 1) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) tma_load_2d(sS + 65536 + g * 16384, &mS1, g * 64, tile * 128, &bar_side);
+            }
+        }
+        if (mbar_wait(&bar_ld, 0, status, kErrTma)) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, 256, false, true);
+#pragma unroll
+            for (int part = 0; part < (SPLIT ? 3 : 1); ++part) {
+                const uint64_t ad = smem_desc(smem_u32(sA) + (part == 1 ? L::kA1 : 0), 0, 1024, kSwz128);
+                const uint64_t bd = smem_desc(smem_u32(sB) + (part == 2 ? L::kB1 : 0), 8192, 1024, kSwz128);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_ss(tm, desc_off(ad, k * 32), desc_off(bd, k * 2048), idesc, (part > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&bar_mma);
+        }
+    }
+    bool ok = mbar_wait(&bar_mma, 0, status, kErrMma);
+    if constexpr (L::kSides > 0) ok = ok && mbar_wait(&bar_side, 0, status, kErrTma);
+    ok = __syncthreads_and(ok) != 0;             // one decision for the whole CTA: the epilogue has barriers
+    tc_fence_after();
+    const uint32_t lane_tm = tm + ((uint32_t)((warp % 4) * 32) << 16);
+    const size_t row = (size_t)tile * 128 + rowt;
+    const bool elected = (tid % 128) == 0;
+    auto wg_sync = [&]() {
+        if (wg == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+        else asm volatile("bar.sync 2, 128;" ::: "memory");
+    };
+    if (ok) {
+        if constexpr (EPI == EPI_GELU) {
+            uint8_t* stg = sA + wg * 3 * 16384;
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int c0 = cg * 64 + half * 32;
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float pv[8], g[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            pv[q] = __uint_as_float(u[j + q]) + s_bias[c0 + j + q];
+                            g[q] = (c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
+                        }
+                        tile_put8(stg, rowt, half * 4 + j / 8, pv);
+                        tile_put8_split(stg + 16384, stg + 32768, rowt, half * 4 + j / 8, g);
+                    }
+                }
+                fence_proxy_async_smem();
+                wg_sync();
+                if (elected) {
+                    tma_store_2d(&mO0, stg, cg * 64, tile * 128);
+                    tma_store_2d(&mO1, stg + 16384, cg * 64, tile * 128);
+                    tma_store_2d(&mO2, stg + 32768, cg * 64, tile * 128);
+                    bulk_commit();
+                    bulk_wait_read();
+                }
+                wg_sync();
+            }
+        } else if constexpr (EPI == EPI_LN) {
+            uint8_t* stg = sA + wg * 3 * 16384;
+            float s = 0.f, ss = 0.f;
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int c0 = cg * 64 + half * 32;
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float pv[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            pv[q] = __uint_as_float(u[j + q]) + s_bias[c0 + j + q];
+                            const float g = (c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
+                            s += g; ss = fmaf(g, g, ss);
+                            u[j + q] = __float_as_uint(g);
+                        }
+                        tile_put8(stg, rowt, half * 4 + j / 8, pv);
+                    }
+                    tmem_st32(lane_tm + c0, u);
+                }
+                fence_proxy_async_smem();
+                wg_sync();
+                if (elected) {
+                    tma_store_2d(&mO0, stg, cg * 64, tile * 128);
+                    bulk_commit();
+                    bulk_wait_read();
+                }
+                wg_sync();
+            }
+            tmem_st_wait();
+            s_part[wg][rowt] = make_float2(s, ss);
+            __syncthreads();
+            const float2 p0 = s_part[0][rowt], p1 = s_part[1][rowt];
+            const float inv = 1.f / (float)a.ncols;
+            const float mu = (p0.x + p1.x) * inv;
+            const float rs = rsqrtf(fmaxf((p0.y + p1.y) * inv - mu * mu, 0.f) + kLnEps);
+            if (wg == 0) a.rs_out[row] = rs;
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int c0 = cg * 64 + half * 32;
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float nrm[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) nrm[q] = (c0 + j + q < a.ncols) ? (__uint_as_float(u[j + q]) - mu) * rs : 0.f;
+                        tile_put8_split(stg + 16384, stg + 32768, rowt, half * 4 + j / 8, nrm);
+                    }
+                }
+                fence_proxy_async_smem();
+                wg_sync();
+                if (elected) {
+                    tma_store_2d(&mO1, stg + 16384, cg * 64, tile * 128);
+                    tma_store_2d(&mO2, stg + 32768, cg * 64, tile * 128);
+                    bulk_commit();
+                    bulk_wait_read();
+                }
+                wg_sync();
+            }
+        } else if constexpr (EPI == EPI_DGELU) {
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+                uint8_t* side = sS + cg * 16384;          // p3's tile, overwritten by dp3
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int c0 = cg * 64 + half * 32;
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float pv[8], o[8];
+                        tile_get8(side, rowt, half * 4 + j / 8, pv);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) o[q] = (c0 + j + q < a.ncols) ? __uint_as_float(u[j + q]) * gelu_grad_f(pv[q]) : 0.f;
+                        tile_put8(side, rowt, half * 4 + j / 8, o);
+                    }
+                }
+                fence_proxy_async_smem();
+                wg_sync();
+                if (elected) { tma_store_2d(&mO0, side, cg * 64, tile * 128); bulk_commit(); }
+            }
+            if (elected) bulk_wait_read();
+        } else {   // EPI_LNBWD: back through n = (g - mu) / sigma and g = gelu(p)
+            float s1 = 0.f, s2 = 0.f;
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + cg * 64 + half * 32, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float nrm[8];
+                        tile_get8(sS + cg * 16384, rowt, half * 4 + j / 8, nrm);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) { const float dn = __uint_as_float(u[j + q]); s1 += dn; s2 = fmaf(dn, nrm[q], s2); }
+                    }
+                }
+            }
+            s_part[wg][rowt] = make_float2(s1, s2);
+            __syncthreads();
+            const float2 p0 = s_part[0][rowt], p1 = s_part[1][rowt];
+            const float inv = 1.f / (float)a.ncols;
+            const float m1 = (p0.x + p1.x) * inv, m2 = (p0.y + p1.y) * inv, rs = a.rs_in[row];
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                const int cg = wg * 2 + i;
+                uint8_t* side = sS + 65536 + cg * 16384;  // p1's tile, overwritten by dp1
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int c0 = cg * 64 + half * 32;
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + c0, u);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        float nrm[8], pv[8], o[8];
+                        tile_get8(sS + cg * 16384, rowt, half * 4 + j / 8, nrm);
+                        tile_get8(side, rowt, half * 4 + j / 8, pv);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            o[q] = (c0 + j + q < a.ncols) ? rs * (__uint_as_float(u[j + q]) - m1 - nrm[q] * m2) * gelu_grad_f(pv[q]) : 0.f;
+                        tile_put8(side, rowt, half * 4 + j / 8, o);
+                    }
+                }
+                fence_proxy_async_smem();
+                wg_sync();
+                if (elected) { tma_store_2d(&mO0, side, cg * 64, tile * 128); bulk_commit(); }
+            }
+            if (elected) bulk_wait_read();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 256);
 }
 
 // ---------------------------------------------------------------------------
@@ -684,27 +891,47 @@ bool build_maps(const LtcWs& w, char* ws, bool backward, Maps* M) {
     return ok;
 }
 
-// backward's layers: single bf16 operands, side tiles S0, S1 where the epilogue needs them
+// names under which the instances appear in the per-kernel timing records
+const char* const kDenseName[6] = {"", "ltc_dense_bwd_mid_kernel", "", "ltc_dense_bwd_in_kernel", "ltc_dense_bwd_gelu_kernel",
+                                   "ltc_dense_bwd_norm_kernel"};
+const char* const kDenseSplitName[6] = {"ltc_dense_norm_kernel", "ltc_dense_mid_kernel", "ltc_dense_gelu_kernel",
+                                        "ltc_dense_out_kernel", "", ""};
+
+// wide layers (64 -> 256)
+template <int EPI, bool SPLIT>
+cudaError_t wide(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
+                 const CUtensorMap& mS0, const CUtensorMap& mS1, const CUtensorMap& mO0, const CUtensorMap& mO1,
+                 const CUtensorMap& mO2, const WideArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
+    auto kern = ltc_wide_kernel<EPI, SPLIT>;
+    constexpr int smem = WideSmem<EPI, SPLIT>::bytes;
+    PSK_TRY(set_smem(kern, smem));
+    prof_begin(SPLIT ? kDenseSplitName[EPI] : kDenseName[EPI], s);
+    kern<<<tiles, 256, smem, s>>>(mA, mA2, mB, mB2, mS0, mS1, mO0, mO1, mO2, a, status);
+    prof_end(s);
+    ++*launches;
+    return cudaGetLastError();
+}
+// narrow layers (256 -> 64) of the backward: single bf16 operands
 template <int KD, int ND, int EPI>
 cudaError_t dense(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mS0, const CUtensorMap& mS1,
                   const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
     auto kern = ltc_dense_kernel<KD, ND, EPI, false>;
     constexpr int smem = DenseSmem<KD, ND, EPI, false>::bytes;
     PSK_TRY(set_smem(kern, smem));
-    prof_begin("ltc_dense_kernel", s);
+    prof_begin(kDenseName[EPI], s);
     kern<<<tiles, 128, smem, s>>>(mA, mA, mB, mB, mS0, mS1, a, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
 }
-// forward's layers: hi + lo operand pairs
+// narrow layers of the forward: hi + lo operand pairs
 template <int KD, int ND, int EPI>
 cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
                         const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
     auto kern = ltc_dense_kernel<KD, ND, EPI, true>;
     constexpr int smem = DenseSmem<KD, ND, EPI, true>::bytes;
     PSK_TRY(set_smem(kern, smem));
-    prof_begin("ltc_dense_kernel", s);
+    prof_begin(kDenseSplitName[EPI], s);
     kern<<<tiles, 128, smem, s>>>(mA, mA2, mB, mB2, mA, mA, a, status);
     prof_end(s);
     ++*launches;
@@ -746,12 +973,12 @@ cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const vo
         const NetBuf& nb = w.net[t];
         const float* vec = (const float*)(ws + w.vec) + (size_t)t * kVec;
         DenseArgs a{};
-        a = DenseArgs{vec, (bf16*)(ws + nb.p1), (bf16*)(ws + nb.n1), (bf16*)(ws + nb.n1_lo), (float*)(ws + nb.rs1), nullptr, m, 0};
-        PSK_TRY((dense_split<64, 256, EPI_LN>(M.n0, M.n0_lo, M.bank[t][0], M.bank[t][8], a, tiles, status, s, launches)));
+        PSK_TRY((wide<EPI_LN, true>(M.n0, M.n0_lo, M.bank[t][0], M.bank[t][8], M.n0, M.n0, M.p1[t], M.n1[t], M.n1_lo[t],
+                                    WideArgs{vec, (float*)(ws + nb.rs1), nullptr, m}, tiles, status, s, launches)));
         a = DenseArgs{vec + 256, (bf16*)(ws + nb.a2), (bf16*)(ws + nb.a2_lo), nullptr, nullptr, nullptr, 0, 0};
         PSK_TRY((dense_split<256, 64, EPI_B64>(M.n1[t], M.n1_lo[t], M.bank[t][1], M.bank[t][9], a, tiles, status, s, launches)));
-        a = DenseArgs{vec + 320, (bf16*)(ws + nb.p3), (bf16*)(ws + nb.a3), (bf16*)(ws + nb.a3_lo), nullptr, nullptr, m, 0};
-        PSK_TRY((dense_split<64, 256, EPI_GELU>(M.a2[t], M.a2_lo[t], M.bank[t][2], M.bank[t][10], a, tiles, status, s, launches)));
+        PSK_TRY((wide<EPI_GELU, true>(M.a2[t], M.a2_lo[t], M.bank[t][2], M.bank[t][10], M.n0, M.n0, M.p3[t], M.a3[t], M.a3_lo[t],
+                                      WideArgs{vec + 320, nullptr, nullptr, m}, tiles, status, s, launches)));
         a = DenseArgs{vec + 576, nullptr, nullptr, nullptr, (float*)(ws + nb.f), nullptr, d.r, 0};
         PSK_TRY((dense_split<256, 64, EPI_F32>(M.a3[t], M.a3_lo[t], M.bank[t][3], M.bank[t][11], a, tiles, status, s, launches)));
     }
@@ -823,8 +1050,8 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             float* sums = (float*)(ws + w.sums) + (size_t)t * kSums;
             DenseArgs a{};
             // dp3 = (df W4^T) * gelu'(p3);  dW4 ~ a3^T df
-            a = DenseArgs{nullptr, (bf16*)(ws + w.dp3), nullptr, nullptr, nullptr, nullptr, m, 0};
-            PSK_TRY((dense<64, 256, EPI_DGELU>(M.df[t], M.bank[t][4], M.p3[t], M.p3[t], a, tiles, status, s, launches)));
+            PSK_TRY((wide<EPI_DGELU, false>(M.df[t], M.df[t], M.bank[t][4], M.bank[t][4], M.p3[t], M.p3[t], M.dp3, M.dp3, M.dp3,
+                                            WideArgs{nullptr, nullptr, nullptr, m}, tiles, status, s, launches)));
             PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, tiles, status, s, launches));
             PSK_TRY(colsum((const bf16*)(ws + w.df[t]), 64, c, sums + 576, s, launches));
             // da2 = dp3 W3^T;  dW3 ~ dp3^T a2
@@ -835,8 +1062,8 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             // dp1 = LN1 backward(da2 (g1 W2)^T) * gelu'(p1);  dW2 ~ n1^T da2
             PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, tiles, status, s, launches));
             PSK_TRY(colsum((const bf16*)(ws + w.da2), 64, c, sums + 256, s, launches));
-            a = DenseArgs{nullptr, (bf16*)(ws + w.dp1), nullptr, nullptr, nullptr, (const float*)(ws + nb.rs1), m, 0};
-            PSK_TRY((dense<64, 256, EPI_LNBWD>(M.da2, M.bank[t][6], M.n1[t], M.p1[t], a, tiles, status, s, launches)));
+            PSK_TRY((wide<EPI_LNBWD, false>(M.da2, M.da2, M.bank[t][6], M.bank[t][6], M.n1[t], M.p1[t], M.dp1, M.dp1, M.dp1,
+                                            WideArgs{nullptr, nullptr, (const float*)(ws + nb.rs1), m}, tiles, status, s, launches)));
             // dn0 (+)= dp1 (g0 W1)^T;  dW1 ~ dp1^T n0
             PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, tiles, status, s, launches));
             PSK_TRY(colsum((const bf16*)(ws + w.dp1), 256, c, sums + 0, s, launches));

@@ -114,3 +114,22 @@ def small_workload(name="tiny", B=1, H=2, n=384, h=64, r=16, b=128, dtype="f32",
 def head_slice_f64(t: torch.Tensor, bi: int, hi: int):
     """One (batch, head) slice of a stored tensor, widened to float64 on the host."""
     return t[bi, hi].detach().to("cpu").to(torch.float64).numpy()
+
+
+def learned_network_params(h: int, r: int, seed: int):
+    """Seeded parameters of the learnable sketch's two dense networks (Algorithm 2 of the appendix) as two
+    dicts of float64 numpy arrays: gains near one, small biases, weights scaled so that every layer
+    keeps its input's scale.  Draws only; none of the method's arithmetic."""
+    import numpy as np
+    g = np.random.default_rng(seed)
+    m = 8 * r
+
+    def net():
+        return {"g0": 1.0 + 0.1 * g.standard_normal(h), "c0": 0.1 * g.standard_normal(h),
+                "W1": g.standard_normal((h, m)) / np.sqrt(h), "b1": 0.1 * g.standard_normal(m),
+                "g1": 1.0 + 0.1 * g.standard_normal(m), "c1": 0.1 * g.standard_normal(m),
+                "W2": g.standard_normal((m, r)) / np.sqrt(m), "b2": 0.1 * g.standard_normal(r),
+                "W3": g.standard_normal((r, m)) / np.sqrt(r), "b3": 0.1 * g.standard_normal(m),
+                "W4": 1.5 * g.standard_normal((m, r)) / np.sqrt(m), "b4": 0.1 * g.standard_normal(r)}
+
+    return net(), net()

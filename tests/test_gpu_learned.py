@@ -71,7 +71,7 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
     on_tc = dtype == "bf16" and r <= 32 and not local and path != psk.PATH_CUDA_CORES
     assert ("tc_bwd_k_kernel" in kernels) == on_tc
     # on that route the networks run on the tensor cores too (dense layers and weight gradients)
-    assert ("ltc_dense_kernel" in kernels and "ltc_wgrad_kernel" in kernels) == on_tc
+    assert ({"ltc_dense_norm_kernel", "ltc_dense_bwd_norm_kernel", "ltc_wgrad_kernel"} <= kernels) == on_tc
     assert ("learned_sketch_bwd_kernel" in kernels) == (not on_tc)
     tol = TOL[dtype]
     diag = "exact" if local else "LR"
