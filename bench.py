@@ -266,12 +266,50 @@ def time_other_config(psk, wl, name, steps, warmup, local, pk, device_index):
             "clocks": clocks}
 
 
+def time_lt_multiply(psk, base, steps, warmup, device_index):
+    """psk_lt_multiply_bf16 (Section 3.1's block algorithm on GIVEN feature matrices, tensor cores) on a
+    quarter of the headline's (batch, head) slices with m = r^2 = 1024 features of unit-variance rows:
+    memory-bound by construction (the features are read, not generated), so the figure of merit is
+    bytes: compulsory = A, B, C once + Out."""
+    import torch
+    batch, n, m, b = max(1, base.B * base.H // 4), base.n, 1024, 256
+    gen = torch.Generator(device="cuda").manual_seed(base.data_seed)
+    A, B = ((torch.randn(batch, n, m, generator=gen, device="cuda") / 32).bfloat16() for _ in range(2))
+    C = torch.randn(batch, n, 64, generator=gen, device="cuda").bfloat16()
+    ws = None
+    for _ in range(warmup):
+        out, ws = psk.lt_multiply_bf16(A, B, C, b, ws)
+    torch.cuda.synchronize()
+    psk.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        out, ws = psk.lt_multiply_bf16(A, B, C, b, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    agg = {}
+    for kname, t in psk.profile_records():
+        agg[kname] = agg.get(kname, 0.0) + t
+    psk.profile_enable(False)
+    if psk.check(ws) != 0:
+        raise RuntimeError("device-side error while timing lt_multiply_bf16")
+    compulsory = 2 * A.numel() * 2 + C.numel() * 2 + out.numel() * 4
+    hbm = peaks()["hbm_gbs"]
+    gbs = compulsory / (ms / 1e3) / 1e9
+    return {"batch": batch, "n": n, "m": m, "k": 64, "b": b, "passes": "fwd", "steps": steps, "warmup": warmup, "ms_per_step": ms,
+            "compulsory_bytes": compulsory, "compulsory_gbs": gbs, "frac_hbm_peak": gbs / hbm,
+            "kernels_ms_per_step": {k: round(v / steps, 3) for k, v in sorted(agg.items(), key=lambda kv: -kv[1])}}
+
+
 def time_variant(psk, wl, name, base, steps, warmup, device_index):
     """A short timed run of another member of the family at the headline configuration's B, H, n
     (forward + backward, bf16): "learned" = the learnable sketch of the appendix (r = 32, b = 256, parameter
     gradients included), "p2" = exact degree-2 attention (r = h = 64, b = 512), "p8" = degree 8 (r = 32)."""
     import torch
     binding = psk.binding
+    if name == "lt":
+        return time_lt_multiply(psk, base, steps, warmup, device_index)
     r, b, p = {"learned": (32, 256, 4), "p2": (64, 512, 2), "p8": (32, 256, 8)}[name]
     w = wl.Workload(name, base.B, base.H, base.n, base.h, r, 4, b, "bf16", True, base.data_seed, base.g_seed)
     inp = wl.make_inputs(w, "cuda", with_dO=True)
@@ -346,7 +384,7 @@ def main():
     ap.add_argument("--others", default="c1,c3,c4",
                     help="other configurations timed briefly after the headline one (N = 1 only); '' for none")
     ap.add_argument("--other-steps", type=int, default=5)
-    ap.add_argument("--variants", default="learned,p2,p8",
+    ap.add_argument("--variants", default="learned,p2,p8,lt",
                     help="other members of the family timed briefly at the headline's B, H, n (N=1 only; '' = none)")
     ap.add_argument("--variant-steps", type=int, default=2)
     ap.add_argument("--seq-segments", type=int, default=0,

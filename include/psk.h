@@ -200,10 +200,12 @@ int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void
  * The other arguments, the workspace rules and the error codes are those of psk_sketch,
  * psk_causal_attn_fwd and psk_causal_attn_bwd; `shape` needs p = 4, g_heads is ignored,
  * PSK_FLAG_LOCAL_EXACT is honoured (the paper's "learned + local" variant), PSK_FLAG_NONCAUSAL is
- * not supported here.  The networks always run on the CUDA cores in fp32; the attention on their half
- * sketches runs on the tensor cores for bf16 storage with r <= 32 and sketched same-block weights
- * (`path` = PSK_PATH_CUDA_CORES forces the CUDA-core kernels, PSK_PATH_TENSOR_CORES refuses what the
- * tensor-core route does not serve), else on the CUDA cores.  Workspace size from
+ * not supported here.  For bf16 storage with r <= 32 and sketched same-block weights everything runs
+ * on the tensor cores: the networks' dense layers (forward with hi + lo pairs of bf16 operands, so
+ * the half sketch keeps 2^-17; backward and weight gradients with single bf16 operands) and the
+ * attention on their half sketches (`path` = PSK_PATH_CUDA_CORES forces the CUDA-core kernels,
+ * PSK_PATH_TENSOR_CORES refuses what the tensor-core route does not serve).  Everything else, and
+ * psk_learned_sketch itself, runs on the CUDA cores in fp32.  Workspace size from
  * psk_learned_workspace_bytes. */
 size_t psk_learned_param_count(int h, int r);
 size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward);
@@ -228,6 +230,18 @@ int psk_learned_attn_bwd(const psk_shape* shape, const void* Q, const void* K, c
 size_t psk_lt_multiply_workspace_bytes(int batch, int n, int m, int k, int b);
 int psk_lt_multiply(int batch, int n, int m, int k, int b, const float* A, const float* B, const float* C,
                     float* Out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same block algorithm (Section 3.1) on the tensor cores for bf16 feature matrices:
+ *   Out = lt(A B^T) C,   A, B: [batch, n, m] bf16,  C: [batch, n, 64] bf16,  Out: [batch, n, 64] fp32,
+ * all contiguous, DEVICE, 16-byte aligned.  Products of bf16 entries are exact and summed in fp32; the
+ * prefix states Z_l and the masked same-block scores are rounded to bf16 once (relative 2^-9)
+ * before they are multiplied, as in the attention calls.  Needs m % 64 == 0, k == 64, b = 128 or 256,
+ * n % b == 0 (else PSK_ERR_SHAPE).  `workspace` (DEVICE, 256-byte aligned) of at least
+ * psk_lt_multiply_bf16_workspace_bytes() bytes (0 for a bad shape): a status word for psk_check,
+ * then the t = n / b prefix states of every batch entry.  Enqueues on `stream` and returns. */
+size_t psk_lt_multiply_bf16_workspace_bytes(int batch, int n, int m, int k, int b);
+int psk_lt_multiply_bf16(int batch, int n, int m, int k, int b, const void* A, const void* B, const void* C,
+                         float* Out, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Recurrent form: one new token per (batch, head) per call (inference at O(r^2 h) per token,
  * whatever the context length).  With the running state S (r^2 x 65 per head, fp32)

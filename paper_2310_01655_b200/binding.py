@@ -71,6 +71,10 @@ def lib():
     L.psk_lt_multiply_workspace_bytes.argtypes = [c_int] * 5
     L.psk_lt_multiply.restype = c_int
     L.psk_lt_multiply.argtypes = [c_int] * 5 + [c_void_p] * 5 + [c_size_t, c_void_p]
+    L.psk_lt_multiply_bf16_workspace_bytes.restype = c_size_t
+    L.psk_lt_multiply_bf16_workspace_bytes.argtypes = [c_int] * 5
+    L.psk_lt_multiply_bf16.restype = c_int
+    L.psk_lt_multiply_bf16.argtypes = [c_int] * 5 + [c_void_p] * 5 + [c_size_t, c_void_p]
     L.psk_decode_state_bytes.restype = c_size_t
     L.psk_decode_state_bytes.argtypes = [POINTER(Shape)]
     L.psk_decode_step.restype = c_int
@@ -322,6 +326,28 @@ def lt_multiply(A, B, C, b, workspace=None):
     if st != 0:
         raise PskError(st, "psk_lt_multiply")
     return out
+
+
+def lt_multiply_bf16(A, B, C, b, workspace=None):
+    """psk_lt_multiply_bf16: lt(A B^T) C on the tensor cores for bf16 CUDA tensors A, B [batch, n, m] and
+    C [batch, n, 64]; returns (Out fp32 [batch, n, 64], workspace) - pass the workspace to check()."""
+    _require_cuda(A, B, C)
+    for t in (A, B, C):
+        if t.dtype != torch.bfloat16 or t.dim() != 3 or not t.is_contiguous():
+            raise ValueError("lt_multiply_bf16 expects contiguous bf16 [batch, n, *] tensors")
+    batch, n, m = A.shape
+    k = C.shape[2]
+    if B.shape != A.shape or C.shape[:2] != A.shape[:2]:
+        raise ValueError("lt_multiply_bf16: A, B [batch, n, m] and C [batch, n, k] must agree")
+    need = int(lib().psk_lt_multiply_bf16_workspace_bytes(batch, n, m, k, b))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=A.device)
+    out = torch.empty((batch, n, k), dtype=torch.float32, device=A.device)
+    st = lib().psk_lt_multiply_bf16(batch, n, m, k, b, _ptr(A), _ptr(B), _ptr(C), _ptr(out), _ptr(workspace),
+                                    workspace.numel() if need else 0, _stream())
+    if st != 0:
+        raise PskError(st, "psk_lt_multiply_bf16")
+    return out, workspace
 
 
 # ---- learnable sketch (Algorithm 2): parameter packing and the three calls ----

@@ -64,6 +64,17 @@ bool tc_map_2d(CUtensorMap* m, const void* base, int cols, int64_t rows, int box
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// [outer][rows][cols] bf16, contiguous; box = box_rows rows x box_cols columns of one outer index.
+bool tc_map_3d(CUtensorMap* m, const void* base, int cols, int64_t rows, int64_t outer, int box_cols, int box_rows) {
+    EncodeFn enc = encoder();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)outer};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)rows * cols * 2};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1}, es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 // States S[nblk][FP][80] bf16 (feature-major rows: 64 state columns, the last column, 15 zeros).
 // Box = 64 features x 64 columns; a second box at column 64 brings the last column (columns
 // beyond 80 lie outside the tensor and arrive as zeros).

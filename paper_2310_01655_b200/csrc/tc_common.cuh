@@ -17,6 +17,8 @@ bool tc_map_rows(CUtensorMap* m, const void* base, int B, int H, int n, int64_t 
 bool tc_map_states(CUtensorMap* m, const void* base, int FP, int64_t nblk);
 // row-major [rows][cols] bf16 matrix, box box_rows x 64 columns
 bool tc_map_2d(CUtensorMap* m, const void* base, int cols, int64_t rows, int box_rows);
+// contiguous [outer][rows][cols] bf16, box box_rows x box_cols
+bool tc_map_3d(CUtensorMap* m, const void* base, int cols, int64_t rows, int64_t outer, int box_cols, int box_rows);
 // per-block states of every head + prefix (reverse = false) or suffix (reverse = true) scan
 // center_mode 0: states as they are; 1: values centred by the per-head vector cmean
 // (columns < 64 become H[:, c] - cmean[c] H[:, 64]); 2: last column becomes H[:, 64] - H[:, :64] cmean.

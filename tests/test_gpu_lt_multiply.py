@@ -48,3 +48,39 @@ def test_bad_arguments():
     with pytest.raises(psk.PskError) as e:
         psk.lt_multiply(A, A, torch.zeros(1, 64, 129, device="cuda"), 32)     # k > 128
     assert e.value.code == -3
+
+
+# ---- the tensor-core instance (bf16 feature matrices) ----
+@pytest.mark.parametrize("batch,n,m,b", [(2, 512, 128, 128), (1, 768, 192, 256), (2, 256, 64, 256), (1, 1024, 512, 256),
+                                         (1, 128, 64, 128)])
+def test_tensor_core_instance_matches_oracle(batch, n, m, b):
+    g = torch.Generator(device="cpu").manual_seed(2000 + n + m)
+    A, B = ((torch.randn(batch, n, m, generator=g) / m ** 0.5).bfloat16() for _ in range(2))
+    C = torch.randn(batch, n, 64, generator=g).bfloat16()
+    psk.profile_enable(True)
+    out, ws = psk.lt_multiply_bf16(A.cuda(), B.cuda(), C.cuda(), b)
+    torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    assert psk.check(ws) == 0
+    assert "lt_tc_rows_kernel" in kernels and ("lt_tc_state_kernel" in kernels) == (n > b)
+    out = out.cpu().double().numpy()
+    for i in range(batch):
+        a, bb, c = (x[i].double().numpy() for x in (A, B, C))      # the bf16 values the kernels read
+        ref = orc.lt_multiply_blocked(a, bb, c, b)
+        # states and masked scores are rounded to bf16 once before they are multiplied: 2^-9 each
+        assert orc.rel_l2(out[i], ref) < 1e-2
+        assert orc.rel_l2(out[i], np.tril(a @ bb.T) @ c) < 1e-2
+        # a row's first entries depend on few terms: check a tile's worth row by row as well
+        for row in (0, 1, 127, min(128, n - 1), n - 1):
+            assert np.allclose(out[i][row], ref[row], rtol=3e-2, atol=3e-2 * np.abs(ref[row]).max() + 1e-6)
+
+
+def test_tensor_core_instance_bad_arguments():
+    A = torch.zeros(1, 256, 64, device="cuda", dtype=torch.bfloat16)
+    C = torch.zeros(1, 256, 64, device="cuda", dtype=torch.bfloat16)
+    for args, code in (((A, A, C, 64), -3), ((A[:, :, :32].contiguous(), A[:, :, :32].contiguous(), C, 128), -3),
+                       ((A, A, C[:, :, :32].contiguous(), 128), -3), ((A[:, :192].contiguous(), A[:, :192].contiguous(), C[:, :192].contiguous(), 128), -3)):
+        with pytest.raises(psk.PskError) as e:
+            psk.lt_multiply_bf16(*args)
+        assert e.value.code == code
