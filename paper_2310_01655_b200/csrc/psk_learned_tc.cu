@@ -18,6 +18,8 @@
 // shapes, 64 -> 256 and 256 -> 64, serve all sixteen layer passes.
 #include "tc_common.cuh"
 
+#include <cstdlib>
+
 namespace psk {
 
 namespace {
@@ -826,10 +828,23 @@ struct LtcWs {
     size_t C;
 };
 
+// Rows per pass.  PSK_LEARNED_CHUNK_ROWS in the environment overrides the default (a multiple of
+// 128; read at every call, so that workspace queries and calls of one process agree as long as
+// it is not changed between them): for tests of the chunk loop on small inputs, and for tuning.
+size_t chunk_rows() {
+    const char* e = std::getenv("PSK_LEARNED_CHUNK_ROWS");
+    if (e != nullptr) {
+        const long long v = std::atoll(e);
+        if (v >= 128 && v % 128 == 0) return (size_t)v;
+    }
+    return kChunkRows;
+}
+
 LtcWs ltc_ws(const Dims& d, bool backward) {
     LtcWs w{};
     const size_t rows = (size_t)d.BH() * d.n;
-    w.C = rows < kChunkRows ? rows : kChunkRows;
+    const size_t chunk = chunk_rows();
+    w.C = rows < chunk ? rows : chunk;
     const size_t C = w.C;
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes); return o; };

@@ -97,6 +97,59 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
             check("net %d %s" % (which + 1, k), got[k], ref[k], 5 * tol if dtype == "bf16" else 2e-3)
 
 
+def _run_and_check(inp, w, flat, P1, P2, r, b, heads, tol, with_params, bwd_heads=None):
+    Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
+    psk.profile_enable(True)
+    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b)
+    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b)
+    torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    assert {"ltc_dense_norm_kernel", "ltc_wgrad_kernel", "tc_bwd_k_kernel"} <= kernels
+    for t in (O, den, dQ, dK, dV, dflat):
+        assert torch.isfinite(t.float()).all()
+    g1_sum = {k: 0.0 for k in orc.NET_KEYS}
+    g2_sum = {k: 0.0 for k in orc.NET_KEYS}
+    for bi, hi in heads:
+        f = lambda k: head_slice_f64(inp[k], bi, hi)
+        O_ref, d_ref = orc.causal_learned_polysketch_attention_blocked(f("Q"), f("K"), f("V"), P1, P2, b, diagonal="LR")
+        check("O[%d,%d]" % (bi, hi), O[bi, hi], O_ref, tol)
+        check("denom[%d,%d]" % (bi, hi), den[bi, hi], d_ref, tol)
+        if bwd_heads is not None and (bi, hi) not in bwd_heads:
+            continue
+        gq, gk, gv, g1, g2 = orc.causal_learned_polysketch_attention_backward(f("Q"), f("K"), f("V"), P1, P2, f("dO"), b, "LR")
+        for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), (gq, gk, gv)):
+            check("%s[%d,%d]" % (nm, bi, hi), got[bi, hi], ref, tol)
+        for k in orc.NET_KEYS:
+            g1_sum[k] = g1_sum[k] + g1[k]
+            g2_sum[k] = g2_sum[k] + g2[k]
+    if with_params:
+        d1, d2 = binding.unpack_learned_params(dflat, 64, r)
+        for which, (got, ref) in enumerate(((d1, g1_sum), (d2, g2_sum))):
+            for k in orc.NET_KEYS:
+                check("net %d %s" % (which + 1, k), got[k], ref[k], 5 * tol)
+
+
+def test_networks_in_several_passes_over_the_rows(monkeypatch):
+    # the tensor-core networks walk the rows in chunks (2^20 by default); with 256-row chunks this small
+    # input takes six passes per tensor, and the weight-gradient accumulators add up across them
+    monkeypatch.setenv("PSK_LEARNED_CHUNK_ROWS", "256")
+    r, b = 32, 128
+    w = wl.small_workload(B=2, H=2, n=384, r=r, b=b, dtype="bf16", seed=91)
+    inp = wl.make_inputs(w, "cuda")
+    flat, P1, P2 = nets(r, 4)
+    _run_and_check(inp, w, flat, P1, P2, r, b, [(bi, hi) for bi in range(2) for hi in range(2)], TOL["bf16"], True)
+
+
+def test_networks_across_the_default_chunk_boundary():
+    # 4 x 12 heads of 32768 rows: 1.5 M rows per tensor, so the second pass starts at head (2, 8)
+    r, b = 32, 256
+    w = wl.small_workload(B=4, H=12, n=32768, r=r, b=b, dtype="bf16", seed=92)
+    inp = wl.make_inputs(w, "cuda")
+    flat, P1, P2 = nets(r, 5)
+    _run_and_check(inp, w, flat, P1, P2, r, b, [(2, 7), (2, 8), (3, 11)], TOL["bf16"], False, bwd_heads=[(2, 8)])
+
+
 def test_refusals():
     w = wl.small_workload(B=1, H=1, n=256, r=32, b=128, dtype="f32", seed=5)
     inp = wl.make_inputs(w, "cuda")
