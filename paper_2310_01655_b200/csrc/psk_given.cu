@@ -7,17 +7,20 @@
 // together in fp32 (tc_common.cuh, read_half_sketch).  Backward: the kernels return the gradient
 // with respect to the [hi | lo] columns, whose first r columns are dL/dm; the existing
 // sketch-backward kernels take it from there.  r <= 32 (both terms fit the 64 columns), bf16 storage.
+// Exact same-block weights (learnable sketch only): the kernels also get the raw rows, for the
+// same-block scores, and return those rows' same-block gradient next to the half sketch's.
 #include "tc_common.cuh"
 
 namespace psk {
 
 namespace {
 
-struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, ltc, total; };
+struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, dXq, dXk, ltc, total; };
 
 Dims linear_dims(const Dims& d) {
     Dims l = d;
-    l.p = 4; l.learned = false; l.lparams = nullptr; l.dlparams = nullptr; l.local = false;
+    l.p = 4; l.learned = false; l.lparams = nullptr; l.dlparams = nullptr;
+    l.local = d.local && d.learned;         // exact same-block weights: the kernels also get the raw rows
     l.sketch_linear = true;
     l.g_heads = 1;
     l.xsn = 64; l.xsh = (int64_t)d.n * 64; l.xsb = (int64_t)d.H * d.n * 64;      // [B, H, n, 64] contiguous
@@ -36,6 +39,10 @@ GivenWs given_ws(const Dims& d, bool backward) {
     if (backward) {
         w.dSq = off; off += align_up(rows * 64 * sizeof(bf16));                     // gradient of the [hi | lo] columns
         w.dSk = off; off += align_up(rows * 64 * sizeof(bf16));
+        if (d.local) {                                                              // same-block gradients of the raw rows
+            w.dXq = off; off += align_up(rows * 64 * sizeof(bf16));
+            w.dXk = off; off += align_up(rows * 64 * sizeof(bf16));
+        }
     }
     if (d.learned && learned_tc_supported(d)) { w.ltc = off; off += align_up(learned_tc_workspace_bytes(d, backward)); }
     w.total = off;
@@ -100,8 +107,10 @@ cudaError_t half_sketches(const Dims& d, const void* Q, const void* K, const voi
 }  // namespace
 
 bool given_supported(const Dims& d) {
-    return d.bf16 && (d.p == 8 || d.learned) && d.r <= 32 && !d.local && !d.noncausal &&
-           tc_supported(linear_dims(d), false);
+    // exact same-block weights: only with the learnable sketch on the tensor-core networks (the
+    // same-block gradient of the raw rows joins the networks' gradient there)
+    return d.bf16 && (d.p == 8 || d.learned) && d.r <= 32 && !d.noncausal &&
+           (!d.local || (d.learned && learned_tc_supported(d))) && tc_supported(linear_dims(d), false);
 }
 
 size_t given_workspace_bytes(const Dims& d, bool backward) { return given_ws(d, backward || d.keep_states).total; }
@@ -110,7 +119,9 @@ cudaError_t given_fwd(const Dims& d, const void* Q, const void* K, const void* V
                       void* O, float* denom, char* ws, cudaStream_t s, int* launches) {
     const GivenWs w = given_ws(d, d.keep_states);
     PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, false, s, launches));
-    return tc_fwd(linear_dims(d), ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, ws + w.tc, s, launches);
+    Dims l = linear_dims(d);
+    l.rawQ = Q; l.rawK = K;
+    return tc_fwd(l, ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, ws + w.tc, s, launches);
 }
 
 cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
@@ -119,11 +130,13 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
     const GivenWs w = given_ws(d, true);
     const size_t rows = (size_t)d.BH() * d.n;
     PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, true, s, launches));
-    PSK_TRY(tc_bwd(linear_dims(d), ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, dO, ws + w.dSq, ws + w.dSk, dV,
-                   ws + w.tc, s, launches));
+    Dims l = linear_dims(d);
+    l.rawQ = Q; l.rawK = K;
+    if (l.local) { l.rawdQ = ws + w.dXq; l.rawdK = ws + w.dXk; }
+    PSK_TRY(tc_bwd(l, ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, dO, ws + w.dSq, ws + w.dSk, dV, ws + w.tc, s, launches));
     const void* X[2] = {Q, K};
     void* dX[2] = {dQ, dK};
-    const size_t mo[2] = {w.Mq, w.Mk}, go[2] = {w.dSq, w.dSk};
+    const size_t mo[2] = {w.Mq, w.Mk}, go[2] = {w.dSq, w.dSk}, xo[2] = {w.dXq, w.dXk};
     const bool nets_on_tc = d.learned && learned_tc_supported(d);
     for (int i = 0; i < 2; ++i) {
         float* dM = reinterpret_cast<float*>(ws + mo[i]);       // m itself is no longer needed
@@ -132,7 +145,8 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
-        if (nets_on_tc) PSK_TRY(learned_tc_sketch_bwd(d, X[i], dM, nullptr, dX[i], ws + w.ltc, reinterpret_cast<int*>(ws + w.tc), s, launches));
+        if (nets_on_tc)
+            PSK_TRY(learned_tc_sketch_bwd(d, X[i], dM, l.local ? ws + xo[i] : nullptr, dX[i], ws + w.ltc, reinterpret_cast<int*>(ws + w.tc), s, launches));
         else PSK_TRY(cc_sketch_bwd(d, X[i], G1, G2, dM, nullptr, dX[i], s, launches));
     }
     if (nets_on_tc) PSK_TRY(learned_tc_finish(d, ws + w.ltc, s, launches));

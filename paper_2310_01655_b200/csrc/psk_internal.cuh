@@ -25,6 +25,13 @@ struct Dims {
     // read_half_sketch); `xsb, xsh, xsn` are the strides of those tensors and of their gradients
     bool sketch_linear = false;
     int64_t xsb = 0, xsh = 0, xsn = 0;
+    // given half sketches WITH exact same-block weights: the raw rows (strides sb, sh, sn) next to
+    // the half sketches, and where the same-block part of their gradients goes (contiguous
+    // [B,H,n,64] bf16); the sketch part of the gradient goes to the tensors "dQ", "dK" as always
+    const void* rawQ = nullptr;
+    const void* rawK = nullptr;
+    void* rawdQ = nullptr;
+    void* rawdK = nullptr;
     // learnable sketch (Algorithm 2): the half sketch comes from two dense networks instead of G1, G2
     bool learned = false;
     const float* lparams = nullptr;   // packed parameters of both networks (psk_learned.cu)
@@ -81,7 +88,7 @@ bool learned_tc_supported(const Dims& d);
 size_t learned_tc_workspace_bytes(const Dims& d, bool backward);
 cudaError_t learned_tc_prepare(const Dims& d, bool backward, char* ws, cudaStream_t s, int* launches);
 cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* M, char* ws, int* status, cudaStream_t s, int* launches);
-cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const float* add, void* dX, char* ws,
+cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const void* add, void* dX, char* ws,
                                   int* status, cudaStream_t s, int* launches);
 cudaError_t learned_tc_finish(const Dims& d, char* ws, cudaStream_t s, int* launches);
 

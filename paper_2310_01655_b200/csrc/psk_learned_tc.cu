@@ -706,7 +706,7 @@ ltc_ln0_kernel(Slice sl, const bf16* __restrict__ X, size_t row0, int rows, bf16
 // dX = back through the first normalisation of the summed gradient of n0 (+ add)
 __global__ void __launch_bounds__(256)
 ltc_ln0_bwd_kernel(Slice sl, size_t row0, int rows, const float* __restrict__ dn0, const bf16* __restrict__ n0,
-                   const float* __restrict__ rs0, const float* __restrict__ add, bf16* __restrict__ dX) {
+                   const float* __restrict__ rs0, const bf16* __restrict__ add, bf16* __restrict__ dX) {
     const int lane = threadIdx.x % 32;
     const int i = blockIdx.x * 8 + threadIdx.x / 32;
     if (i >= rows) return;
@@ -718,8 +718,8 @@ ltc_ln0_bwd_kernel(Slice sl, size_t row0, int rows, const float* __restrict__ dn
     const float m1 = s1 * (1.f / 64.f), m2 = s2 * (1.f / 64.f), rs = rs0[i];
     float oa = rs * (d.x - m1 - na * m2), ob = rs * (d.y - m1 - nb * m2);
     if (add != nullptr) {
-        const float2 q = *reinterpret_cast<const float2*>(add + (row0 + i) * 64 + 2 * lane);
-        oa += q.x; ob += q.y;
+        const __nv_bfloat162 q = *reinterpret_cast<const __nv_bfloat162*>(add + (row0 + i) * 64 + 2 * lane);
+        oa += __low2float(q); ob += __high2float(q);
     }
     *reinterpret_cast<uint32_t*>(dX + sl.row(row0 + i) + 2 * lane) = pack_bf16(oa, ob);
 }
@@ -1037,10 +1037,11 @@ cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* Mout, char* w
     return cudaSuccess;
 }
 
-// dX = chain rule of sum(dM * M) through both networks (+ add); the weight-gradient
+// dX = chain rule of sum(dM * M) through both networks (+ add, a contiguous [rows][64] bf16 array
+// or null: the part of the gradient that reached X directly); the weight-gradient
 // accumulators in the workspace grow by this tensor's share (learned_tc_finish turns them into
 // parameter gradients)
-cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const float* add, void* dX, char* ws,
+cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const void* add, void* dX, char* ws,
                                   int* status, cudaStream_t s, int* launches) {
     const LtcWs w = ltc_ws(d, true);
     Maps M;
@@ -1087,7 +1088,7 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
         }
         prof_begin("ltc_ln0_bwd_kernel", s);
         ltc_ln0_bwd_kernel<<<(c + 7) / 8, 256, 0, s>>>(sl, row0, c, (const float*)(ws + w.dn0), (const bf16*)(ws + w.n0),
-                                                      (const float*)(ws + w.rs0), add, (bf16*)dX);
+                                                      (const float*)(ws + w.rs0), (const bf16*)add, (bf16*)dX);
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());

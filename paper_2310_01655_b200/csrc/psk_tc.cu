@@ -158,9 +158,12 @@ struct OutSmem {
 // (bf16 operands, exact products, fp32 sums) in place of m(q_i) . m(k_j); squared like those,
 // they give the exact weights (q_i . k_j)^4.  No key sketches, no split operands.
 // LIN: the rows hold a given half sketch (tc_common.cuh, read_half_sketch).
+// LIN and LOCAL: mapQ is the given half sketch, mapQraw the raw query rows (fetched into the query
+// tile's buffer once the sketch GEMM has read it), mapK the raw key rows.
 template <int R, int MODE, bool LOCAL, bool LIN>
 __global__ void __launch_bounds__(kOutThreads, ((R <= 32 || LOCAL) ? 2 : 1))
-tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapQraw,
+                  const __grid_constant__ CUtensorMap mapK,
                   const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapZ,
                   const __grid_constant__ CUtensorMap mapO, const __grid_constant__ CUtensorMap mapOc,
                   const uint8_t* __restrict__ gimg, int g_heads, int H, int n, int b, int t,
@@ -272,6 +275,11 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             issue_sketch<R>(tm + cSk, smem + L::Q, smem + L::G);
             umma_commit(&bar_sk);
             FTR(3, 0);
+            if constexpr (LIN && LOCAL) {
+                ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);
+                mbar_expect_tx(&bar_q, 16384);
+                tma_load_4d(smem + L::Q, &mapQraw, 0, row0, hi, bi, &bar_q);
+            }
             if (has_prefix && kZStages - 1 < F::NC) {
                 // the query tile has been consumed: its buffer becomes the ring's last stage
                 ok = ok && mbar_spin(&bar_sk, 0, status, kErrMma);
@@ -317,6 +325,7 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 tc_fence_after();
                 if constexpr (LOCAL) {
                     // scores = Q_tile K_tile^T over the head dimension
+                    if constexpr (LIN) ok = ok && mbar_spin(&bar_q, 1, status, kErrTma);     // the raw query rows
                     constexpr uint32_t idesc = idesc_bf16(128, 128, false, false);
                     const uint64_t qr = smem_desc(smem_u32(smem + L::Q), 0, 1024, kSwz128);
                     const uint64_t kr = smem_desc(smem_u32(smem + L::K), 0, 1024, kSwz128);
@@ -659,23 +668,37 @@ cudaError_t fwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
     PSK_TRY(tc_states(d, mK, mV, gimg, nullptr, nullptr, cmean, cmean ? 1 : 0, Z, false,
                       reinterpret_cast<float*>(ws + w.tot), status, s, launches));
     prof_begin("tc_fwd_out_kernel", s);
-    if (d.local) {
+    if (d.local && d.sketch_linear) {
+        if constexpr (R <= 32) {
+            CUtensorMap mQraw, mKraw;
+            if (d.rawQ == nullptr || d.rawK == nullptr || !tc_map_rows(&mQraw, d.rawQ, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+                !tc_map_rows(&mKraw, d.rawK, d.B, d.H, d.n, d.sb, d.sh, d.sn))
+                return cudaErrorInvalidValue;
+            constexpr size_t smem = OutSmem<R, true>::total + 1024;
+            PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true, true>, smem)));
+            tc_fwd_out_kernel<R, 0, true, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+                mQ, mQraw, mKraw, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+                denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, 0, status);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    } else if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, true, false>, smem)));
         tc_fwd_out_kernel<R, 0, true, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     } else if (d.sketch_linear) {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false, true>, smem)));
         tc_fwd_out_kernel<R, 0, false, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 0, false, false>, smem)));
         tc_fwd_out_kernel<R, 0, false, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mO, mOc, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             denom, nullptr, nullptr, nullptr, Oc != nullptr ? 1 : 0, d.noncausal ? 1 : 0, status);
     }
     prof_end(s);
@@ -720,28 +743,38 @@ cudaError_t tc_fwd(const Dims& d, const void* Q, const void* K, const void* V, c
 }
 
 template <int R>
-static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mQraw, const CUtensorMap& mK, const CUtensorMap& mV,
                                   const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean,
                                   const float* denom, const bf16* dO, float* y65, float* e65h, int* status,
                                   cudaStream_t s, int* launches) {
     prof_begin("tc_bwd_recompute_kernel", s);
-    if (d.local) {
+    if (d.local && d.sketch_linear) {
+        if constexpr (R <= 32) {
+            constexpr size_t smem = OutSmem<R, true>::total + 1024;
+            PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true, true>, smem)));
+            tc_fwd_out_kernel<R, 1, true, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
+                mQ, mQraw, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+                const_cast<float*>(denom), dO, y65, e65h, 0, 0, status);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    } else if (d.local) {
         constexpr size_t smem = OutSmem<R, true>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, true, false>, smem)));
         tc_fwd_out_kernel<R, 1, true, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     } else if (d.sketch_linear) {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false, true>, smem)));
         tc_fwd_out_kernel<R, 1, false, true><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     } else {
         constexpr size_t smem = OutSmem<R, false>::total + 1024;
         PSK_TRY((set_smem(tc_fwd_out_kernel<R, 1, false, false>, smem)));
         tc_fwd_out_kernel<R, 1, false, false><<<dim3(d.b / 128, d.t, d.BH()), kOutThreads, smem, s>>>(
-            mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
+            mQ, mQ, mK, mV, mZ, mZ, mZ, gimg, d.g_heads, d.H, d.n, d.b, d.t, cmean, d.sb, d.sh, d.sn,
             const_cast<float*>(denom), dO, y65, e65h, 0, d.noncausal ? 1 : 0, status);
     }
     prof_end(s);
@@ -749,13 +782,13 @@ static cudaError_t recompute_impl(const Dims& d, const CUtensorMap& mQ, const CU
     return cudaGetLastError();
 }
 
-cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mQraw, const CUtensorMap& mK, const CUtensorMap& mV,
                          const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
                          const bf16* dO, float* y65, float* e65h, int* status, cudaStream_t s, int* launches) {
     switch (d.r) {
-        case 16: return recompute_impl<16>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
-        case 32: return recompute_impl<32>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
-        case 64: return recompute_impl<64>(d, mQ, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
+        case 16: return recompute_impl<16>(d, mQ, mQraw, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
+        case 32: return recompute_impl<32>(d, mQ, mQraw, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
+        case 64: return recompute_impl<64>(d, mQ, mQraw, mK, mV, mZ, gimg, cmean, denom, dO, y65, e65h, status, s, launches);
     }
     return cudaErrorInvalidValue;
 }

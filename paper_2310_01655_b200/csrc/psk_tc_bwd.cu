@@ -153,7 +153,8 @@ __global__ void __launch_bounds__(128, ((R <= 32 || (LOCAL && QSIDE)) ? 2 : 1))
 tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_constant__ CUtensorMap mapYown,
                    const __grid_constant__ CUtensorMap mapXoth, const __grid_constant__ CUtensorMap mapYoth,
                    const __grid_constant__ CUtensorMap mapS, const __grid_constant__ CUtensorMap mapDX,
-                   const __grid_constant__ CUtensorMap mapDV, const uint8_t* __restrict__ gimg,
+                   const __grid_constant__ CUtensorMap mapDV, const __grid_constant__ CUtensorMap mapXownRaw,
+                   const __grid_constant__ CUtensorMap mapDXraw, const uint8_t* __restrict__ gimg,
                    int g_heads, int H, int n, int b, int t,
                    const float* __restrict__ y65g, const float* __restrict__ e65h, const float* __restrict__ denom,
                    int noncausal, int* status) {
@@ -259,6 +260,14 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     tc_fence_after();
     float m[R], dm[R];
     read_half_sketch<R>(lane_tm + cSk, m, 1.f, lin != 0);
+    if constexpr (LIN && LOCAL) {
+        // The own tile held the given half sketch; the exact same-block scores need the raw rows.
+        // The sketch GEMM has completed: fetch them into the same buffer (phase C waits for them).
+        if (tid == 0) {
+            mbar_expect_tx(&bar_own, 16384);
+            tma_load_4d(smem + L::Xown, &mapXownRaw, 0, row0, hi, bi, &bar_own);
+        }
+    }
 #pragma unroll
     for (int c = 0; c < R; ++c) dm[c] = 0.f;
     bool dv_started = false;
@@ -458,6 +467,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     uint32_t oth_uses = 0;
     float2* oth_col = reinterpret_cast<float2*>(smem + L::Eoth);   // other rows: (1/d, -(g . O)/d)
     const float y65h_inv = y65h * inv_own;
+    if constexpr (LIN && LOCAL) ok = ok && mbar_wait(&bar_own, 1, status, kErrTma);      // the raw own rows
 #pragma unroll 1
     for (int tp = tp_begin; tp < tp_end && ok; ++tp) {
         const int orow0 = l * b + tp * 128;
@@ -636,16 +646,18 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
                 for (int j = 0; j < 16; ++j) dm[c0 + j] = (dm[c0 + j] + (dm_started ? __uint_as_float(v[j]) : 0.f)) * rs;
             }
         }
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+        if constexpr (!LIN) {      // (a given half sketch: dX = dM "G1"^T needs neither A1 nor A2)
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);   // A1, A2 again
+                umma_commit(&bar_mma);
+            }
+            ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
+            ++mma_uses;
             tc_fence_after();
-            issue_sketch<R>(tm + cSk, smem + L::Xown, smem + L::G);   // A1, A2 again
-            umma_commit(&bar_mma);
         }
-        ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
-        ++mma_uses;
-        tc_fence_after();
     }
     if (ok) {
         // U = [dM*A2 | dM*A1] as a bf16 A operand in tensor memory (2R values -> R columns at cdM).
@@ -654,6 +666,34 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
         // GEMM adds to that accumulator.
         constexpr uint32_t cU1 = LOCAL ? cSk : cdM, cU2 = LOCAL ? cSk + R : cdM + R / 2;
         constexpr uint32_t cDX = LOCAL ? cXl : cS;
+        if constexpr (LIN && LOCAL) {
+            // Two gradients leave this kernel: the same-block tiles' one belongs to the raw rows and
+            // goes out now; the sketch's belongs to the given half sketch and takes the
+            // accumulator over afterwards.  (Every MMA has completed: the staging tile is free.)
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(lane_tm + cXl + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; j += 8)
+                    *reinterpret_cast<uint4*>(smem + L::Sx + swz128_offset(tid, (c0 + j) / 8)) =
+                        make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+                                   pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
+                                   pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
+                                   pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tma_store_4d(&mapDXraw, smem + L::Sx, 0, row0, hi, bi);
+                bulk_commit();
+                bulk_wait_read();
+            }
+            __syncthreads();
+            tc_fence_after();
+        }
 #pragma unroll
         for (int c0 = 0; c0 < R; c0 += 16) {
             uint32_t a1[16], a2[16], u1[8], u2[8];
@@ -680,7 +720,7 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
 #pragma unroll
             for (int k = 0; k < 2 * R / 16; ++k)    // contraction over the 2R sketch columns
                 umma_ts(tm + cDX, tm + (k < R / 16 ? cU1 + k * 8 : cU2 + (k - R / 16) * 8),
-                        desc_off(smem_desc(smem_u32(smem + L::G), 0, 1024, kSwz128), k * 2048), idesc, (LOCAL || k > 0) ? 1u : 0u);
+                        desc_off(smem_desc(smem_u32(smem + L::G), 0, 1024, kSwz128), k * 2048), idesc, ((LOCAL && !LIN) || k > 0) ? 1u : 0u);
             umma_commit(&bar_mma);
         }
         ok = mbar_wait(&bar_mma, mma_uses & 1, status, kErrMma);
@@ -756,6 +796,16 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         !tc_map_rows(&mdQ, dQ, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) || !tc_map_rows(&mdK, dK, d.B, d.H, d.n, d.xsb, d.xsh, d.xsn) ||
         !tc_map_rows(&mdV, dV, d.B, d.H, d.n, d.sb, d.sh, d.sn))
         return cudaErrorInvalidValue;
+    // given half sketches with exact same-block weights: raw rows in, their gradients out
+    CUtensorMap mQraw = mQ, mKraw = mK, mdQraw = mdQ, mdKraw = mdK;
+    const bool linloc = d.sketch_linear && d.local;
+    if (linloc) {
+        const int64_t hs = (int64_t)d.n * 64, bs = (int64_t)d.H * hs;
+        if (!d.rawQ || !d.rawK || !d.rawdQ || !d.rawdK || !tc_map_rows(&mQraw, d.rawQ, d.B, d.H, d.n, d.sb, d.sh, d.sn) ||
+            !tc_map_rows(&mKraw, d.rawK, d.B, d.H, d.n, d.sb, d.sh, d.sn) || !tc_map_rows(&mdQraw, d.rawdQ, d.B, d.H, d.n, bs, hs, 64) ||
+            !tc_map_rows(&mdKraw, d.rawdK, d.B, d.H, d.n, bs, hs, 64))
+            return cudaErrorInvalidValue;
+    }
     uint8_t* gimg = reinterpret_cast<uint8_t*>(ws + w.gimg);
     PSK_TRY(tc_gimage(d, G1, G2, gimg, s, launches));
     // prefix states of centred values; forward rows again in fp32 -> y65, e65h; suffix states
@@ -770,7 +820,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         ++*launches;
         PSK_TRY(cudaGetLastError());
     } else {
-        PSK_TRY(tc_recompute(d, mQ, mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, y65, e65h, status, s, launches));
+        PSK_TRY(tc_recompute(d, mQ, mQraw, linloc ? mKraw : mK, mV, mZ, gimg, cmean, denom, (const bf16*)dO, y65, e65h, status, s, launches));
     }
     const dim3 grid(d.b / 128, d.t, d.BH());
     auto rows = [&](auto local_c, auto lin_c) -> cudaError_t {
@@ -782,7 +832,7 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // query side first: it needs only the prefix states, and the row scalars just written are
         // still in L2; the suffix states (5 GB through L2) come after it
         prof_begin("tc_bwd_q_kernel", s);
-        tc_bwd_rows_kernel<R, true, LOCAL, LIN><<<grid, 128, smem, s>>>(mQ, mG, mK, mV, mZ, mdQ, mdQ, gimg, d.g_heads, d.H, d.n,
+        tc_bwd_rows_kernel<R, true, LOCAL, LIN><<<grid, 128, smem, s>>>(mQ, mG, (LOCAL && LIN) ? mKraw : mK, mV, mZ, mdQ, mdQ, mQraw, mdQraw, gimg, d.g_heads, d.H, d.n,
                                                                    d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
@@ -790,13 +840,17 @@ cudaError_t bwd_impl(const Dims& d, const void* Q, const void* K, const void* V,
         // suffix states: phi(q_i) / d_i against [dO_i | y65_i]
         PSK_TRY(tc_states(d, mQ, mG, gimg, y65, denom, cmean, 2, Rs, true, tot, status, s, launches));
         prof_begin("tc_bwd_k_kernel", s);
-        tc_bwd_rows_kernel<R, false, LOCAL, LIN><<<grid, 128, smem_k, s>>>(mK, mV, mQ, mG, mR, mdK, mdV, gimg, d.g_heads, d.H, d.n,
+        tc_bwd_rows_kernel<R, false, LOCAL, LIN><<<grid, 128, smem_k, s>>>(mK, mV, (LOCAL && LIN) ? mQraw : mQ, mG, mR, mdK, mdV, mKraw, mdKraw, gimg, d.g_heads, d.H, d.n,
                                                                     d.b, d.t, y65, e65h, denom, d.noncausal ? 1 : 0, status);
         prof_end(s);
         ++*launches;
         return cudaGetLastError();
     };
-    if (d.sketch_linear) return rows(std::false_type{}, std::true_type{});      // (never with exact same-block weights)
+    if (linloc) {
+        if constexpr (R <= 32) return rows(std::true_type{}, std::true_type{});
+        else return cudaErrorInvalidValue;
+    }
+    if (d.sketch_linear) return rows(std::false_type{}, std::true_type{});
     return d.local ? rows(std::true_type{}, std::false_type{}) : rows(std::false_type{}, std::false_type{});
 }
 

@@ -31,7 +31,8 @@ cudaError_t tc_states(const Dims& d, const CUtensorMap& mX, const CUtensorMap& m
 int tc_state_segments(const Dims& d);
 size_t tc_state_total_bytes(const Dims& d);
 // the backward's recomputation of the forward rows: writes y65, e65h (see tc_fwd_out_kernel)
-cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mK, const CUtensorMap& mV,
+// (mQraw, and mK = the raw key rows: only with a given half sketch and exact same-block weights)
+cudaError_t tc_recompute(const Dims& d, const CUtensorMap& mQ, const CUtensorMap& mQraw, const CUtensorMap& mK, const CUtensorMap& mV,
                          const CUtensorMap& mZ, const uint8_t* gimg, const float* cmean, const float* denom,
                          const bf16* dO, float* y65, float* e65h, int* status, cudaStream_t s, int* launches);
 // gimg[g] = [G1 | G2]^T of sketch-matrix set g as the shared-memory image of the sketch GEMM's B operand

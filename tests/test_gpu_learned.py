@@ -52,8 +52,8 @@ def test_half_sketch(r, dtype):
 @pytest.mark.parametrize("dtype,path", [("f32", psk.PATH_AUTO), ("bf16", psk.PATH_CUDA_CORES), ("bf16", psk.PATH_AUTO)])
 @pytest.mark.parametrize("local", [False, True])
 def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype, path, local):
-    # (bf16 storage, r <= 32, sketched same-block weights: PATH_AUTO is the tensor-core route on half
-    # sketches formed by the networks; everything else runs on the CUDA cores)
+    # (bf16 storage, r <= 32: PATH_AUTO is the tensor-core route, networks and attention, with sketched
+    # or exact same-block weights; everything else runs on the CUDA cores)
     w = wl.small_workload(B=2, H=2, n=n, r=r, b=b, dtype=dtype, seed=70 + r)
     inp = wl.make_inputs(w, "cuda")
     if local:
@@ -68,7 +68,7 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
     torch.cuda.synchronize()
     kernels = {name for name, _ in psk.profile_records()}
     psk.profile_enable(False)
-    on_tc = dtype == "bf16" and r <= 32 and not local and path != psk.PATH_CUDA_CORES
+    on_tc = dtype == "bf16" and r <= 32 and path != psk.PATH_CUDA_CORES
     assert ("tc_bwd_k_kernel" in kernels) == on_tc
     # on that route the networks run on the tensor cores too (dense layers and weight gradients)
     assert ({"ltc_dense_norm_kernel", "ltc_dense_bwd_norm_kernel", "ltc_wgrad_kernel"} <= kernels) == on_tc
