@@ -305,12 +305,13 @@ def time_lt_multiply(psk, base, steps, warmup, device_index):
 def time_variant(psk, wl, name, base, steps, warmup, device_index):
     """A short timed run of another member of the family at the headline configuration's B, H, n
     (forward + backward, bf16): "learned" = the learnable sketch of the appendix (r = 32, b = 256, parameter
-    gradients included), "p2" = exact degree-2 attention (r = h = 64, b = 512), "p8" = degree 8 (r = 32)."""
+    gradients included), "learned_local" = the same with exact same-block weights (the paper's
+    "learned + local"), "p2" = exact degree-2 attention (r = h = 64, b = 512), "p8" = degree 8 (r = 32)."""
     import torch
     binding = psk.binding
     if name == "lt":
         return time_lt_multiply(psk, base, steps, warmup, device_index)
-    r, b, p = {"learned": (32, 256, 4), "p2": (64, 512, 2), "p8": (32, 256, 8)}[name]
+    r, b, p = {"learned": (32, 256, 4), "learned_local": (32, 256, 4), "p2": (64, 512, 2), "p8": (32, 256, 8)}[name]
     w = wl.Workload(name, base.B, base.H, base.n, base.h, r, 4, b, "bf16", True, base.data_seed, base.g_seed)
     inp = wl.make_inputs(w, "cuda", with_dO=True)
     Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
@@ -318,13 +319,16 @@ def time_variant(psk, wl, name, base, steps, warmup, device_index):
     O = torch.empty_like(Q)
     den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
     grads = tuple(torch.empty_like(Q) for _ in range(3))
-    if name == "learned":
+    if name in ("learned", "learned_local"):
+        lflags = psk.FLAG_LOCAL_EXACT if name == "learned_local" else 0
+        if lflags:
+            Q.mul_(0.35); K.mul_(0.35)      # (q.k)^4 next to sketch weights bounded by r^2: the same scale
         flat = binding.pack_learned_params(*wl.learned_network_params(w.h, r, base.g_seed))
-        ws = torch.empty(binding.learned_workspace_bytes(Q, r, b), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(binding.learned_workspace_bytes(Q, r, b, lflags), dtype=torch.uint8, device="cuda")
 
         def step():
-            o, d = binding.learned_attn_fwd(Q, K, V, flat, r, b, 0, ws)
-            binding.learned_attn_bwd(Q, K, V, flat, o, d, dO, r, b, 0, ws)
+            o, d = binding.learned_attn_fwd(Q, K, V, flat, r, b, lflags, ws)
+            binding.learned_attn_bwd(Q, K, V, flat, o, d, dO, r, b, lflags, ws)
     else:
         if p == 2:
             Q.mul_(0.5); K.mul_(0.5)        # (q.k)^2 with |q|^2 = 64: keep the weights on the headline's scale
@@ -384,7 +388,7 @@ def main():
     ap.add_argument("--others", default="c1,c3,c4",
                     help="other configurations timed briefly after the headline one (N = 1 only); '' for none")
     ap.add_argument("--other-steps", type=int, default=5)
-    ap.add_argument("--variants", default="learned,p2,p8,lt",
+    ap.add_argument("--variants", default="learned,learned_local,p2,p8,lt",
                     help="other members of the family timed briefly at the headline's B, H, n (N=1 only; '' = none)")
     ap.add_argument("--variant-steps", type=int, default=2)
     ap.add_argument("--seq-segments", type=int, default=0,

@@ -200,8 +200,8 @@ int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void
  * The other arguments, the workspace rules and the error codes are those of psk_sketch,
  * psk_causal_attn_fwd and psk_causal_attn_bwd; `shape` needs p = 4, g_heads is ignored,
  * PSK_FLAG_LOCAL_EXACT is honoured (the paper's "learned + local" variant), PSK_FLAG_NONCAUSAL is
- * not supported here.  For bf16 storage with r <= 32 and sketched same-block weights everything runs
- * on the tensor cores: the networks' dense layers (forward with hi + lo pairs of bf16 operands, so
+ * not supported here.  For bf16 storage with r <= 32 (sketched or exact same-block weights) everything
+ * runs on the tensor cores: the networks' dense layers (forward with hi + lo pairs of bf16 operands, so
  * the half sketch keeps 2^-17; backward and weight gradients with single bf16 operands) and the
  * attention on their half sketches (`path` = PSK_PATH_CUDA_CORES forces the CUDA-core kernels,
  * PSK_PATH_TENSOR_CORES refuses what the tensor-core route does not serve).  Everything else, and
