@@ -1,7 +1,7 @@
 // Attention on GIVEN half sketches, on the tensor cores: degree 8 (one more level of Algorithm 1)
 // and the learnable sketch (Algorithm 2) only change how the half sketch m(x) is formed; features
-// m (x) m, block states and row kernels are the ones of degree 4.  So the existing sketch kernels
-// (CUDA cores) write m for Q and K, a small kernel splits it into two bf16 terms side by side,
+// m (x) m, block states and row kernels are the ones of degree 4.  So sketch kernels of their own
+// (psk_sketch8_tc.cu, psk_learned_tc.cu) form m for Q and K as two bf16 terms side by side,
 // [hi | lo] (64 columns, zero-padded), and the tensor-core kernels run in their "linear" sketch mode
 // on those arrays in place of Q and K: their sketch GEMM against [I; I] adds the two terms back
 // together in fp32 (tc_common.cuh, read_half_sketch).  Backward: the kernels return the gradient
@@ -15,7 +15,7 @@ namespace psk {
 
 namespace {
 
-struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, dXq, dXk, ltc, total; };
+struct GivenWs { size_t tc, Mq, Mk, Sq, Sk, dSq, dSk, dXq, dXk, ltc, sk8, total; };
 
 Dims linear_dims(const Dims& d) {
     Dims l = d;
@@ -32,8 +32,12 @@ GivenWs given_ws(const Dims& d, bool backward) {
     const size_t rows = (size_t)d.BH() * d.n;
     size_t off = 0;
     w.tc = off; off += align_up(tc_workspace_bytes(linear_dims(d), backward));     // first: its status word is the call's
-    w.Mq = off; off += align_up(rows * d.r * sizeof(float));                        // m, later dL/dm (fp32)
-    w.Mk = off; off += align_up(rows * d.r * sizeof(float));
+    if (sketch8_tc_supported(d)) {                                                  // degree 8: the sketch kernels write [hi | lo] themselves
+        w.sk8 = off; off += sketch8_tc_bank_bytes(d);
+    } else {
+        w.Mq = off; off += align_up(rows * d.r * sizeof(float));                    // m, later dL/dm (fp32)
+        w.Mk = off; off += align_up(rows * d.r * sizeof(float));
+    }
     w.Sq = off; off += align_up(rows * 64 * sizeof(bf16));                          // [hi | lo]
     w.Sk = off; off += align_up(rows * 64 * sizeof(bf16));
     if (backward) {
@@ -91,6 +95,12 @@ cudaError_t half_sketches(const Dims& d, const void* Q, const void* K, const voi
     const size_t mo[2] = {w.Mq, w.Mk}, so[2] = {w.Sq, w.Sk};
     const bool nets_on_tc = d.learned && learned_tc_supported(d);
     if (nets_on_tc) PSK_TRY(learned_tc_prepare(d, backward, ws + w.ltc, s, launches));
+    if (sketch8_tc_supported(d)) {
+        PSK_TRY(sketch8_tc_prepare(d, G1, G2, ws + w.sk8, s, launches));
+        for (int i = 0; i < 2; ++i)
+            PSK_TRY(sketch8_tc_fwd(d, X[i], ws + so[i], ws + w.sk8, reinterpret_cast<int*>(ws + w.tc), s, launches));
+        return cudaSuccess;
+    }
     for (int i = 0; i < 2; ++i) {
         float* M = reinterpret_cast<float*>(ws + mo[i]);
         if (nets_on_tc) PSK_TRY(learned_tc_sketch(d, X[i], M, ws + w.ltc, reinterpret_cast<int*>(ws + w.tc), s, launches));
@@ -138,6 +148,11 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
     void* dX[2] = {dQ, dK};
     const size_t mo[2] = {w.Mq, w.Mk}, go[2] = {w.dSq, w.dSk}, xo[2] = {w.dXq, w.dXk};
     const bool nets_on_tc = d.learned && learned_tc_supported(d);
+    if (sketch8_tc_supported(d)) {
+        for (int i = 0; i < 2; ++i)
+            PSK_TRY(sketch8_tc_bwd(d, X[i], ws + go[i], dX[i], ws + w.sk8, reinterpret_cast<int*>(ws + w.tc), s, launches));
+        return cudaSuccess;
+    }
     for (int i = 0; i < 2; ++i) {
         float* dM = reinterpret_cast<float*>(ws + mo[i]);       // m itself is no longer needed
         prof_begin("unsplit_kernel", s);

@@ -92,6 +92,15 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
                                   int* status, cudaStream_t s, int* launches);
 cudaError_t learned_tc_finish(const Dims& d, char* ws, cudaStream_t s, int* launches);
 
+// Degree 8's half sketch on the tensor cores (psk_sketch8_tc.cu): bf16, r <= 32.  `prepare` once per
+// call; `fwd` writes the [hi | lo] rows the attention kernels read, `bwd` takes their gradient.
+bool sketch8_tc_supported(const Dims& d);
+size_t sketch8_tc_bank_bytes(const Dims& d);
+cudaError_t sketch8_tc_prepare(const Dims& d, const void* G1, const void* G2, char* bank, cudaStream_t s, int* launches);
+cudaError_t sketch8_tc_fwd(const Dims& d, const void* X, void* S, char* bank, int* status, cudaStream_t s, int* launches);
+cudaError_t sketch8_tc_bwd(const Dims& d, const void* X, const void* dS, void* dX, char* bank, int* status, cudaStream_t s,
+                           int* launches);
+
 // Tensor-core (bf16 operands, fp32 accumulation) launchers.
 size_t tc_workspace_bytes(const Dims& d, bool backward);
 bool tc_supported(const Dims& d, bool backward);

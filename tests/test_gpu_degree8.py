@@ -27,7 +27,7 @@ def _oracle_gaussians(G1, G2, hi, h):
 @pytest.mark.parametrize("r,b,n,dtype,path", [
     (16, 128, 384, "f32", psk.PATH_AUTO), (32, 256, 512, "f32", psk.PATH_AUTO), (64, 128, 256, "f32", psk.PATH_AUTO),
     (32, 128, 128, "f32", psk.PATH_AUTO), (32, 256, 768, "bf16", psk.PATH_CUDA_CORES), (64, 256, 512, "bf16", psk.PATH_AUTO),
-    # bf16 storage, r <= 32: half sketches by the sketch kernels, attention on them by the tensor-core kernels
+    # bf16 storage, r <= 32: half sketches and the attention on them by tensor-core kernels
     (32, 256, 768, "bf16", psk.PATH_TENSOR_CORES), (16, 128, 640, "bf16", psk.PATH_AUTO), (32, 512, 1024, "bf16", psk.PATH_AUTO),
 ])
 def test_forward_and_backward(r, b, n, dtype, path):
@@ -45,7 +45,9 @@ def test_forward_and_backward(r, b, n, dtype, path):
     kernels = {name for name, _ in psk.profile_records()}
     psk.profile_enable(False)
     on_tc = dtype == "bf16" and r <= 32 and path != psk.PATH_CUDA_CORES
-    assert ("tc_fwd_out_kernel" in kernels) == on_tc and ("sketch8_kernel" in kernels) and (("fwd_out_kernel" in kernels) != on_tc)
+    assert ("tc_fwd_out_kernel" in kernels) == on_tc and (("fwd_out_kernel" in kernels) != on_tc)
+    # on that route the deeper sketch runs on the tensor cores too, forward and backward
+    assert ({"sk8_tc_fwd_kernel", "sk8_tc_bwd_kernel"} <= kernels) == on_tc and ("sketch8_kernel" in kernels) != on_tc
     for hi in range(w.H):
         q, k, v, g = (x[0, hi].double().cpu().numpy() for x in (Q, K, V, dO))
         Gs = _oracle_gaussians(G1, G2, hi, 64)
