@@ -45,8 +45,8 @@
  *     so the weights approximate (q_i . k_j)^8.  G1 then holds [Ga1; Gb1; Gc1] and G2 holds
  *     [Ga2; Gb2; Gc2], each [g_heads, 2h + r, r] contiguous.  Not with PSK_FLAG_LOCAL_EXACT
  *     (PSK_ERR_UNSUPPORTED).  fp32 storage and r = 64: CUDA-core kernels.  bf16 storage with
- *     r <= 32: the half sketches are formed by the CUDA-core sketch kernels and the attention on
- *     them runs on the tensor cores (PSK_PATH_CUDA_CORES forces the CUDA-core kernels throughout).
+ *     r <= 32: the half sketches and the attention on them run on the tensor cores
+ *     (PSK_PATH_CUDA_CORES forces the CUDA-core kernels throughout).
  */
 #ifndef PSK_H_
 #define PSK_H_
