@@ -591,9 +591,9 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
 constexpr int kWgStage = 65536 + 16384;
 constexpr int kWgSmem = 2 * kWgStage + 1024;
 
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(160)
 ltc_wgrad_kernel(const __grid_constant__ CUtensorMap mP, const __grid_constant__ CUtensorMap mS, float* __restrict__ Gt,
-                 int ntiles, int tiles_per_cta, int* status) {
+                 float* __restrict__ colsum, int sum_wide, int ntiles, int tiles_per_cta, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align1024(smem_raw);
     __shared__ uint64_t bar_full[2], bar_free[2], bar_done;
@@ -604,7 +604,7 @@ ltc_wgrad_kernel(const __grid_constant__ CUtensorMap mP, const __grid_constant__
     if (tid == 0) {
         cta_giveup_init();
         mbar_init(&bar_full[0], 1); mbar_init(&bar_full[1], 1);
-        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1);
+        mbar_init(&bar_free[0], 5); mbar_init(&bar_free[1], 5);        // the tile's MMAs and the four summing warps
         mbar_init(&bar_done, 1);
         mbar_fence_init();
     }
@@ -647,10 +647,46 @@ ltc_wgrad_kernel(const __grid_constant__ CUtensorMap mP, const __grid_constant__
             }
         }
         if (ok) umma_commit(&bar_done);
+    } else if (warp >= 1) {
+        // Warps 1-4: column sums of the delta operand (the wide one's 256 columns, two per thread,
+        // or the narrow one's 64) from the tiles while they sit in shared memory: the bias
+        // gradients, and what the folded normalisation gains need.
+        const int j0 = tid - 32;
+        float acc0 = 0.f, acc1 = 0.f;
+        bool ok = true;
+        for (int j = 0; j < T; ++j) {
+            const int s = j & 1;
+            if (ok) ok = mbar_wait(&bar_full[s], (j >> 1) & 1, status, kErrTma);
+            if (ok) {
+                const uint8_t* st = smem + s * kWgStage;
+                if (sum_wide) {
+                    const uint8_t* c0p = st + (j0 / 64) * 16384 + (j0 % 8) * 2;
+                    const uint8_t* c1p = c0p + 32768;
+                    const uint32_t ch = (j0 % 64) / 8;
+#pragma unroll 8
+                    for (int row = 0; row < 128; ++row) {
+                        const uint32_t o = swz128_offset(row, ch);
+                        acc0 += __bfloat162float(*reinterpret_cast<const bf16*>(c0p + o));
+                        acc1 += __bfloat162float(*reinterpret_cast<const bf16*>(c1p + o));
+                    }
+                } else if (j0 < 64) {
+                    const uint8_t* cp = st + 65536 + (j0 % 8) * 2;
+                    const uint32_t ch = j0 / 8;
+#pragma unroll 8
+                    for (int row = 0; row < 128; ++row) acc0 += __bfloat162float(*reinterpret_cast<const bf16*>(cp + swz128_offset(row, ch)));
+                }
+            }
+            __syncwarp();
+            if (tid % 32 == 0) mbar_arrive(&bar_free[s]);      // (also after a failed wait: the issuer must not be left waiting)
+        }
+        if (ok && colsum != nullptr) {
+            if (sum_wide) { atomicAdd(colsum + j0, acc0); atomicAdd(colsum + j0 + 128, acc1); }
+            else if (j0 < 64) atomicAdd(colsum + j0, acc0);
+        }
     }
     const bool ok = mbar_wait(&bar_done, 0, status, kErrMma);
     tc_fence_after();
-    if (ok) {
+    if (ok && warp < 4) {
         const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -750,16 +786,6 @@ ltc_combine_bwd_kernel(const float* __restrict__ f1, const float* __restrict__ f
     }
     df1[e] = __float2bfloat16_rn(o1);
     df2[e] = __float2bfloat16_rn(o2);
-}
-
-// out[c] += sum over rows of A[row][c]   (A: [rows][W] bf16, W = 64 or 256; 256 rows per CTA)
-__global__ void __launch_bounds__(256)
-ltc_colsum_kernel(const bf16* __restrict__ A, int W, int rows, float* __restrict__ out) {
-    const int c = threadIdx.x % W, sub = threadIdx.x / W, step = 256 / W;
-    const int r0 = blockIdx.x * 256, r1 = min(rows, r0 + 256);
-    float acc = 0.f;
-    for (int i = r0 + sub; i < r1; i += step) acc += __bfloat162float(A[(size_t)i * W + c]);
-    atomicAdd(out + c, acc);
 }
 
 // parameter gradients of one network from the four accumulators and the column sums
@@ -953,22 +979,15 @@ cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUt
     return cudaGetLastError();
 }
 
-cudaError_t wgrad(const CUtensorMap& mP, const CUtensorMap& mS, float* Gt, int tiles, int* status, cudaStream_t s,
-                  int* launches) {
+// (colsum: where the column sums of the delta operand are added; wide = that operand is P)
+cudaError_t wgrad(const CUtensorMap& mP, const CUtensorMap& mS, float* Gt, float* colsum, bool wide, int tiles, int* status,
+                  cudaStream_t s, int* launches) {
     PSK_TRY(set_smem(ltc_wgrad_kernel, kWgSmem));
     int per = (tiles + 295) / 296;            // about two CTAs per SM, but at least four tiles per result added
     if (per < 4) per = tiles < 4 ? tiles : 4;
     const int grid = (tiles + per - 1) / per;
     prof_begin("ltc_wgrad_kernel", s);
-    ltc_wgrad_kernel<<<grid, 128, kWgSmem, s>>>(mP, mS, Gt, tiles, per, status);
-    prof_end(s);
-    ++*launches;
-    return cudaGetLastError();
-}
-
-cudaError_t colsum(const bf16* A, int W, int rows, float* out, cudaStream_t s, int* launches) {
-    prof_begin("ltc_colsum_kernel", s);
-    ltc_colsum_kernel<<<(rows + 255) / 256, 256, 0, s>>>(A, W, rows, out);
+    ltc_wgrad_kernel<<<grid, 160, kWgSmem, s>>>(mP, mS, Gt, colsum, wide ? 1 : 0, tiles, per, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -1068,21 +1087,17 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             // dp3 = (df W4^T) * gelu'(p3);  dW4 ~ a3^T df
             PSK_TRY((wide<EPI_DGELU, false>(M.df[t], M.df[t], M.bank[t][4], M.bank[t][4], M.p3[t], M.p3[t], M.dp3, M.dp3, M.dp3,
                                             WideArgs{nullptr, nullptr, nullptr, m}, tiles, status, s, launches)));
-            PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, tiles, status, s, launches));
-            PSK_TRY(colsum((const bf16*)(ws + w.df[t]), 64, c, sums + 576, s, launches));
+            PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, sums + 576, false, tiles, status, s, launches));
             // da2 = dp3 W3^T;  dW3 ~ dp3^T a2
-            PSK_TRY(wgrad(M.dp3, M.a2[t], G + 2 * kMat, tiles, status, s, launches));
-            PSK_TRY(colsum((const bf16*)(ws + w.dp3), 256, c, sums + 320, s, launches));
+            PSK_TRY(wgrad(M.dp3, M.a2[t], G + 2 * kMat, sums + 320, true, tiles, status, s, launches));
             a = DenseArgs{nullptr, (bf16*)(ws + w.da2), nullptr, nullptr, nullptr, nullptr, 0, 0};
             PSK_TRY((dense<256, 64, EPI_B64>(M.dp3, M.bank[t][5], M.n0, M.n0, a, tiles, status, s, launches)));
             // dp1 = LN1 backward(da2 (g1 W2)^T) * gelu'(p1);  dW2 ~ n1^T da2
-            PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, tiles, status, s, launches));
-            PSK_TRY(colsum((const bf16*)(ws + w.da2), 64, c, sums + 256, s, launches));
+            PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, sums + 256, false, tiles, status, s, launches));
             PSK_TRY((wide<EPI_LNBWD, false>(M.da2, M.da2, M.bank[t][6], M.bank[t][6], M.n1[t], M.p1[t], M.dp1, M.dp1, M.dp1,
                                             WideArgs{nullptr, nullptr, (const float*)(ws + nb.rs1), m}, tiles, status, s, launches)));
             // dn0 (+)= dp1 (g0 W1)^T;  dW1 ~ dp1^T n0
-            PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, tiles, status, s, launches));
-            PSK_TRY(colsum((const bf16*)(ws + w.dp1), 256, c, sums + 0, s, launches));
+            PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, sums + 0, true, tiles, status, s, launches));
             a = DenseArgs{nullptr, nullptr, nullptr, nullptr, (float*)(ws + w.dn0), nullptr, 64, t};
             PSK_TRY((dense<256, 64, EPI_F32>(M.dp1, M.bank[t][7], M.n0, M.n0, a, tiles, status, s, launches)));
         }
