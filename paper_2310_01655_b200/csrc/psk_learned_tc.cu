@@ -272,6 +272,141 @@ ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------
+// narrow layers of the forward (256 -> 64, hi + lo pairs): persistent, one CTA per SM.  The layer's
+// weights stay in shared memory; the activation tiles stream through a four-stage ring of
+// 64-column chunks (hi and lo, 32 KB a stage) that the producer thread keeps full across tile
+// boundaries; the accumulator is double-buffered in tensor memory, so the rows' epilogue of one
+// tile runs under the loads and MMAs of the next.  Warps 0-3: epilogue (thread = row); warp 4: TMA
+// producer; warp 5: MMA issuer.
+// ---------------------------------------------------------------------------
+constexpr int kNrStages = 4, kNrStage = 32768;
+constexpr int kNrSmem = 65536 + kNrStages * kNrStage + 1024;
+
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+ltc_narrow_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mA2,
+                  const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2, DenseArgs a, int tiles,
+                  int* status) {
+    static_assert(EPI == EPI_B64 || EPI == EPI_F32, "the 256 -> 64 layers");
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* sB = align1024(smem_raw);
+    uint8_t* sR = sB + 65536;
+    __shared__ uint64_t bar_b, bar_full[kNrStages], bar_empty[kNrStages], bar_accfull[2], bar_accfree[2];
+    __shared__ uint32_t tm_slot;
+    __shared__ float s_bias[64];
+    const int tid = threadIdx.x, warp = tid / 32;
+    const int ntl = (tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (tid == 0) {
+        cta_giveup_init();
+        mbar_init(&bar_b, 1);
+        for (int s = 0; s < kNrStages; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+        mbar_init(&bar_accfull[0], 1); mbar_init(&bar_accfull[1], 1);
+        mbar_init(&bar_accfree[0], 128); mbar_init(&bar_accfree[1], 128);
+        mbar_fence_init();
+    }
+    if (warp == 0) { tmem_alloc(&tm_slot, 128); tmem_relinquish(); }
+    if (tid < 64) s_bias[tid] = a.bias != nullptr ? a.bias[tid] : 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tm_slot;
+    if (tid == 128) {
+        // ---- producer ----
+        mbar_expect_tx(&bar_b, 65536);
+        tma_load_2d(sB, &mB, 0, 0, &bar_b);
+        tma_load_2d(sB + 32768, &mB2, 0, 0, &bar_b);
+        bool ok = true;
+        int it = 0;
+        for (int i = 0; i < ntl && ok; ++i) {
+            const int tile = blockIdx.x + i * gridDim.x;
+            for (int c = 0; c < 4 && ok; ++c, ++it) {
+                const int s = it % kNrStages;
+                if (it >= kNrStages) ok = mbar_spin(&bar_empty[s], ((it / kNrStages) - 1) & 1, status, kErrMma);
+                if (!ok) break;
+                mbar_expect_tx(&bar_full[s], kNrStage);
+                tma_load_2d(sR + s * kNrStage, &mA, c * 64, tile * 128, &bar_full[s]);
+                tma_load_2d(sR + s * kNrStage + 16384, &mA2, c * 64, tile * 128, &bar_full[s]);
+            }
+        }
+    } else if (tid == 160) {
+        // ---- MMA issuer ----
+        constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+        bool ok = mbar_spin(&bar_b, 0, status, kErrTma);
+        const uint64_t bhi = smem_desc(smem_u32(sB), 0, 1024, kSwz128);
+        const uint64_t blo = smem_desc(smem_u32(sB) + 32768, 0, 1024, kSwz128);
+        int it = 0;
+        for (int i = 0; i < ntl && ok; ++i) {
+            const int buf = i & 1;
+            if (i >= 2) ok = mbar_spin(&bar_accfree[buf], ((i / 2) - 1) & 1, status, kErrMma);
+            for (int c = 0; c < 4 && ok; ++c, ++it) {
+                const int s = it % kNrStages;
+                ok = mbar_spin(&bar_full[s], (it / kNrStages) & 1, status, kErrTma);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t ahi = smem_desc(smem_u32(sR) + s * kNrStage, 0, 1024, kSwz128);
+                const uint64_t alo = smem_desc(smem_u32(sR) + s * kNrStage + 16384, 0, 1024, kSwz128);
+#pragma unroll
+                for (int part = 0; part < 3; ++part) {
+                    const uint64_t ad = part == 1 ? alo : ahi;
+                    const uint64_t bd = part == 2 ? blo : bhi;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_ss(tm + buf * 64, desc_off(ad, k * 32), desc_off(bd, c * 8192 + k * 2048), idesc,
+                                (c > 0 || part > 0 || k > 0) ? 1u : 0u);
+                }
+                umma_commit(&bar_empty[s]);
+            }
+            if (ok) umma_commit(&bar_accfull[buf]);
+        }
+    } else if (warp < 4) {
+        // ---- epilogue ----
+        const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        for (int i = 0; i < ntl && ok; ++i) {
+            const int buf = i & 1;
+            const size_t row = (size_t)(blockIdx.x + i * gridDim.x) * 128 + tid;
+            ok = mbar_wait(&bar_accfull[buf], (i / 2) & 1, status, kErrMma);
+            if (!ok) break;
+            tc_fence_after();
+            if constexpr (EPI == EPI_B64) {
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t u[32];
+                    tmem_ld32(lane_tm + buf * 64 + c0, u);
+                    tmem_ld_wait();
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) store8_split(a.out0 + row * 64 + c0 + j, a.out1 + row * 64 + c0 + j, v + j);
+                }
+            } else {
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    if (c0 < a.ncols) {
+                        uint32_t u[32];
+                        tmem_ld32(lane_tm + buf * 64 + c0, u);
+                        tmem_ld_wait();
+                        float* dst = a.outf + row * a.ncols + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (c0 + j < a.ncols)
+                                *reinterpret_cast<float4*>(dst + j) =
+                                    make_float4(__uint_as_float(u[j]) + s_bias[c0 + j], __uint_as_float(u[j + 1]) + s_bias[c0 + j + 1],
+                                                __uint_as_float(u[j + 2]) + s_bias[c0 + j + 2], __uint_as_float(u[j + 3]) + s_bias[c0 + j + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&bar_accfree[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 128);
+}
+
+// ---------------------------------------------------------------------------
 // wide layer: Out[128 rows x 256] = epilogue(A[128 x 64] B[64 x 256]).  256 threads: the two
 // warpgroups share the rows (thread = row) and take two 64-column groups each; every output
 // leaves as TMA stores of [128 x 64] tiles staged in shared memory.  SPLIT (forward): hi + lo
@@ -969,11 +1104,17 @@ cudaError_t dense(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMa
 template <int KD, int ND, int EPI>
 cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
                         const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
-    auto kern = ltc_dense_kernel<KD, ND, EPI, true>;
-    constexpr int smem = DenseSmem<KD, ND, EPI, true>::bytes;
-    PSK_TRY(set_smem(kern, smem));
+    static_assert(KD == 256 && ND == 64, "the narrow layers");
+    auto kern = ltc_narrow_kernel<EPI>;
+    PSK_TRY(set_smem(kern, kNrSmem));
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
     prof_begin(kDenseSplitName[EPI], s);
-    kern<<<tiles, 128, smem, s>>>(mA, mA2, mB, mB2, mA, mA, a, status);
+    kern<<<tiles < sms ? tiles : sms, 192, kNrSmem, s>>>(mA, mA2, mB, mB2, a, tiles, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
