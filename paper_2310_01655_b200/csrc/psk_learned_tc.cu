@@ -458,7 +458,8 @@ __device__ __forceinline__ void tile_get8(const uint8_t* tile, int row, int chun
     }
 }
 
-template <int EPI, bool SPLIT>
+// FULL: all 256 columns are live (8r = 256), no masks
+template <int EPI, bool SPLIT, bool FULL>
 __global__ void __launch_bounds__(256)
 ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mA2,
                 const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2,
@@ -472,7 +473,7 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
     uint8_t* sS = sB + L::kB;
     __shared__ uint64_t bar_ld, bar_side, bar_mma;
     __shared__ uint32_t tm_slot;
-    __shared__ float s_bias[256];
+    __shared__ __align__(16) float s_bias[256];
     __shared__ float2 s_part[2][128];
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int wg = warp / 4, rowt = (warp % 4) * 32 + lane;
@@ -546,10 +547,12 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
                         float pv[8], g[8];
+                        const float4 b0 = *reinterpret_cast<const float4*>(s_bias + c0 + j), b1 = *reinterpret_cast<const float4*>(s_bias + c0 + j + 4);
+                        const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
-                            pv[q] = __uint_as_float(u[j + q]) + s_bias[c0 + j + q];
-                            g[q] = (c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
+                            pv[q] = __uint_as_float(u[j + q]) + bv[q];
+                            g[q] = (FULL || c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
                         }
                         tile_put8(stg, rowt, half * 4 + j / 8, pv);
                         tile_put8_split(stg + 16384, stg + 32768, rowt, half * 4 + j / 8, g);
@@ -581,10 +584,12 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
                         float pv[8];
+                        const float4 b0 = *reinterpret_cast<const float4*>(s_bias + c0 + j), b1 = *reinterpret_cast<const float4*>(s_bias + c0 + j + 4);
+                        const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
-                            pv[q] = __uint_as_float(u[j + q]) + s_bias[c0 + j + q];
-                            const float g = (c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
+                            pv[q] = __uint_as_float(u[j + q]) + bv[q];
+                            const float g = (FULL || c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
                             s += g; ss = fmaf(g, g, ss);
                             u[j + q] = __float_as_uint(g);
                         }
@@ -622,7 +627,7 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
                     for (int j = 0; j < 32; j += 8) {
                         float nrm[8];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) nrm[q] = (c0 + j + q < a.ncols) ? (__uint_as_float(u[j + q]) - mu) * rs : 0.f;
+                        for (int q = 0; q < 8; ++q) nrm[q] = (FULL || c0 + j + q < a.ncols) ? (__uint_as_float(u[j + q]) - mu) * rs : 0.f;
                         tile_put8_split(stg + 16384, stg + 32768, rowt, half * 4 + j / 8, nrm);
                     }
                 }
@@ -652,7 +657,7 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
                         float pv[8], o[8];
                         tile_get8(side, rowt, half * 4 + j / 8, pv);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) o[q] = (c0 + j + q < a.ncols) ? __uint_as_float(u[j + q]) * gelu_grad_f(pv[q]) : 0.f;
+                        for (int q = 0; q < 8; ++q) o[q] = (FULL || c0 + j + q < a.ncols) ? __uint_as_float(u[j + q]) * gelu_grad_f(pv[q]) : 0.f;
                         tile_put8(side, rowt, half * 4 + j / 8, o);
                     }
                 }
@@ -702,7 +707,7 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
                         tile_get8(side, rowt, half * 4 + j / 8, pv);
 #pragma unroll
                         for (int q = 0; q < 8; ++q)
-                            o[q] = (c0 + j + q < a.ncols) ? rs * (__uint_as_float(u[j + q]) - m1 - nrm[q] * m2) * gelu_grad_f(pv[q]) : 0.f;
+                            o[q] = (FULL || c0 + j + q < a.ncols) ? rs * (__uint_as_float(u[j + q]) - m1 - nrm[q] * m2) * gelu_grad_f(pv[q]) : 0.f;
                         tile_put8(side, rowt, half * 4 + j / 8, o);
                     }
                 }
@@ -1078,11 +1083,12 @@ template <int EPI, bool SPLIT>
 cudaError_t wide(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
                  const CUtensorMap& mS0, const CUtensorMap& mS1, const CUtensorMap& mO0, const CUtensorMap& mO1,
                  const CUtensorMap& mO2, const WideArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
-    auto kern = ltc_wide_kernel<EPI, SPLIT>;
     constexpr int smem = WideSmem<EPI, SPLIT>::bytes;
-    PSK_TRY(set_smem(kern, smem));
+    PSK_TRY(set_smem(ltc_wide_kernel<EPI, SPLIT, true>, smem));
+    PSK_TRY(set_smem(ltc_wide_kernel<EPI, SPLIT, false>, smem));
     prof_begin(SPLIT ? kDenseSplitName[EPI] : kDenseName[EPI], s);
-    kern<<<tiles, 256, smem, s>>>(mA, mA2, mB, mB2, mS0, mS1, mO0, mO1, mO2, a, status);
+    if (a.ncols == 256) ltc_wide_kernel<EPI, SPLIT, true><<<tiles, 256, smem, s>>>(mA, mA2, mB, mB2, mS0, mS1, mO0, mO1, mO2, a, status);
+    else ltc_wide_kernel<EPI, SPLIT, false><<<tiles, 256, smem, s>>>(mA, mA2, mB, mB2, mS0, mS1, mO0, mO1, mO2, a, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
