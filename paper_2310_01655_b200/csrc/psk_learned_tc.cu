@@ -33,23 +33,33 @@ constexpr int kBank = 12;                             // operand matrices per ne
 constexpr int kVec = 256 + 64 + 256 + 64;             // folded biases of one network: b1' | b2' | b3 | b4
 constexpr int kSums = 256 + 64 + 256 + 64;            // column sums of one network: dp1 | da2 | dp3 | df
 
-// Phi(x) and the normal density at x.  erf by a five-term rational approximation in
-// t = 1 / (1 + 0.3275911 z), z = |x| / sqrt(2) (absolute error 1.5e-7), whose exponential
-// exp(-z^2) = exp(-x^2 / 2) is the density's too.
-__device__ __forceinline__ void normal_parts(float x, float& cdf, float& pdf) {
-    const float z = fabsf(x) * 0.70710678118654752f;
-    const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
-    const float e = __expf(-z * z);
-    float poly = fmaf(1.061405429f, t, -1.453152027f);
-    poly = fmaf(poly, t, 1.421413741f);
-    poly = fmaf(poly, t, -0.284496736f);
-    poly = fmaf(poly, t, 0.254829592f);
-    const float q = 0.5f * poly * t * e;                 // 1 - Phi(|x|)
-    cdf = x >= 0.f ? 1.f - q : q;
-    pdf = 0.3989422804014327f * e;
+// gelu(x) = x Phi(x) and its derivative Phi(x) + x phi(x).  erfc(z), z = |x| / sqrt(2), by the
+// five-term rational approximation in t = 1 / (1 + 0.3275911 z) (absolute error 1.5e-7); its
+// exponential exp(-z^2) = exp(-x^2 / 2) is the normal density's too.  With E = erfc(z):
+//   gelu(x) = max(x, 0) - |x| E / 2,     Phi(x) = 1/2 + copysign(1/2 - E/2, x).
+__device__ __forceinline__ float rcp_approx(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// half of erfc(|x| / sqrt(2)) and exp(-x^2 / 2)
+__device__ __forceinline__ float half_erfc(float ax, float& e) {
+    const float z = ax * 0.70710678118654752f;
+    const float t = rcp_approx(fmaf(0.3275911f, z, 1.f));
+    e = ex2_approx(z * z * -1.4426950408889634f);
+    float poly = fmaf(0.5f * 1.061405429f, t, 0.5f * -1.453152027f);
+    poly = fmaf(poly, t, 0.5f * 1.421413741f);
+    poly = fmaf(poly, t, 0.5f * -0.284496736f);
+    poly = fmaf(poly, t, 0.5f * 0.254829592f);
+    return poly * t * e;
 }
-__device__ __forceinline__ float gelu_f(float x) { float c, d; normal_parts(x, c, d); return x * c; }
-__device__ __forceinline__ float gelu_grad_f(float x) { float c, d; normal_parts(x, c, d); return fmaf(x, d, c); }
+__device__ __forceinline__ float gelu_f(float x) {
+    float e;
+    const float ax = fabsf(x);
+    return fmaf(-ax, half_erfc(ax, e), fmaxf(x, 0.f));
+}
+__device__ __forceinline__ float gelu_grad_f(float x) {
+    float e;
+    const float q = half_erfc(fabsf(x), e);
+    return fmaf(x, 0.3989422804014327f * e, 0.5f + copysignf(0.5f - q, x));
+}
 
 struct NetLayout {
     int h, r, m;
@@ -441,12 +451,17 @@ __device__ __forceinline__ void tile_put8(uint8_t* tile, int row, int chunk, con
     *reinterpret_cast<uint4*>(tile + swz128_offset(row, chunk)) =
         make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
 }
+// v = hi + lo: one packed conversion gives two hi terms, whose float values are the halves of that word
 __device__ __forceinline__ void tile_put8_split(uint8_t* hi_tile, uint8_t* lo_tile, int row, int chunk, const float* v) {
-    float h[8], l[8];
+    uint32_t h[4], l[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { h[i] = __bfloat162float(__float2bfloat16_rn(v[i])); l[i] = v[i] - h[i]; }
-    tile_put8(hi_tile, row, chunk, h);
-    tile_put8(lo_tile, row, chunk, l);
+    for (int i = 0; i < 4; ++i) {
+        h[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+        l[i] = pack_bf16(v[2 * i] - __uint_as_float(h[i] << 16), v[2 * i + 1] - __uint_as_float(h[i] & 0xffff0000u));
+    }
+    const uint32_t o = swz128_offset(row, chunk);
+    *reinterpret_cast<uint4*>(hi_tile + o) = make_uint4(h[0], h[1], h[2], h[3]);
+    *reinterpret_cast<uint4*>(lo_tile + o) = make_uint4(l[0], l[1], l[2], l[3]);
 }
 __device__ __forceinline__ void tile_get8(const uint8_t* tile, int row, int chunk, float* v) {
     const uint4 q = *reinterpret_cast<const uint4*>(tile + swz128_offset(row, chunk));
