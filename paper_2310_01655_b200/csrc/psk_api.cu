@@ -94,7 +94,7 @@ size_t path_workspace(int path, const Dims& d, bool backward) {
 
 extern "C" {
 
-int psk_version(void) { return 100; }
+int psk_version(void) { return 200; }
 
 const char* psk_status_string(int status) {
     switch (status) {

@@ -4,16 +4,18 @@
 //   f(x) = W4^T gelu(W3^T (W2^T LN1(gelu(W1^T LN0(x) + b1)) + b2) + b3) + b4      (two such networks)
 //   M    = sqrt(r) tanh(f_1(x) * f_2(x) / sqrt(r))
 //
-// Rows are processed in chunks; inside a chunk every layer is one launch of tc_dense_kernel
-// (128 rows per CTA: activations by TMA, the layer's weights as the MN-major B operand, the
-// accumulator read back by thread = row, where bias, gelu and the layer normalisations are plain
-// per-thread loops), with the activations the backward needs kept in the workspace as bf16.
+// Rows are processed in chunks; inside a chunk every layer is one launch (ltc_wide_kernel,
+// ltc_narrow_kernel, ltc_dense_kernel; 128 rows per tile: activations by TMA, the layer's weights
+// as the MN-major B operand, the accumulator read back by thread = row, where bias, gelu and the
+// layer normalisations are plain per-thread loops), with the activations the backward needs
+// kept in the workspace as bf16.
 // The gains of the normalisations are folded into the following layer's weights
 // (z W = n (diag(g) W) + c W), so the normalised activations n are the GEMM operands and
 // their gradients come out of the GEMM with the gain already applied.  Weight gradients are
-// sums over ALL rows of outer products: tc_wgrad_kernel accumulates P^T S over a slab of rows in
-// tensor memory and adds the result to an fp32 accumulator once per slab; gains, biases and the
-// folded terms are taken from those accumulators and from column sums by a last small kernel.
+// sums over ALL rows of outer products: ltc_wgrad_kernel accumulates P^T S over a slab of rows in
+// tensor memory and adds the result to an fp32 accumulator once per slab, and sums the delta
+// operand's columns from the same tiles; gains, biases and the folded terms are taken from those
+// accumulators and sums by a last small kernel.
 // Every r-wide array is padded to 64 columns and every 8r-wide one to 256 (zeros), so two GEMM
 // shapes, 64 -> 256 and 256 -> 64, serve all sixteen layer passes.
 #include "tc_common.cuh"
