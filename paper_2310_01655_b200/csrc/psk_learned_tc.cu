@@ -137,14 +137,12 @@ ltc_bank_kernel(int h, int r, const float* __restrict__ params, bf16* __restrict
 enum { EPI_LN = 0, EPI_B64 = 1, EPI_GELU = 2, EPI_F32 = 3, EPI_DGELU = 4, EPI_LNBWD = 5 };
 
 struct DenseArgs {
-    const float* bias;      // [ND] or null
-    bf16* out0;             // bf16 outputs, [rows][ND]
-    bf16* out1;
-    bf16* out2;
+    const float* bias;      // [64] or null
+    bf16* out0;             // EPI_B64: [rows][64] bf16 (the forward's narrow layers: the hi terms)
+    bf16* out1;             //          the lo terms (forward only)
     float* outf;            // EPI_F32: [rows][ncols]
-    const float* rs;        // (unused by the narrow layers)
     int ncols;              // EPI_F32: columns stored
-    int accumulate;         // EPI_F32: add to what is there
+    int accumulate;         // EPI_F32: add to what is there (backward only)
 };
 
 __device__ __forceinline__ void store8(bf16* dst, const float* v) {
@@ -158,83 +156,54 @@ __device__ __forceinline__ void store8_split(bf16* hi, bf16* lo, const float* v)
     store8(hi, h);
     store8(lo, l);
 }
-// SPLIT (the forward's layers): activations and weights are both hi + lo pairs of bf16 arrays and
-// the product is A_hi B_hi + A_lo B_hi + A_hi B_lo.  A half sketch feeds fourth powers of
-// cancelling sums; single bf16 operands (2^-9 per entry, four layers deep) would leave percents of
-// error on the attention's output, the pairs leave 2^-17.
-template <int KD, int ND, int EPI, bool SPLIT>
-struct DenseSmem {
-    static constexpr int kA1 = 128 * KD * 2, kB1 = KD * ND * 2;
-    static constexpr int kA = kA1 * (SPLIT ? 2 : 1), kB = kB1 * (SPLIT ? 2 : 1);
-    static constexpr int kSides = 0;
-    static constexpr int bytes = kA + kB + 1024;
-};
+// (The forward's layers multiply hi + lo pairs of bf16 arrays for both activations and weights,
+// A_hi B_hi + A_lo B_hi + A_hi B_lo: a half sketch feeds fourth powers of cancelling sums, and
+// single bf16 operands, 2^-9 per entry and four layers deep, would leave percents of error on the
+// attention's output; the pairs leave 2^-17.  The backward's deltas are single bf16.)
+//
+// Narrow layers of the backward (256 -> 64, single operands): one tile per CTA, 128 threads.
+constexpr int kDenseSmem = 128 * 256 * 2 + 256 * 64 * 2 + 1024;
 
-template <int KD, int ND, int EPI, bool SPLIT>
+template <int EPI>
 __global__ void __launch_bounds__(128)
-ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mA2,
-                 const __grid_constant__ CUtensorMap mB, const __grid_constant__ CUtensorMap mB2,
-                 const __grid_constant__ CUtensorMap mS0, const __grid_constant__ CUtensorMap mS1, DenseArgs a,
-                 int* status) {
-    static_assert(KD == 256 && ND == 64 && (EPI == EPI_B64 || EPI == EPI_F32), "the 256 -> 64 layers");
-    using L = DenseSmem<KD, ND, EPI, SPLIT>;
+ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mB, DenseArgs a, int* status) {
+    static_assert(EPI == EPI_B64 || EPI == EPI_F32, "the 256 -> 64 layers");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sA = align1024(smem_raw);
-    uint8_t* sB = sA + L::kA;
-    uint8_t* sS = sB + L::kB;
-    __shared__ uint64_t bar_ld, bar_side, bar_mma;
+    uint8_t* sB = sA + 65536;
+    __shared__ uint64_t bar_ld, bar_mma;
     __shared__ uint32_t tm_slot;
-    __shared__ float s_bias[ND];
+    __shared__ float s_bias[64];
     const int tid = threadIdx.x, warp = tid / 32;
     const int tile = blockIdx.x;
     if (tid == 0) {
         cta_giveup_init();
-        mbar_init(&bar_ld, 1); mbar_init(&bar_side, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_ld, 1); mbar_init(&bar_mma, 1);
         mbar_fence_init();
     }
-    if (warp == 0) { tmem_alloc(&tm_slot, ND); tmem_relinquish(); }
-    for (int j = tid; j < ND; j += 128) s_bias[j] = a.bias != nullptr ? a.bias[j] : 0.f;
+    if (warp == 0) { tmem_alloc(&tm_slot, 64); tmem_relinquish(); }
+    if (tid < 64) s_bias[tid] = a.bias != nullptr ? a.bias[tid] : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tm = tm_slot;
     if (tid == 0) {
-        mbar_expect_tx(&bar_ld, L::kA + L::kB);
+        mbar_expect_tx(&bar_ld, 65536 + 32768);
 #pragma unroll
-        for (int s = 0; s < KD / 64; ++s) tma_load_2d(sA + s * 16384, &mA, s * 64, tile * 128, &bar_ld);
-#pragma unroll
-        for (int g = 0; g < ND / 64; ++g) tma_load_2d(sB + g * KD * 128, &mB, g * 64, 0, &bar_ld);
-        if constexpr (SPLIT) {
-#pragma unroll
-            for (int s = 0; s < KD / 64; ++s) tma_load_2d(sA + L::kA1 + s * 16384, &mA2, s * 64, tile * 128, &bar_ld);
-#pragma unroll
-            for (int g = 0; g < ND / 64; ++g) tma_load_2d(sB + L::kB1 + g * KD * 128, &mB2, g * 64, 0, &bar_ld);
-        }
-        if constexpr (L::kSides > 0) {
-            mbar_expect_tx(&bar_side, L::kSides * 65536);
-#pragma unroll
-            for (int g = 0; g < 4; ++g) tma_load_2d(sS + g * 16384, &mS0, g * 64, tile * 128, &bar_side);
-            if constexpr (L::kSides > 1) {
-#pragma unroll
-                for (int g = 0; g < 4; ++g) tma_load_2d(sS + 65536 + g * 16384, &mS1, g * 64, tile * 128, &bar_side);
-            }
-        }
+        for (int s = 0; s < 4; ++s) tma_load_2d(sA + s * 16384, &mA, s * 64, tile * 128, &bar_ld);
+        tma_load_2d(sB, &mB, 0, 0, &bar_ld);
         if (mbar_wait(&bar_ld, 0, status, kErrTma)) {
             tc_fence_after();
-            constexpr uint32_t idesc = idesc_bf16(128, ND, false, true);
+            constexpr uint32_t idesc = idesc_bf16(128, 64, false, true);
+            const uint64_t ad = smem_desc(smem_u32(sA), 0, 1024, kSwz128);
+            const uint64_t bd = smem_desc(smem_u32(sB), 0, 1024, kSwz128);
 #pragma unroll
-            for (int part = 0; part < (SPLIT ? 3 : 1); ++part) {
-                const uint64_t ad = smem_desc(smem_u32(sA) + (part == 1 ? L::kA1 : 0), 0, 1024, kSwz128);
-                const uint64_t bd = smem_desc(smem_u32(sB) + (part == 2 ? L::kB1 : 0), KD * 128, 1024, kSwz128);
-#pragma unroll
-                for (int k = 0; k < KD / 16; ++k)
-                    umma_ss(tm, desc_off(ad, (k / 4) * 16384 + (k % 4) * 32), desc_off(bd, k * 2048), idesc, (part > 0 || k > 0) ? 1u : 0u);
-            }
+            for (int k = 0; k < 16; ++k)
+                umma_ss(tm, desc_off(ad, (k / 4) * 16384 + (k % 4) * 32), desc_off(bd, k * 2048), idesc, k > 0);
             umma_commit(&bar_mma);
         }
     }
-    bool ok = mbar_wait(&bar_mma, 0, status, kErrMma);
-    if constexpr (L::kSides > 0) ok = ok && mbar_wait(&bar_side, 0, status, kErrTma);
+    const bool ok = mbar_wait(&bar_mma, 0, status, kErrMma);
     tc_fence_after();
     const uint32_t lane_tm = tm + ((uint32_t)(warp * 32) << 16);
     const size_t row = (size_t)tile * 128 + tid;
@@ -249,12 +218,9 @@ ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(u[j]) + s_bias[c0 + j];
 #pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    if constexpr (SPLIT) store8_split(a.out0 + row * 64 + c0 + j, a.out1 + row * 64 + c0 + j, v + j);
-                    else store8(a.out0 + row * 64 + c0 + j, v + j);
-                }
+                for (int j = 0; j < 32; j += 8) store8(a.out0 + row * 64 + c0 + j, v + j);
             }
-        } else if constexpr (EPI == EPI_F32) {
+        } else {
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 if (c0 < a.ncols) {
@@ -280,7 +246,7 @@ ltc_dense_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, ND);
+    if (warp == 0) tmem_dealloc(tm, 64);
 }
 
 // ---------------------------------------------------------------------------
@@ -1111,25 +1077,21 @@ cudaError_t wide(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMa
     return cudaGetLastError();
 }
 // narrow layers (256 -> 64) of the backward: single bf16 operands
-template <int KD, int ND, int EPI>
-cudaError_t dense(const CUtensorMap& mA, const CUtensorMap& mB, const CUtensorMap& mS0, const CUtensorMap& mS1,
-                  const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
-    auto kern = ltc_dense_kernel<KD, ND, EPI, false>;
-    constexpr int smem = DenseSmem<KD, ND, EPI, false>::bytes;
-    PSK_TRY(set_smem(kern, smem));
+template <int EPI>
+cudaError_t dense(const CUtensorMap& mA, const CUtensorMap& mB, const DenseArgs& a, int tiles, int* status, cudaStream_t s,
+                  int* launches) {
+    PSK_TRY(set_smem(ltc_dense_kernel<EPI>, kDenseSmem));
     prof_begin(kDenseName[EPI], s);
-    kern<<<tiles, 128, smem, s>>>(mA, mA, mB, mB, mS0, mS1, a, status);
+    ltc_dense_kernel<EPI><<<tiles, 128, kDenseSmem, s>>>(mA, mB, a, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
 }
-// narrow layers of the forward: hi + lo operand pairs
-template <int KD, int ND, int EPI>
-cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
-                        const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
-    static_assert(KD == 256 && ND == 64, "the narrow layers");
-    auto kern = ltc_narrow_kernel<EPI>;
-    PSK_TRY(set_smem(kern, kNrSmem));
+// narrow layers of the forward: hi + lo operand pairs, persistent kernel
+template <int EPI>
+cudaError_t narrow(const CUtensorMap& mA, const CUtensorMap& mA2, const CUtensorMap& mB, const CUtensorMap& mB2,
+                   const DenseArgs& a, int tiles, int* status, cudaStream_t s, int* launches) {
+    PSK_TRY(set_smem(ltc_narrow_kernel<EPI>, kNrSmem));
     static int sms = 0;
     if (sms == 0) {
         int dev = 0;
@@ -1137,7 +1099,7 @@ cudaError_t dense_split(const CUtensorMap& mA, const CUtensorMap& mA2, const CUt
             sms = 148;
     }
     prof_begin(kDenseSplitName[EPI], s);
-    kern<<<tiles < sms ? tiles : sms, 192, kNrSmem, s>>>(mA, mA2, mB, mB2, a, tiles, status);
+    ltc_narrow_kernel<EPI><<<tiles < sms ? tiles : sms, 192, kNrSmem, s>>>(mA, mA2, mB, mB2, a, tiles, status);
     prof_end(s);
     ++*launches;
     return cudaGetLastError();
@@ -1170,15 +1132,14 @@ cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const vo
     for (int t = 0; t < 2; ++t) {
         const NetBuf& nb = w.net[t];
         const float* vec = (const float*)(ws + w.vec) + (size_t)t * kVec;
-        DenseArgs a{};
         PSK_TRY((wide<EPI_LN, true>(M.n0, M.n0_lo, M.bank[t][0], M.bank[t][8], M.n0, M.n0, M.p1[t], M.n1[t], M.n1_lo[t],
                                     WideArgs{vec, (float*)(ws + nb.rs1), nullptr, m}, tiles, status, s, launches)));
-        a = DenseArgs{vec + 256, (bf16*)(ws + nb.a2), (bf16*)(ws + nb.a2_lo), nullptr, nullptr, nullptr, 0, 0};
-        PSK_TRY((dense_split<256, 64, EPI_B64>(M.n1[t], M.n1_lo[t], M.bank[t][1], M.bank[t][9], a, tiles, status, s, launches)));
+        PSK_TRY(narrow<EPI_B64>(M.n1[t], M.n1_lo[t], M.bank[t][1], M.bank[t][9],
+                                DenseArgs{vec + 256, (bf16*)(ws + nb.a2), (bf16*)(ws + nb.a2_lo), nullptr, 0, 0}, tiles, status, s, launches));
         PSK_TRY((wide<EPI_GELU, true>(M.a2[t], M.a2_lo[t], M.bank[t][2], M.bank[t][10], M.n0, M.n0, M.p3[t], M.a3[t], M.a3_lo[t],
                                       WideArgs{vec + 320, nullptr, nullptr, m}, tiles, status, s, launches)));
-        a = DenseArgs{vec + 576, nullptr, nullptr, nullptr, (float*)(ws + nb.f), nullptr, d.r, 0};
-        PSK_TRY((dense_split<256, 64, EPI_F32>(M.a3[t], M.a3_lo[t], M.bank[t][3], M.bank[t][11], a, tiles, status, s, launches)));
+        PSK_TRY(narrow<EPI_F32>(M.a3[t], M.a3_lo[t], M.bank[t][3], M.bank[t][11],
+                                DenseArgs{vec + 576, nullptr, nullptr, (float*)(ws + nb.f), d.r, 0}, tiles, status, s, launches));
     }
     return cudaSuccess;
 }
@@ -1247,23 +1208,20 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             const NetBuf& nb = w.net[t];
             float* G = (float*)(ws + w.G) + (size_t)t * 4 * kMat;
             float* sums = (float*)(ws + w.sums) + (size_t)t * kSums;
-            DenseArgs a{};
             // dp3 = (df W4^T) * gelu'(p3);  dW4 ~ a3^T df
             PSK_TRY((wide<EPI_DGELU, false>(M.df[t], M.df[t], M.bank[t][4], M.bank[t][4], M.p3[t], M.p3[t], M.dp3, M.dp3, M.dp3,
                                             WideArgs{nullptr, nullptr, nullptr, m}, tiles, status, s, launches)));
             PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, sums + 576, false, tiles, status, s, launches));
             // da2 = dp3 W3^T;  dW3 ~ dp3^T a2
             PSK_TRY(wgrad(M.dp3, M.a2[t], G + 2 * kMat, sums + 320, true, tiles, status, s, launches));
-            a = DenseArgs{nullptr, (bf16*)(ws + w.da2), nullptr, nullptr, nullptr, nullptr, 0, 0};
-            PSK_TRY((dense<256, 64, EPI_B64>(M.dp3, M.bank[t][5], M.n0, M.n0, a, tiles, status, s, launches)));
+            PSK_TRY(dense<EPI_B64>(M.dp3, M.bank[t][5], DenseArgs{nullptr, (bf16*)(ws + w.da2), nullptr, nullptr, 0, 0}, tiles, status, s, launches));
             // dp1 = LN1 backward(da2 (g1 W2)^T) * gelu'(p1);  dW2 ~ n1^T da2
             PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, sums + 256, false, tiles, status, s, launches));
             PSK_TRY((wide<EPI_LNBWD, false>(M.da2, M.da2, M.bank[t][6], M.bank[t][6], M.n1[t], M.p1[t], M.dp1, M.dp1, M.dp1,
                                             WideArgs{nullptr, nullptr, (const float*)(ws + nb.rs1), m}, tiles, status, s, launches)));
             // dn0 (+)= dp1 (g0 W1)^T;  dW1 ~ dp1^T n0
             PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, sums + 0, true, tiles, status, s, launches));
-            a = DenseArgs{nullptr, nullptr, nullptr, nullptr, (float*)(ws + w.dn0), nullptr, 64, t};
-            PSK_TRY((dense<256, 64, EPI_F32>(M.dp1, M.bank[t][7], M.n0, M.n0, a, tiles, status, s, launches)));
+            PSK_TRY(dense<EPI_F32>(M.dp1, M.bank[t][7], DenseArgs{nullptr, nullptr, nullptr, (float*)(ws + w.dn0), 64, t}, tiles, status, s, launches));
         }
         prof_begin("ltc_ln0_bwd_kernel", s);
         ltc_ln0_bwd_kernel<<<(c + 7) / 8, 256, 0, s>>>(sl, row0, c, (const float*)(ws + w.dn0), (const bf16*)(ws + w.n0),
