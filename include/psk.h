@@ -205,7 +205,10 @@ int psk_causal_attn_fwd_static(const psk_shape* shape, const void* Q, const void
  * the half sketch keeps 2^-17; backward and weight gradients with single bf16 operands) and the
  * attention on their half sketches (`path` = PSK_PATH_CUDA_CORES forces the CUDA-core kernels,
  * PSK_PATH_TENSOR_CORES refuses what the tensor-core route does not serve).  Everything else, and
- * psk_learned_sketch itself, runs on the CUDA cores in fp32.  Workspace size from
+ * psk_learned_sketch itself, runs on the CUDA cores in fp32.  On the tensor-core route the rows pass
+ * through the networks' layers 2^20 at a time (the activations of one such pass are part of the
+ * workspace); the environment variable PSK_LEARNED_CHUNK_ROWS (a multiple of 128) overrides that
+ * number, provided it does not change between the workspace query and the calls that use it.  Workspace size from
  * psk_learned_workspace_bytes. */
 size_t psk_learned_param_count(int h, int r);
 size_t psk_learned_workspace_bytes(const psk_shape* shape, int for_backward);
