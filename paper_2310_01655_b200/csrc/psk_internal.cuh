@@ -83,12 +83,13 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
                       cudaStream_t s, int* launches);
 
 // The learnable sketch's networks on the tensor cores (psk_learned_tc.cu): bf16, r <= 32.
-// `prepare` once per call, `sketch` / `sketch_bwd` per tensor, `finish` once after the last sketch_bwd.
+// `prepare` once per call, `sketch` / `sketch_bwd` per tensor (they write the [hi | lo] rows the
+// attention kernels read, and take their gradient), `finish` once after the last sketch_bwd.
 bool learned_tc_supported(const Dims& d);
 size_t learned_tc_workspace_bytes(const Dims& d, bool backward);
 cudaError_t learned_tc_prepare(const Dims& d, bool backward, char* ws, cudaStream_t s, int* launches);
-cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* M, char* ws, int* status, cudaStream_t s, int* launches);
-cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const void* add, void* dX, char* ws,
+cudaError_t learned_tc_sketch(const Dims& d, const void* X, void* S, char* ws, int* status, cudaStream_t s, int* launches);
+cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const void* dS, const void* add, void* dX, char* ws,
                                   int* status, cudaStream_t s, int* launches);
 cudaError_t learned_tc_finish(const Dims& d, char* ws, cudaStream_t s, int* launches);
 

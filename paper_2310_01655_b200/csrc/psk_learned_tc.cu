@@ -397,6 +397,7 @@ struct WideArgs {
     float* rs_out;          // EPI_LN: 1 / sigma of every row
     const float* rs_in;     // EPI_LNBWD
     int ncols;              // live columns (8r)
+    int keep_pre;           // EPI_LN, EPI_GELU: also store the pre-activation (output 0), which only the backward reads
 };
 
 template <int EPI, bool SPLIT>
@@ -537,14 +538,14 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
                             pv[q] = __uint_as_float(u[j + q]) + bv[q];
                             g[q] = (FULL || c0 + j + q < a.ncols) ? gelu_f(pv[q]) : 0.f;
                         }
-                        tile_put8(stg, rowt, half * 4 + j / 8, pv);
+                        if (a.keep_pre) tile_put8(stg, rowt, half * 4 + j / 8, pv);
                         tile_put8_split(stg + 16384, stg + 32768, rowt, half * 4 + j / 8, g);
                     }
                 }
                 fence_proxy_async_smem();
                 wg_sync();
                 if (elected) {
-                    tma_store_2d(&mO0, stg, cg * 64, tile * 128);
+                    if (a.keep_pre) tma_store_2d(&mO0, stg, cg * 64, tile * 128);
                     tma_store_2d(&mO1, stg + 16384, cg * 64, tile * 128);
                     tma_store_2d(&mO2, stg + 32768, cg * 64, tile * 128);
                     bulk_commit();
@@ -576,18 +577,20 @@ ltc_wide_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
                             s += g; ss = fmaf(g, g, ss);
                             u[j + q] = __float_as_uint(g);
                         }
-                        tile_put8(stg, rowt, half * 4 + j / 8, pv);
+                        if (a.keep_pre) tile_put8(stg, rowt, half * 4 + j / 8, pv);
                     }
                     tmem_st32(lane_tm + c0, u);
                 }
-                fence_proxy_async_smem();
-                wg_sync();
-                if (elected) {
-                    tma_store_2d(&mO0, stg, cg * 64, tile * 128);
-                    bulk_commit();
-                    bulk_wait_read();
+                if (a.keep_pre) {
+                    fence_proxy_async_smem();
+                    wg_sync();
+                    if (elected) {
+                        tma_store_2d(&mO0, stg, cg * 64, tile * 128);
+                        bulk_commit();
+                        bulk_wait_read();
+                    }
+                    wg_sync();
                 }
-                wg_sync();
             }
             tmem_st_wait();
             s_part[wg][rowt] = make_float2(s, ss);
@@ -883,18 +886,40 @@ ltc_ln0_bwd_kernel(Slice sl, size_t row0, int rows, const float* __restrict__ dn
     *reinterpret_cast<uint32_t*>(dX + sl.row(row0 + i) + 2 * lane) = pack_bf16(oa, ob);
 }
 
-// M = sqrt(r) tanh(f1 f2 / sqrt(r))
+// M = sqrt(r) tanh(f1 f2 / sqrt(r)), written as the [hi | lo] rows (64 bf16 columns, zero beyond 2r) the
+// attention kernels read in their linear sketch mode; one thread = 8 consecutive columns of a row
 __global__ void __launch_bounds__(256)
-ltc_combine_kernel(const float* __restrict__ f1, const float* __restrict__ f2, int r, size_t count, float* __restrict__ M) {
+ltc_combine_kernel(const float* __restrict__ f1, const float* __restrict__ f2, int r, size_t rows, bf16* __restrict__ S) {
     const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
-    if (e >= count) return;
-    const float sr = sqrtf((float)r);
-    M[e] = sr * tanhf(f1[e] * f2[e] / sr);
+    if (e >= rows * 8) return;
+    const size_t row = e / 8;
+    const int c0 = (int)(e % 8) * 8;
+    const float sr = sqrtf((float)r), isr = rsqrtf((float)r);
+    uint32_t pk[4];
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+        float x[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int c = c0 + j + q;
+            float v = 0.f;
+            if (c < 2 * r) {
+                const size_t o = row * r + (c % r);
+                const float m = sr * tanhf(f1[o] * f2[o] * isr);
+                const float hi = __bfloat162float(__float2bfloat16_rn(m));
+                v = c < r ? hi : m - hi;
+            }
+            x[q] = v;
+        }
+        pk[j / 2] = pack_bf16(x[0], x[1]);
+    }
+    *reinterpret_cast<uint4*>(S + row * 64 + c0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
 }
 
-// df1 = dM (1 - t^2) f2, df2 = dM (1 - t^2) f1 as bf16 rows of 64 columns (zero beyond r)
+// df1 = dM (1 - t^2) f2, df2 = dM (1 - t^2) f1 as bf16 rows of 64 columns (zero beyond r); dM = the
+// first r columns of dS, the gradient of the [hi | lo] rows (M = hi + lo)
 __global__ void __launch_bounds__(256)
-ltc_combine_bwd_kernel(const float* __restrict__ f1, const float* __restrict__ f2, const float* __restrict__ dM, int r,
+ltc_combine_bwd_kernel(const float* __restrict__ f1, const float* __restrict__ f2, const bf16* __restrict__ dS, int r,
                        size_t rows, bf16* __restrict__ df1, bf16* __restrict__ df2) {
     const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (e >= rows * 64) return;
@@ -904,7 +929,7 @@ ltc_combine_bwd_kernel(const float* __restrict__ f1, const float* __restrict__ f
     if (c < r) {
         const float a = f1[row * r + c], b = f2[row * r + c];
         const float t = tanhf(a * b * rsqrtf((float)r));
-        const float du = dM[row * r + c] * (1.f - t * t);
+        const float du = __bfloat162float(dS[e]) * (1.f - t * t);
         o1 = du * b; o2 = du * a;
     }
     df1[e] = __float2bfloat16_rn(o1);
@@ -1120,7 +1145,8 @@ cudaError_t wgrad(const CUtensorMap& mP, const CUtensorMap& mS, float* Gt, float
 }
 
 // forward of both networks on `c` rows starting at row0: activations and f into the chunk buffers
-cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const void* X, size_t row0, int c, char* ws,
+// (keep_pre: also the pre-activations p1, p3, which only the backward reads)
+cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const void* X, size_t row0, int c, bool keep_pre, char* ws,
                           int* status, cudaStream_t s, int* launches) {
     const Slice sl{d.H, d.n, d.sb, d.sh, d.sn};
     const int tiles = c / 128, m = 8 * d.r;
@@ -1133,11 +1159,11 @@ cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const vo
         const NetBuf& nb = w.net[t];
         const float* vec = (const float*)(ws + w.vec) + (size_t)t * kVec;
         PSK_TRY((wide<EPI_LN, true>(M.n0, M.n0_lo, M.bank[t][0], M.bank[t][8], M.n0, M.n0, M.p1[t], M.n1[t], M.n1_lo[t],
-                                    WideArgs{vec, (float*)(ws + nb.rs1), nullptr, m}, tiles, status, s, launches)));
+                                    WideArgs{vec, (float*)(ws + nb.rs1), nullptr, m, keep_pre ? 1 : 0}, tiles, status, s, launches)));
         PSK_TRY(narrow<EPI_B64>(M.n1[t], M.n1_lo[t], M.bank[t][1], M.bank[t][9],
                                 DenseArgs{vec + 256, (bf16*)(ws + nb.a2), (bf16*)(ws + nb.a2_lo), nullptr, 0, 0}, tiles, status, s, launches));
         PSK_TRY((wide<EPI_GELU, true>(M.a2[t], M.a2_lo[t], M.bank[t][2], M.bank[t][10], M.n0, M.n0, M.p3[t], M.a3[t], M.a3_lo[t],
-                                      WideArgs{vec + 320, nullptr, nullptr, m}, tiles, status, s, launches)));
+                                      WideArgs{vec + 320, nullptr, nullptr, m, keep_pre ? 1 : 0}, tiles, status, s, launches)));
         PSK_TRY(narrow<EPI_F32>(M.a3[t], M.a3_lo[t], M.bank[t][3], M.bank[t][11],
                                 DenseArgs{vec + 576, nullptr, nullptr, (float*)(ws + nb.f), d.r, 0}, tiles, status, s, launches));
     }
@@ -1162,18 +1188,18 @@ cudaError_t learned_tc_prepare(const Dims& d, bool backward, char* ws, cudaStrea
     return cudaSuccess;
 }
 
-cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* Mout, char* ws, int* status, cudaStream_t s, int* launches) {
+// S = the [hi | lo] rows of the half sketch of X (contiguous [rows][64] bf16)
+cudaError_t learned_tc_sketch(const Dims& d, const void* X, void* S, char* ws, int* status, cudaStream_t s, int* launches) {
     const LtcWs w = ltc_ws(d, false);            // the forward's buffers come first in either layout
     Maps M;
     if (!build_maps(w, ws, false, &M)) return cudaErrorInvalidValue;
     const size_t rows = (size_t)d.BH() * d.n;
     for (size_t row0 = 0; row0 < rows; row0 += w.C) {
         const int c = (int)(rows - row0 < w.C ? rows - row0 : w.C);
-        PSK_TRY(forward_chunk(d, w, M, X, row0, c, ws, status, s, launches));
-        const size_t cnt = (size_t)c * d.r;
+        PSK_TRY(forward_chunk(d, w, M, X, row0, c, false, ws, status, s, launches));
         prof_begin("ltc_combine_kernel", s);
-        ltc_combine_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, s>>>((const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f),
-                                                                         d.r, cnt, Mout + row0 * d.r);
+        ltc_combine_kernel<<<(unsigned)(((size_t)c * 8 + 255) / 256), 256, 0, s>>>((const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f),
+                                                                              d.r, (size_t)c, (bf16*)S + row0 * 64);
         prof_end(s);
         ++*launches;
         PSK_TRY(cudaGetLastError());
@@ -1181,11 +1207,11 @@ cudaError_t learned_tc_sketch(const Dims& d, const void* X, float* Mout, char* w
     return cudaSuccess;
 }
 
-// dX = chain rule of sum(dM * M) through both networks (+ add, a contiguous [rows][64] bf16 array
+// dX = chain rule through both networks of the gradient dS of the [hi | lo] rows (+ add, a contiguous [rows][64] bf16 array
 // or null: the part of the gradient that reached X directly); the weight-gradient
 // accumulators in the workspace grow by this tensor's share (learned_tc_finish turns them into
 // parameter gradients)
-cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM, const void* add, void* dX, char* ws,
+cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const void* dS, const void* add, void* dX, char* ws,
                                   int* status, cudaStream_t s, int* launches) {
     const LtcWs w = ltc_ws(d, true);
     Maps M;
@@ -1196,10 +1222,10 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
     for (size_t row0 = 0; row0 < rows; row0 += w.C) {
         const int c = (int)(rows - row0 < w.C ? rows - row0 : w.C);
         const int tiles = c / 128;
-        PSK_TRY(forward_chunk(d, w, M, X, row0, c, ws, status, s, launches));
+        PSK_TRY(forward_chunk(d, w, M, X, row0, c, true, ws, status, s, launches));
         prof_begin("ltc_combine_bwd_kernel", s);
         ltc_combine_bwd_kernel<<<(unsigned)(((size_t)c * 64 + 255) / 256), 256, 0, s>>>(
-            (const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f), dM + row0 * d.r, d.r, (size_t)c,
+            (const float*)(ws + w.net[0].f), (const float*)(ws + w.net[1].f), (const bf16*)dS + row0 * 64, d.r, (size_t)c,
             (bf16*)(ws + w.df[0]), (bf16*)(ws + w.df[1]));
         prof_end(s);
         ++*launches;
@@ -1210,7 +1236,7 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             float* sums = (float*)(ws + w.sums) + (size_t)t * kSums;
             // dp3 = (df W4^T) * gelu'(p3);  dW4 ~ a3^T df
             PSK_TRY((wide<EPI_DGELU, false>(M.df[t], M.df[t], M.bank[t][4], M.bank[t][4], M.p3[t], M.p3[t], M.dp3, M.dp3, M.dp3,
-                                            WideArgs{nullptr, nullptr, nullptr, m}, tiles, status, s, launches)));
+                                            WideArgs{nullptr, nullptr, nullptr, m, 0}, tiles, status, s, launches)));
             PSK_TRY(wgrad(M.a3[t], M.df[t], G + 3 * kMat, sums + 576, false, tiles, status, s, launches));
             // da2 = dp3 W3^T;  dW3 ~ dp3^T a2
             PSK_TRY(wgrad(M.dp3, M.a2[t], G + 2 * kMat, sums + 320, true, tiles, status, s, launches));
@@ -1218,7 +1244,7 @@ cudaError_t learned_tc_sketch_bwd(const Dims& d, const void* X, const float* dM,
             // dp1 = LN1 backward(da2 (g1 W2)^T) * gelu'(p1);  dW2 ~ n1^T da2
             PSK_TRY(wgrad(M.n1[t], M.da2, G + 1 * kMat, sums + 256, false, tiles, status, s, launches));
             PSK_TRY((wide<EPI_LNBWD, false>(M.da2, M.da2, M.bank[t][6], M.bank[t][6], M.n1[t], M.p1[t], M.dp1, M.dp1, M.dp1,
-                                            WideArgs{nullptr, nullptr, (const float*)(ws + nb.rs1), m}, tiles, status, s, launches)));
+                                            WideArgs{nullptr, nullptr, (const float*)(ws + nb.rs1), m, 0}, tiles, status, s, launches)));
             // dn0 (+)= dp1 (g0 W1)^T;  dW1 ~ dp1^T n0
             PSK_TRY(wgrad(M.dp1, M.n0, G + 0 * kMat, sums + 0, true, tiles, status, s, launches));
             PSK_TRY(dense<EPI_F32>(M.dp1, M.bank[t][7], DenseArgs{nullptr, nullptr, nullptr, (float*)(ws + w.dn0), 64, t}, tiles, status, s, launches));
