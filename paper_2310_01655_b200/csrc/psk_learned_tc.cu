@@ -843,26 +843,36 @@ struct Slice {
     }
 };
 
-// n0 = (x - mean) / sigma of every row (one warp per row, two columns per lane), 1 / sigma kept
+// n0 = (x - mean) / sigma of every row as hi + lo, 1 / sigma kept.  One warp per row, two columns
+// per lane, eight rows per warp with their loads issued together.
+constexpr int kLnRowsPerWarp = 8;
 __global__ void __launch_bounds__(256)
 ltc_ln0_kernel(Slice sl, const bf16* __restrict__ X, size_t row0, int rows, bf16* __restrict__ n0, bf16* __restrict__ n0_lo,
                float* __restrict__ rs0) {
     const int lane = threadIdx.x % 32;
-    const int i = blockIdx.x * 8 + threadIdx.x / 32;
-    if (i >= rows) return;
-    const __nv_bfloat162 x2 = *reinterpret_cast<const __nv_bfloat162*>(X + sl.row(row0 + i) + 2 * lane);
-    const float a = __low2float(x2), b = __high2float(x2);
-    float s = a + b;
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float mu = s * (1.f / 64.f);
-    float v = (a - mu) * (a - mu) + (b - mu) * (b - mu);
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    const float rs = rsqrtf(v * (1.f / 64.f) + kLnEps);
-    const float na = (a - mu) * rs, nb = (b - mu) * rs;
-    const float ha = __bfloat162float(__float2bfloat16_rn(na)), hb = __bfloat162float(__float2bfloat16_rn(nb));
-    *reinterpret_cast<uint32_t*>(n0 + (size_t)i * 64 + 2 * lane) = pack_bf16(ha, hb);
-    *reinterpret_cast<uint32_t*>(n0_lo + (size_t)i * 64 + 2 * lane) = pack_bf16(na - ha, nb - hb);
-    if (lane == 0) rs0[i] = rs;
+    const int i0 = (blockIdx.x * 8 + threadIdx.x / 32) * kLnRowsPerWarp;
+    __nv_bfloat162 x2[kLnRowsPerWarp];
+#pragma unroll
+    for (int q = 0; q < kLnRowsPerWarp; ++q)
+        if (i0 + q < rows) x2[q] = *reinterpret_cast<const __nv_bfloat162*>(X + sl.row(row0 + i0 + q) + 2 * lane);
+#pragma unroll
+    for (int q = 0; q < kLnRowsPerWarp; ++q) {
+        const int i = i0 + q;
+        if (i >= rows) break;
+        const float a = __low2float(x2[q]), b = __high2float(x2[q]);
+        float s = a + b;
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float mu = s * (1.f / 64.f);
+        float v = (a - mu) * (a - mu) + (b - mu) * (b - mu);
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        const float rs = rsqrtf(v * (1.f / 64.f) + kLnEps);
+        const float na = (a - mu) * rs, nb = (b - mu) * rs;
+        const uint32_t h = pack_bf16(na, nb);
+        *reinterpret_cast<uint32_t*>(n0 + (size_t)i * 64 + 2 * lane) = h;
+        *reinterpret_cast<uint32_t*>(n0_lo + (size_t)i * 64 + 2 * lane) =
+            pack_bf16(na - __uint_as_float(h << 16), nb - __uint_as_float(h & 0xffff0000u));
+        if (lane == 0) rs0[i] = rs;
+    }
 }
 
 // dX = back through the first normalisation of the summed gradient of n0 (+ add)
@@ -1151,7 +1161,7 @@ cudaError_t forward_chunk(const Dims& d, const LtcWs& w, const Maps& M, const vo
     const Slice sl{d.H, d.n, d.sb, d.sh, d.sn};
     const int tiles = c / 128, m = 8 * d.r;
     prof_begin("ltc_ln0_kernel", s);
-    ltc_ln0_kernel<<<(c + 7) / 8, 256, 0, s>>>(sl, (const bf16*)X, row0, c, (bf16*)(ws + w.n0), (bf16*)(ws + w.n0_lo), (float*)(ws + w.rs0));
+    ltc_ln0_kernel<<<(c + 8 * kLnRowsPerWarp - 1) / (8 * kLnRowsPerWarp), 256, 0, s>>>(sl, (const bf16*)X, row0, c, (bf16*)(ws + w.n0), (bf16*)(ws + w.n0_lo), (float*)(ws + w.rs0));
     prof_end(s);
     ++*launches;
     PSK_TRY(cudaGetLastError());
