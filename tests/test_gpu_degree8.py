@@ -101,3 +101,32 @@ def test_kept_states_on_the_tensor_cores():
         check("denom", den[bi, hi], d_ref, TOL["bf16"])
         for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), orc.causal_polysketch8_attention_backward(q, k, v, Gs, g)):
             check(name, got[bi, hi], ref, TOL["bf16"])
+
+
+def test_strided_views_and_one_shared_sketch_on_the_tensor_cores():
+    # [B, n, H, h] storage viewed as [B, H, n, h]; one packed Gaussian set for all heads
+    B, H, n, r, b = 2, 3, 512, 32, 256
+    w = wl.small_workload(B=B, H=H, n=n, r=r, b=b, dtype="bf16", seed=520)
+    inp = wl.make_inputs(w, "cuda")
+    view = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    Q, K = (view((inp[k].float() * 0.25).bfloat16()) for k in ("Q", "K"))
+    V, dO = view(inp["V"]), view(inp["dO"])
+    assert not Q.is_contiguous()
+    G1, G2 = _packed_gaussians(1, 64, r, 621, torch.bfloat16)
+    psk.profile_enable(True)
+    O, den = psk.causal_attn_fwd(Q, K, V, G1, G2, b, p=8)
+    dQ, dK, dV = psk.causal_attn_bwd(Q, K, V, G1, G2, O, den, dO, b, p=8)
+    torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    assert {"sk8_tc_fwd_kernel", "sk8_tc_bwd_kernel", "tc_bwd_k_kernel"} <= kernels
+    assert O.stride() == Q.stride() and dQ.stride() == Q.stride()
+    Gs = _oracle_gaussians(G1, G2, 0, 64)
+    for bi, hi in ((0, 0), (1, 2)):
+        q, k, v, g = (x[bi, hi].double().cpu().numpy() for x in (Q, K, V, dO))
+        Mq, Mk = orc.half_sketch_degree4(q, Gs), orc.half_sketch_degree4(k, Gs)
+        O_ref, d_ref = orc.causal_attention_blocked_from_half_sketches(Mq, Mk, v, b)
+        check("O", O[bi, hi], O_ref, TOL["bf16"])
+        check("denom", den[bi, hi], d_ref, TOL["bf16"])
+        for name, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), orc.causal_polysketch8_attention_backward(q, k, v, Gs, g)):
+            check(name, got[bi, hi], ref, TOL["bf16"])

@@ -141,6 +141,35 @@ def test_networks_in_several_passes_over_the_rows(monkeypatch):
     _run_and_check(inp, w, flat, P1, P2, r, b, [(bi, hi) for bi in range(2) for hi in range(2)], TOL["bf16"], True)
 
 
+@pytest.mark.parametrize("local", [False, True])
+def test_strided_views_on_the_tensor_cores(local):
+    # [B, n, H, h] storage viewed as [B, H, n, h]: the networks read and write rows by their strides,
+    # the attention kernels through tensor maps with non-dense strides
+    r, b = 32, 128
+    w = wl.small_workload(B=2, H=3, n=384, r=r, b=b, dtype="bf16", seed=93)
+    inp = wl.make_inputs(w, "cuda")
+    view = lambda t: t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    scale = 0.35 if local else 1.0
+    inp = dict(inp, Q=view((scale * inp["Q"].float()).bfloat16()), K=view((scale * inp["K"].float()).bfloat16()),
+               V=view(inp["V"]), dO=view(inp["dO"]))
+    assert not inp["Q"].is_contiguous()
+    flat, P1, P2 = nets(r, 6)
+    flags = psk.FLAG_LOCAL_EXACT if local else 0
+    Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
+    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags)
+    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags)
+    assert O.stride() == Q.stride() and dQ.stride() == Q.stride()
+    diag = "exact" if local else "LR"
+    for bi, hi in ((0, 0), (1, 2)):
+        f = lambda k: head_slice_f64(inp[k], bi, hi)
+        O_ref, d_ref = orc.causal_learned_polysketch_attention_blocked(f("Q"), f("K"), f("V"), P1, P2, b, diagonal=diag)
+        check("O", O[bi, hi], O_ref, TOL["bf16"])
+        check("denom", den[bi, hi], d_ref, TOL["bf16"])
+        gq, gk, gv, _, _ = orc.causal_learned_polysketch_attention_backward(f("Q"), f("K"), f("V"), P1, P2, f("dO"), b, diag)
+        for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), (gq, gk, gv)):
+            check(nm, got[bi, hi], ref, TOL["bf16"])
+
+
 def test_networks_across_the_default_chunk_boundary():
     # 4 x 12 heads of 32768 rows: 1.5 M rows per tensor, so the second pass starts at head (2, 8)
     r, b = 32, 256
