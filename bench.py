@@ -320,8 +320,8 @@ def time_variant(psk, wl, name, base, steps, warmup, device_index):
     den = torch.empty((w.B, w.H, w.n), dtype=torch.float32, device="cuda")
     grads = tuple(torch.empty_like(Q) for _ in range(3))
     if name in ("learned", "learned_local"):
-        lflags = psk.FLAG_LOCAL_EXACT if name == "learned_local" else 0
-        if lflags:
+        lflags = flags | (psk.FLAG_LOCAL_EXACT if name == "learned_local" else 0)      # kept states, like the headline
+        if name == "learned_local":
             Q.mul_(0.35); K.mul_(0.35)      # (q.k)^4 next to sketch weights bounded by r^2: the same scale
         flat = binding.pack_learned_params(*wl.learned_network_params(w.h, r, base.g_seed))
         ws = torch.empty(binding.learned_workspace_bytes(Q, r, b, lflags), dtype=torch.uint8, device="cuda")

@@ -170,6 +170,37 @@ def test_strided_views_on_the_tensor_cores(local):
             check(nm, got[bi, hi], ref, TOL["bf16"])
 
 
+@pytest.mark.parametrize("local", [False, True])
+def test_kept_states_on_the_tensor_cores(local):
+    # one workspace for both calls: the backward reads the states the forward left there
+    r, b = 32, 256
+    w = wl.small_workload(B=2, H=2, n=1024, r=r, b=b, dtype="bf16", seed=94)
+    inp = wl.make_inputs(w, "cuda")
+    if local:
+        inp["Q"], inp["K"] = (0.35 * inp["Q"].float()).bfloat16(), (0.35 * inp["K"].float()).bfloat16()
+    flat, P1, P2 = nets(r, 7)
+    flags = psk.FLAG_KEEP_STATES | (psk.FLAG_LOCAL_EXACT if local else 0)
+    Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
+    ws = torch.empty(binding.learned_workspace_bytes(Q, r, b, flags), dtype=torch.uint8, device="cuda")
+    psk.profile_enable(True)
+    O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags, ws)
+    dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags, ws)
+    torch.cuda.synchronize()
+    kernels = {name for name, _ in psk.profile_records()}
+    psk.profile_enable(False)
+    assert psk.check(ws) == 0
+    assert "tc_bwd_prep_kernel" in kernels and "tc_bwd_recompute_kernel" not in kernels      # the kept states were used
+    diag = "exact" if local else "LR"
+    for bi, hi in ((0, 1), (1, 0)):
+        f = lambda k: head_slice_f64(inp[k], bi, hi)
+        O_ref, d_ref = orc.causal_learned_polysketch_attention_blocked(f("Q"), f("K"), f("V"), P1, P2, b, diagonal=diag)
+        check("O", O[bi, hi], O_ref, TOL["bf16"])
+        check("denom", den[bi, hi], d_ref, TOL["bf16"])
+        gq, gk, gv, _, _ = orc.causal_learned_polysketch_attention_backward(f("Q"), f("K"), f("V"), P1, P2, f("dO"), b, diag)
+        for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), (gq, gk, gv)):
+            check(nm, got[bi, hi], ref, TOL["bf16"])
+
+
 def test_networks_across_the_default_chunk_boundary():
     # 4 x 12 heads of 32768 rows: 1.5 M rows per tensor, so the second pass starts at head (2, 8)
     r, b = 32, 256
