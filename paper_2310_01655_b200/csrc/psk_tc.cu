@@ -190,16 +190,19 @@ tc_fwd_out_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     const bool has_prefix = noncausal || l > 0;
 
     if (tid == 0) {
-        mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_sk, 1); mbar_init(&bar_s, 1); mbar_init(&bar_pv, 1);
+        // the query tile is what everything waits for: its request goes out before anything else
+        mbar_init(&bar_q, 1);
+        mbar_fence_init();
+        mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
+        tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
+        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
+        mbar_init(&bar_kv, 1); mbar_init(&bar_sk, 1); mbar_init(&bar_s, 1); mbar_init(&bar_pv, 1);
         mbar_init(&bar_mk, 128); mbar_init(&bar_p, 128); mbar_init(&bar_go, 128);
         for (int s = 0; s < kZStages; ++s) mbar_init(&bar_z[s], 1);
         for (int s = 0; s < kFeatBufs; ++s) { mbar_init(&bar_feat[s], 128); mbar_init(&bar_a[s], 1); }
         cta_giveup_init();
         mbar_fence_init();
-        tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV); tma_prefetch_desc(&mapZ);
-        mbar_expect_tx(&bar_q, 16384 + GImage<R>::bytes);
-        tma_load_4d(smem + L::Q, &mapQ, 0, row0, hi, bi, &bar_q);
-        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_q);
+        tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV); tma_prefetch_desc(&mapZ);
     }
     // The same-block key/value tiles are loaded late (their buffers hold state chunks first, and a
     // tile's buffers are free only when the previous tile's MMAs are done): ask for them in L2 now,
