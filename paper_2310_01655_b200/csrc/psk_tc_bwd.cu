@@ -176,17 +176,19 @@ tc_bwd_rows_kernel(const __grid_constant__ CUtensorMap mapXown, const __grid_con
     const bool has_state = noncausal || (QSIDE ? (l > 0) : (l < t - 1));
 
     if (tid == 0) {
-        mbar_init(&bar_own, 1); mbar_init(&bar_xoth, 1); mbar_init(&bar_yoth, 1); mbar_init(&bar_mma, 1);
+        // the own tiles are what everything waits for: their requests go out before anything else
+        mbar_init(&bar_own, 1);
+        mbar_fence_init();
+        mbar_expect_tx(&bar_own, 32768 + GImage<R>::bytes);
+        tma_load_4d(smem + L::Xown, &mapXown, 0, row0, hi, bi, &bar_own);
+        tma_load_4d(smem + L::Yown, &mapYown, 0, row0, hi, bi, &bar_own);
+        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_own);
+        mbar_init(&bar_xoth, 1); mbar_init(&bar_yoth, 1); mbar_init(&bar_mma, 1);
         mbar_init(&bar_phi[0], 1); mbar_init(&bar_phi[1], 1);
         for (int s = 0; s < kStages; ++s) mbar_init(&bar_box[s], 1);
         cta_giveup_init();
         mbar_fence_init();
-        tma_prefetch_desc(&mapXown); tma_prefetch_desc(&mapYown); tma_prefetch_desc(&mapXoth);
-        tma_prefetch_desc(&mapYoth); tma_prefetch_desc(&mapS);
-        mbar_expect_tx(&bar_own, 32768 + GImage<R>::bytes);
-        bulk_load(smem + L::G, gimg + (size_t)g * GImage<R>::bytes, GImage<R>::bytes, &bar_own);
-        tma_load_4d(smem + L::Xown, &mapXown, 0, row0, hi, bi, &bar_own);
-        tma_load_4d(smem + L::Yown, &mapYown, 0, row0, hi, bi, &bar_own);
+        tma_prefetch_desc(&mapXoth); tma_prefetch_desc(&mapYoth); tma_prefetch_desc(&mapS);
         if (has_state) {
             for (int c = 0; c < kStages && c < F::NC; ++c) {
                 mbar_expect_tx(&bar_box[c], kBoxBytes);
