@@ -92,7 +92,8 @@ typedef struct {
 /* PSK_FLAG_KEEP_STATES (tensor-core path; ignored by the CUDA-core path): set on BOTH the
  * forward and the backward call of one training step.  The forward then leaves in its
  * workspace the prefix states Z_l of Section 3.1, the per-head value centres c they are centred
- * by, and O - c (rounded after the subtraction: the caller's rounded O cannot supply it); the
+ * by, and O - c (rounded after the subtraction: the caller's rounded O cannot supply it) - for
+ * p = 8 and the learnable sketch also the half sketches of Q and K; the
  * backward, given the SAME workspace memory (not written in between) with the same shape and inputs, reads them instead
  * of rebuilding the states from K and V and recomputing the forward rows.  With the flag set
  * psk_workspace_bytes() returns the backward's size for both calls.  Without the flag each

@@ -49,14 +49,16 @@ GivenWs given_ws(const Dims& d, bool backward) {
     return w;
 }
 
+// the sketch kernels' operand banks, then (unless `kept`: the forward left them in this workspace)
 // the [hi | lo] rows of both tensors' half sketches
 cudaError_t half_sketches(const Dims& d, const void* Q, const void* K, const void* G1, const void* G2, char* ws,
-                          const GivenWs& w, bool backward, cudaStream_t s, int* launches) {
+                          const GivenWs& w, bool backward, bool kept, cudaStream_t s, int* launches) {
     const void* X[2] = {Q, K};
     const size_t so[2] = {w.Sq, w.Sk};
     int* status = reinterpret_cast<int*>(ws + w.tc);
     if (d.learned) PSK_TRY(learned_tc_prepare(d, backward, ws + w.sketch, s, launches));
     else PSK_TRY(sketch8_tc_prepare(d, G1, G2, ws + w.sketch, s, launches));
+    if (kept) return cudaSuccess;
     for (int i = 0; i < 2; ++i) {
         if (d.learned) PSK_TRY(learned_tc_sketch(d, X[i], ws + so[i], ws + w.sketch, status, s, launches));
         else PSK_TRY(sketch8_tc_fwd(d, X[i], ws + so[i], ws + w.sketch, status, s, launches));
@@ -78,7 +80,7 @@ size_t given_workspace_bytes(const Dims& d, bool backward) { return given_ws(d, 
 cudaError_t given_fwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
                       void* O, float* denom, char* ws, cudaStream_t s, int* launches) {
     const GivenWs w = given_ws(d, d.keep_states);
-    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, false, s, launches));
+    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, false, false, s, launches));
     Dims l = linear_dims(d);
     l.rawQ = Q; l.rawK = K;
     return tc_fwd(l, ws + w.Sq, ws + w.Sk, V, nullptr, nullptr, O, denom, ws + w.tc, s, launches);
@@ -88,7 +90,8 @@ cudaError_t given_bwd(const Dims& d, const void* Q, const void* K, const void* V
                       const void* O, const float* denom, const void* dO, void* dQ, void* dK, void* dV, char* ws,
                       cudaStream_t s, int* launches) {
     const GivenWs w = given_ws(d, true);
-    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, true, s, launches));
+    // PSK_FLAG_KEEP_STATES: the half sketches are part of what the forward left in the workspace
+    PSK_TRY(half_sketches(d, Q, K, G1, G2, ws, w, true, d.keep_states, s, launches));
     Dims l = linear_dims(d);
     l.rawQ = Q; l.rawK = K;
     if (l.local) { l.rawdQ = ws + w.dXq; l.rawdK = ws + w.dXk; }

@@ -97,15 +97,20 @@ def test_attention_forward_and_backward_with_parameter_gradients(r, b, n, dtype,
             check("net %d %s" % (which + 1, k), got[k], ref[k], 5 * tol if dtype == "bf16" else 2e-3)
 
 
-def _run_and_check(inp, w, flat, P1, P2, r, b, heads, tol, with_params, bwd_heads=None):
+def _run_and_check(inp, w, flat, P1, P2, r, b, heads, tol, with_params, bwd_heads=None, passes=None):
     Q, K, V, dO = (inp[k] for k in ("Q", "K", "V", "dO"))
     psk.profile_enable(True)
     O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b)
     dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b)
     torch.cuda.synchronize()
-    kernels = {name for name, _ in psk.profile_records()}
+    records = [name for name, _ in psk.profile_records()]
+    kernels = set(records)
     psk.profile_enable(False)
     assert {"ltc_dense_norm_kernel", "ltc_wgrad_kernel", "tc_bwd_k_kernel"} <= kernels
+    if passes is not None:
+        # one first-normalisation launch per pass and tensor (Q, K), three times: the forward call, the
+        # backward call's half sketches (no kept states here) and its recomputation inside the chain rule
+        assert records.count("ltc_ln0_kernel") == 6 * passes
     for t in (O, den, dQ, dK, dV, dflat):
         assert torch.isfinite(t.float()).all()
     g1_sum = {k: 0.0 for k in orc.NET_KEYS}
@@ -138,7 +143,7 @@ def test_networks_in_several_passes_over_the_rows(monkeypatch):
     w = wl.small_workload(B=2, H=2, n=384, r=r, b=b, dtype="bf16", seed=91)
     inp = wl.make_inputs(w, "cuda")
     flat, P1, P2 = nets(r, 4)
-    _run_and_check(inp, w, flat, P1, P2, r, b, [(bi, hi) for bi in range(2) for hi in range(2)], TOL["bf16"], True)
+    _run_and_check(inp, w, flat, P1, P2, r, b, [(bi, hi) for bi in range(2) for hi in range(2)], TOL["bf16"], True, passes=6)
 
 
 @pytest.mark.parametrize("local", [False, True])
@@ -186,10 +191,13 @@ def test_kept_states_on_the_tensor_cores(local):
     O, den = binding.learned_attn_fwd(Q, K, V, flat, r, b, flags, ws)
     dQ, dK, dV, dflat = binding.learned_attn_bwd(Q, K, V, flat, O, den, dO, r, b, flags, ws)
     torch.cuda.synchronize()
-    kernels = {name for name, _ in psk.profile_records()}
+    records = [name for name, _ in psk.profile_records()]
+    kernels = set(records)
     psk.profile_enable(False)
     assert psk.check(ws) == 0
     assert "tc_bwd_prep_kernel" in kernels and "tc_bwd_recompute_kernel" not in kernels      # the kept states were used
+    # ... and the kept half sketches: they were formed once per tensor, by the forward call
+    assert records.count("ltc_combine_kernel") == 2
     diag = "exact" if local else "LR"
     for bi, hi in ((0, 1), (1, 0)):
         f = lambda k: head_slice_f64(inp[k], bi, hi)
@@ -207,7 +215,7 @@ def test_networks_across_the_default_chunk_boundary():
     w = wl.small_workload(B=4, H=12, n=32768, r=r, b=b, dtype="bf16", seed=92)
     inp = wl.make_inputs(w, "cuda")
     flat, P1, P2 = nets(r, 5)
-    _run_and_check(inp, w, flat, P1, P2, r, b, [(2, 7), (2, 8), (3, 11)], TOL["bf16"], False, bwd_heads=[(2, 8)])
+    _run_and_check(inp, w, flat, P1, P2, r, b, [(2, 7), (2, 8), (3, 11)], TOL["bf16"], False, bwd_heads=[(2, 8)], passes=2)
 
 
 def test_refusals():
