@@ -75,8 +75,8 @@ int make_dims(const psk_shape* sh, Dims* d) {
     return PSK_OK;
 }
 
-// 0 = CUDA cores, 1 = tensor cores, 2 = tensor cores on half sketches formed by the CUDA-core sketch
-// kernels (degree 8, learnable sketch), <0 = error
+// 0 = CUDA cores, 1 = tensor cores, 2 = tensor cores on half sketches formed by sketch kernels of
+// their own (degree 8, learnable sketch: psk_given.cu), <0 = error
 int pick_path(const psk_shape* sh, const Dims& d, bool backward) {
     if (sh->path == PSK_PATH_CUDA_CORES) return 0;
     if (given_supported(d)) return 2;

@@ -72,8 +72,8 @@ cudaError_t learned_sketch_bwd(const Dims& d, const void* X, const float* dM, co
 cudaError_t cc_sketch_bwd(const Dims& d, const void* X, const void* G1, const void* G2, const float* dM,
                           const float* add, void* dX, cudaStream_t s, int* launches);
 
-// Degree 8 and the learnable sketch on the tensor cores: half sketches by the CUDA-core sketch
-// kernels, attention on them by the tensor-core kernels (psk_given.cu).
+// Degree 8 and the learnable sketch on the tensor cores: half sketches by their own tensor-core
+// sketch kernels, attention on them by the tensor-core kernels in linear sketch mode (psk_given.cu).
 bool given_supported(const Dims& d);
 size_t given_workspace_bytes(const Dims& d, bool backward);
 cudaError_t given_fwd(const Dims& d, const void* Q, const void* K, const void* V, const void* G1, const void* G2,
